@@ -1,0 +1,160 @@
+"""ctypes wrapper around the C oracle (oracle/kroquant_oracle.c).
+
+TEST INFRASTRUCTURE: see the header of the C file.  Arrays are NumPy; bf16
+tensors are uint16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes as C
+
+import numpy as np
+
+from .build import build
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        i64, i32, vp = C.c_int64, C.c_int, C.c_void_p
+        L.kq_oracle_lu_to_factors.argtypes = [vp, i32, vp]
+        L.kq_oracle_lu_to_factors.restype = None
+        L.kq_oracle_dense_k.argtypes = [vp, vp]
+        L.kq_oracle_dense_k.restype = None
+        L.kq_oracle_dense_kinv.argtypes = [vp, vp]
+        L.kq_oracle_dense_kinv.restype = None
+        L.kq_oracle_transform.argtypes = [vp, i64, i32, vp, i32, vp]
+        L.kq_oracle_scale_transform.argtypes = [vp, i64, i32, vp, vp]
+        L.kq_oracle_widen.argtypes = [vp, i64, i32, vp]
+        L.kq_oracle_encode_block.argtypes = [vp, vp, vp]
+        L.kq_oracle_encode_block.restype = None
+        L.kq_oracle_mx_encode.argtypes = [vp, i64, i32, vp, vp]
+        L.kq_oracle_quantize.argtypes = [vp, i64, i32, vp, i32, vp, vp, vp]
+        L.kq_oracle_scale_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
+        L.kq_oracle_dequantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, i32]
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise ValueError("oracle: bad shape (d must be a positive multiple of 32, "
+                         "n_sets must be 1 or d/32)")
+
+
+def _x(X):
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    assert X.ndim == 2
+    return X
+
+
+def _g(G):
+    G = np.ascontiguousarray(G, dtype=np.float32)
+    assert G.ndim == 4 and G.shape[1:] == (5, 2, 2)
+    return G
+
+
+def lu_to_factors(abc) -> np.ndarray:
+    abc = np.ascontiguousarray(abc, dtype=np.float32)
+    assert abc.ndim == 3 and abc.shape[1:] == (5, 3)
+    G = np.empty((abc.shape[0], 5, 2, 2), np.float32)
+    lib().kq_oracle_lu_to_factors(_p(abc), abc.shape[0], _p(G))
+    return G
+
+
+def dense_k(G1) -> np.ndarray:
+    G1 = np.ascontiguousarray(G1, dtype=np.float32).reshape(5, 2, 2)
+    K = np.empty((32, 32), np.float64)
+    lib().kq_oracle_dense_k(_p(G1), _p(K))
+    return K
+
+
+def dense_kinv(G1) -> np.ndarray:
+    G1 = np.ascontiguousarray(G1, dtype=np.float32).reshape(5, 2, 2)
+    K = np.empty((32, 32), np.float64)
+    lib().kq_oracle_dense_kinv(_p(G1), _p(K))
+    return K
+
+
+def transform(X, G) -> np.ndarray:
+    X, G = _x(X), _g(G)
+    Y = np.empty(X.shape, np.float32)
+    _check(lib().kq_oracle_transform(_p(X), X.shape[0], X.shape[1], _p(G), G.shape[0], _p(Y)))
+    return Y
+
+
+def scale_transform(X, s) -> np.ndarray:
+    X = _x(X)
+    s = np.ascontiguousarray(s, dtype=np.float32)
+    assert s.shape == (X.shape[1],)
+    Y = np.empty(X.shape, np.float32)
+    _check(lib().kq_oracle_scale_transform(_p(X), X.shape[0], X.shape[1], _p(s), _p(Y)))
+    return Y
+
+
+def widen(X) -> np.ndarray:
+    X = _x(X)
+    Y = np.empty(X.shape, np.float32)
+    _check(lib().kq_oracle_widen(_p(X), X.shape[0], X.shape[1], _p(Y)))
+    return Y
+
+
+def encode_block(y32) -> tuple[np.ndarray, int]:
+    y = np.ascontiguousarray(y32, dtype=np.float32)
+    assert y.shape == (32,)
+    q = np.empty(16, np.uint8)
+    s = np.empty(1, np.uint8)
+    lib().kq_oracle_encode_block(_p(y), _p(q), _p(s))
+    return q, int(s[0])
+
+
+def mx_encode(Y) -> tuple[np.ndarray, np.ndarray]:
+    Y = np.ascontiguousarray(Y, dtype=np.float32)
+    t, d = Y.shape
+    if d <= 0 or d % 32:
+        _check(-1)
+    q = np.empty((t, d // 2), np.uint8)
+    s = np.empty((t, d // 32), np.uint8)
+    _check(lib().kq_oracle_mx_encode(_p(Y), t, d, _p(q), _p(s)))
+    return q, s
+
+
+def quantize(X, G):
+    """-> (q_packed, scales, Y) with Y the float pre-rounding values."""
+    Y = transform(X, G)
+    q, s = mx_encode(Y)
+    return q, s, Y
+
+
+def scale_quantize(X, svec):
+    Y = scale_transform(X, svec)
+    q, s = mx_encode(Y)
+    return q, s, Y
+
+
+def plain_quantize(X):
+    Y = widen(X)
+    q, s = mx_encode(Y)
+    return q, s, Y
+
+
+def dequantize(q, scales, G=None, out_bf16: bool = False) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    t, half = q.shape
+    d = half * 2
+    assert scales.shape == (t, d // 32)
+    out = np.empty((t, d), np.uint16 if out_bf16 else np.float32)
+    if G is None:
+        gp, ns = None, 0
+    else:
+        G = _g(G)
+        gp, ns = _p(G), G.shape[0]
+    _check(lib().kq_oracle_dequantize(_p(q), _p(scales), t, d, gp, ns, _p(out), int(out_bf16)))
+    return out
