@@ -1,0 +1,138 @@
+/*
+ * kroquant.h -- C ABI of the B200 (sm_100a) KroQuant online activation quantizer.
+ *
+ * The operation (paper Sections 3.1, 3.2, 3.5, 4.1; Appendix D):
+ *   X[tokens][d] (bf16, row-major)  is split, row by row, into d/32 blocks of 32
+ *   consecutive channels.  Block j of every row is multiplied from the left into
+ *   a 32x32 matrix  K^(j) = G1 (x) G2 (x) G3 (x) G4 (x) G5  (five 2x2 factors;
+ *   factor k reads bit 5-k of the row/column index:  K[r][c] = prod_k
+ *   G_k[r_{5-k}][c_{5-k}],  y_c = sum_r x_r K[r][c]),  and the 32 transformed
+ *   values are encoded as MXFP4: one E8M0 scale byte  S = clamp(floor(log2 amax)
+ *   - 2 + 127, 0, 254)  (0 for an all-zero block) and 32 E2M1 codes of
+ *   y_c * 2^(127-S), round-to-nearest-even, saturating at +-6, sign bit kept.
+ *
+ * Layouts (all row-major, contiguous, caller-owned DEVICE memory unless marked host):
+ *   X         bf16   [tokens][d]
+ *   q_packed  uint8  [tokens][d/2]    byte i of a row = code[2i] | code[2i+1] << 4
+ *   scales    uint8  [tokens][d/32]   one E8M0 byte per block
+ *   factors   float  [n_sets][5][2][2] (HOST), G_k[r][c] row-major, k = 1..5;
+ *             n_sets == 1 (one set shared by every block of the layer) or
+ *             n_sets == d/32 (set j belongs to block j).
+ *
+ * Conventions:
+ *   - every hot call is asynchronous on `stream` (a cudaStream_t passed as void*,
+ *     NULL = the legacy default stream), never synchronizes, never allocates,
+ *     never throws; errors are return codes and nothing is launched on error;
+ *   - tokens == 0 is KQ_OK and launches nothing;
+ *   - X, q_packed and float outputs must be 16-byte aligned (KQ_ERR_ALIGN);
+ *   - inputs must be finite; non-finite input gives unspecified codes, no fault;
+ *   - there is no CPU fallback: without a CUDA device every hot call returns
+ *     KQ_ERR_CUDA.
+ */
+#ifndef KROQUANT_H
+#define KROQUANT_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KQ_OK = 0,
+    KQ_ERR_NULL = 1,         /* a required pointer is NULL */
+    KQ_ERR_SHAPE = 2,        /* d <= 0, d % 32 != 0, tokens < 0, tokens*d/32 >= 2^31 */
+    KQ_ERR_ALIGN = 3,        /* a device pointer is not 16-byte aligned */
+    KQ_ERR_FACTORS = 4,      /* n_sets not in {1, d/32}, non-finite or singular factor */
+    KQ_ERR_UNSUPPORTED = 5,  /* unknown enum value */
+    KQ_ERR_CUDA = 6          /* a CUDA call or launch failed (no device, bad pointer kind, ...) */
+} kq_status_t;
+
+typedef enum { KQ_OUT_F32 = 0, KQ_OUT_BF16 = 1 } kq_dtype_t;
+
+/* Which device code applies the transform in kroquant_quantize / kroquant_transform_f32.
+ * KQ_PATH_AUTO picks the tensor-core kernel (tcgen05 + TMA) whenever it applies. */
+typedef enum { KQ_PATH_AUTO = 0, KQ_PATH_TENSOR = 1, KQ_PATH_ALU = 2 } kq_path_t;
+
+/* Opaque, immutable after creation; belongs to the device that was current at creation. */
+typedef struct kroquant_factors kroquant_factors_t;
+
+/* Section 3.2 (Kronecker product construction).  Copies G_host (HOST,
+ * [n_sets][5][2][2]) and uploads what the kernels need (the factors, their 2x2
+ * inverses, and a 3-term bf16 image of every dense K).  Allocates device memory;
+ * synchronizes the device once.  A factor with |det| < 1e-12 * ||G||_F^2 or a
+ * non-finite entry gives KQ_ERR_FACTORS. */
+kq_status_t kroquant_factors_create(const float *G_host, int n_sets, kroquant_factors_t **out);
+
+/* Section 3.2 (unit-determinant LU parametrisation): abc_host (HOST, [n_sets][5][3])
+ * holds (a_k, b_k, c_k);  G_k = [[1,0],[c,1]] * [[a,b],[0,-1/a]] = [[a, b],[a c, b c - 1/a]].
+ * a == 0 gives KQ_ERR_FACTORS. */
+kq_status_t kroquant_factors_create_lu(const float *abc_host, int n_sets, kroquant_factors_t **out);
+
+/* Frees host and device storage.  NULL is allowed.  No kernel using it may be in flight. */
+void kroquant_factors_destroy(kroquant_factors_t *f);
+
+/* Copies the factor matrices G[n_sets][5][2][2] back to HOST memory (for checking the LU helper). */
+kq_status_t kroquant_factors_get(const kroquant_factors_t *f, float *G_host_out);
+int kroquant_factors_n_sets(const kroquant_factors_t *f);
+
+/* Sections 3.1 + 3.5: the online quantizer  (X, factors) -> MXFP4(X T),
+ * T = diag(K^(1) .. K^(d/32)).  One kernel launch. */
+kq_status_t kroquant_quantize(const void *X, int64_t tokens, int d, const kroquant_factors_t *f,
+                              uint8_t *q_packed, uint8_t *scales, void *stream);
+
+/* Same, with the transform code path chosen by the caller (tests and ablations). */
+kq_status_t kroquant_quantize_path(const void *X, int64_t tokens, int d,
+                                   const kroquant_factors_t *f, uint8_t *q_packed,
+                                   uint8_t *scales, kq_path_t path, void *stream);
+
+/* Section 3.1 (quantize-then-DEquantize operator Q_b), decode half.
+ * f == NULL: out = decoded transformed values  grid[code & 7] * sign * 2^(S-127)
+ * (what a W4A4 GEMM consumes).  With factors: additionally multiplied by
+ * K^-1 = G1^-1 (x) .. (x) G5^-1 (Section 3.2), so out ~ X.  out: [tokens][d] of out_dtype. */
+kq_status_t kroquant_dequantize(const uint8_t *q_packed, const uint8_t *scales, int64_t tokens,
+                                int d, const kroquant_factors_t *f_or_null, void *out,
+                                kq_dtype_t out_dtype, void *stream);
+
+/* Appendix D "Smoothing" / Section 4.4 "Scale": per-channel multiply y = x * s_i
+ * (s: DEVICE float [d], the diagonal of T; SmoothQuant's 1/gamma) followed by the
+ * same MXFP4 encoder.  The in-run comparison kernel. */
+kq_status_t kroquant_scale_quantize(const void *X, int64_t tokens, int d, const float *s,
+                                    uint8_t *q_packed, uint8_t *scales, void *stream);
+
+/* Section 4.4 "Q4": the bare fused MXFP4 encoder (no transform), the lower bound
+ * every transform variant is compared with. */
+kq_status_t kroquant_mxfp4_quantize(const void *X, int64_t tokens, int d, uint8_t *q_packed,
+                                    uint8_t *scales, void *stream);
+
+/* Debug/parity export of the pre-rounding values: Y[tokens][d] (DEVICE float) =
+ * X T, produced by the same device code as kroquant_quantize_path up to the
+ * encoder. */
+kq_status_t kroquant_transform_f32(const void *X, int64_t tokens, int d,
+                                   const kroquant_factors_t *f, float *Y, kq_path_t path,
+                                   void *stream);
+
+/* Section 4.1 "Data format": exhaustive self-check of the hardware float -> E2M1
+ * convert used by the encoder.  Writes, for each of the n float inputs v (DEVICE),
+ * the 4-bit code the encoder's convert instruction gives (DEVICE uint8 [n]). */
+kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes, void *stream);
+
+/* Tuning hook for the tensor-core kernel: config 0..3 selects (smem stages, TMEM
+ * accumulator slots, epilogue warpgroups) = (8,8,1), (8,8,2), (12,16,2), (12,16,4);
+ * ctas_per_sm in 1..4 caps the persistent grid.  Process-wide. */
+kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm);
+
+/* Number of kernels this library has launched in the calling process (all streams). */
+int64_t kroquant_launch_count(void);
+
+/* Device-side error word of the tensor-core kernel: 0 = none; otherwise the code
+ * of the bounded wait that gave up (the kernel then returns early and the output
+ * of that call is unspecified).  Reads and clears it; synchronizes `stream`. */
+kq_status_t kroquant_last_device_error(void *stream, int *code_out);
+
+const char *kroquant_status_string(kq_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KROQUANT_H */

@@ -113,3 +113,23 @@ def decode(q: np.ndarray, scales: np.ndarray) -> np.ndarray:
     sign = np.where(code & 8, -1.0, 1.0)
     sc = np.exp2(np.asarray(scales, dtype=np.float64) - 127.0)
     return (mag * sign).reshape(t, d // BLOCK, BLOCK) * sc[:, :, None]
+
+
+def encode_with_scale(Y: np.ndarray, S: np.ndarray) -> np.ndarray:
+    """Codes (one per element, uint8 [t, d]) of float32 Y when the scale bytes S
+    [t, d/32] are imposed instead of derived from the block amax.  Used by the
+    parity rule that lets a block whose amax sits within rounding distance of a
+    power of two take the neighbouring scale."""
+    Y = np.asarray(Y, dtype=np.float32)
+    t, d = Y.shape
+    nb = d // BLOCK
+    v = Y.reshape(t, nb, BLOCK).astype(np.float64) * np.exp2(127.0 - np.asarray(S, np.float64))[:, :, None]
+    av = np.abs(v)
+    bounds = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0])
+    # ties to the even code: boundaries 0.25, 1.25, 2.5, 5.0 round down (<=), the others up
+    mag = np.zeros(av.shape, np.int64)
+    for i, b in enumerate(bounds):
+        down = i % 2 == 0           # boundary between code i (even when i even) and i+1
+        mag += (av > b) if down else (av >= b)
+    code = mag | (np.signbit(v).astype(np.int64) << 3)
+    return code.reshape(t, d).astype(np.uint8)

@@ -1,0 +1,237 @@
+"""Thin ctypes binding over libkroquant.so (include/kroquant.h).
+
+Argument marshalling only: every step of the quantizer runs in the CUDA
+kernels behind the C ABI.  torch is used for device memory and streams.  There
+is no CPU fallback: if the library cannot be loaded, or a call returns a
+non-zero status, a :class:`KroQuantError` is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libkroquant.so")
+
+KQ_OK = 0
+PATHS = {"auto": 0, "tensor": 1, "alu": 2}
+EXPORTS = [
+    "kroquant_factors_create", "kroquant_factors_create_lu", "kroquant_factors_destroy",
+    "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize",
+    "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
+    "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
+    "kroquant_debug_set_umma_config", "kroquant_launch_count", "kroquant_last_device_error",
+    "kroquant_status_string",
+]
+
+
+class KroQuantError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def load_library() -> C.CDLL:
+    """Load libkroquant.so (built in-tree by ``paper_2607_21446_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2607_21446_b200.build` "
+            "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int
+    L.kroquant_factors_create.argtypes = [vp, i32, C.POINTER(vp)]
+    L.kroquant_factors_create_lu.argtypes = [vp, i32, C.POINTER(vp)]
+    L.kroquant_factors_destroy.argtypes = [vp]
+    L.kroquant_factors_destroy.restype = None
+    L.kroquant_factors_get.argtypes = [vp, vp]
+    L.kroquant_factors_n_sets.argtypes = [vp]
+    L.kroquant_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
+    L.kroquant_quantize_path.argtypes = [vp, i64, i32, vp, vp, vp, i32, vp]
+    L.kroquant_dequantize.argtypes = [vp, vp, i64, i32, vp, vp, i32, vp]
+    L.kroquant_scale_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
+    L.kroquant_mxfp4_quantize.argtypes = [vp, i64, i32, vp, vp, vp]
+    L.kroquant_transform_f32.argtypes = [vp, i64, i32, vp, vp, i32, vp]
+    L.kroquant_debug_e2m1_codes.argtypes = [vp, i64, vp, vp]
+    L.kroquant_debug_set_umma_config.argtypes = [i32, i32]
+    L.kroquant_launch_count.argtypes = []
+    L.kroquant_launch_count.restype = i64
+    L.kroquant_last_device_error.argtypes = [vp, C.POINTER(i32)]
+    L.kroquant_status_string.argtypes = [i32]
+    L.kroquant_status_string.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return load_library().kroquant_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != KQ_OK:
+        raise KroQuantError(status, where)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _x_shape(X: torch.Tensor) -> tuple[int, int]:
+    if X.dim() != 2 or X.dtype != torch.bfloat16 or not X.is_cuda or not X.is_contiguous():
+        raise ValueError("X must be a contiguous 2-D CUDA bfloat16 tensor [tokens, d]")
+    return X.shape[0], X.shape[1]
+
+
+class Factors:
+    """Handle of a kroquant_factors_t.  G: float32 [n_sets, 5, 2, 2] (host)."""
+
+    def __init__(self, handle: int, n_sets: int):
+        self._h = C.c_void_p(handle)
+        self.n_sets = n_sets
+
+    @classmethod
+    def create(cls, G) -> "Factors":
+        G = np.ascontiguousarray(G, dtype=np.float32)
+        if G.ndim != 4 or G.shape[1:] != (5, 2, 2):
+            raise ValueError("G must have shape [n_sets, 5, 2, 2]")
+        out = C.c_void_p()
+        _check(load_library().kroquant_factors_create(G.ctypes.data_as(C.c_void_p), G.shape[0],
+                                                      C.byref(out)), "kroquant_factors_create")
+        return cls(out.value, G.shape[0])
+
+    @classmethod
+    def create_lu(cls, abc) -> "Factors":
+        abc = np.ascontiguousarray(abc, dtype=np.float32)
+        if abc.ndim != 3 or abc.shape[1:] != (5, 3):
+            raise ValueError("abc must have shape [n_sets, 5, 3]")
+        out = C.c_void_p()
+        _check(load_library().kroquant_factors_create_lu(abc.ctypes.data_as(C.c_void_p), abc.shape[0],
+                                                         C.byref(out)), "kroquant_factors_create_lu")
+        return cls(out.value, abc.shape[0])
+
+    def get(self) -> np.ndarray:
+        G = np.empty((self.n_sets, 5, 2, 2), np.float32)
+        _check(load_library().kroquant_factors_get(self._h, G.ctypes.data_as(C.c_void_p)),
+               "kroquant_factors_get")
+        return G
+
+    def destroy(self) -> None:
+        if self._h:
+            load_library().kroquant_factors_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def kroquant_quantize(X: torch.Tensor, factors: Factors, q_packed: Optional[torch.Tensor] = None,
+                      scales: Optional[torch.Tensor] = None, path: str = "auto", stream=None):
+    """(X bf16 [tokens, d], factors) -> (q_packed uint8 [tokens, d/2], scales uint8 [tokens, d/32])."""
+    tokens, d = _x_shape(X)
+    if q_packed is None:
+        q_packed = torch.empty((tokens, max(d // 2, 0)), dtype=torch.uint8, device=X.device)
+    if scales is None:
+        scales = torch.empty((tokens, max(d // 32, 0)), dtype=torch.uint8, device=X.device)
+    _check(load_library().kroquant_quantize_path(_ptr(X), tokens, d, factors._h, _ptr(q_packed),
+                                                 _ptr(scales), PATHS[path], C.c_void_p(_stream(stream))),
+           "kroquant_quantize")
+    return q_packed, scales
+
+
+def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, scales=None, stream=None):
+    tokens, d = _x_shape(X)
+    if s.dtype != torch.float32 or not s.is_cuda or s.numel() != d or not s.is_contiguous():
+        raise ValueError("s must be a contiguous CUDA float32 tensor [d]")
+    if q_packed is None:
+        q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
+    if scales is None:
+        scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
+    _check(load_library().kroquant_scale_quantize(_ptr(X), tokens, d, _ptr(s), _ptr(q_packed),
+                                                  _ptr(scales), C.c_void_p(_stream(stream))),
+           "kroquant_scale_quantize")
+    return q_packed, scales
+
+
+def kroquant_mxfp4_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=None):
+    tokens, d = _x_shape(X)
+    if q_packed is None:
+        q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
+    if scales is None:
+        scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
+    _check(load_library().kroquant_mxfp4_quantize(_ptr(X), tokens, d, _ptr(q_packed), _ptr(scales),
+                                                  C.c_void_p(_stream(stream))), "kroquant_mxfp4_quantize")
+    return q_packed, scales
+
+
+def kroquant_transform_f32(X: torch.Tensor, factors: Factors, Y=None, path: str = "auto", stream=None):
+    tokens, d = _x_shape(X)
+    if Y is None:
+        Y = torch.empty((tokens, d), dtype=torch.float32, device=X.device)
+    _check(load_library().kroquant_transform_f32(_ptr(X), tokens, d, factors._h, _ptr(Y), PATHS[path],
+                                                 C.c_void_p(_stream(stream))), "kroquant_transform_f32")
+    return Y
+
+
+def kroquant_dequantize(q_packed: torch.Tensor, scales: torch.Tensor, factors: Optional[Factors] = None,
+                        out_dtype=torch.float32, out=None, stream=None):
+    tokens, half = q_packed.shape
+    d = half * 2
+    if out is None:
+        out = torch.empty((tokens, d), dtype=out_dtype, device=q_packed.device)
+    code = {torch.float32: 0, torch.bfloat16: 1}[out.dtype]
+    _check(load_library().kroquant_dequantize(_ptr(q_packed), _ptr(scales), tokens, d,
+                                              factors._h if factors is not None else None, _ptr(out), code,
+                                              C.c_void_p(_stream(stream))), "kroquant_dequantize")
+    return out
+
+
+def kroquant_debug_e2m1_codes(v: torch.Tensor, stream=None) -> torch.Tensor:
+    codes = torch.empty(v.numel(), dtype=torch.uint8, device=v.device)
+    _check(load_library().kroquant_debug_e2m1_codes(_ptr(v), v.numel(), _ptr(codes),
+                                                    C.c_void_p(_stream(stream))), "kroquant_debug_e2m1_codes")
+    return codes
+
+
+def kroquant_debug_set_umma_config(config: int, ctas_per_sm: int) -> None:
+    _check(load_library().kroquant_debug_set_umma_config(config, ctas_per_sm),
+           "kroquant_debug_set_umma_config")
+
+
+def kroquant_launch_count() -> int:
+    return int(load_library().kroquant_launch_count())
+
+
+def kroquant_last_device_error(stream=None) -> int:
+    code = C.c_int(0)
+    _check(load_library().kroquant_last_device_error(C.c_void_p(_stream(stream)), C.byref(code)),
+           "kroquant_last_device_error")
+    return int(code.value)
+
+
+# ---- host-buffer convenience used for end-to-end timing -------------------------
+def quantize_from_host(X_host: torch.Tensor, factors: Factors, X_dev: torch.Tensor, q_dev: torch.Tensor,
+                       s_dev: torch.Tensor, q_host: torch.Tensor, s_host: torch.Tensor, stream=None):
+    """Pinned host X -> device, quantize, codes + scales -> pinned host.  All async on `stream`."""
+    X_dev.copy_(X_host, non_blocking=True)
+    kroquant_quantize(X_dev, factors, q_dev, s_dev, stream=stream)
+    q_host.copy_(q_dev, non_blocking=True)
+    s_host.copy_(s_dev, non_blocking=True)
+    return q_host, s_host

@@ -1,0 +1,197 @@
+// Streaming CUDA-core kernels: four threads own one 32-channel block (8 channels =
+// one 16-byte load each), so every global access is a fully coalesced 128-bit
+// vector and the block amax is two quad shuffles.
+//
+//   quantize_stream<MODE>   MODE_PLAIN  bare MXFP4 encoder ("Q4", Section 4.4)
+//                           MODE_SCALE  per-channel multiply + encoder ("Scale")
+//                           MODE_KRON   five-stage 2x2 butterfly + encoder: the
+//                                       transform y = x (G1 (x) .. (x) G5) applied
+//                                       factor by factor (Section 3.2 / 3.5)
+//   transform_stream        the butterfly alone, float output (parity export)
+//   dequantize_stream       decode (+ optional inverse butterfly, Section 3.2)
+#pragma once
+#include "kq_common.cuh"
+
+namespace kq {
+
+enum { MODE_PLAIN = 0, MODE_SCALE = 1, MODE_KRON = 2 };
+
+// One factor set as the kernels read it: g[k] = {G_k[0][0], G_k[0][1], G_k[1][0], G_k[1][1]}.
+struct FactorSet { float4 g[5]; };
+
+// y = x K for the 8 channels of this thread (channel index c = 8*quad + i).
+// Factors 3,4,5 mix index bits 2,1,0 (inside the thread); factors 1,2 mix bits 4,3
+// (across the quad, by shuffle).  Stage order k = 1..5 is free (the stages commute).
+__device__ __forceinline__ void kron_butterfly(float (&x)[8], const FactorSet& F, int quad) {
+    // in-thread stages: bit b of i, factor index k = 4 - b (0-based)
+#pragma unroll
+    for (int b = 2; b >= 0; --b) {
+        const float4 g = F.g[4 - b];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (!(i & (1 << b))) {
+                const int lo = i, hi = i | (1 << b);
+                const float xl = x[lo], xh = x[hi];
+                x[lo] = fmaf(xh, g.z, xl * g.x);   // x_lo G[0][0] + x_hi G[1][0]
+                x[hi] = fmaf(xh, g.w, xl * g.y);   // x_lo G[0][1] + x_hi G[1][1]
+            }
+        }
+    }
+    // cross-thread stages: quad bit 0 <-> index bit 3 (factor 2), quad bit 1 <-> bit 4 (factor 1)
+#pragma unroll
+    for (int qb = 0; qb < 2; ++qb) {
+        const float4 g = F.g[1 - qb];
+        const int tb = (quad >> qb) & 1;
+        // mine is the lo element when tb == 0, the hi element when tb == 1
+        const float g_mine = tb ? g.w : g.x;     // G[tb][tb]
+        const float g_other = tb ? g.y : g.z;    // G[1-tb][tb]
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float other = __shfl_xor_sync(0xFFFFFFFFu, x[i], 1 << qb);
+            x[i] = fmaf(other, g_other, x[i] * g_mine);
+        }
+    }
+}
+
+// Encode the thread's 8 values given the quad's block amax; lane quad==0 also writes the scale.
+__device__ __forceinline__ uint32_t encode8(const float (&y)[8], float amax_block, uint32_t& S_out) {
+    const uint32_t S = e8m0_from_amax(amax_block);
+    const float inv = inv_scale_from_e8m0(S);
+    S_out = S;
+    return e2m1x8(y[0] * inv, y[1] * inv, y[2] * inv, y[3] * inv,
+                  y[4] * inv, y[5] * inv, y[6] * inv, y[7] * inv);
+}
+
+// n_quads = tokens * d / 8 work items; item q: block = q / 4, quad = q % 4.
+// factors: n_sets FactorSet (MODE_KRON); chan_scale: float[d] (MODE_SCALE).
+template <int MODE, bool WRITE_Y>
+__global__ void __launch_bounds__(256)
+quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row,
+                const FactorSet* __restrict__ factors, int n_sets,
+                const float* __restrict__ chan_scale,
+                uint32_t* __restrict__ q_packed, uint8_t* __restrict__ scales,
+                float* __restrict__ Y) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;   // multiple of 32: quads stay lane-aligned
+    const int quad = threadIdx.x & 3;
+    FactorSet F;
+    if (MODE == MODE_KRON && n_sets == 1) F = factors[0];
+    // the trip count is uniform across the warp: all lanes run the shuffles together
+    const int64_t n_iter = (n_quads + stride - 1) / stride;
+    int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t it = 0; it < n_iter; ++it, q += stride) {
+        const bool live = q < n_quads;
+        float y[8];
+        if (live) {
+            widen8(ld_stream_16(X + q), y);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) y[i] = 0.f;
+        }
+        const int64_t blk = q >> 2;
+        if (MODE == MODE_SCALE) {
+            if (live) {
+                const int j = (int)(blk % blocks_per_row);
+                const float4* sp = reinterpret_cast<const float4*>(chan_scale + j * kBlock + quad * 8);
+                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
+                y[0] *= s0.x; y[1] *= s0.y; y[2] *= s0.z; y[3] *= s0.w;
+                y[4] *= s1.x; y[5] *= s1.y; y[6] *= s1.z; y[7] *= s1.w;
+            }
+        } else if (MODE == MODE_KRON) {
+            if (n_sets != 1) {
+                const int j = live ? (int)(blk % blocks_per_row) : 0;
+                const float4* gp = reinterpret_cast<const float4*>(factors + j);
+#pragma unroll
+                for (int k = 0; k < 5; ++k) F.g[k] = __ldg(gp + k);
+            }
+            kron_butterfly(y, F, quad);
+        }
+        if (WRITE_Y) {
+            if (live) {
+                float4* yp = reinterpret_cast<float4*>(Y) + 2 * q;
+                yp[0] = make_float4(y[0], y[1], y[2], y[3]);
+                yp[1] = make_float4(y[4], y[5], y[6], y[7]);
+            }
+        } else {
+            float amax = absmax8(y);
+            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+            uint32_t S;
+            const uint32_t codes = encode8(y, amax, S);
+            if (live) {
+                st_stream_4(q_packed + q, codes);
+                if (quad == 0) scales[blk] = (uint8_t)S;
+            }
+        }
+    }
+}
+
+// codes + scales -> values.  Ginv: inverse factor sets (or nullptr: no inverse transform).
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(256)
+dequantize_stream(const uint32_t* __restrict__ q_packed, const uint8_t* __restrict__ scales,
+                  int64_t n_quads, int blocks_per_row, const FactorSet* __restrict__ Ginv,
+                  int n_sets, void* __restrict__ out) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int quad = threadIdx.x & 3;
+    FactorSet F;
+    if (Ginv != nullptr && n_sets == 1) F = Ginv[0];
+    const int64_t n_iter = (n_quads + stride - 1) / stride;
+    int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t it = 0; it < n_iter; ++it, q += stride) {
+        const bool live = q < n_quads;
+        const int64_t blk = q >> 2;
+        float y[8];
+        uint32_t codes = 0, S = 127;
+        if (live) {
+            codes = __ldg(q_packed + q);
+            S = __ldg(scales + blk);
+        }
+        const float sc = scale_from_e8m0(S);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t c = (codes >> (4 * i)) & 15u;
+            const uint32_t m = c & 7u;
+            // E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6: code 1 is the only subnormal
+            const float mag = (m < 2u) ? 0.5f * (float)m
+                                       : __uint_as_float(((126u + (m >> 1)) << 23) | ((m & 1u) << 22));
+            const float v = mag * sc;
+            y[i] = (c & 8u) ? -v : v;
+        }
+        if (Ginv != nullptr) {
+            if (n_sets != 1) {
+                const int j = live ? (int)(blk % blocks_per_row) : 0;
+                const float4* gp = reinterpret_cast<const float4*>(Ginv + j);
+#pragma unroll
+                for (int k = 0; k < 5; ++k) F.g[k] = __ldg(gp + k);
+            }
+            kron_butterfly(y, F, quad);
+        }
+        if (live) {
+            if (OUT_BF16) {
+                uint4 o;
+                uint32_t* w = &o.x;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    // round-to-nearest-even float -> bf16 on the bit pattern (finite inputs)
+                    uint32_t a = __float_as_uint(y[2 * i]), b = __float_as_uint(y[2 * i + 1]);
+                    a = (a + 0x7FFFu + ((a >> 16) & 1u)) >> 16;
+                    b = (b + 0x7FFFu + ((b >> 16) & 1u)) >> 16;
+                    w[i] = a | (b << 16);
+                }
+                reinterpret_cast<uint4*>(out)[q] = o;
+            } else {
+                float4* op = reinterpret_cast<float4*>(out) + 2 * q;
+                op[0] = make_float4(y[0], y[1], y[2], y[3]);
+                op[1] = make_float4(y[4], y[5], y[6], y[7]);
+            }
+        }
+    }
+}
+
+// float v[n] -> the 4-bit code the encoder's convert instruction gives for each.
+__global__ void e2m1_codes_kernel(const float* __restrict__ v, int64_t n, uint8_t* __restrict__ codes) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) codes[i] = (uint8_t)(e2m1x8(v[i], 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f) & 15u);
+}
+
+}  // namespace kq

@@ -1,0 +1,331 @@
+// Tensor-core KroQuant quantizer for sm_100a: TMA -> shared memory -> tcgen05.mma
+// (accumulators in TMEM) -> tcgen05.ld -> fused MXFP4 encoder in registers.
+//
+// Shared factor set (one K per layer).  Because every 32-channel block of every
+// token is multiplied by the same K (paper Section 3.5: "many column blocks share
+// the same Kronecker factors"), X[tokens][d] is viewed as a flat matrix of
+// n_blocks = tokens*d/32 rows of 32 bf16 (64 contiguous bytes each), and the whole
+// layer is one tall GEMM  Y[n_blocks][32] = Xflat[n_blocks][32] * K[32][32]
+// (Section 3.5: y = x K per block).  In this view the inputs, the 16-byte code
+// groups and the scale bytes of consecutive rows are all contiguous in HBM.
+//
+// Exactness.  X is bf16 and feeds the MMA unconverted.  K (a product of five floats,
+// formed in double on the host) is split into three bf16 terms K = K0 + K1 + K2
+// (8 + 8 + 8 significand bits), so every product x*K_t is exact in the fp32
+// accumulator and only the accumulation rounds.  The three terms are three
+// accumulating MMAs into the same TMEM tile.
+//
+// One CTA = 1 TMA producer warp, 1 MMA warp (one elected thread issues), and
+// NG epilogue warpgroups of 4 warps; thread t of an epilogue warpgroup owns TMEM
+// lane t = one 32-channel block: it reads its 32 accumulators with one
+// tcgen05.ld.32x32b.x32, takes the block amax without any shuffle, and stores one
+// 16-byte code vector + one scale byte (coalesced across the warp).
+//
+// Every mbarrier wait is bounded; a wait that gives up records a code in
+// g_kq_device_error, raises the CTA's abort flag and the CTA drains and frees
+// its TMEM before returning.
+#pragma once
+#include <cuda.h>
+#include "kq_common.cuh"
+
+namespace kq {
+
+__device__ int g_kq_device_error = 0;
+
+constexpr int kTileRows = 128;                    // blocks (flat rows) per MMA tile = TMEM lanes
+constexpr int kTileBytes = kTileRows * 64;        // 8 KB of bf16 per tile
+constexpr int kBTermBytes = 32 * 64;              // one bf16 term of K^T: 32 rows (n) x 64 B (k)
+constexpr int kBImageBytes = 3 * kBTermBytes;     // 6 KB per factor set
+constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // every mbarrier wait gives up after 1 s
+
+enum {
+    KQ_DEV_OK = 0,
+    KQ_DEV_TIMEOUT_PRODUCER = 1,
+    KQ_DEV_TIMEOUT_MMA_FULL = 2,
+    KQ_DEV_TIMEOUT_MMA_TMEM = 3,
+    KQ_DEV_TIMEOUT_EPILOGUE = 4,
+    KQ_DEV_TIMEOUT_B = 5,
+    KQ_DEV_TIMEOUT_DRAIN = 6
+};
+
+// ---- PTX wrappers --------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false once kWaitLimitNs has passed (checked every 256 failed
+// tries, and at most 2^26 tries in any case) or when the CTA has aborted.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t i = 1; i < (1u << 26); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+        }
+    }
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]; bf16 inputs, fp32 accumulate; M=128, N=32, K=16.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b,
+                                            uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 columns of 32-bit: thread i of the warp gets lane (base + i), columns 0..31.
+// The load and its completion wait are one asm statement, so no use of the registers can
+// be scheduled between them.
+__device__ __forceinline__ void tc_ld_32x32_wait(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+
+// K-major operand tile with 64-byte rows in the 64-byte-swizzle layout: 8-row groups
+// 512 bytes apart (stride byte offset), descriptor version 1 (sm_100), swizzle code 4.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)1 << 16;                 // leading byte offset (unused for one swizzle atom in K)
+    d |= (uint64_t)(512 >> 4) << 32;        // stride byte offset
+    d |= (uint64_t)1 << 46;                 // descriptor version
+    d |= (uint64_t)4 << 61;                 // SWIZZLE_64B
+    return d;
+}
+// kind::f16 instruction descriptor: D=f32, A=B=bf16, both K-major, N=32, M=128.
+constexpr uint32_t kIdescBf16M128N32 =
+    (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+
+// ---- shared memory plan ----------------------------------------------------------
+template <int NS, int NA>
+struct UmmaSmem {
+    static constexpr int kBOff = 0;                                  // 6 KB, 1024-aligned
+    static constexpr int kAOff = 8192;                               // NS stages of 8 KB
+    static constexpr int kBarOff = kAOff + NS * kTileBytes;
+    // barriers: full[NS], empty[NS], tfull[NA], tempty[NA], bfull
+    static constexpr int kNumBars = 2 * NS + 2 * NA + 1;
+    static constexpr int kTmemSlotOff = kBarOff + 8 * kNumBars;
+    static constexpr int kAbortOff = kTmemSlotOff + 4;
+    static constexpr int kBytes = kAbortOff + 4;
+    static constexpr int kDynBytes = kBytes + 1024;                  // slack for manual alignment
+};
+
+// The fused epilogue math of one 32-channel block held in registers.
+__device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uint4& codes, uint32_t& S) {
+    float amax = 0.f;
+#pragma unroll
+    for (int c = 0; c < 32; ++c) amax = fmaxf(amax, fabsf(__uint_as_float(acc[c])));
+    S = e8m0_from_amax(amax);
+    const float inv = inv_scale_from_e8m0(S);
+    uint32_t w[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        w[g] = e2m1x8(__uint_as_float(acc[8 * g + 0]) * inv, __uint_as_float(acc[8 * g + 1]) * inv,
+                      __uint_as_float(acc[8 * g + 2]) * inv, __uint_as_float(acc[8 * g + 3]) * inv,
+                      __uint_as_float(acc[8 * g + 4]) * inv, __uint_as_float(acc[8 * g + 5]) * inv,
+                      __uint_as_float(acc[8 * g + 6]) * inv, __uint_as_float(acc[8 * g + 7]) * inv);
+    }
+    codes = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// NS smem stages, NA TMEM accumulator slots (NA*32 columns, a power of two >= 32),
+// NG epilogue warpgroups.  Grid: any size <= number of tiles; CTA b takes tiles
+// b, b + gridDim.x, ...
+template <int NS, int NA, int NG, bool WRITE_Y>
+__global__ void __launch_bounds__(64 + 128 * NG, 1)
+quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ b_image,
+                     int64_t n_blocks, uint4* __restrict__ q_packed, uint8_t* __restrict__ scales,
+                     float* __restrict__ Y) {
+    using L = UmmaSmem<NS, NA>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* base_ptr = smem_raw + (base - raw);
+    const uint32_t bar0 = base + L::kBarOff;
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar0 + 8u * (NS + s); };
+    auto bar_tfull = [&](int a) { return bar0 + 8u * (2 * NS + a); };
+    auto bar_tempty = [&](int a) { return bar0 + 8u * (2 * NS + NA + a); };
+    const uint32_t bar_b = bar0 + 8u * (2 * NS + 2 * NA);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTmemSlotOff);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kAbortOff);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int64_t n_tiles = (n_blocks + kTileRows - 1) / kTileRows;
+    // local tile count of this CTA
+    const int my_tiles = (int)((n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int a = 0; a < NA; ++a) { mbar_init(bar_tfull(a), 1); mbar_init(bar_tempty(a), 4); }
+        mbar_init(bar_b, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + (uint32_t)L::kTmemSlotOff), "r"((uint32_t)(NA * 32)) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    int issued = 0;   // tiles whose TMA load this thread has issued (producer lane only)
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+            mbar_expect_tx(bar_b, kBImageBytes);
+            bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
+            for (int n = 0; n < my_tiles; ++n) {
+                const int s = n % NS;
+                if (n >= NS && !mbar_wait(bar_empty(s), ((n / NS) - 1) & 1, abort_flag)) {
+                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
+                    break;
+                }
+                const int64_t tile = blockIdx.x + (int64_t)n * gridDim.x;
+                mbar_expect_tx(bar_full(s), kTileBytes);
+                tma_load_2d(base + L::kAOff + s * kTileBytes, &tmap_x, 0, (int)(tile * kTileRows), bar_full(s));
+                issued = n + 1;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            bool ok = mbar_wait(bar_b, 0, abort_flag);
+            if (!ok && !*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
+            for (int n = 0; ok && n < my_tiles; ++n) {
+                const int s = n % NS, a = n % NA;
+                if (!mbar_wait(bar_full(s), (n / NS) & 1, abort_flag)) {
+                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_MMA_FULL); *abort_flag = 1; }
+                    break;
+                }
+                if (n >= NA && !mbar_wait(bar_tempty(a), ((n / NA) - 1) & 1, abort_flag)) {
+                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_MMA_TMEM); *abort_flag = 1; }
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t a_addr = base + L::kAOff + s * kTileBytes;
+                const uint32_t d_addr = tmem_base + (uint32_t)(a * 32);
+#pragma unroll
+                for (int t = 0; t < 3; ++t) {
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) {
+                        tc_mma_bf16(d_addr, smem_desc_sw64(a_addr + kk * 32),
+                                    smem_desc_sw64(base + L::kBOff + t * kBTermBytes + kk * 32),
+                                    kIdescBf16M128N32, (uint32_t)((t | kk) != 0));
+                    }
+                }
+                tc_commit(bar_empty(s));     // smem stage reusable once these MMAs have read it
+                tc_commit(bar_tfull(a));     // accumulator complete
+            }
+        }
+    } else {
+        // ---------------- epilogue warpgroups ----------------
+        const int g = (warp - 2) >> 2;             // warpgroup index
+        const int quarter = warp & 3;              // TMEM lane quarter this warp may read
+        for (int n = g; n < my_tiles; n += NG) {
+            const int a = n % NA;
+            if (!mbar_wait(bar_tfull(a), (n / NA) & 1, abort_flag)) {
+                if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_EPILOGUE); *abort_flag = 1; }
+                break;
+            }
+            tc_fence_after();
+            uint32_t acc[32];
+            tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * 32), acc);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty(a));
+            const int64_t tile = blockIdx.x + (int64_t)n * gridDim.x;
+            const int64_t row = tile * kTileRows + quarter * 32 + lane;
+            if (row < n_blocks) {
+                if (WRITE_Y) {
+                    float4* yp = reinterpret_cast<float4*>(Y + row * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        yp[i] = make_float4(__uint_as_float(acc[4 * i]), __uint_as_float(acc[4 * i + 1]),
+                                            __uint_as_float(acc[4 * i + 2]), __uint_as_float(acc[4 * i + 3]));
+                } else {
+                    uint4 codes;
+                    uint32_t S;
+                    encode_block_regs(acc, codes, S);
+                    st_stream_16(q_packed + row, codes);
+                    scales[row] = (uint8_t)S;
+                }
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) {
+        // abort path only: let the copies this thread issued land before the CTA's shared
+        // memory goes away (load m went to stage m % NS and completes phase (m / NS) & 1)
+        int never = 0;
+        (void)mbar_wait(bar_b, 0, &never);
+        for (int m = (issued > NS ? issued - NS : 0); m < issued; ++m)
+            if (!mbar_wait(bar_full(m % NS), (m / NS) & 1, &never))
+                atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_DRAIN);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"((uint32_t)(NA * 32)) : "memory");
+    }
+}
+
+}  // namespace kq

@@ -1,0 +1,402 @@
+// C ABI of the KroQuant quantizer (see include/kroquant.h): argument validation,
+// the factor object, kernel selection and launches.  No hot call allocates,
+// synchronizes or throws.
+#include "../../include/kroquant.h"
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "kq_stream.cuh"
+#include "kq_umma.cuh"
+
+struct kroquant_factors {
+    int n_sets = 0;
+    int device = -1;
+    bool identity = false;
+    std::vector<float> G;             // host copy [n_sets][5][2][2]
+    kq::FactorSet* d_G = nullptr;     // device [n_sets]
+    kq::FactorSet* d_Ginv = nullptr;  // device [n_sets], 2x2 inverses
+    uint8_t* d_bimage = nullptr;      // device [n_sets][6 KB]: 3-term bf16 image of K^T, 64B-swizzled
+};
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+
+// ---- tensor-core kernel configuration ----------------------------------------
+struct UmmaConfig { int id; int ns, na, ng; };
+std::atomic<int> g_umma_cfg{0};
+std::atomic<int> g_umma_ctas_per_sm{2};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+kq_status_t check_shape(int64_t tokens, int d) {
+    if (d <= 0 || d % 32 != 0 || tokens < 0) return KQ_ERR_SHAPE;
+    if (tokens > 0 && tokens > ((int64_t)1 << 31) / (d / 32) - 1) return KQ_ERR_SHAPE;  // tokens*d/32 < 2^31
+    return KQ_OK;
+}
+
+int stream_grid(int64_t n_quads) {
+    const int sms = sm_count();
+    if (sms <= 0) return 0;
+    const int64_t want = (n_quads + 255) / 256;
+    const int64_t cap = (int64_t)sms * 8;    // 8 x 256 threads = 2048 resident threads per SM
+    return (int)(want < cap ? want : cap);
+}
+
+// bf16 round-to-nearest-even of a double, returned as the bf16 bit pattern and its value
+uint16_t bf16_of(double v, double* back) {
+    float f = (float)v;
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    float g;
+    std::memcpy(&g, &u, 4);
+    *back = (double)g;
+    return (uint16_t)(u >> 16);
+}
+
+// K^T as three bf16 terms in the 64-byte-swizzled K-major operand layout the MMA reads:
+// element (n = c, k = r) of term t at byte  t*2048 + swz(c*64 + 2r),  swz(o) = o ^ (((o >> 7) & 3) << 4).
+void build_b_image(const float* G20, uint8_t* img) {
+    std::memset(img, 0, kq::kBImageBytes);
+    for (int r = 0; r < 32; ++r)
+        for (int c = 0; c < 32; ++c) {
+            double k = 1.0;
+            for (int f = 0; f < 5; ++f) {
+                const int bit = 4 - f;
+                k *= (double)G20[f * 4 + ((r >> bit) & 1) * 2 + ((c >> bit) & 1)];
+            }
+            double rest = k;
+            for (int t = 0; t < 3; ++t) {
+                double back;
+                const uint16_t b = bf16_of(rest, &back);
+                rest -= back;
+                uint32_t off = (uint32_t)(c * 64 + 2 * r);
+                off ^= ((off >> 7) & 3u) << 4;
+                std::memcpy(img + t * kq::kBTermBytes + off, &b, 2);
+            }
+        }
+}
+
+template <int NS, int NA, int NG, bool WRITE_Y>
+kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, int64_t n_blocks, uint4* q,
+                        uint8_t* scales, float* Y, int ctas_per_sm, cudaStream_t st) {
+    using L = kq::UmmaSmem<NS, NA>;
+    auto kern = kq::quantize_umma_shared<NS, NA, NG, WRITE_Y>;
+    static std::once_flag once;
+    static cudaError_t attr_rc = cudaSuccess;
+    std::call_once(once, [&] {
+        attr_rc = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynBytes);
+    });
+    if (attr_rc != cudaSuccess) return KQ_ERR_CUDA;
+    const int sms = sm_count();
+    if (sms <= 0) return KQ_ERR_CUDA;
+    const int64_t n_tiles = (n_blocks + kq::kTileRows - 1) / kq::kTileRows;
+    const int64_t cap = (int64_t)sms * ctas_per_sm;
+    const int grid = (int)(n_tiles < cap ? n_tiles : cap);
+    kern<<<grid, 64 + 128 * NG, L::kDynBytes, st>>>(tmap, bimg, n_blocks, q, scales, Y);
+    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
+}
+
+template <bool WRITE_Y>
+kq_status_t run_umma(const void* X, int64_t n_blocks, const kroquant_factors_t* f, uint8_t* q,
+                     uint8_t* scales, float* Y, cudaStream_t st) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return KQ_ERR_CUDA;
+    CUtensorMap tmap;
+    const cuuint64_t dims[2] = {32, (cuuint64_t)n_blocks};
+    const cuuint64_t strides[1] = {64};
+    const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return KQ_ERR_CUDA;
+    uint4* q4 = reinterpret_cast<uint4*>(q);
+    const int cps = g_umma_ctas_per_sm.load();
+    switch (g_umma_cfg.load()) {
+        default:
+        case 0: return launch_umma<8, 8, 1, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
+        case 1: return launch_umma<8, 8, 2, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
+        case 2: return launch_umma<12, 16, 2, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
+        case 3: return launch_umma<12, 16, 4, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
+    }
+}
+
+template <int MODE, bool WRITE_Y>
+kq_status_t run_stream(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, const float* s,
+                       uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
+    const int64_t n_quads = tokens * (int64_t)(d / 8);
+    const int grid = stream_grid(n_quads);
+    if (grid <= 0) return KQ_ERR_CUDA;
+    kq::quantize_stream<MODE, WRITE_Y><<<grid, 256, 0, st>>>(
+        reinterpret_cast<const uint4*>(X), n_quads, d / 32, f ? f->d_G : nullptr, f ? f->n_sets : 0, s,
+        reinterpret_cast<uint32_t*>(q), scales, Y);
+    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
+}
+
+kq_status_t check_factors_for(const kroquant_factors_t* f, int d) {
+    if (!f) return KQ_ERR_NULL;
+    if (f->n_sets != 1 && f->n_sets != d / 32) return KQ_ERR_FACTORS;
+    return KQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+kq_status_t kroquant_factors_create(const float* G_host, int n_sets, kroquant_factors_t** out) {
+    if (!G_host || !out) return KQ_ERR_NULL;
+    *out = nullptr;
+    if (n_sets <= 0) return KQ_ERR_FACTORS;
+    bool identity = true;
+    std::vector<kq::FactorSet> inv(n_sets), fwd(n_sets);
+    for (int s = 0; s < n_sets; ++s)
+        for (int k = 0; k < 5; ++k) {
+            const float* g = G_host + ((size_t)s * 5 + k) * 4;
+            for (int i = 0; i < 4; ++i)
+                if (!std::isfinite(g[i])) return KQ_ERR_FACTORS;
+            const double a = g[0], b = g[1], c = g[2], e = g[3];
+            const double det = a * e - b * c;
+            const double fro2 = a * a + b * b + c * c + e * e;
+            if (!(std::fabs(det) >= 1e-12 * fro2) || fro2 == 0.0) return KQ_ERR_FACTORS;
+            if (!(g[0] == 1.f && g[1] == 0.f && g[2] == 0.f && g[3] == 1.f)) identity = false;
+            fwd[s].g[k] = make_float4(g[0], g[1], g[2], g[3]);
+            inv[s].g[k] = make_float4((float)(e / det), (float)(-b / det), (float)(-c / det), (float)(a / det));
+        }
+    kroquant_factors_t* f = new (std::nothrow) kroquant_factors_t;
+    if (!f) return KQ_ERR_CUDA;
+    f->n_sets = n_sets;
+    f->identity = identity;
+    f->G.assign(G_host, G_host + (size_t)n_sets * 20);
+    std::vector<uint8_t> img((size_t)n_sets * kq::kBImageBytes);
+    for (int s = 0; s < n_sets; ++s) build_b_image(G_host + (size_t)s * 20, img.data() + (size_t)s * kq::kBImageBytes);
+    bool ok = cudaGetDevice(&f->device) == cudaSuccess;
+    ok = ok && cudaMalloc(&f->d_G, sizeof(kq::FactorSet) * n_sets) == cudaSuccess;
+    ok = ok && cudaMalloc(&f->d_Ginv, sizeof(kq::FactorSet) * n_sets) == cudaSuccess;
+    ok = ok && cudaMalloc(&f->d_bimage, img.size()) == cudaSuccess;
+    ok = ok && cudaMemcpy(f->d_G, fwd.data(), sizeof(kq::FactorSet) * n_sets, cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(f->d_Ginv, inv.data(), sizeof(kq::FactorSet) * n_sets, cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(f->d_bimage, img.data(), img.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        kroquant_factors_destroy(f);
+        return KQ_ERR_CUDA;
+    }
+    *out = f;
+    return KQ_OK;
+}
+
+kq_status_t kroquant_factors_create_lu(const float* abc_host, int n_sets, kroquant_factors_t** out) {
+    if (!abc_host || !out) return KQ_ERR_NULL;
+    *out = nullptr;
+    if (n_sets <= 0) return KQ_ERR_FACTORS;
+    std::vector<float> G((size_t)n_sets * 20);
+    for (int i = 0; i < n_sets * 5; ++i) {
+        const double a = abc_host[3 * i], b = abc_host[3 * i + 1], c = abc_host[3 * i + 2];
+        if (a == 0.0 || !std::isfinite(a) || !std::isfinite(b) || !std::isfinite(c)) return KQ_ERR_FACTORS;
+        G[4 * i + 0] = (float)a;
+        G[4 * i + 1] = (float)b;
+        G[4 * i + 2] = (float)(a * c);
+        G[4 * i + 3] = (float)(b * c - 1.0 / a);
+    }
+    return kroquant_factors_create(G.data(), n_sets, out);
+}
+
+void kroquant_factors_destroy(kroquant_factors_t* f) {
+    if (!f) return;
+    if (f->d_G) cudaFree(f->d_G);
+    if (f->d_Ginv) cudaFree(f->d_Ginv);
+    if (f->d_bimage) cudaFree(f->d_bimage);
+    delete f;
+}
+
+kq_status_t kroquant_factors_get(const kroquant_factors_t* f, float* G_host_out) {
+    if (!f || !G_host_out) return KQ_ERR_NULL;
+    std::memcpy(G_host_out, f->G.data(), f->G.size() * sizeof(float));
+    return KQ_OK;
+}
+
+int kroquant_factors_n_sets(const kroquant_factors_t* f) { return f ? f->n_sets : 0; }
+
+kq_status_t kroquant_quantize_path(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
+                                   uint8_t* q_packed, uint8_t* scales, kq_path_t path, void* stream) {
+    if (!X || !q_packed || !scales) return KQ_ERR_NULL;
+    kq_status_t rc = check_shape(tokens, d);
+    if (rc != KQ_OK) return rc;
+    rc = check_factors_for(f, d);
+    if (rc != KQ_OK) return rc;
+    if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
+    if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
+    if (tokens == 0) return KQ_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool shared = f->n_sets == 1;
+    if (path == KQ_PATH_TENSOR && !shared) return KQ_ERR_UNSUPPORTED;
+    if (path == KQ_PATH_AUTO && f->identity)
+        return run_stream<kq::MODE_PLAIN, false>(X, tokens, d, nullptr, nullptr, q_packed, scales, nullptr, st);
+    if (shared && path != KQ_PATH_ALU)
+        return run_umma<false>(X, tokens * (int64_t)(d / 32), f, q_packed, scales, nullptr, st);
+    return run_stream<kq::MODE_KRON, false>(X, tokens, d, f, nullptr, q_packed, scales, nullptr, st);
+}
+
+kq_status_t kroquant_quantize(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
+                              uint8_t* q_packed, uint8_t* scales, void* stream) {
+    return kroquant_quantize_path(X, tokens, d, f, q_packed, scales, KQ_PATH_AUTO, stream);
+}
+
+kq_status_t kroquant_transform_f32(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
+                                   float* Y, kq_path_t path, void* stream) {
+    if (!X || !Y) return KQ_ERR_NULL;
+    kq_status_t rc = check_shape(tokens, d);
+    if (rc != KQ_OK) return rc;
+    rc = check_factors_for(f, d);
+    if (rc != KQ_OK) return rc;
+    if (!aligned16(X) || !aligned16(Y)) return KQ_ERR_ALIGN;
+    if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
+    if (tokens == 0) return KQ_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool shared = f->n_sets == 1;
+    if (path == KQ_PATH_TENSOR && !shared) return KQ_ERR_UNSUPPORTED;
+    if (path == KQ_PATH_AUTO && f->identity)
+        return run_stream<kq::MODE_PLAIN, true>(X, tokens, d, nullptr, nullptr, nullptr, nullptr, Y, st);
+    if (shared && path != KQ_PATH_ALU)
+        return run_umma<true>(X, tokens * (int64_t)(d / 32), f, nullptr, nullptr, Y, st);
+    return run_stream<kq::MODE_KRON, true>(X, tokens, d, f, nullptr, nullptr, nullptr, Y, st);
+}
+
+kq_status_t kroquant_scale_quantize(const void* X, int64_t tokens, int d, const float* s, uint8_t* q_packed,
+                                    uint8_t* scales, void* stream) {
+    if (!X || !s || !q_packed || !scales) return KQ_ERR_NULL;
+    kq_status_t rc = check_shape(tokens, d);
+    if (rc != KQ_OK) return rc;
+    if (!aligned16(X) || !aligned16(q_packed) || !aligned16(s)) return KQ_ERR_ALIGN;
+    if (tokens == 0) return KQ_OK;
+    return run_stream<kq::MODE_SCALE, false>(X, tokens, d, nullptr, s, q_packed, scales, nullptr,
+                                             static_cast<cudaStream_t>(stream));
+}
+
+kq_status_t kroquant_mxfp4_quantize(const void* X, int64_t tokens, int d, uint8_t* q_packed, uint8_t* scales,
+                                    void* stream) {
+    if (!X || !q_packed || !scales) return KQ_ERR_NULL;
+    kq_status_t rc = check_shape(tokens, d);
+    if (rc != KQ_OK) return rc;
+    if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
+    if (tokens == 0) return KQ_OK;
+    return run_stream<kq::MODE_PLAIN, false>(X, tokens, d, nullptr, nullptr, q_packed, scales, nullptr,
+                                             static_cast<cudaStream_t>(stream));
+}
+
+kq_status_t kroquant_dequantize(const uint8_t* q_packed, const uint8_t* scales, int64_t tokens, int d,
+                                const kroquant_factors_t* f, void* out, kq_dtype_t out_dtype, void* stream) {
+    if (!q_packed || !scales || !out) return KQ_ERR_NULL;
+    kq_status_t rc = check_shape(tokens, d);
+    if (rc != KQ_OK) return rc;
+    if (f && f->n_sets != 1 && f->n_sets != d / 32) return KQ_ERR_FACTORS;
+    if (!aligned16(q_packed) || !aligned16(out)) return KQ_ERR_ALIGN;
+    if (out_dtype != KQ_OUT_F32 && out_dtype != KQ_OUT_BF16) return KQ_ERR_UNSUPPORTED;
+    if (tokens == 0) return KQ_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t n_quads = tokens * (int64_t)(d / 8);
+    const int grid = stream_grid(n_quads);
+    if (grid <= 0) return KQ_ERR_CUDA;
+    const kq::FactorSet* gi = (f && !f->identity) ? f->d_Ginv : nullptr;
+    const int ns = f ? f->n_sets : 0;
+    const uint32_t* q32 = reinterpret_cast<const uint32_t*>(q_packed);
+    if (out_dtype == KQ_OUT_BF16)
+        kq::dequantize_stream<true><<<grid, 256, 0, st>>>(q32, scales, n_quads, d / 32, gi, ns, out);
+    else
+        kq::dequantize_stream<false><<<grid, 256, 0, st>>>(q32, scales, n_quads, d / 32, gi, ns, out);
+    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
+}
+
+kq_status_t kroquant_debug_e2m1_codes(const float* v, int64_t n, uint8_t* codes, void* stream) {
+    if (!v || !codes) return KQ_ERR_NULL;
+    if (n < 0) return KQ_ERR_SHAPE;
+    if (n == 0) return KQ_OK;
+    kq::e2m1_codes_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(v, n, codes);
+    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
+}
+
+kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm) {
+    if (config < 0 || config > 3 || ctas_per_sm < 1 || ctas_per_sm > 4) return KQ_ERR_UNSUPPORTED;
+    g_umma_cfg.store(config);
+    g_umma_ctas_per_sm.store(ctas_per_sm);
+    return KQ_OK;
+}
+
+int64_t kroquant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+kq_status_t kroquant_last_device_error(void* stream, int* code_out) {
+    if (!code_out) return KQ_ERR_NULL;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KQ_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, kq::g_kq_device_error, sizeof(int)) != cudaSuccess) return KQ_ERR_CUDA;
+    if (v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(kq::g_kq_device_error, &zero, sizeof(int)) != cudaSuccess) return KQ_ERR_CUDA;
+    }
+    *code_out = v;
+    return KQ_OK;
+}
+
+const char* kroquant_status_string(kq_status_t s) {
+    switch (s) {
+        case KQ_OK: return "ok";
+        case KQ_ERR_NULL: return "null pointer";
+        case KQ_ERR_SHAPE: return "bad shape (d must be a positive multiple of 32, tokens >= 0)";
+        case KQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case KQ_ERR_FACTORS: return "bad factors (n_sets must be 1 or d/32; factors finite and non-singular)";
+        case KQ_ERR_UNSUPPORTED: return "unsupported option";
+        case KQ_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+"""Parity rules between the CUDA quantizer and the CPU oracle.
+
+P0  exact kernels (bare MXFP4, per-channel scale, identity factors): every code
+    and scale byte identical (a zero's sign may differ only where the oracle's
+    value is exactly +-0).
+P1  pre-rounding values: |y_gpu - y| <= 1e-5 * max(|y|, amax_block / 32).
+P2  codes: a mismatch is allowed only where the oracle's scaled value lies within
+    1e-5 relative of a rounding boundary, must be one adjacent magnitude step
+    with the same sign, and at most 1e-4 of all codes may differ.
+P3  scales: identical, except blocks whose oracle amax lies within 1e-5 relative
+    of a power of two, which may be off by one; their codes are then checked
+    against the oracle re-encoded with the GPU's scale; at most 1e-4 of blocks.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import np_oracle as no
+
+BOUNDS = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0])
+REL = 1e-5
+MAX_FRACTION = 1e-4
+
+
+def unpack(q: np.ndarray) -> np.ndarray:
+    t, half = q.shape
+    c = np.empty((t, half * 2), np.uint8)
+    c[:, 0::2] = q & 15
+    c[:, 1::2] = q >> 4
+    return c
+
+
+def check_values(Y_gpu: np.ndarray, Y_or: np.ndarray) -> dict:
+    t, d = Y_or.shape
+    yo = Y_or.astype(np.float64).reshape(t, d // 32, 32)
+    yg = Y_gpu.astype(np.float64).reshape(t, d // 32, 32)
+    amax = np.abs(yo).max(axis=2, keepdims=True)
+    tol = REL * np.maximum(np.abs(yo), amax / 32.0)
+    err = np.abs(yg - yo)
+    bad = err > tol
+    ratio = np.where(tol > 0, err / np.where(tol > 0, tol, 1), np.where(err > 0, np.inf, 0))
+    assert not bad.any(), f"P1: {bad.sum()} values outside tolerance, worst err/tol = {ratio.max():.3g}"
+    return {"max_err_over_tol": float(ratio.max())}
+
+
+def check_codes(q_gpu, s_gpu, q_or, s_or, Y_or, exact: bool) -> dict:
+    q_gpu, s_gpu = np.asarray(q_gpu), np.asarray(s_gpu)
+    t, d = Y_or.shape
+    nb = d // 32
+    cg, co = unpack(q_gpu), unpack(q_or)
+    Y = Y_or.astype(np.float64)
+    # ---- scales (P3)
+    sdiff = s_gpu != s_or
+    n_sdiff = int(sdiff.sum())
+    expect_codes = co
+    if n_sdiff:
+        assert not exact, f"P0: {n_sdiff} scale bytes differ"
+        amax = np.abs(Y.reshape(t, nb, 32)).max(axis=2)
+        m, _ = np.frexp(amax[sdiff])                  # amax = m 2^e, m in [0.5, 1)
+        near_pow2 = np.minimum(np.abs(m - 0.5) / 0.5, np.abs(m - 1.0)) <= REL
+        assert near_pow2.all(), "P3: a scale differs on a block whose amax is not at a power of two"
+        assert (np.abs(s_gpu[sdiff].astype(int) - s_or[sdiff].astype(int)) == 1).all()
+        assert n_sdiff <= max(1, MAX_FRACTION * t * nb), f"P3: {n_sdiff} scale mismatches"
+        expect_codes = no.encode_with_scale(Y_or, np.where(sdiff, s_gpu, s_or))
+    # ---- codes (P0 / P2)
+    diff = cg != expect_codes
+    # zero-sign exemption: the oracle's value is exactly +-0 and only the sign bit differs
+    zero_sign = diff & (Y == 0.0) & ((cg & 7) == 0) & ((expect_codes & 7) == 0)
+    diff &= ~zero_sign
+    n_diff = int(diff.sum())
+    if exact:
+        assert n_diff == 0, f"P0: {n_diff} codes differ"
+    elif n_diff:
+        S_used = np.where(sdiff, s_gpu, s_or).astype(np.float64)
+        v = np.abs(Y.reshape(t, nb, 32) * np.exp2(127.0 - S_used)[:, :, None]).reshape(t, d)
+        vd = v[diff]
+        near = (np.abs(vd[:, None] - BOUNDS[None, :]) <= REL * BOUNDS[None, :]).any(axis=1)
+        assert near.all(), f"P2: {int((~near).sum())} code mismatches away from any rounding boundary"
+        g, o = cg[diff].astype(int), expect_codes[diff].astype(int)
+        assert ((g & 8) == (o & 8)).all(), "P2: sign differs"
+        assert (np.abs((g & 7) - (o & 7)) == 1).all(), "P2: more than one step"
+        assert n_diff <= max(1, MAX_FRACTION * t * d), f"P2: {n_diff} code mismatches"
+    return {"code_mismatches": n_diff, "scale_mismatches": n_sdiff,
+            "zero_sign_only": int(zero_sign.sum())}
