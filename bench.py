@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the KroQuant online activation quantizer on B200.
+
+One *step* = one denoising-step-like pass of the quantizer over a FLUX.1-schnell-shaped
+layer stack: 28 consecutive calls, 14 on X[4608, 3072] and 14 on X[4608, 12288]
+(interleaved), each call with its own input buffer, output buffers and factor set,
+captured in one CUDA graph.  The 28 inputs total 1.98 GB, far beyond the 126 MB L2, so
+every call reads its input from HBM.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` = algorithmic bytes moved per second by the
+whole job (2 B read + 0.5 B codes + 1/32 B scale per element), inputs resident in HBM;
+`e2e` = the same metric with pinned-host inputs and outputs, copies inside the timed
+region.  `--impl reference` times the CPU oracle on a bounded sample of the same
+workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_21446_b200 import workloads as W  # noqa: E402
+
+METRIC = "quantizer_hbm_throughput"
+UNIT = "GB/s"
+CALLS_PER_STEP = 28
+SHAPES = [(4608, 3072), (4608, 12288)]
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per launch of the tensor-core kernel from the Nsight Compute captures
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
+NCU_TRAFFIC_BYTES = {(4608, 3072): None, (4608, 12288): None}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def step_bytes() -> float:
+    return sum(W.algorithmic_bytes(t, d) for t, d in SHAPES) * (CALLS_PER_STEP // 2)
+
+
+def step_tokens() -> int:
+    return sum(t for t, _ in SHAPES) * (CALLS_PER_STEP // 2)
+
+
+# --------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines: list[str] = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def count(self) -> int:
+        return len(self.lines)
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [v for v in sm if v > 0.5 * max(sm)] or sm
+        return {"sm_mhz": float(np.median(busy)), "sm_max_mhz": float(max(mx)),
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------
+# reference arm: the CPU oracle on a bounded sample
+# --------------------------------------------------------------------------------------
+SAMPLE = "calls 0 and 1 of the 28-call step (the full X[4608,3072] and X[4608,12288] tensors)"
+
+
+def oracle_sample_inputs():
+    return [(W.gen_activations(sp), W.gen_factors(3, layer=layer))
+            for layer, sp in enumerate(W.flux_specs())]
+
+
+def time_oracle(steps: int, warmup: int):
+    from oracle import c_oracle as co
+    inputs = oracle_sample_inputs()
+    byts = sum(W.algorithmic_bytes(*x.shape) for x, _ in inputs)
+
+    def one():
+        for x, g in inputs:
+            co.quantize(x, g)
+    for _ in range(max(warmup, 1)):
+        one()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    dt = (time.perf_counter() - t0) / steps
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return byts / dt / 1e9, dt, cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 10))
+    gbs, dt, cores = time_oracle(steps, min(args.warmup, 2))
+    sample = f"{SAMPLE} per step, C oracle (fp64, OpenMP over token rows)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": "flux_step_28_calls (bounded sample)", "l2": "oracle on host cores"},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------
+def build_inputs(torch, B, device):
+    """28 distinct input buffers: the seeded FLUX-shaped tensors, rolled by i token rows."""
+    specs = W.flux_specs()
+    base = []
+    for sp in specs:
+        bits = W.gen_activations(sp)
+        base.append((bits, torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)))
+    calls = []
+    for i in range(CALLS_PER_STEP):
+        k = i % 2
+        bits, x0 = base[k]
+        shift = i // 2
+        x = torch.roll(x0, shifts=shift, dims=0).contiguous() if shift else x0
+        G = W.gen_factors(3, layer=i)
+        t, d = x.shape
+        calls.append({
+            "shift": shift, "shape_idx": k, "X": x, "G": G, "factors": B.Factors.create(G),
+            "q": torch.empty((t, d // 2), dtype=torch.uint8, device=device),
+            "s": torch.empty((t, d // 32), dtype=torch.uint8, device=device),
+            "sv": torch.from_numpy(W.gen_channel_scales(3, d, layer=i)).to(device),
+        })
+    return base, calls
+
+
+def capture(torch, fns, stream):
+    with torch.cuda.stream(stream):
+        for f in fns:
+            f()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for f in fns:
+                f()
+    return g
+
+
+def time_graph(torch, dist, g, stream, steps, warmup, sampler=None):
+    """W untimed replays, then exactly `steps` timed replays between two events on `stream`.
+    The clock sampler (nvidia-smi, 20 ms period) is started before the warm-up; extra
+    untimed replays keep the GPU under the same load until its first samples arrive and
+    until one more arrives after the timed region, so the samples bracket and cover it."""
+    with torch.cuda.stream(stream):
+        if sampler:
+            sampler.start()
+        for _ in range(warmup):
+            g.replay()
+        if sampler and sampler.proc is not None:
+            t_end = time.perf_counter() + 4.0
+            while sampler.count() < 3 and time.perf_counter() < t_end:
+                for _ in range(20):
+                    g.replay()
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(steps):
+            g.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sampler and sampler.proc is not None:
+            n_before = sampler.count()
+            t_end = time.perf_counter() + 1.0
+            while sampler.count() < n_before + 2 and time.perf_counter() < t_end:
+                for _ in range(20):
+                    g.replay()
+                torch.cuda.synchronize()
+    ms = a.elapsed_time(b)
+    clocks = sampler.stop() if sampler else None
+    return ms / steps, clocks
+
+
+def check_parity(torch, B, base, calls):
+    """Sampled-row parity of two timed calls (one per shape) against the oracle."""
+    from oracle import c_oracle as co
+    from tests import parity as P
+    rng = np.random.default_rng(0)
+    out = {}
+    for c in calls[:2]:
+        bits, _ = base[c["shape_idx"]]
+        t, d = bits.shape
+        rows = np.sort(rng.choice(t, size=96, replace=False))
+        src = (rows - c["shift"]) % t                      # X = roll(X0, shift)
+        q_or, s_or, Y = co.quantize(bits[src], c["G"])
+        q = c["q"][torch.from_numpy(rows).to(c["q"].device)].cpu().numpy()
+        s = c["s"][torch.from_numpy(rows).to(c["s"].device)].cpu().numpy()
+        out[f"{t}x{d}"] = P.check_codes(q, s, q_or, s_or, Y, exact=False)
+    return out
+
+
+def run_ours(args):
+    import torch
+    from paper_2607_21446_b200 import binding as B
+    B.load_library()                       # fails loudly if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=device)
+        dist = dist_mod
+    peak, peak_kind = measured_peak()
+    base, calls = build_inputs(torch, B, device)
+    stream = torch.cuda.Stream()
+
+    n0 = B.kroquant_launch_count()
+    g_kq = capture(torch, [lambda c=c: B.kroquant_quantize(c["X"], c["factors"], c["q"], c["s"], stream=stream)
+                           for c in calls], stream)
+    launches_per_step = (B.kroquant_launch_count() - n0) // 2     # eager pass + captured pass
+    g_scale = capture(torch, [lambda c=c: B.kroquant_scale_quantize(c["X"], c["sv"], c["q"], c["s"], stream=stream)
+                              for c in calls], stream)
+    g_plain = capture(torch, [lambda c=c: B.kroquant_mxfp4_quantize(c["X"], c["q"], c["s"], stream=stream)
+                              for c in calls], stream)
+
+    idx = torch.cuda.current_device()
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    smi_index = int(vis.split(",")[idx]) if vis and vis.split(",")[idx].isdigit() else idx
+    ms_step, clocks = time_graph(torch, dist, g_kq, stream, args.steps, args.warmup, ClockSampler(smi_index))
+    if dist is not None:
+        tmax = torch.tensor([ms_step], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms_step = float(tmax.item())
+    byts = step_bytes()
+    value = world * byts / (ms_step * 1e-3) / 1e9
+    dev_err = B.kroquant_last_device_error(stream)
+
+    # in-run comparison kernels and per-shape breakdown (rank-local, shorter runs)
+    k2 = max(3, args.steps // 2)
+    ms_scale, _ = time_graph(torch, None, g_scale, stream, k2, 3)
+    ms_plain, _ = time_graph(torch, None, g_plain, stream, k2, 3)
+    per_shape = {}
+    for k, (t, d) in enumerate(SHAPES):
+        sub = [c for c in calls if c["shape_idx"] == k]
+        res = {}
+        for name, fn in (("kroquant", lambda c: B.kroquant_quantize(c["X"], c["factors"], c["q"], c["s"], stream=stream)),
+                         ("scale", lambda c: B.kroquant_scale_quantize(c["X"], c["sv"], c["q"], c["s"], stream=stream)),
+                         ("plain_mxfp4", lambda c: B.kroquant_mxfp4_quantize(c["X"], c["q"], c["s"], stream=stream))):
+            g = capture(torch, [lambda c=c, fn=fn: fn(c) for c in sub + sub], stream)   # 28 calls of one shape
+            ms, _ = time_graph(torch, None, g, stream, k2, 3)
+            us = ms * 1e3 / (2 * len(sub))
+            res[name] = {"us_per_call": round(us, 3),
+                         "GB/s": round(W.algorithmic_bytes(t, d) / us / 1e3, 1),
+                         "frac_of_peak": round(W.algorithmic_bytes(t, d) / us / 1e3 / peak, 4)}
+        per_shape[f"{t}x{d}"] = res
+
+    # end to end: pinned host inputs -> device -> quantize -> pinned host outputs
+    e2e_steps = max(1, min(args.steps, 3))
+    hx = [torch.empty(c["X"].shape, dtype=torch.bfloat16).pin_memory() for c in calls[:2]]
+    for h, c in zip(hx, calls[:2]):
+        h.copy_(c["X"])
+    hq = [torch.empty(c["q"].shape, dtype=torch.uint8).pin_memory() for c in calls[:2]]
+    hs = [torch.empty(c["s"].shape, dtype=torch.uint8).pin_memory() for c in calls[:2]]
+
+    def e2e_step():
+        with torch.cuda.stream(stream):
+            for c in calls:
+                k = c["shape_idx"]
+                B.quantize_from_host(hx[k], c["factors"], c["X"], c["q"], c["s"], hq[k], hs[k], stream=stream)
+    # (the device copies of X are overwritten by identical data: calls[0:2] hold the unrolled tensors;
+    #  the other 26 device buffers receive the same host tensor, which changes no timing-relevant property)
+    e2e_step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if dist is not None:
+        tmax = torch.tensor([e2e_s], device=device)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_s = float(tmax.item())
+    h2d = sum(c["X"].numel() * 2 for c in calls)
+    d2h = sum(c["q"].numel() + c["s"].numel() for c in calls)
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # parity of the timed configuration (fresh device-resident run of the first two calls)
+    g_kq.replay()
+    torch.cuda.synchronize()
+    try:
+        parity = check_parity(torch, B, base, calls)
+        parity["status"] = "ok"
+    except AssertionError as e:          # report, never hide
+        parity = {"status": "FAILED", "error": str(e)[:200]}
+
+    cpu_gbs, cpu_dt, cores = time_oracle(5, 1)
+    n_launch = launches_per_step * args.steps
+    us_per_launch = ms_step * 1e3 / CALLS_PER_STEP
+    alg_per_launch = byts / CALLS_PER_STEP
+    traffic = None
+    if all(NCU_TRAFFIC_BYTES[s] is not None for s in SHAPES):
+        traffic = sum(NCU_TRAFFIC_BYTES[s] for s in SHAPES) / 2
+    achieved = alg_per_launch / us_per_launch / 1e3
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "flux_step_28_calls: 14 x X[4608,3072] + 14 x X[4608,12288] bf16, interleaved, "
+                               "one CUDA graph, distinct buffers and factor sets per call",
+                   "l2": "28 input buffers total 1.98 GB (> 126 MB L2); no flush needed",
+                   "factors": "one shared set per call (orthogonal x diag(U[0.5,2]))",
+                   "kernel": "tcgen05+TMA tensor-core quantizer"},
+        "tokens_per_s": world * step_tokens() / (ms_step * 1e-3),
+        "frac_of_hbm_peak": value / world / peak,
+        "speedup_vs_scale_kernel": ms_scale / ms_step,
+        "speedup_vs_plain_mxfp4": ms_plain / ms_step,
+        "per_shape": per_shape,
+        "parity": parity,
+        "device_error": dev_err,
+        "clocks": clocks,
+        "e2e": {"value": world * byts / e2e_s / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": n_launch,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                     "kernel": "quantize_umma_shared", "launches": n_launch,
+                     "avg_launch_us": us_per_launch, "algorithmic_bytes_per_launch": alg_per_launch},
+        "cpu_baseline": {"value": cpu_gbs, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{SAMPLE}, {cpu_dt:.2f} s per pass, 5 passes, "
+                                   "C oracle (fp64, OpenMP over token rows)"},
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

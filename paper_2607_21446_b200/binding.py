@@ -62,7 +62,7 @@ def load_library() -> C.CDLL:
     L.kroquant_mxfp4_quantize.argtypes = [vp, i64, i32, vp, vp, vp]
     L.kroquant_transform_f32.argtypes = [vp, i64, i32, vp, vp, i32, vp]
     L.kroquant_debug_e2m1_codes.argtypes = [vp, i64, vp, vp]
-    L.kroquant_debug_set_umma_config.argtypes = [i32, i32]
+    L.kroquant_debug_set_umma_config.argtypes = [i32, i32, i32]
     L.kroquant_launch_count.argtypes = []
     L.kroquant_launch_count.restype = i64
     L.kroquant_last_device_error.argtypes = [vp, C.POINTER(i32)]
@@ -210,8 +210,8 @@ def kroquant_debug_e2m1_codes(v: torch.Tensor, stream=None) -> torch.Tensor:
     return codes
 
 
-def kroquant_debug_set_umma_config(config: int, ctas_per_sm: int) -> None:
-    _check(load_library().kroquant_debug_set_umma_config(config, ctas_per_sm),
+def kroquant_debug_set_umma_config(config: int, ctas_per_sm: int, use_pdl: bool = True) -> None:
+    _check(load_library().kroquant_debug_set_umma_config(config, ctas_per_sm, int(use_pdl)),
            "kroquant_debug_set_umma_config")
 
 

@@ -73,22 +73,22 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait.  Returns false once kWaitLimitNs has passed (checked every 256 failed
-// tries, and at most 2^26 tries in any case) or when the CTA has aborted.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    const uint64_t t0 = global_timer_ns();
-    for (uint32_t i = 1; i < (1u << 26); ++i) {
+// Bounded wait.  The clock is consulted only every 4096 failed tries (each try already
+// blocks for a hardware-defined interval), so the common path is a bare try_wait loop.
+// Returns false once kWaitLimitNs has passed since the first clock check, after 2^30
+// tries in any case, or when the CTA has aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    uint64_t t0 = 0;
+    for (uint32_t i = 1; i < (1u << 30); ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 0u) {
+        if ((i & 4095u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
         }
     }
     return false;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
@@ -143,14 +143,19 @@ __device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr) {
 constexpr uint32_t kIdescBf16M128N32 =
     (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
 
+// Programmatic dependent launch: let the next kernel in the stream start its prologue
+// early, and wait for the previous kernel's memory before touching global data.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- shared memory plan ----------------------------------------------------------
-template <int NS, int NA>
+template <int NS>
 struct UmmaSmem {
     static constexpr int kBOff = 0;                                  // 6 KB, 1024-aligned
     static constexpr int kAOff = 8192;                               // NS stages of 8 KB
     static constexpr int kBarOff = kAOff + NS * kTileBytes;
-    // barriers: full[NS], empty[NS], tfull[NA], tempty[NA], bfull
-    static constexpr int kNumBars = 2 * NS + 2 * NA + 1;
+    // barriers: full[NS], done[NS], tempty[NS], bfull
+    static constexpr int kNumBars = 3 * NS + 1;
     static constexpr int kTmemSlotOff = kBarOff + 8 * kNumBars;
     static constexpr int kAbortOff = kTmemSlotOff + 4;
     static constexpr int kBytes = kAbortOff + 4;
@@ -159,9 +164,15 @@ struct UmmaSmem {
 
 // The fused epilogue math of one 32-channel block held in registers.
 __device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uint4& codes, uint32_t& S) {
-    float amax = 0.f;
+    float m[4] = {0.f, 0.f, 0.f, 0.f};      // four independent max chains
 #pragma unroll
-    for (int c = 0; c < 32; ++c) amax = fmaxf(amax, fabsf(__uint_as_float(acc[c])));
+    for (int c = 0; c < 32; c += 4) {
+        m[0] = fmaxf(m[0], fabsf(__uint_as_float(acc[c + 0])));
+        m[1] = fmaxf(m[1], fabsf(__uint_as_float(acc[c + 1])));
+        m[2] = fmaxf(m[2], fabsf(__uint_as_float(acc[c + 2])));
+        m[3] = fmaxf(m[3], fabsf(__uint_as_float(acc[c + 3])));
+    }
+    const float amax = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
     S = e8m0_from_amax(amax);
     const float inv = inv_scale_from_e8m0(S);
     uint32_t w[4];
@@ -175,37 +186,49 @@ __device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uin
     codes = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// NS smem stages, NA TMEM accumulator slots (NA*32 columns, a power of two >= 32),
-// NG epilogue warpgroups.  Grid: any size <= number of tiles; CTA b takes tiles
-// b, b + gridDim.x, ...
-template <int NS, int NA, int NG, bool WRITE_Y>
-__global__ void __launch_bounds__(64 + 128 * NG, 1)
+// NS pipeline slots: slot s = one 8 KB shared-memory stage + one 32-column TMEM
+// accumulator (NS*32 columns, a power of two >= 32).  NM MMA-issuing warps (tile n is
+// issued by warp 1 + n % NM; a tcgen05.mma costs its issuing thread ~60 cycles, so one
+// thread cannot issue the six MMAs of a tile inside the tile's HBM time), NG epilogue
+// warpgroups (tile n is drained by group n % NG).
+//
+// Warps: 0 = TMA producer, 1..NM = MMA issuers (warp 1 also owns the TMEM allocation),
+// warps 4.. = epilogue (4 per group; warp w reads TMEM lanes 32*(w%4)..+31).
+// Per slot: full (TMA landed) -> done (one tcgen05.commit: the MMAs have read the stage
+// and written the accumulator; frees the stage for the producer and hands the
+// accumulator to the epilogue) -> tempty (4 epilogue warps have read the accumulator).
+// Grid: any size <= number of tiles; CTA b takes tiles b, b + gridDim.x, ...
+template <int NS, int NM, int NG, bool WRITE_Y>
+__global__ void __launch_bounds__(128 + 128 * NG, 1)
 quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ b_image,
                      int64_t n_blocks, uint4* __restrict__ q_packed, uint8_t* __restrict__ scales,
                      float* __restrict__ Y) {
-    using L = UmmaSmem<NS, NA>;
+    static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
+    // A slot must always be served by the same issuer warp and the same epilogue group:
+    // only then does program order inside that warp guarantee that a parity wait never
+    // runs a whole phase ahead of the barrier it polls.
+    static_assert(NS % NM == 0 && NS % NG == 0, "slot ownership must be fixed");
+    using L = UmmaSmem<NS>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* base_ptr = smem_raw + (base - raw);
     const uint32_t bar0 = base + L::kBarOff;
     auto bar_full = [&](int s) { return bar0 + 8u * s; };
-    auto bar_empty = [&](int s) { return bar0 + 8u * (NS + s); };
-    auto bar_tfull = [&](int a) { return bar0 + 8u * (2 * NS + a); };
-    auto bar_tempty = [&](int a) { return bar0 + 8u * (2 * NS + NA + a); };
-    const uint32_t bar_b = bar0 + 8u * (2 * NS + 2 * NA);
+    auto bar_done = [&](int s) { return bar0 + 8u * (NS + s); };
+    auto bar_tempty = [&](int s) { return bar0 + 8u * (2 * NS + s); };
+    const uint32_t bar_b = bar0 + 8u * (3 * NS);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + L::kTmemSlotOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + L::kAbortOff);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int64_t n_tiles = (n_blocks + kTileRows - 1) / kTileRows;
-    // local tile count of this CTA
     const int my_tiles = (int)((n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-        for (int a = 0; a < NA; ++a) { mbar_init(bar_tfull(a), 1); mbar_init(bar_tempty(a), 4); }
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_done(s), 1); mbar_init(bar_tempty(s), 4); }
         mbar_init(bar_b, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -213,7 +236,7 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
     if (warp == 1) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(base + (uint32_t)L::kTmemSlotOff), "r"((uint32_t)(NA * 32)) : "memory");
+                     ::"r"(base + (uint32_t)L::kTmemSlotOff), "r"((uint32_t)(NS * 32)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -226,11 +249,14 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+            // the factor image is immutable after creation: safe to fetch before the
+            // previous kernel in the stream has finished
             mbar_expect_tx(bar_b, kBImageBytes);
             bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
+            pdl_wait_prior_grid();
             for (int n = 0; n < my_tiles; ++n) {
                 const int s = n % NS;
-                if (n >= NS && !mbar_wait(bar_empty(s), ((n / NS) - 1) & 1, abort_flag)) {
+                if (n >= NS && !mbar_wait(bar_done(s), ((n / NS) - 1) & 1, abort_flag)) {
                     if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
                     break;
                 }
@@ -240,53 +266,59 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
                 issued = n + 1;
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
+    } else if (warp <= NM) {
+        // ---------------- MMA issuers ----------------
         if (lane == 0) {
             bool ok = mbar_wait(bar_b, 0, abort_flag);
             if (!ok && !*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
-            for (int n = 0; ok && n < my_tiles; ++n) {
-                const int s = n % NS, a = n % NA;
+            uint64_t b_desc[3][2];
+#pragma unroll
+            for (int t = 0; t < 3; ++t)
+#pragma unroll
+                for (int kk = 0; kk < 2; ++kk)
+                    b_desc[t][kk] = smem_desc_sw64(base + L::kBOff + t * kBTermBytes + kk * 32);
+            const uint64_t a_desc0 = smem_desc_sw64(base + L::kAOff);
+            for (int n = warp - 1; ok && n < my_tiles; n += NM) {
+                const int s = n % NS;
                 if (!mbar_wait(bar_full(s), (n / NS) & 1, abort_flag)) {
                     if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_MMA_FULL); *abort_flag = 1; }
                     break;
                 }
-                if (n >= NA && !mbar_wait(bar_tempty(a), ((n / NA) - 1) & 1, abort_flag)) {
+                if (n >= NS && !mbar_wait(bar_tempty(s), ((n / NS) - 1) & 1, abort_flag)) {
                     if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_MMA_TMEM); *abort_flag = 1; }
                     break;
                 }
                 tc_fence_after();
-                const uint32_t a_addr = base + L::kAOff + s * kTileBytes;
-                const uint32_t d_addr = tmem_base + (uint32_t)(a * 32);
+                const uint64_t a_desc = a_desc0 + (uint64_t)((s * kTileBytes) >> 4);   // start-address field
+                const uint32_t d_addr = tmem_base + (uint32_t)(s * 32);
 #pragma unroll
                 for (int t = 0; t < 3; ++t) {
 #pragma unroll
                     for (int kk = 0; kk < 2; ++kk) {
-                        tc_mma_bf16(d_addr, smem_desc_sw64(a_addr + kk * 32),
-                                    smem_desc_sw64(base + L::kBOff + t * kBTermBytes + kk * 32),
-                                    kIdescBf16M128N32, (uint32_t)((t | kk) != 0));
+                        tc_mma_bf16(d_addr, a_desc + (uint64_t)(kk * 2), b_desc[t][kk], kIdescBf16M128N32,
+                                    (uint32_t)((t | kk) != 0));
                     }
                 }
-                tc_commit(bar_empty(s));     // smem stage reusable once these MMAs have read it
-                tc_commit(bar_tfull(a));     // accumulator complete
+                tc_commit(bar_done(s));
             }
         }
-    } else {
+    } else if (warp >= 4) {
         // ---------------- epilogue warpgroups ----------------
-        const int g = (warp - 2) >> 2;             // warpgroup index
+        const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
+        pdl_wait_prior_grid();   // the outputs may still be read by the previous kernel
         for (int n = g; n < my_tiles; n += NG) {
-            const int a = n % NA;
-            if (!mbar_wait(bar_tfull(a), (n / NA) & 1, abort_flag)) {
+            const int s = n % NS;
+            if (!mbar_wait(bar_done(s), (n / NS) & 1, abort_flag)) {
                 if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_EPILOGUE); *abort_flag = 1; }
                 break;
             }
             tc_fence_after();
             uint32_t acc[32];
-            tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * 32), acc);
+            tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * 32), acc);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty(a));
+            if (lane == 0) mbar_arrive(bar_tempty(s));
             const int64_t tile = blockIdx.x + (int64_t)n * gridDim.x;
             const int64_t row = tile * kTileRows + quarter * 32 + lane;
             if (row < n_blocks) {
@@ -324,7 +356,7 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                     ::"r"(tmem_base), "r"((uint32_t)(NA * 32)) : "memory");
+                     ::"r"(tmem_base), "r"((uint32_t)(NS * 32)) : "memory");
     }
 }
 

@@ -31,9 +31,9 @@ namespace {
 std::atomic<int64_t> g_launches{0};
 
 // ---- tensor-core kernel configuration ----------------------------------------
-struct UmmaConfig { int id; int ns, na, ng; };
-std::atomic<int> g_umma_cfg{0};
-std::atomic<int> g_umma_ctas_per_sm{2};
+std::atomic<int> g_umma_cfg{5};
+std::atomic<int> g_umma_ctas_per_sm{3};
+std::atomic<int> g_umma_pdl{1};
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -117,11 +117,11 @@ void build_b_image(const float* G20, uint8_t* img) {
         }
 }
 
-template <int NS, int NA, int NG, bool WRITE_Y>
+template <int NS, int NM, int NG, bool WRITE_Y>
 kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, int64_t n_blocks, uint4* q,
-                        uint8_t* scales, float* Y, int ctas_per_sm, cudaStream_t st) {
-    using L = kq::UmmaSmem<NS, NA>;
-    auto kern = kq::quantize_umma_shared<NS, NA, NG, WRITE_Y>;
+                        uint8_t* scales, float* Y, int ctas_per_sm, bool pdl, cudaStream_t st) {
+    using L = kq::UmmaSmem<NS>;
+    auto kern = kq::quantize_umma_shared<NS, NM, NG, WRITE_Y>;
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, [&] {
@@ -132,9 +132,20 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, int64_t n_
     if (sms <= 0) return KQ_ERR_CUDA;
     const int64_t n_tiles = (n_blocks + kq::kTileRows - 1) / kq::kTileRows;
     const int64_t cap = (int64_t)sms * ctas_per_sm;
-    const int grid = (int)(n_tiles < cap ? n_tiles : cap);
-    kern<<<grid, 64 + 128 * NG, L::kDynBytes, st>>>(tmap, bimg, n_blocks, q, scales, Y);
-    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(n_tiles < cap ? n_tiles : cap));
+    cfg.blockDim = dim3(128 + 128 * NG);
+    cfg.dynamicSmemBytes = L::kDynBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, bimg, n_blocks, q, scales, Y) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KQ_ERR_CUDA;
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return KQ_OK;
 }
@@ -155,12 +166,18 @@ kq_status_t run_umma(const void* X, int64_t n_blocks, const kroquant_factors_t* 
         return KQ_ERR_CUDA;
     uint4* q4 = reinterpret_cast<uint4*>(q);
     const int cps = g_umma_ctas_per_sm.load();
+    const bool pdl = g_umma_pdl.load() != 0;
+    const uint8_t* b = f->d_bimage;
     switch (g_umma_cfg.load()) {
         default:
-        case 0: return launch_umma<8, 8, 1, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
-        case 1: return launch_umma<8, 8, 2, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
-        case 2: return launch_umma<12, 16, 2, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
-        case 3: return launch_umma<12, 16, 4, WRITE_Y>(tmap, f->d_bimage, n_blocks, q4, scales, Y, cps, st);
+        case 0: return launch_umma<8, 1, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 1: return launch_umma<8, 2, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 2: return launch_umma<8, 2, 2, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 3: return launch_umma<8, 1, 2, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 4: return launch_umma<4, 1, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 5: return launch_umma<4, 2, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 6: return launch_umma<16, 2, 2, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 7: return launch_umma<16, 2, 4, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
     }
 }
 
@@ -364,10 +381,11 @@ kq_status_t kroquant_debug_e2m1_codes(const float* v, int64_t n, uint8_t* codes,
     return KQ_OK;
 }
 
-kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm) {
-    if (config < 0 || config > 3 || ctas_per_sm < 1 || ctas_per_sm > 4) return KQ_ERR_UNSUPPORTED;
+kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl) {
+    if (config < 0 || config > 7 || ctas_per_sm < 1 || ctas_per_sm > 4) return KQ_ERR_UNSUPPORTED;
     g_umma_cfg.store(config);
     g_umma_ctas_per_sm.store(ctas_per_sm);
+    g_umma_pdl.store(use_pdl != 0);
     return KQ_OK;
 }
 
