@@ -411,15 +411,54 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_single(args):
+    """Small case for profilers: a few eager launches of one shape on rotating buffers
+    (no CUDA graph, no comparison kernels).  Prints a short JSON line; never a bench value."""
+    import torch
+    from paper_2607_21446_b200 import binding as B
+    B.load_library()
+    t, d = (int(v) for v in args.single.lower().split("x"))
+    nbuf = max(2, int(400e6 // (t * d * 2)) + 1)          # > 3 x L2 of distinct inputs
+    sp = W.ActivationSpec("single", t, d, seed=3, outlier_channels=max(1, d // 200), outlier_gain=100.0)
+    x0 = torch.from_numpy(W.gen_activations(sp).view(np.int16)).cuda().view(torch.bfloat16)
+    Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, nbuf)]
+    q = torch.empty((t, d // 2), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((t, d // 32), dtype=torch.uint8, device="cuda")
+    f = B.Factors.create(W.gen_factors(3))
+    sv = torch.from_numpy(W.gen_channel_scales(3, d)).cuda()
+    fn = {"kroquant": lambda x: B.kroquant_quantize(x, f, q, sc),
+          "scale": lambda x: B.kroquant_scale_quantize(x, sv, q, sc),
+          "plain": lambda x: B.kroquant_mxfp4_quantize(x, q, sc)}[args.kernel]
+    torch.cuda.synchronize()
+    evs = []
+    for i in range(args.calls):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn(Xs[i % nbuf])
+        b.record()
+        evs.append((a, b))
+    torch.cuda.synchronize()
+    us = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+    print(json.dumps({"single": args.single, "kernel": args.kernel, "calls": args.calls,
+                      "median_us_eager": us[len(us) // 2], "buffers": nbuf,
+                      "device_error": B.kroquant_last_device_error()}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--single", default=None, metavar="TOKENSxD",
+                    help="profiling aid: a few eager launches of one shape, e.g. 4608x12288")
+    ap.add_argument("--kernel", default="kroquant", choices=["kroquant", "scale", "plain"])
+    ap.add_argument("--calls", type=int, default=8)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.single:
+        run_single(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
