@@ -1,8 +1,8 @@
 // Tensor-core KroQuant quantizer for sm_100a: TMA -> shared memory -> tcgen05.mma
 // (accumulators in TMEM) -> tcgen05.ld -> fused MXFP4 encoder in registers.
 //
-// Shared factor set (one K per layer).  Because every 32-channel block of every
-// token is multiplied by the same K (paper Section 3.5: "many column blocks share
+// Shared factor set (one K per layer; the per-block variant is described at the
+// kernel).  Because every 32-channel block of every token is multiplied by the same K (paper Section 3.5: "many column blocks share
 // the same Kronecker factors"), X[tokens][d] is viewed as a flat matrix of
 // n_blocks = tokens*d/32 rows of 32 bf16 (64 contiguous bytes each), and the whole
 // layer is one tall GEMM  Y[n_blocks][32] = Xflat[n_blocks][32] * K[32][32]
@@ -149,11 +149,14 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ---- shared memory plan ----------------------------------------------------------
-template <int NS>
+// PB = false: one factor image for the whole launch at offset 0, stages of 8 KB (A only).
+// PB = true : every stage carries its own factor image: 8 KB of A + 6 KB of B.
+template <int NS, bool PB>
 struct UmmaSmem {
-    static constexpr int kBOff = 0;                                  // 6 KB, 1024-aligned
-    static constexpr int kAOff = 8192;                               // NS stages of 8 KB
-    static constexpr int kBarOff = kAOff + NS * kTileBytes;
+    static constexpr int kStageBytes = kTileBytes + (PB ? kBImageBytes : 0);   // multiple of 1024
+    static constexpr int kBOff = 0;                                  // shared image (PB = false)
+    static constexpr int kAOff = PB ? 0 : 8192;                      // NS stages
+    static constexpr int kBarOff = kAOff + NS * kStageBytes;
     // barriers: full[NS], done[NS], tempty[NS], bfull
     static constexpr int kNumBars = 3 * NS + 1;
     static constexpr int kTmemSlotOff = kBarOff + 8 * kNumBars;
@@ -186,10 +189,25 @@ __device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uin
     codes = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// NS pipeline slots: slot s = one 8 KB shared-memory stage + one 32-column TMEM
-// accumulator (NS*32 columns, a power of two >= 32).  NM MMA-issuing warps (tile n is
-// issued by warp 1 + n % NM; a tcgen05.mma costs its issuing thread ~60 cycles, so one
-// thread cannot issue the six MMAs of a tile inside the tile's HBM time), NG epilogue
+// Work decomposition.
+//   PB = false (one shared factor set): X is the flat matrix [n_rows = tokens*d/32][32];
+//     tile w = flat rows 128w .. 128w+127; outputs of flat row r: 16 B of codes at
+//     q_packed + 16 r, scale byte at scales + r.
+//   PB = true (factor set j for block column j): tile w = (column j = w / n_ttiles,
+//     token tile tt = w % n_ttiles): 128 tokens x 32 channels of column j, fetched as a
+//     strided 2-D box from X[tokens][d]; its B operand is image j.  Output of token t:
+//     codes at q_packed + t*(d/2) + 16 j, scale byte at scales + t*(d/32) + j.
+struct UmmaProblem {
+    int64_t n_rows;      // PB=false: tokens*d/32 ; PB=true: tokens
+    int64_t n_tiles;     // total 128-row tiles
+    int n_ttiles;        // PB=true: token tiles per column (ceil(tokens/128))
+    int blocks_per_row;  // d/32
+};
+
+// NS pipeline slots: slot s = one shared-memory stage + one 32-column TMEM accumulator
+// (NS*32 columns, a power of two >= 32).  NM MMA-issuing warps (tile n is issued by
+// warp 1 + n % NM; a tcgen05.mma costs its issuing thread ~60 cycles, so one thread
+// cannot issue the six MMAs of a tile inside the tile's HBM time), NG epilogue
 // warpgroups (tile n is drained by group n % NG).
 //
 // Warps: 0 = TMA producer, 1..NM = MMA issuers (warp 1 also owns the TMEM allocation),
@@ -198,17 +216,17 @@ __device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uin
 // and written the accumulator; frees the stage for the producer and hands the
 // accumulator to the epilogue) -> tempty (4 epilogue warps have read the accumulator).
 // Grid: any size <= number of tiles; CTA b takes tiles b, b + gridDim.x, ...
-template <int NS, int NM, int NG, bool WRITE_Y>
+template <int NS, int NM, int NG, bool PB, bool WRITE_Y>
 __global__ void __launch_bounds__(128 + 128 * NG, 1)
-quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ b_image,
-                     int64_t n_blocks, uint4* __restrict__ q_packed, uint8_t* __restrict__ scales,
-                     float* __restrict__ Y) {
+quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ b_image,
+              const UmmaProblem prob, uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales,
+              float* __restrict__ Y) {
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
     // A slot must always be served by the same issuer warp and the same epilogue group:
     // only then does program order inside that warp guarantee that a parity wait never
     // runs a whole phase ahead of the barrier it polls.
     static_assert(NS % NM == 0 && NS % NG == 0, "slot ownership must be fixed");
-    using L = UmmaSmem<NS>;
+    using L = UmmaSmem<NS, PB>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -223,15 +241,44 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int64_t n_tiles = (n_blocks + kTileRows - 1) / kTileRows;
-    const int my_tiles = (int)((n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    const int my_tiles = (int)((prob.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+
+    // issue the TMA copies of local tile n into slot n % NS (producer thread only)
+    auto issue_tile = [&](int n) {
+        const int s = n % NS;
+        const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
+        const uint32_t dst = base + L::kAOff + s * L::kStageBytes;
+        mbar_expect_tx(bar_full(s), L::kStageBytes);
+        if (PB) {
+            const int j = (int)(w / prob.n_ttiles), tt = (int)(w % prob.n_ttiles);
+            tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));
+            bulk_load(dst + kTileBytes, b_image + (size_t)j * kBImageBytes, kBImageBytes, bar_full(s));
+        } else {
+            tma_load_2d(dst, &tmap_x, 0, (int)(w * kTileRows), bar_full(s));
+        }
+    };
 
     pdl_launch_dependents();
+    int issued = 0;   // tiles whose TMA load the producer thread has issued
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_done(s), 1); mbar_init(bar_tempty(s), 4); }
         mbar_init(bar_b, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // The producer starts the pipeline before the CTA-wide sync: only this thread
+        // touches the barriers until then.  The factor image is immutable after creation,
+        // so it may be fetched before the previous kernel in the stream has finished; X
+        // (and, in the epilogue, the outputs) may not.
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+        if (!PB) {
+            mbar_expect_tx(bar_b, kBImageBytes);
+            bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
+        }
+        pdl_wait_prior_grid();
+        const int first = my_tiles < NS ? my_tiles : NS;
+        for (int n = 0; n < first; ++n) issue_tile(n);
+        issued = first;
     }
     if (warp == 1) {
         __syncwarp();
@@ -244,39 +291,34 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    int issued = 0;   // tiles whose TMA load this thread has issued (producer lane only)
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
-            // the factor image is immutable after creation: safe to fetch before the
-            // previous kernel in the stream has finished
-            mbar_expect_tx(bar_b, kBImageBytes);
-            bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
-            pdl_wait_prior_grid();
-            for (int n = 0; n < my_tiles; ++n) {
-                const int s = n % NS;
-                if (n >= NS && !mbar_wait(bar_done(s), ((n / NS) - 1) & 1, abort_flag)) {
+            for (int n = NS; n < my_tiles; ++n) {
+                if (!mbar_wait(bar_done(n % NS), ((n / NS) - 1) & 1, abort_flag)) {
                     if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
                     break;
                 }
-                const int64_t tile = blockIdx.x + (int64_t)n * gridDim.x;
-                mbar_expect_tx(bar_full(s), kTileBytes);
-                tma_load_2d(base + L::kAOff + s * kTileBytes, &tmap_x, 0, (int)(tile * kTileRows), bar_full(s));
+                issue_tile(n);
                 issued = n + 1;
             }
         }
     } else if (warp <= NM) {
         // ---------------- MMA issuers ----------------
         if (lane == 0) {
-            bool ok = mbar_wait(bar_b, 0, abort_flag);
-            if (!ok && !*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
+            bool ok = true;
+            if (!PB) {
+                ok = mbar_wait(bar_b, 0, abort_flag);
+                if (!ok && !*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
+            }
+            // descriptors of slot 0; slot s adds s*kStageBytes to the start-address field
             uint64_t b_desc[3][2];
 #pragma unroll
             for (int t = 0; t < 3; ++t)
 #pragma unroll
                 for (int kk = 0; kk < 2; ++kk)
-                    b_desc[t][kk] = smem_desc_sw64(base + L::kBOff + t * kBTermBytes + kk * 32);
+                    b_desc[t][kk] = smem_desc_sw64(base + (PB ? L::kAOff + kTileBytes : L::kBOff) +
+                                                   t * kBTermBytes + kk * 32);
             const uint64_t a_desc0 = smem_desc_sw64(base + L::kAOff);
             for (int n = warp - 1; ok && n < my_tiles; n += NM) {
                 const int s = n % NS;
@@ -289,14 +331,15 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
                     break;
                 }
                 tc_fence_after();
-                const uint64_t a_desc = a_desc0 + (uint64_t)((s * kTileBytes) >> 4);   // start-address field
+                const uint64_t slot_off = (uint64_t)((s * L::kStageBytes) >> 4);
+                const uint64_t a_desc = a_desc0 + slot_off;
                 const uint32_t d_addr = tmem_base + (uint32_t)(s * 32);
 #pragma unroll
                 for (int t = 0; t < 3; ++t) {
 #pragma unroll
                     for (int kk = 0; kk < 2; ++kk) {
-                        tc_mma_bf16(d_addr, a_desc + (uint64_t)(kk * 2), b_desc[t][kk], kIdescBf16M128N32,
-                                    (uint32_t)((t | kk) != 0));
+                        tc_mma_bf16(d_addr, a_desc + (uint64_t)(kk * 2), b_desc[t][kk] + (PB ? slot_off : 0),
+                                    kIdescBf16M128N32, (uint32_t)((t | kk) != 0));
                     }
                 }
                 tc_commit(bar_done(s));
@@ -306,7 +349,7 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
         // ---------------- epilogue warpgroups ----------------
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
-        pdl_wait_prior_grid();   // the outputs may still be read by the previous kernel
+        pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
         for (int n = g; n < my_tiles; n += NG) {
             const int s = n % NS;
             if (!mbar_wait(bar_done(s), (n / NS) & 1, abort_flag)) {
@@ -319,11 +362,19 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tempty(s));
-            const int64_t tile = blockIdx.x + (int64_t)n * gridDim.x;
-            const int64_t row = tile * kTileRows + quarter * 32 + lane;
-            if (row < n_blocks) {
+            const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
+            int64_t row, blk;       // row inside the tiled dimension; flat index of the 32-channel block
+            if (PB) {
+                const int j = (int)(w / prob.n_ttiles), tt = (int)(w % prob.n_ttiles);
+                row = (int64_t)tt * kTileRows + quarter * 32 + lane;
+                blk = row * prob.blocks_per_row + j;
+            } else {
+                row = w * kTileRows + quarter * 32 + lane;
+                blk = row;
+            }
+            if (row < prob.n_rows) {
                 if (WRITE_Y) {
-                    float4* yp = reinterpret_cast<float4*>(Y + row * 32);
+                    float4* yp = reinterpret_cast<float4*>(Y + blk * 32);
 #pragma unroll
                     for (int i = 0; i < 8; ++i)
                         yp[i] = make_float4(__uint_as_float(acc[4 * i]), __uint_as_float(acc[4 * i + 1]),
@@ -332,8 +383,8 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
                     uint4 codes;
                     uint32_t S;
                     encode_block_regs(acc, codes, S);
-                    st_stream_16(q_packed + row, codes);
-                    scales[row] = (uint8_t)S;
+                    st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
+                    scales[blk] = (uint8_t)S;
                 }
             }
         }
@@ -344,9 +395,9 @@ quantize_umma_shared(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* 
     __syncthreads();
     if (*abort_flag && threadIdx.x == 0) {
         // abort path only: let the copies this thread issued land before the CTA's shared
-        // memory goes away (load m went to stage m % NS and completes phase (m / NS) & 1)
+        // memory goes away (load m went to slot m % NS and completes phase (m / NS) & 1)
         int never = 0;
-        (void)mbar_wait(bar_b, 0, &never);
+        if (!PB) (void)mbar_wait(bar_b, 0, &never);
         for (int m = (issued > NS ? issued - NS : 0); m < issued; ++m)
             if (!mbar_wait(bar_full(m % NS), (m / NS) & 1, &never))
                 atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_DRAIN);

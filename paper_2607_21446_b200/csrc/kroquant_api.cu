@@ -117,11 +117,11 @@ void build_b_image(const float* G20, uint8_t* img) {
         }
 }
 
-template <int NS, int NM, int NG, bool WRITE_Y>
-kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, int64_t n_blocks, uint4* q,
-                        uint8_t* scales, float* Y, int ctas_per_sm, bool pdl, cudaStream_t st) {
-    using L = kq::UmmaSmem<NS>;
-    auto kern = kq::quantize_umma_shared<NS, NM, NG, WRITE_Y>;
+template <int NS, int NM, int NG, bool PB, bool WRITE_Y>
+kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, const kq::UmmaProblem& prob,
+                        uint8_t* q, uint8_t* scales, float* Y, int ctas_per_sm, bool pdl, cudaStream_t st) {
+    using L = kq::UmmaSmem<NS, PB>;
+    auto kern = kq::quantize_umma<NS, NM, NG, PB, WRITE_Y>;
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, [&] {
@@ -130,10 +130,9 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, int64_t n_
     if (attr_rc != cudaSuccess) return KQ_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
-    const int64_t n_tiles = (n_blocks + kq::kTileRows - 1) / kq::kTileRows;
     const int64_t cap = (int64_t)sms * ctas_per_sm;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(n_tiles < cap ? n_tiles : cap));
+    cfg.gridDim = dim3((unsigned)(prob.n_tiles < cap ? prob.n_tiles : cap));
     cfg.blockDim = dim3(128 + 128 * NG);
     cfg.dynamicSmemBytes = L::kDynBytes;
     cfg.stream = st;
@@ -142,7 +141,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, int64_t n_
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap, bimg, n_blocks, q, scales, Y) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, bimg, prob, q, scales, Y) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -150,34 +149,57 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, int64_t n_
     return KQ_OK;
 }
 
+// Tensor-core path.  Shared factor set: flat [tokens*d/32][32] view of X.  Per-block
+// factor sets: 2-D view [tokens][d] with one 32-channel column per tile.
 template <bool WRITE_Y>
-kq_status_t run_umma(const void* X, int64_t n_blocks, const kroquant_factors_t* f, uint8_t* q,
+kq_status_t run_umma(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, uint8_t* q,
                      uint8_t* scales, float* Y, cudaStream_t st) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
+    const bool pb = f->n_sets != 1;
+    const int nb = d / 32;
+    kq::UmmaProblem prob;
+    prob.blocks_per_row = nb;
     CUtensorMap tmap;
-    const cuuint64_t dims[2] = {32, (cuuint64_t)n_blocks};
-    const cuuint64_t strides[1] = {64};
+    cuuint64_t dims[2], strides[1];
+    if (pb) {
+        prob.n_rows = tokens;
+        prob.n_ttiles = (int)((tokens + kq::kTileRows - 1) / kq::kTileRows);
+        prob.n_tiles = (int64_t)prob.n_ttiles * nb;
+        dims[0] = (cuuint64_t)d; dims[1] = (cuuint64_t)tokens; strides[0] = (cuuint64_t)d * 2;
+    } else {
+        prob.n_rows = tokens * (int64_t)nb;
+        prob.n_ttiles = 1;
+        prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
+        dims[0] = 32; dims[1] = (cuuint64_t)prob.n_rows; strides[0] = 64;
+    }
     const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
-    uint4* q4 = reinterpret_cast<uint4*>(q);
     const int cps = g_umma_ctas_per_sm.load();
     const bool pdl = g_umma_pdl.load() != 0;
     const uint8_t* b = f->d_bimage;
+    if (pb) {
+        switch (g_umma_cfg.load()) {
+            default:
+            case 5: return launch_umma<4, 2, 1, true, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+            case 4: return launch_umma<4, 1, 1, true, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+            case 2: return launch_umma<8, 2, 2, true, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        }
+    }
     switch (g_umma_cfg.load()) {
         default:
-        case 0: return launch_umma<8, 1, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
-        case 1: return launch_umma<8, 2, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
-        case 2: return launch_umma<8, 2, 2, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
-        case 3: return launch_umma<8, 1, 2, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
-        case 4: return launch_umma<4, 1, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
-        case 5: return launch_umma<4, 2, 1, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
-        case 6: return launch_umma<16, 2, 2, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
-        case 7: return launch_umma<16, 2, 4, WRITE_Y>(tmap, b, n_blocks, q4, scales, Y, cps, pdl, st);
+        case 0: return launch_umma<8, 1, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 1: return launch_umma<8, 2, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 2: return launch_umma<8, 2, 2, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 3: return launch_umma<8, 1, 2, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 4: return launch_umma<4, 1, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 5: return launch_umma<4, 2, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 6: return launch_umma<16, 2, 2, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 7: return launch_umma<16, 2, 4, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
     }
 }
 
@@ -290,12 +312,10 @@ kq_status_t kroquant_quantize_path(const void* X, int64_t tokens, int d, const k
     if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool shared = f->n_sets == 1;
-    if (path == KQ_PATH_TENSOR && !shared) return KQ_ERR_UNSUPPORTED;
     if (path == KQ_PATH_AUTO && f->identity)
         return run_stream<kq::MODE_PLAIN, false>(X, tokens, d, nullptr, nullptr, q_packed, scales, nullptr, st);
-    if (shared && path != KQ_PATH_ALU)
-        return run_umma<false>(X, tokens * (int64_t)(d / 32), f, q_packed, scales, nullptr, st);
+    if (path != KQ_PATH_ALU)
+        return run_umma<false>(X, tokens, d, f, q_packed, scales, nullptr, st);
     return run_stream<kq::MODE_KRON, false>(X, tokens, d, f, nullptr, q_packed, scales, nullptr, st);
 }
 
@@ -315,12 +335,10 @@ kq_status_t kroquant_transform_f32(const void* X, int64_t tokens, int d, const k
     if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool shared = f->n_sets == 1;
-    if (path == KQ_PATH_TENSOR && !shared) return KQ_ERR_UNSUPPORTED;
     if (path == KQ_PATH_AUTO && f->identity)
         return run_stream<kq::MODE_PLAIN, true>(X, tokens, d, nullptr, nullptr, nullptr, nullptr, Y, st);
-    if (shared && path != KQ_PATH_ALU)
-        return run_umma<true>(X, tokens * (int64_t)(d / 32), f, nullptr, nullptr, Y, st);
+    if (path != KQ_PATH_ALU)
+        return run_umma<true>(X, tokens, d, f, nullptr, nullptr, Y, st);
     return run_stream<kq::MODE_KRON, true>(X, tokens, d, f, nullptr, nullptr, nullptr, Y, st);
 }
 

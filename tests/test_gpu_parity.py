@@ -124,10 +124,11 @@ def test_hadamard_and_lu_factors(B, path):
         P.check_codes(host(q), host(s), q_or, s_or, Y, exact=False)
 
 
-@pytest.mark.parametrize("tokens,d", [(64, 320), (33, 2240), (128, 5600)])
-def test_per_block_factor_sets(B, tokens, d):
+@pytest.mark.parametrize("path", ["tensor", "alu"])
+@pytest.mark.parametrize("tokens,d", [(1, 32), (64, 320), (33, 2240), (128, 5600), (300, 1152)])
+def test_per_block_factor_sets(B, path, tokens, d):
     Xb = W.gen_activations(spec(tokens, d, seed=2))
-    run_kroquant(B, Xb, W.gen_factors(2, n_sets=d // 32), "auto")
+    run_kroquant(B, Xb, W.gen_factors(2, n_sets=d // 32), path)
 
 
 def test_outputs_stay_inside_their_buffers(B):
