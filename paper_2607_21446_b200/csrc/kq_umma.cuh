@@ -143,6 +143,19 @@ __device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr) {
 constexpr uint32_t kIdescBf16M128N32 =
     (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
 
+// TMA store of a 2-D box from shared memory (bulk async group of the issuing thread).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(tmap), "r"(x), "r"(y), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// wait until at most N of this thread's bulk groups still READ their shared-memory source
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // Programmatic dependent launch: let the next kernel in the stream start its prologue
 // early, and wait for the previous kernel's memory before touching global data.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -156,7 +169,11 @@ struct UmmaSmem {
     static constexpr int kStageBytes = kTileBytes + (PB ? kBImageBytes : 0);   // multiple of 1024
     static constexpr int kBOff = 0;                                  // shared image (PB = false)
     static constexpr int kAOff = PB ? 0 : 8192;                      // NS stages
-    static constexpr int kBarOff = kAOff + NS * kStageBytes;
+    // PB only: staging of one column group's outputs: 128 rows x 64 B of codes (64-byte
+    // swizzle, leaves by TMA store) and 128 x 4 scale bytes
+    static constexpr int kStoreOff = kAOff + NS * kStageBytes;
+    static constexpr int kStoreBytes = PB ? (kTileRows * 64 + kTileRows * 4) : 0;
+    static constexpr int kBarOff = kStoreOff + kStoreBytes;
     // barriers: full[NS], done[NS], tempty[NS], bfull
     static constexpr int kNumBars = 3 * NS + 1;
     static constexpr int kTmemSlotOff = kBarOff + 8 * kNumBars;
@@ -189,18 +206,22 @@ __device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uin
     codes = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// Work decomposition.
+// Work decomposition.  CTA b takes work units b, b + gridDim.x, ...
 //   PB = false (one shared factor set): X is the flat matrix [n_rows = tokens*d/32][32];
-//     tile w = flat rows 128w .. 128w+127; outputs of flat row r: 16 B of codes at
+//     unit = tile w = flat rows 128w .. 128w+127; outputs of flat row r: 16 B of codes at
 //     q_packed + 16 r, scale byte at scales + r.
-//   PB = true (factor set j for block column j): tile w = (column j = w / n_ttiles,
-//     token tile tt = w % n_ttiles): 128 tokens x 32 channels of column j, fetched as a
-//     strided 2-D box from X[tokens][d]; its B operand is image j.  Output of token t:
-//     codes at q_packed + t*(d/2) + 16 j, scale byte at scales + t*(d/32) + j.
+//   PB = true (factor set j for block column j): unit u = (column group jg = u / n_ttiles,
+//     token tile tt = u % n_ttiles) = kPbCols consecutive MMA tiles, one per column
+//     j = kPbCols*jg + c: 128 tokens x 32 channels fetched as a strided 2-D box from
+//     X[tokens][d], multiplied by image j.  The group's codes (128 rows x 64 B, row pitch
+//     d/2) and scale bytes (128 x 4) are staged in shared memory and written once per
+//     group, because 16-byte and 1-byte pieces scattered at a row pitch cost one L2 write
+//     transaction each (measured: they halve the kernel's throughput).
+constexpr int kPbCols = 4;
 struct UmmaProblem {
     int64_t n_rows;      // PB=false: tokens*d/32 ; PB=true: tokens
-    int64_t n_tiles;     // total 128-row tiles
-    int n_ttiles;        // PB=true: token tiles per column (ceil(tokens/128))
+    int64_t n_units;     // PB=false: 128-row tiles ; PB=true: column groups x token tiles
+    int n_ttiles;        // PB=true: token tiles (ceil(tokens/128))
     int blocks_per_row;  // d/32
 };
 
@@ -218,9 +239,9 @@ struct UmmaProblem {
 // Grid: any size <= number of tiles; CTA b takes tiles b, b + gridDim.x, ...
 template <int NS, int NM, int NG, bool PB, bool WRITE_Y>
 __global__ void __launch_bounds__(128 + 128 * NG, 1)
-quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restrict__ b_image,
-              const UmmaProblem prob, uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales,
-              float* __restrict__ Y) {
+quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
+              const uint8_t* __restrict__ b_image, const UmmaProblem prob, uint8_t* __restrict__ q_packed,
+              uint8_t* __restrict__ scales, float* __restrict__ Y) {
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
     // A slot must always be served by the same issuer warp and the same epilogue group:
     // only then does program order inside that warp guarantee that a parity wait never
@@ -241,19 +262,31 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int my_tiles = (int)((prob.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    const int my_units = (int)((prob.n_units - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    const int my_tiles = PB ? my_units * kPbCols : my_units;
+    static_assert(!PB || NG == 1, "a column group is staged by one epilogue warpgroup");
 
     // issue the TMA copies of local tile n into slot n % NS (producer thread only)
+    // PB: local tile n -> column j (may be >= blocks_per_row in the last, ragged group: such a
+    // tile loads zeros and stores nothing), column group jg, token tile tt
+    auto pb_coords = [&](int n, int& j, int& jg, int& tt) {
+        const int64_t u = blockIdx.x + (int64_t)(n / kPbCols) * gridDim.x;
+        jg = (int)(u / prob.n_ttiles);
+        tt = (int)(u % prob.n_ttiles);
+        j = jg * kPbCols + (n % kPbCols);
+    };
     auto issue_tile = [&](int n) {
         const int s = n % NS;
-        const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
         const uint32_t dst = base + L::kAOff + s * L::kStageBytes;
         mbar_expect_tx(bar_full(s), L::kStageBytes);
         if (PB) {
-            const int j = (int)(w / prob.n_ttiles), tt = (int)(w % prob.n_ttiles);
-            tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));
-            bulk_load(dst + kTileBytes, b_image + (size_t)j * kBImageBytes, kBImageBytes, bar_full(s));
+            int j, jg, tt;
+            pb_coords(n, j, jg, tt);
+            const int jb = j < prob.blocks_per_row ? j : prob.blocks_per_row - 1;
+            tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));      // zero-filled if j is out of range
+            bulk_load(dst + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(s));
         } else {
+            const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
             tma_load_2d(dst, &tmap_x, 0, (int)(w * kTileRows), bar_full(s));
         }
     };
@@ -271,6 +304,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
         // so it may be fetched before the previous kernel in the stream has finished; X
         // (and, in the epilogue, the outputs) may not.
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+        if (PB && !WRITE_Y) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
         if (!PB) {
             mbar_expect_tx(bar_b, kBImageBytes);
             bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
@@ -362,32 +396,81 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const uint8_t* __restr
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tempty(s));
-            const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
-            int64_t row, blk;       // row inside the tiled dimension; flat index of the 32-channel block
-            if (PB) {
-                const int j = (int)(w / prob.n_ttiles), tt = (int)(w % prob.n_ttiles);
-                row = (int64_t)tt * kTileRows + quarter * 32 + lane;
-                blk = row * prob.blocks_per_row + j;
-            } else {
-                row = w * kTileRows + quarter * 32 + lane;
-                blk = row;
-            }
-            if (row < prob.n_rows) {
-                if (WRITE_Y) {
-                    float4* yp = reinterpret_cast<float4*>(Y + blk * 32);
+            if (PB && !WRITE_Y) {
+                int j, jg, tt;
+                pb_coords(n, j, jg, tt);
+                const int c = n % kPbCols;
+                const int r = quarter * 32 + lane;                 // token row inside the tile
+                const uint32_t st_codes = base + L::kStoreOff;
+                const uint32_t st_scale = st_codes + kTileRows * 64;
+                const bool elected = threadIdx.x == 128;
+                uint4 codes;
+                uint32_t S;
+                encode_block_regs(acc, codes, S);
+                if (c == 0) {
+                    // the previous group's TMA store must have finished reading the staging tile
+                    if (elected) bulk_wait_group_read<0>();
+                    named_barrier_sync(1, 128);
+                }
+                // 64-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3)
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                             ::"r"(st_codes + 64u * r + 16u * (uint32_t)(c ^ ((r >> 1) & 3))),
+                               "r"(codes.x), "r"(codes.y), "r"(codes.z), "r"(codes.w) : "memory");
+                asm volatile("st.shared.u8 [%0], %1;" ::"r"(st_scale + 4u * r + c), "r"(S) : "memory");
+                if (c == kPbCols - 1) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    named_barrier_sync(1, 128);
+                    if (elected) {
+                        tma_store_2d(&tmap_q, st_codes, 16 * kPbCols * jg, tt * kTileRows);   // clips ragged edges
+                        bulk_commit_group();
+                    }
+                    // scale bytes: lane l writes byte (l & 3) of row 8i + (l >> 2): 8 rows x 4 bytes per store
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        yp[i] = make_float4(__uint_as_float(acc[4 * i]), __uint_as_float(acc[4 * i + 1]),
-                                            __uint_as_float(acc[4 * i + 2]), __uint_as_float(acc[4 * i + 3]));
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = quarter * 32 + i * 8 + (lane >> 2);
+                        const int cc = lane & 3;
+                        const int64_t t = (int64_t)tt * kTileRows + rr;
+                        const int jj = jg * kPbCols + cc;
+                        uint32_t v;
+                        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(st_scale + 4u * rr + cc) : "memory");
+                        if (t < prob.n_rows && jj < prob.blocks_per_row)
+                            scales[t * prob.blocks_per_row + jj] = (uint8_t)v;
+                    }
+                }
+            } else {
+                int64_t row, blk;       // row inside the tiled dimension; flat index of the 32-channel block
+                bool valid;
+                if (PB) {
+                    int j, jg, tt;
+                    pb_coords(n, j, jg, tt);
+                    row = (int64_t)tt * kTileRows + quarter * 32 + lane;
+                    blk = row * prob.blocks_per_row + j;
+                    valid = row < prob.n_rows && j < prob.blocks_per_row;
                 } else {
-                    uint4 codes;
-                    uint32_t S;
-                    encode_block_regs(acc, codes, S);
-                    st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
-                    scales[blk] = (uint8_t)S;
+                    const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
+                    row = w * kTileRows + quarter * 32 + lane;
+                    blk = row;
+                    valid = row < prob.n_rows;
+                }
+                if (valid) {
+                    if (WRITE_Y) {
+                        float4* yp = reinterpret_cast<float4*>(Y + blk * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            yp[i] = make_float4(__uint_as_float(acc[4 * i]), __uint_as_float(acc[4 * i + 1]),
+                                                __uint_as_float(acc[4 * i + 2]), __uint_as_float(acc[4 * i + 3]));
+                    } else {
+                        uint4 codes;
+                        uint32_t S;
+                        encode_block_regs(acc, codes, S);
+                        st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
+                        scales[blk] = (uint8_t)S;
+                    }
                 }
             }
         }
+        // the staging tile must not be released while a TMA store still reads it
+        if (PB && !WRITE_Y && threadIdx.x == 128) bulk_wait_group_read<0>();
     }
 
     // ---------------- teardown ----------------

@@ -118,7 +118,8 @@ void build_b_image(const float* G20, uint8_t* img) {
 }
 
 template <int NS, int NM, int NG, bool PB, bool WRITE_Y>
-kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, const kq::UmmaProblem& prob,
+kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
+                        const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, int ctas_per_sm, bool pdl, cudaStream_t st) {
     using L = kq::UmmaSmem<NS, PB>;
     auto kern = kq::quantize_umma<NS, NM, NG, PB, WRITE_Y>;
@@ -130,9 +131,13 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, const kq::
     if (attr_rc != cudaSuccess) return KQ_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
+    // persistent grid: at most ctas_per_sm CTAs per SM (shrinking it further so that every CTA
+    // gets the same number of units was measured and is no faster: fewer resident CTAs hide
+    // less latency than the shorter last round saves)
     const int64_t cap = (int64_t)sms * ctas_per_sm;
+    const int64_t grid = prob.n_units < cap ? prob.n_units : cap;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(prob.n_tiles < cap ? prob.n_tiles : cap));
+    cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(128 + 128 * NG);
     cfg.dynamicSmemBytes = L::kDynBytes;
     cfg.stream = st;
@@ -141,7 +146,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const uint8_t* bimg, const kq::
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap, bimg, prob, q, scales, Y) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, prob, q, scales, Y) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -165,12 +170,12 @@ kq_status_t run_umma(const void* X, int64_t tokens, int d, const kroquant_factor
     if (pb) {
         prob.n_rows = tokens;
         prob.n_ttiles = (int)((tokens + kq::kTileRows - 1) / kq::kTileRows);
-        prob.n_tiles = (int64_t)prob.n_ttiles * nb;
+        prob.n_units = (int64_t)prob.n_ttiles * ((nb + kq::kPbCols - 1) / kq::kPbCols);
         dims[0] = (cuuint64_t)d; dims[1] = (cuuint64_t)tokens; strides[0] = (cuuint64_t)d * 2;
     } else {
         prob.n_rows = tokens * (int64_t)nb;
         prob.n_ttiles = 1;
-        prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
+        prob.n_units = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
         dims[0] = 32; dims[1] = (cuuint64_t)prob.n_rows; strides[0] = 64;
     }
     const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
@@ -179,27 +184,38 @@ kq_status_t run_umma(const void* X, int64_t tokens, int d, const kroquant_factor
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
+    // per-block variant: the codes of a column group (128 tokens x 64 B, row pitch d/2) leave by TMA store
+    CUtensorMap tmap_q = tmap;
+    if (pb && !WRITE_Y) {
+        const cuuint64_t qdims[2] = {(cuuint64_t)(d / 2), (cuuint64_t)tokens};
+        const cuuint64_t qstrides[1] = {(cuuint64_t)(d / 2)};
+        const cuuint32_t qbox[2] = {16 * kq::kPbCols, (cuuint32_t)kq::kTileRows};
+        if (enc(&tmap_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, q, qdims, qstrides, qbox, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return KQ_ERR_CUDA;
+    }
     const int cps = g_umma_ctas_per_sm.load();
     const bool pdl = g_umma_pdl.load() != 0;
     const uint8_t* b = f->d_bimage;
     if (pb) {
         switch (g_umma_cfg.load()) {
             default:
-            case 5: return launch_umma<4, 2, 1, true, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-            case 4: return launch_umma<4, 1, 1, true, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-            case 2: return launch_umma<8, 2, 2, true, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+            case 4: return launch_umma<4, 1, 1, true, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+            case 0: return launch_umma<4, 2, 1, true, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+            case 1: return launch_umma<8, 2, 1, true, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
         }
     }
     switch (g_umma_cfg.load()) {
         default:
-        case 0: return launch_umma<8, 1, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-        case 1: return launch_umma<8, 2, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-        case 2: return launch_umma<8, 2, 2, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-        case 3: return launch_umma<8, 1, 2, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-        case 4: return launch_umma<4, 1, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-        case 5: return launch_umma<4, 2, 1, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-        case 6: return launch_umma<16, 2, 2, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
-        case 7: return launch_umma<16, 2, 4, false, WRITE_Y>(tmap, b, prob, q, scales, Y, cps, pdl, st);
+        case 0: return launch_umma<8, 1, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 1: return launch_umma<8, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 2: return launch_umma<8, 2, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 3: return launch_umma<8, 1, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 4: return launch_umma<4, 1, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 5: return launch_umma<4, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 6: return launch_umma<16, 2, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 7: return launch_umma<16, 2, 4, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
     }
 }
 
