@@ -64,6 +64,11 @@ __device__ __forceinline__ uint32_t encode8(const float (&y)[8], float amax_bloc
 
 // n_quads = tokens * d / 8 work items; item q: block = q / 4, quad = q % 4.
 // factors: n_sets FactorSet (MODE_KRON); chan_scale: float[d] (MODE_SCALE).
+// Every thread keeps kStreamUnroll independent 16-byte loads in flight per iteration
+// (2048 resident threads x 16 B alone would be 32 KB per SM, below the ~40 KB the HBM
+// latency-bandwidth product asks for).
+constexpr int kStreamUnroll = 4;
+
 template <int MODE, bool WRITE_Y>
 __global__ void __launch_bounds__(256)
 quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row,
@@ -71,56 +76,118 @@ quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row
                 const float* __restrict__ chan_scale,
                 uint32_t* __restrict__ q_packed, uint8_t* __restrict__ scales,
                 float* __restrict__ Y) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;   // multiple of 32: quads stay lane-aligned
     const int quad = threadIdx.x & 3;
     FactorSet F;
     if (MODE == MODE_KRON && n_sets == 1) F = factors[0];
     // the trip count is uniform across the warp: all lanes run the shuffles together
-    const int64_t n_iter = (n_quads + stride - 1) / stride;
-    int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    for (int64_t it = 0; it < n_iter; ++it, q += stride) {
-        const bool live = q < n_quads;
-        float y[8];
-        if (live) {
-            widen8(ld_stream_16(X + q), y);
-        } else {
+    const int64_t n_iter = (n_quads + stride * kStreamUnroll - 1) / (stride * kStreamUnroll);
+    int64_t q0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // position inside the token row, in quads (8 channels), kept incrementally: one 64-bit
+    // remainder per thread instead of one per item
+    const int quads_per_row = blocks_per_row * 4;
+    const int step = (int)(stride % quads_per_row);
+    int pos = (int)(q0 % quads_per_row);
+    for (int64_t it = 0; it < n_iter; ++it, q0 += stride * kStreamUnroll) {
+        uint4 raw[kStreamUnroll];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) y[i] = 0.f;
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            const int64_t q = q0 + u * stride;
+            raw[u] = q < n_quads ? ld_stream_16(X + q) : make_uint4(0u, 0u, 0u, 0u);
         }
-        const int64_t blk = q >> 2;
-        if (MODE == MODE_SCALE) {
-            if (live) {
-                const int j = (int)(blk % blocks_per_row);
-                const float4* sp = reinterpret_cast<const float4*>(chan_scale + j * kBlock + quad * 8);
-                const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
-                y[0] *= s0.x; y[1] *= s0.y; y[2] *= s0.z; y[3] *= s0.w;
-                y[4] *= s1.x; y[5] *= s1.y; y[6] *= s1.z; y[7] *= s1.w;
-            }
-        } else if (MODE == MODE_KRON) {
-            if (n_sets != 1) {
-                const int j = live ? (int)(blk % blocks_per_row) : 0;
-                const float4* gp = reinterpret_cast<const float4*>(factors + j);
 #pragma unroll
-                for (int k = 0; k < 5; ++k) F.g[k] = __ldg(gp + k);
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            const int64_t q = q0 + u * stride;
+            const bool live = q < n_quads;
+            float y[8];
+            widen8(raw[u], y);
+            const int64_t blk = q >> 2;
+            const int j = pos >> 2;                 // block column of this item
+            pos += step;
+            if (pos >= quads_per_row) pos -= quads_per_row;
+            if (MODE == MODE_SCALE) {
+                if (live) {
+                    const float4* sp = reinterpret_cast<const float4*>(chan_scale + j * kBlock + quad * 8);
+                    const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
+                    y[0] *= s0.x; y[1] *= s0.y; y[2] *= s0.z; y[3] *= s0.w;
+                    y[4] *= s1.x; y[5] *= s1.y; y[6] *= s1.z; y[7] *= s1.w;
+                }
+            } else if (MODE == MODE_KRON) {
+                if (n_sets != 1) {
+                    const float4* gp = reinterpret_cast<const float4*>(factors + j);
+#pragma unroll
+                    for (int k = 0; k < 5; ++k) F.g[k] = __ldg(gp + k);
+                }
+                kron_butterfly(y, F, quad);
             }
-            kron_butterfly(y, F, quad);
+            if (WRITE_Y) {
+                if (live) {
+                    float4* yp = reinterpret_cast<float4*>(Y) + 2 * q;
+                    yp[0] = make_float4(y[0], y[1], y[2], y[3]);
+                    yp[1] = make_float4(y[4], y[5], y[6], y[7]);
+                }
+            } else {
+                float amax = absmax8(y);
+                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+                uint32_t S;
+                const uint32_t codes = encode8(y, amax, S);
+                if (live) {
+                    st_stream_4(q_packed + q, codes);
+                    if (quad == 0) scales[blk] = (uint8_t)S;
+                }
+            }
         }
-        if (WRITE_Y) {
-            if (live) {
-                float4* yp = reinterpret_cast<float4*>(Y) + 2 * q;
-                yp[0] = make_float4(y[0], y[1], y[2], y[3]);
-                yp[1] = make_float4(y[4], y[5], y[6], y[7]);
-            }
-        } else {
+    }
+}
+
+// Per-channel scale + MXFP4 with the thread's eight multipliers held in registers: thread t
+// owns quad column p = t % (d/8) of the token rows r0, r0 + R, r0 + 2R, ... (R = rows in
+// flight = threads / (d/8)), so the scale vector is read once per thread instead of once
+// per item.  Requires gridDim.x * blockDim.x >= d/8.  The four lanes of a quad always
+// work on the same row, so the amax shuffles use a per-quad mask (trip counts may differ
+// between quads of one warp).
+__global__ void __launch_bounds__(256)
+scale_quantize_rows(const uint4* __restrict__ X, int64_t tokens, int quads_per_row,
+                    const float* __restrict__ chan_scale, uint32_t* __restrict__ q_packed,
+                    uint8_t* __restrict__ scales) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t n_threads = (int64_t)gridDim.x * blockDim.x;
+    const int64_t R = n_threads / quads_per_row;          // token rows in flight
+    const int p = (int)(t % quads_per_row);
+    const int64_t r0 = t / quads_per_row;
+    const int quad = threadIdx.x & 3;
+    const uint32_t qmask = 0xFu << (threadIdx.x & 28);
+    const float4* sp = reinterpret_cast<const float4*>(chan_scale + (int64_t)p * 8);
+    const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);      // the scale vector is immutable input
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (r0 >= R) return;                                  // leftover threads of the last partial row group
+    for (int64_t r = r0; r < tokens; r += R * kStreamUnroll) {
+        uint4 raw[kStreamUnroll];
+#pragma unroll
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            const int64_t rr = r + u * R;
+            raw[u] = rr < tokens ? ld_stream_16(X + rr * quads_per_row + p) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            const int64_t rr = r + u * R;
+            if (rr >= tokens) break;                      // uniform inside the quad
+            float y[8];
+            widen8(raw[u], y);
+            y[0] *= s0.x; y[1] *= s0.y; y[2] *= s0.z; y[3] *= s0.w;
+            y[4] *= s1.x; y[5] *= s1.y; y[6] *= s1.z; y[7] *= s1.w;
             float amax = absmax8(y);
-            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+            amax = fmaxf(amax, __shfl_xor_sync(qmask, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(qmask, amax, 2));
             uint32_t S;
             const uint32_t codes = encode8(y, amax, S);
-            if (live) {
-                st_stream_4(q_packed + q, codes);
-                if (quad == 0) scales[blk] = (uint8_t)S;
-            }
+            const int64_t q = rr * quads_per_row + p;
+            st_stream_4(q_packed + q, codes);
+            if (quad == 0) scales[q >> 2] = (uint8_t)S;
         }
     }
 }

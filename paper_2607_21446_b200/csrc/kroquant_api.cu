@@ -223,12 +223,23 @@ template <int MODE, bool WRITE_Y>
 kq_status_t run_stream(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, const float* s,
                        uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
     const int64_t n_quads = tokens * (int64_t)(d / 8);
-    const int grid = stream_grid(n_quads);
+    const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
-    kq::quantize_stream<MODE, WRITE_Y><<<grid, 256, 0, st>>>(
-        reinterpret_cast<const uint4*>(X), n_quads, d / 32, f ? f->d_G : nullptr, f ? f->n_sets : 0, s,
-        reinterpret_cast<uint32_t*>(q), scales, Y);
-    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kq::quantize_stream<MODE, WRITE_Y>, reinterpret_cast<const uint4*>(X), n_quads,
+                           d / 32, f ? (const kq::FactorSet*)f->d_G : (const kq::FactorSet*)nullptr,
+                           f ? f->n_sets : 0, s, reinterpret_cast<uint32_t*>(q), scales, Y) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KQ_ERR_CUDA;
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return KQ_OK;
 }
@@ -365,8 +376,28 @@ kq_status_t kroquant_scale_quantize(const void* X, int64_t tokens, int d, const 
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed) || !aligned16(s)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
-    return run_stream<kq::MODE_SCALE, false>(X, tokens, d, nullptr, s, q_packed, scales, nullptr,
-                                             static_cast<cudaStream_t>(stream));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t n_quads = tokens * (int64_t)(d / 8);
+    const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
+    if (grid <= 0) return KQ_ERR_CUDA;
+    if ((int64_t)grid * 256 < d / 8)      // fewer threads than quad columns: generic kernel
+        return run_stream<kq::MODE_SCALE, false>(X, tokens, d, nullptr, s, q_packed, scales, nullptr, st);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows, reinterpret_cast<const uint4*>(X), tokens, d / 8, s,
+                           reinterpret_cast<uint32_t*>(q_packed), scales) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KQ_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
 }
 
 kq_status_t kroquant_mxfp4_quantize(const void* X, int64_t tokens, int d, uint8_t* q_packed, uint8_t* scales,
