@@ -118,8 +118,8 @@ kq_status_t kroquant_transform_f32(const void *X, int64_t tokens, int d,
 kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes, void *stream);
 
 /* Tuning hook for the tensor-core kernel.  config 0..7 selects (pipeline slots, MMA
- * issuer warps, epilogue warpgroups) = (8,1,1) (8,2,1) (8,2,2) (8,1,2) (4,1,1) (4,2,1)
- * (16,2,2) (16,2,4); the default is config 5 with 3 CTAs per SM; ctas_per_sm in 1..4 caps the persistent grid; use_pdl != 0
+ * issuer warps, epilogue warpgroups) = (2,2,1) (8,2,1) (8,2,2) (2,1,1) (4,1,1) (4,2,1)
+ * (16,2,2) (16,2,4); the default is config 5 with 3 CTAs per SM; ctas_per_sm in 1..8 caps the persistent grid; use_pdl != 0
  * launches with programmatic stream serialization.  Process-wide. */
 kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl);
 

@@ -208,10 +208,10 @@ kq_status_t run_umma(const void* X, int64_t tokens, int d, const kroquant_factor
     }
     switch (g_umma_cfg.load()) {
         default:
-        case 0: return launch_umma<8, 1, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 0: return launch_umma<2, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
         case 1: return launch_umma<8, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
         case 2: return launch_umma<8, 2, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 3: return launch_umma<8, 1, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 3: return launch_umma<2, 1, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
         case 4: return launch_umma<4, 1, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
         case 5: return launch_umma<4, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
         case 6: return launch_umma<16, 2, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
@@ -447,7 +447,7 @@ kq_status_t kroquant_debug_e2m1_codes(const float* v, int64_t n, uint8_t* codes,
 }
 
 kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl) {
-    if (config < 0 || config > 7 || ctas_per_sm < 1 || ctas_per_sm > 4) return KQ_ERR_UNSUPPORTED;
+    if (config < 0 || config > 7 || ctas_per_sm < 1 || ctas_per_sm > 8) return KQ_ERR_UNSUPPORTED;
     g_umma_cfg.store(config);
     g_umma_ctas_per_sm.store(ctas_per_sm);
     g_umma_pdl.store(use_pdl != 0);
