@@ -444,8 +444,57 @@ def run_single(args):
                       "device_error": B.kroquant_last_device_error()}), flush=True)
 
 
+def run_sweep(args):
+    """The sweep config: tokens x d grid; KroQuant (one shared set), Scale and bare MXFP4 on the
+    same input, each as a CUDA graph of back-to-back calls over rotating buffers (> 3 x L2);
+    CPU oracle timed on the first 2048 rows and scaled linearly.  One JSON line per point."""
+    import torch
+    from oracle import c_oracle as co
+    from paper_2607_21446_b200 import binding as B
+    B.load_library()
+    peak, peak_kind = measured_peak()
+    stream = torch.cuda.Stream()
+    for tokens in W.SWEEP_TOKENS:
+        for d in W.SWEEP_D:
+            nbuf = min(28, max(3, int(400e6 // (tokens * d * 2)) + 1))
+            sp = W.sweep_spec(min(tokens, 4096), d)          # host generator on <= 4096 rows, tiled on the device
+            bits = W.gen_activations(sp)
+            x0 = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+            x0 = x0.repeat((tokens + x0.shape[0] - 1) // x0.shape[0], 1)[:tokens].contiguous()
+            Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, nbuf)]
+            q = torch.empty((tokens, d // 2), dtype=torch.uint8, device="cuda")
+            sc = torch.empty((tokens, d // 32), dtype=torch.uint8, device="cuda")
+            G = W.gen_factors(4)
+            f = B.Factors.create(G)
+            sv = torch.from_numpy(W.gen_channel_scales(4, d)).cuda()
+            res = {}
+            for name, fn in (("kroquant", lambda x: B.kroquant_quantize(x, f, q, sc, stream=stream)),
+                             ("scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
+                             ("plain_mxfp4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream))):
+                g = capture(torch, [lambda x=x, fn=fn: fn(x) for x in Xs], stream)
+                ms, _ = time_graph(torch, None, g, stream, max(5, args.steps // 10), 3)
+                res[name] = ms * 1e3 / nbuf
+            rows = min(tokens, 2048)
+            t0 = time.perf_counter()
+            co.quantize(bits[:rows], G)
+            cpu_s = (time.perf_counter() - t0) * tokens / rows
+            byt = W.algorithmic_bytes(tokens, d)
+            print(json.dumps({
+                "sweep": f"{tokens}x{d}", "us": {k: round(v, 2) for k, v in res.items()},
+                "GB/s": {k: round(byt / v / 1e3, 1) for k, v in res.items()},
+                "frac_of_hbm_peak": {k: round(byt / v / 1e3 / peak, 4) for k, v in res.items()},
+                "tokens_per_s": round(tokens / (res["kroquant"] * 1e-6)),
+                "scale_over_kroquant": round(res["scale"] / res["kroquant"], 3),
+                "plain_over_kroquant": round(res["plain_mxfp4"] / res["kroquant"], 3),
+                "cpu_oracle_s": round(cpu_s, 3), "cpu_oracle_extrapolated_from_rows": rows,
+                "cpu_cores": os.cpu_count(), "peak": f"{peak} GB/s of {peak_kind}", "buffers": nbuf}), flush=True)
+            del Xs, x0, q, sc
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--sweep", action="store_true",
+                    help="tokens x d sweep of KroQuant / Scale / bare MXFP4 (one JSON line per point)")
     ap.add_argument("--single", default=None, metavar="TOKENSxD",
                     help="profiling aid: a few eager launches of one shape, e.g. 4608x12288")
     ap.add_argument("--kernel", default="kroquant", choices=["kroquant", "scale", "plain"])
@@ -456,7 +505,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.single:
+    if args.sweep:
+        run_sweep(args)
+    elif args.single:
         run_single(args)
     elif args.impl == "reference":
         run_reference(args)
