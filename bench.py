@@ -424,7 +424,7 @@ def run_single(args):
     Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, nbuf)]
     q = torch.empty((t, d // 2), dtype=torch.uint8, device="cuda")
     sc = torch.empty((t, d // 32), dtype=torch.uint8, device="cuda")
-    f = B.Factors.create(W.gen_factors(3))
+    f = B.Factors.create(W.gen_factors(3, n_sets=d // 32 if args.per_block else 1))
     sv = torch.from_numpy(W.gen_channel_scales(3, d)).cuda()
     fn = {"kroquant": lambda x: B.kroquant_quantize(x, f, q, sc),
           "scale": lambda x: B.kroquant_scale_quantize(x, sv, q, sc),
@@ -499,6 +499,7 @@ def main():
                     help="profiling aid: a few eager launches of one shape, e.g. 4608x12288")
     ap.add_argument("--kernel", default="kroquant", choices=["kroquant", "scale", "plain"])
     ap.add_argument("--calls", type=int, default=8)
+    ap.add_argument("--per-block", action="store_true", help="with --single: one factor set per 32-channel block")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
