@@ -40,7 +40,7 @@ SHAPES = [(4608, 3072), (4608, 12288)]
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch of the tensor-core kernel from the Nsight Compute captures
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
-NCU_TRAFFIC_BYTES = {(4608, 3072): 28.35e6, (4608, 12288): 124.8e6}
+NCU_TRAFFIC_BYTES = {(4608, 3072): 28.35e6, (4608, 12288): 125.5e6}
 
 
 def measured_peak():
@@ -400,7 +400,7 @@ def run_ours(args):
         "gpu_launches": n_launch,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                     "kernel": "quantize_umma_shared", "launches": n_launch,
+                     "kernel": "quantize_umma<4,2,1,false,false>", "launches": n_launch,
                      "avg_launch_us": us_per_launch, "algorithmic_bytes_per_launch": alg_per_launch},
         "cpu_baseline": {"value": cpu_gbs, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{SAMPLE}, {cpu_dt:.2f} s per pass, 5 passes, "
