@@ -26,6 +26,9 @@ def lib() -> C.CDLL:
         L.kq_oracle_dense_kinv.argtypes = [vp, vp]
         L.kq_oracle_dense_kinv.restype = None
         L.kq_oracle_transform.argtypes = [vp, i64, i32, vp, i32, vp]
+        L.kq_oracle_transform_x.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
+        L.kq_oracle_scale_transform_x.argtypes = [vp, i32, i64, i32, vp, vp]
+        L.kq_oracle_widen_x.argtypes = [vp, i32, i64, i32, vp]
         L.kq_oracle_scale_transform.argtypes = [vp, i64, i32, vp, vp]
         L.kq_oracle_widen.argtypes = [vp, i64, i32, vp]
         L.kq_oracle_encode_block.argtypes = [vp, vp, vp]
@@ -82,26 +85,39 @@ def dense_kinv(G1) -> np.ndarray:
     return K
 
 
-def transform(X, G) -> np.ndarray:
-    X, G = _x(X), _g(G)
+X_DTYPES = {"bf16": 0, "fp16": 1}
+
+
+def transform(X, G=None, x_dtype: str = "bf16", K_dense=None) -> np.ndarray:
+    """float32( x K ) per block.  Either factors G [n_sets,5,2,2] or dense K_dense [n_sets,32,32]."""
+    X = _x(X)
     Y = np.empty(X.shape, np.float32)
-    _check(lib().kq_oracle_transform(_p(X), X.shape[0], X.shape[1], _p(G), G.shape[0], _p(Y)))
+    if K_dense is not None:
+        Kd = np.ascontiguousarray(K_dense, dtype=np.float32)
+        assert Kd.ndim == 3 and Kd.shape[1:] == (32, 32)
+        rc = lib().kq_oracle_transform_x(_p(X), X_DTYPES[x_dtype], X.shape[0], X.shape[1], None, _p(Kd),
+                                         Kd.shape[0], _p(Y))
+    else:
+        G = _g(G)
+        rc = lib().kq_oracle_transform_x(_p(X), X_DTYPES[x_dtype], X.shape[0], X.shape[1], _p(G), None,
+                                         G.shape[0], _p(Y))
+    _check(rc)
     return Y
 
 
-def scale_transform(X, s) -> np.ndarray:
+def scale_transform(X, s, x_dtype: str = "bf16") -> np.ndarray:
     X = _x(X)
     s = np.ascontiguousarray(s, dtype=np.float32)
     assert s.shape == (X.shape[1],)
     Y = np.empty(X.shape, np.float32)
-    _check(lib().kq_oracle_scale_transform(_p(X), X.shape[0], X.shape[1], _p(s), _p(Y)))
+    _check(lib().kq_oracle_scale_transform_x(_p(X), X_DTYPES[x_dtype], X.shape[0], X.shape[1], _p(s), _p(Y)))
     return Y
 
 
-def widen(X) -> np.ndarray:
+def widen(X, x_dtype: str = "bf16") -> np.ndarray:
     X = _x(X)
     Y = np.empty(X.shape, np.float32)
-    _check(lib().kq_oracle_widen(_p(X), X.shape[0], X.shape[1], _p(Y)))
+    _check(lib().kq_oracle_widen_x(_p(X), X_DTYPES[x_dtype], X.shape[0], X.shape[1], _p(Y)))
     return Y
 
 
@@ -125,21 +141,21 @@ def mx_encode(Y) -> tuple[np.ndarray, np.ndarray]:
     return q, s
 
 
-def quantize(X, G):
+def quantize(X, G=None, x_dtype: str = "bf16", K_dense=None):
     """-> (q_packed, scales, Y) with Y the float pre-rounding values."""
-    Y = transform(X, G)
+    Y = transform(X, G, x_dtype, K_dense)
     q, s = mx_encode(Y)
     return q, s, Y
 
 
-def scale_quantize(X, svec):
-    Y = scale_transform(X, svec)
+def scale_quantize(X, svec, x_dtype: str = "bf16"):
+    Y = scale_transform(X, svec, x_dtype)
     q, s = mx_encode(Y)
     return q, s, Y
 
 
-def plain_quantize(X):
-    Y = widen(X)
+def plain_quantize(X, x_dtype: str = "bf16"):
+    Y = widen(X, x_dtype)
     q, s = mx_encode(Y)
     return q, s, Y
 

@@ -15,6 +15,8 @@
  *     the tile is multiplied from the left: y = x K            (Section 3.5)
  *   - inverse = Kronecker product of the five 2x2 inverses     (Section 3.2)
  *   - LU form G = [[1,0],[c,1]] [[a,b],[0,-1/a]]                (Section 3.2)
+ *   - dense 32x32 blocks given directly ("K1", Section 3.5) and fp16 activations
+ *     (the paper's kernel benchmarks run in FP16, Section 4.4) use the same sums
  *   - MXFP4: E2M1 elements, one E8M0 scale per 32 block, OCP Microscaling
  *     conversion (Section 4.1 "Data format", Appendix D "Quantization"):
  *     shared exponent = floor(log2 amax) - 2, elements rounded to nearest even
@@ -41,6 +43,23 @@ static float bf16_bits_to_float(uint16_t b)
     float f;
     memcpy(&f, &u, sizeof f);
     return f;
+}
+
+/* exact fp16 (IEEE binary16) widening, subnormals included */
+static float fp16_bits_to_float(uint16_t h)
+{
+    int sign = (h >> 15) & 1, e = (h >> 10) & 31, m = h & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)m, -24);                 /* subnormal: m * 2^-24 */
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)m / 1024.0, e - 15);
+    return (float)(sign ? -v : v);
+}
+
+/* activation element i of X as a float; x_dtype: 0 = bf16 bits, 1 = fp16 bits */
+static float load_x(const uint16_t *X, int64_t i, int x_dtype)
+{
+    return x_dtype ? fp16_bits_to_float(X[i]) : bf16_bits_to_float(X[i]);
 }
 
 /* float -> bf16 bits, round-to-nearest-even (finite inputs). */
@@ -108,10 +127,12 @@ void kq_oracle_dense_kinv(const float *G, double *Kinv)
 }
 
 /* ---- transform: Y[t, 32j + c] = float( sum_r x_r K^(j)[r][c] ) ----------- */
-/* X: bf16 bits [tokens][d]; G: [n_sets][5][2][2], n_sets in {1, d/32};
+/* X: 16-bit patterns [tokens][d] (x_dtype 0 = bf16, 1 = fp16).  The block matrices come either from
+ * factors G: [n_sets][5][2][2] (Kdense == NULL) or directly as dense Kdense: float [n_sets][32][32],
+ * K[r][c] row-major (the paper's "precomputed dense" storage, Section 3.5 K1); n_sets in {1, d/32}.
  * Y: float [tokens][d].  Returns 0, or -1 on a bad shape. */
-int kq_oracle_transform(const uint16_t *X, int64_t tokens, int d,
-                        const float *G, int n_sets, float *Y)
+int kq_oracle_transform_x(const uint16_t *X, int x_dtype, int64_t tokens, int d,
+                          const float *G, const float *Kdense, int n_sets, float *Y)
 {
     if (d <= 0 || d % KQ_BLOCK || tokens < 0) return -1;
     int nb = d / KQ_BLOCK;
@@ -119,13 +140,19 @@ int kq_oracle_transform(const uint16_t *X, int64_t tokens, int d,
 #pragma omp parallel for schedule(static)
     for (int64_t t = 0; t < tokens; ++t) {
         double K[KQ_BLOCK * KQ_BLOCK];
-        if (n_sets == 1) kq_oracle_dense_k(G, K);
         for (int j = 0; j < nb; ++j) {
-            if (n_sets != 1) kq_oracle_dense_k(G + (size_t)j * 20, K);
-            const uint16_t *xb = X + t * d + (int64_t)j * KQ_BLOCK;
+            if (j == 0 || n_sets != 1) {
+                int set = n_sets == 1 ? 0 : j;
+                if (Kdense)
+                    for (int i = 0; i < KQ_BLOCK * KQ_BLOCK; ++i)
+                        K[i] = (double)Kdense[(size_t)set * KQ_BLOCK * KQ_BLOCK + i];
+                else
+                    kq_oracle_dense_k(G + (size_t)set * 20, K);
+            }
             float *yb = Y + t * d + (int64_t)j * KQ_BLOCK;
             double x[KQ_BLOCK];
-            for (int r = 0; r < KQ_BLOCK; ++r) x[r] = (double)bf16_bits_to_float(xb[r]);
+            for (int r = 0; r < KQ_BLOCK; ++r)
+                x[r] = (double)load_x(X, t * d + (int64_t)j * KQ_BLOCK + r, x_dtype);
             for (int c = 0; c < KQ_BLOCK; ++c) {
                 double acc = 0.0;
                 for (int r = 0; r < KQ_BLOCK; ++r) acc += x[r] * K[r * KQ_BLOCK + c];
@@ -136,26 +163,42 @@ int kq_oracle_transform(const uint16_t *X, int64_t tokens, int d,
     return 0;
 }
 
+int kq_oracle_transform(const uint16_t *X, int64_t tokens, int d,
+                        const float *G, int n_sets, float *Y)
+{
+    return kq_oracle_transform_x(X, 0, tokens, d, G, NULL, n_sets, Y);
+}
+
 /* per-channel scaling (SmoothQuant-style diagonal T, Appendix D "Smoothing"):
  * Y[t, i] = float( x * s_i ); the double product is exact, so this is one
  * correctly rounded float product. */
-int kq_oracle_scale_transform(const uint16_t *X, int64_t tokens, int d,
-                              const float *s, float *Y)
+int kq_oracle_scale_transform_x(const uint16_t *X, int x_dtype, int64_t tokens, int d,
+                                const float *s, float *Y)
 {
     if (d <= 0 || d % KQ_BLOCK || tokens < 0) return -1;
 #pragma omp parallel for schedule(static)
     for (int64_t t = 0; t < tokens; ++t)
         for (int i = 0; i < d; ++i)
-            Y[t * d + i] = (float)((double)bf16_bits_to_float(X[t * d + i]) * (double)s[i]);
+            Y[t * d + i] = (float)((double)load_x(X, t * d + i, x_dtype) * (double)s[i]);
     return 0;
 }
 
+int kq_oracle_scale_transform(const uint16_t *X, int64_t tokens, int d, const float *s, float *Y)
+{
+    return kq_oracle_scale_transform_x(X, 0, tokens, d, s, Y);
+}
+
 /* no transform (bare MXFP4 quantizer, the paper's "Q4" column): Y = X widened. */
-int kq_oracle_widen(const uint16_t *X, int64_t tokens, int d, float *Y)
+int kq_oracle_widen_x(const uint16_t *X, int x_dtype, int64_t tokens, int d, float *Y)
 {
     if (d <= 0 || d % KQ_BLOCK || tokens < 0) return -1;
-    for (int64_t i = 0; i < tokens * d; ++i) Y[i] = bf16_bits_to_float(X[i]);
+    for (int64_t i = 0; i < tokens * d; ++i) Y[i] = load_x(X, i, x_dtype);
     return 0;
+}
+
+int kq_oracle_widen(const uint16_t *X, int64_t tokens, int d, float *Y)
+{
+    return kq_oracle_widen_x(X, 0, tokens, d, Y);
 }
 
 /* ---- MXFP4 encode -------------------------------------------------------- */

@@ -45,6 +45,16 @@ def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
     return b.view(np.float32)
 
 
+def f32_to_fp16_bits(x: np.ndarray) -> np.ndarray:
+    """Round float32 values to IEEE binary16 (NumPy's round-to-nearest-even cast) and return
+    the 16-bit patterns.  Inputs must be finite and below 65504 in magnitude."""
+    return np.ascontiguousarray(x, dtype=np.float32).astype(np.float16).view(np.uint16)
+
+
+def fp16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(bits, dtype=np.uint16).view(np.float16).astype(np.float32)
+
+
 # --------------------------------------------------------------------------
 # factors, LU parameters, scales
 # --------------------------------------------------------------------------
@@ -139,9 +149,22 @@ def gen_activations_f32(spec: ActivationSpec) -> np.ndarray:
     return x
 
 
-def gen_activations(spec: ActivationSpec) -> np.ndarray:
-    """bf16 bit patterns (uint16) of the activation tensor, shape [tokens, d]."""
-    return f32_to_bf16_bits(gen_activations_f32(spec))
+def gen_activations(spec: ActivationSpec, dtype: str = "bf16") -> np.ndarray:
+    """16-bit patterns (uint16) of the activation tensor, shape [tokens, d]; bf16 or fp16."""
+    x = gen_activations_f32(spec)
+    return f32_to_fp16_bits(x) if dtype == "fp16" else f32_to_bf16_bits(x)
+
+
+def gen_dense_blocks(seed: int, n_sets: int = 1) -> np.ndarray:
+    """Random well-conditioned dense 32x32 blocks (not Kronecker-structured): orthogonal (QR of a
+    Gaussian) times diag(U[0.5, 2])."""
+    rng = np.random.default_rng(seed + 2000)
+    out = np.empty((n_sets, 32, 32), np.float32)
+    for s in range(n_sets):
+        Q, R = np.linalg.qr(rng.standard_normal((32, 32)))
+        Q = Q * np.sign(np.diag(R))
+        out[s] = (Q * rng.uniform(0.5, 2.0, size=32)[None, :]).astype(np.float32)
+    return out
 
 
 def tiny_spec() -> ActivationSpec:

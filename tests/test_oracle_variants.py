@@ -1,0 +1,72 @@
+"""Pins for the oracle's fp16-input and dense-block variants (CPU only)."""
+import numpy as np
+import pytest
+
+from oracle import c_oracle as co
+from paper_2607_21446_b200 import workloads as W
+
+
+def kron_chain(G1):
+    K = G1[0].astype(np.float64)
+    for k in range(1, 5):
+        K = np.kron(K, G1[k].astype(np.float64))
+    return K
+
+
+def test_fp16_widening_matches_numpy_for_every_finite_pattern():
+    bits = np.arange(0, 1 << 16, dtype=np.uint32).astype(np.uint16)
+    ref = bits.view(np.float16).astype(np.float32)           # library conversion
+    fin = np.isfinite(ref)
+    pad = (-fin.sum()) % 32
+    b = np.concatenate([bits[fin], np.zeros(pad, np.uint16)]).reshape(-1, 32)
+    got = co.widen(b, x_dtype="fp16").reshape(-1)[:fin.sum()]
+    assert np.array_equal(got.view(np.uint32), ref[fin].view(np.uint32))   # also the sign of zero
+
+
+def test_fp16_and_bf16_inputs_agree_on_values_both_formats_hold():
+    # values with <= 8 significant bits and small exponents are exact in both formats
+    rng = np.random.default_rng(0)
+    x = (rng.integers(-255, 256, size=(16, 128)) * 2.0 ** rng.integers(-6, 3, size=(16, 128))).astype(np.float32)
+    G = W.gen_factors(3)
+    a = co.quantize(W.f32_to_bf16_bits(x), G, x_dtype="bf16")
+    b = co.quantize(W.f32_to_fp16_bits(x), G, x_dtype="fp16")
+    for u, v in zip(a, b):
+        assert np.array_equal(u, v)
+
+
+def test_dense_blocks_equal_factor_path_when_the_product_is_exact_in_float():
+    # dyadic factor entries: every K entry is exactly representable in float32
+    rng = np.random.default_rng(5)
+    G = (rng.integers(-3, 4, size=(2, 5, 2, 2)) / 2.0).astype(np.float32)
+    for s in range(2):
+        for k in range(5):
+            if abs(np.linalg.det(G[s, k])) < 0.2:
+                G[s, k] = np.array([[1, 0.5], [-0.5, 1]], np.float32)
+    Kd = np.stack([kron_chain(G[s]) for s in range(2)]).astype(np.float32)
+    assert np.array_equal(Kd.astype(np.float64), np.stack([kron_chain(G[s]) for s in range(2)]))
+    Xb = W.gen_activations(W.ActivationSpec("d", 8, 64, seed=1, outlier_channels=2, outlier_gain=50.0))
+    assert np.array_equal(co.transform(Xb, G), co.transform(Xb, K_dense=Kd))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+def test_dense_transform_equals_library_matmul(dtype):
+    Kd = W.gen_dense_blocks(7, n_sets=3)
+    Xb = W.gen_activations(W.ActivationSpec("m", 24, 96, seed=7, outlier_channels=2, outlier_gain=50.0), dtype)
+    x = (W.fp16_bits_to_f32(Xb) if dtype == "fp16" else W.bf16_bits_to_f32(Xb)).astype(np.float64)
+    Y = co.transform(Xb, K_dense=Kd, x_dtype=dtype)
+    ref = np.einsum("tjr,jrc->tjc", x.reshape(24, 3, 32), Kd.astype(np.float64)).reshape(24, 96)
+    err = np.abs(Y.astype(np.float64) - ref)
+    assert (err <= np.spacing(np.abs(ref).astype(np.float32)).astype(np.float64)).all()
+    # shared dense block = the same block replicated
+    assert np.array_equal(co.transform(Xb, K_dense=Kd[:1]), co.transform(Xb, K_dense=np.repeat(Kd[:1], 3, 0)))
+    with pytest.raises(ValueError):
+        co.transform(Xb, K_dense=Kd[:2])
+
+
+def test_scale_and_plain_paths_with_fp16_input():
+    Xb = W.gen_activations(W.ActivationSpec("s", 8, 64, seed=2, outlier_channels=1, outlier_gain=50.0), "fp16")
+    x = W.fp16_bits_to_f32(Xb)
+    sv = W.gen_channel_scales(2, 64)
+    assert np.array_equal(co.widen(Xb, "fp16"), x)
+    assert np.array_equal(co.scale_transform(Xb, sv, "fp16"),
+                          (x.astype(np.float64) * sv.astype(np.float64)[None, :]).astype(np.float32))
