@@ -50,6 +50,9 @@ typedef enum {
 
 typedef enum { KQ_OUT_F32 = 0, KQ_OUT_BF16 = 1 } kq_dtype_t;
 
+/* Element type of the activations X.  The entry points without `_ex` take bf16. */
+typedef enum { KQ_X_BF16 = 0, KQ_X_FP16 = 1 } kq_xdtype_t;
+
 /* Which device code applies the transform in kroquant_quantize / kroquant_transform_f32.
  * KQ_PATH_AUTO picks the tensor-core kernel (tcgen05 + TMA) whenever it applies. */
 typedef enum { KQ_PATH_AUTO = 0, KQ_PATH_TENSOR = 1, KQ_PATH_ALU = 2 } kq_path_t;
@@ -59,7 +62,7 @@ typedef struct kroquant_factors kroquant_factors_t;
 
 /* Section 3.2 (Kronecker product construction).  Copies G_host (HOST,
  * [n_sets][5][2][2]) and uploads what the kernels need (the factors, their 2x2
- * inverses, and a 3-term bf16 image of every dense K).  Allocates device memory;
+ * inverses, and 3-term bf16 and fp16 images of every dense K).  Allocates device memory;
  * synchronizes the device once.  A factor with |det| < 1e-12 * ||G||_F^2 or a
  * non-finite entry gives KQ_ERR_FACTORS. */
 kq_status_t kroquant_factors_create(const float *G_host, int n_sets, kroquant_factors_t **out);
@@ -68,6 +71,14 @@ kq_status_t kroquant_factors_create(const float *G_host, int n_sets, kroquant_fa
  * holds (a_k, b_k, c_k);  G_k = [[1,0],[c,1]] * [[a,b],[0,-1/a]] = [[a, b],[a c, b c - 1/a]].
  * a == 0 gives KQ_ERR_FACTORS. */
 kq_status_t kroquant_factors_create_lu(const float *abc_host, int n_sets, kroquant_factors_t **out);
+
+/* Section 3.5, "K1 (precomputed dense)": the 32x32 blocks given directly, K_host (HOST,
+ * [n_sets][32][32] row-major K[r][c], y_c = sum_r x_r K[r][c]); they need not be Kronecker
+ * products.  Such a handle serves the tensor-core path of quantize / transform only:
+ * KQ_PATH_ALU and dequantize-with-factors return KQ_ERR_UNSUPPORTED (the blocks' inverses
+ * are not formed), kroquant_factors_get likewise.  A non-finite entry, or a block whose largest
+ * magnitude is 0 or outside [2^-100, 2^100], gives KQ_ERR_FACTORS. */
+kq_status_t kroquant_factors_create_dense(const float *K_host, int n_sets, kroquant_factors_t **out);
 
 /* Frees host and device storage.  NULL is allowed.  No kernel using it may be in flight. */
 void kroquant_factors_destroy(kroquant_factors_t *f);
@@ -85,6 +96,21 @@ kq_status_t kroquant_quantize(const void *X, int64_t tokens, int d, const kroqua
 kq_status_t kroquant_quantize_path(const void *X, int64_t tokens, int d,
                                    const kroquant_factors_t *f, uint8_t *q_packed,
                                    uint8_t *scales, kq_path_t path, void *stream);
+
+/* The same four operations for activations of either 16-bit type (Section 4.4: the paper's
+ * kernel benchmarks run on FP16 activations; Appendix D: PixArt-Sigma runs in FP16, SANA and
+ * FLUX.1 in BF16).  x_dtype outside the enum gives KQ_ERR_UNSUPPORTED. */
+kq_status_t kroquant_quantize_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                 const kroquant_factors_t *f, uint8_t *q_packed, uint8_t *scales,
+                                 kq_path_t path, void *stream);
+kq_status_t kroquant_transform_f32_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                      const kroquant_factors_t *f, float *Y, kq_path_t path,
+                                      void *stream);
+kq_status_t kroquant_scale_quantize_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                       const float *s, uint8_t *q_packed, uint8_t *scales,
+                                       void *stream);
+kq_status_t kroquant_mxfp4_quantize_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                       uint8_t *q_packed, uint8_t *scales, void *stream);
 
 /* Section 3.1 (quantize-then-DEquantize operator Q_b), decode half.
  * f == NULL: out = decoded transformed values  grid[code & 7] * sign * 2^(S-127)

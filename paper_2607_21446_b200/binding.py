@@ -20,7 +20,9 @@ LIB_PATH = os.path.join(_PKG, "libkroquant.so")
 KQ_OK = 0
 PATHS = {"auto": 0, "tensor": 1, "alu": 2}
 EXPORTS = [
-    "kroquant_factors_create", "kroquant_factors_create_lu", "kroquant_factors_destroy",
+    "kroquant_factors_create", "kroquant_factors_create_lu", "kroquant_factors_create_dense",
+    "kroquant_factors_destroy", "kroquant_quantize_ex", "kroquant_transform_f32_ex",
+    "kroquant_scale_quantize_ex", "kroquant_mxfp4_quantize_ex",
     "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize",
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
@@ -51,6 +53,11 @@ def load_library() -> C.CDLL:
     vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int
     L.kroquant_factors_create.argtypes = [vp, i32, C.POINTER(vp)]
     L.kroquant_factors_create_lu.argtypes = [vp, i32, C.POINTER(vp)]
+    L.kroquant_factors_create_dense.argtypes = [vp, i32, C.POINTER(vp)]
+    L.kroquant_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp]
+    L.kroquant_transform_f32_ex.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
+    L.kroquant_scale_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, vp]
+    L.kroquant_mxfp4_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp]
     L.kroquant_factors_destroy.argtypes = [vp]
     L.kroquant_factors_destroy.restype = None
     L.kroquant_factors_get.argtypes = [vp, vp]
@@ -91,9 +98,12 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+X_DTYPES = {torch.bfloat16: 0, torch.float16: 1}
+
+
 def _x_shape(X: torch.Tensor) -> tuple[int, int]:
-    if X.dim() != 2 or X.dtype != torch.bfloat16 or not X.is_cuda or not X.is_contiguous():
-        raise ValueError("X must be a contiguous 2-D CUDA bfloat16 tensor [tokens, d]")
+    if X.dim() != 2 or X.dtype not in X_DTYPES or not X.is_cuda or not X.is_contiguous():
+        raise ValueError("X must be a contiguous 2-D CUDA bfloat16 or float16 tensor [tokens, d]")
     return X.shape[0], X.shape[1]
 
 
@@ -124,6 +134,17 @@ class Factors:
                                                          C.byref(out)), "kroquant_factors_create_lu")
         return cls(out.value, abc.shape[0])
 
+    @classmethod
+    def create_dense(cls, K) -> "Factors":
+        """K: float32 [n_sets, 32, 32] dense blocks, y = x K per block."""
+        K = np.ascontiguousarray(K, dtype=np.float32)
+        if K.ndim != 3 or K.shape[1:] != (32, 32):
+            raise ValueError("K must have shape [n_sets, 32, 32]")
+        out = C.c_void_p()
+        _check(load_library().kroquant_factors_create_dense(K.ctypes.data_as(C.c_void_p), K.shape[0],
+                                                            C.byref(out)), "kroquant_factors_create_dense")
+        return cls(out.value, K.shape[0])
+
     def get(self) -> np.ndarray:
         G = np.empty((self.n_sets, 5, 2, 2), np.float32)
         _check(load_library().kroquant_factors_get(self._h, G.ctypes.data_as(C.c_void_p)),
@@ -150,8 +171,8 @@ def kroquant_quantize(X: torch.Tensor, factors: Factors, q_packed: Optional[torc
         q_packed = torch.empty((tokens, max(d // 2, 0)), dtype=torch.uint8, device=X.device)
     if scales is None:
         scales = torch.empty((tokens, max(d // 32, 0)), dtype=torch.uint8, device=X.device)
-    _check(load_library().kroquant_quantize_path(_ptr(X), tokens, d, factors._h, _ptr(q_packed),
-                                                 _ptr(scales), PATHS[path], C.c_void_p(_stream(stream))),
+    _check(load_library().kroquant_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(q_packed),
+                                               _ptr(scales), PATHS[path], C.c_void_p(_stream(stream))),
            "kroquant_quantize")
     return q_packed, scales
 
@@ -164,8 +185,8 @@ def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, sca
         q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
     if scales is None:
         scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
-    _check(load_library().kroquant_scale_quantize(_ptr(X), tokens, d, _ptr(s), _ptr(q_packed),
-                                                  _ptr(scales), C.c_void_p(_stream(stream))),
+    _check(load_library().kroquant_scale_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(s), _ptr(q_packed),
+                                                     _ptr(scales), C.c_void_p(_stream(stream))),
            "kroquant_scale_quantize")
     return q_packed, scales
 
@@ -176,8 +197,9 @@ def kroquant_mxfp4_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=
         q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
     if scales is None:
         scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
-    _check(load_library().kroquant_mxfp4_quantize(_ptr(X), tokens, d, _ptr(q_packed), _ptr(scales),
-                                                  C.c_void_p(_stream(stream))), "kroquant_mxfp4_quantize")
+    _check(load_library().kroquant_mxfp4_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(q_packed),
+                                                     _ptr(scales), C.c_void_p(_stream(stream))),
+           "kroquant_mxfp4_quantize")
     return q_packed, scales
 
 
@@ -185,8 +207,9 @@ def kroquant_transform_f32(X: torch.Tensor, factors: Factors, Y=None, path: str 
     tokens, d = _x_shape(X)
     if Y is None:
         Y = torch.empty((tokens, d), dtype=torch.float32, device=X.device)
-    _check(load_library().kroquant_transform_f32(_ptr(X), tokens, d, factors._h, _ptr(Y), PATHS[path],
-                                                 C.c_void_p(_stream(stream))), "kroquant_transform_f32")
+    _check(load_library().kroquant_transform_f32_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(Y),
+                                                    PATHS[path], C.c_void_p(_stream(stream))),
+           "kroquant_transform_f32")
     return Y
 
 

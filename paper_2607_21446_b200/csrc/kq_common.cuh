@@ -7,6 +7,7 @@
 //   v_c  = y_c * 2^(127 - S)                        (exact; |v_c| < 8)
 //   code = hardware float -> E2M1 convert (round-to-nearest-even, saturating at 6)
 #pragma once
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -23,6 +24,21 @@ __device__ __forceinline__ void widen8(const uint4& p, float (&x)[8]) {
     x[2] = bf16lo_to_f32(p.y); x[3] = bf16hi_to_f32(p.y);
     x[4] = bf16lo_to_f32(p.z); x[5] = bf16hi_to_f32(p.z);
     x[6] = bf16lo_to_f32(p.w); x[7] = bf16hi_to_f32(p.w);
+}
+
+// 8 fp16 (one 16-byte vector) -> 8 floats (exact), channel order preserved.
+__device__ __forceinline__ void widen8_f16(const uint4& p, float (&x)[8]) {
+    const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+    }
+}
+template <bool XF16>
+__device__ __forceinline__ void widen8_any(const uint4& p, float (&x)[8]) {
+    if (XF16) widen8_f16(p, x); else widen8(p, x);
 }
 
 // E8M0 byte from a block amax (amax >= 0, finite).

@@ -69,7 +69,7 @@ __device__ __forceinline__ uint32_t encode8(const float (&y)[8], float amax_bloc
 // latency-bandwidth product asks for).
 constexpr int kStreamUnroll = 4;
 
-template <int MODE, bool WRITE_Y>
+template <int MODE, bool WRITE_Y, bool XF16>
 __global__ void __launch_bounds__(256)
 quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row,
                 const FactorSet* __restrict__ factors, int n_sets,
@@ -102,7 +102,7 @@ quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row
             const int64_t q = q0 + u * stride;
             const bool live = q < n_quads;
             float y[8];
-            widen8(raw[u], y);
+            widen8_any<XF16>(raw[u], y);
             const int64_t blk = q >> 2;
             const int j = pos >> 2;                 // block column of this item
             pos += step;
@@ -149,6 +149,7 @@ quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row
 // per item.  Requires gridDim.x * blockDim.x >= d/8.  The four lanes of a quad always
 // work on the same row, so the amax shuffles use a per-quad mask (trip counts may differ
 // between quads of one warp).
+template <bool XF16>
 __global__ void __launch_bounds__(256)
 scale_quantize_rows(const uint4* __restrict__ X, int64_t tokens, int quads_per_row,
                     const float* __restrict__ chan_scale, uint32_t* __restrict__ q_packed,
@@ -177,7 +178,7 @@ scale_quantize_rows(const uint4* __restrict__ X, int64_t tokens, int quads_per_r
             const int64_t rr = r + u * R;
             if (rr >= tokens) break;                      // uniform inside the quad
             float y[8];
-            widen8(raw[u], y);
+            widen8_any<XF16>(raw[u], y);
             y[0] *= s0.x; y[1] *= s0.y; y[2] *= s0.z; y[3] *= s0.w;
             y[4] *= s1.x; y[5] *= s1.y; y[6] *= s1.z; y[7] *= s1.w;
             float amax = absmax8(y);

@@ -9,11 +9,16 @@
 // (Section 3.5: y = x K per block).  In this view the inputs, the 16-byte code
 // groups and the scale bytes of consecutive rows are all contiguous in HBM.
 //
-// Exactness.  X is bf16 and feeds the MMA unconverted.  K (a product of five floats,
-// formed in double on the host) is split into three bf16 terms K = K0 + K1 + K2
-// (8 + 8 + 8 significand bits), so every product x*K_t is exact in the fp32
-// accumulator and only the accumulation rounds.  The three terms are three
-// accumulating MMAs into the same TMEM tile.
+// Exactness.  X (bf16 or fp16) feeds the MMA unconverted.  K (a product of five floats
+// formed in double on the host, or a dense block given directly) is split into three
+// 16-bit terms of X's own format (kind::f16 wants equal operand formats), so every product
+// x*K_t is exact in the fp32 accumulator and only the accumulation rounds.  The three terms
+// are three accumulating MMA passes into the same TMEM tile.
+//   bf16: K = K0 + K1 + K2 exactly (8+8+8 significand bits, fp32's exponent range).
+//   fp16: K is first scaled by 2^e so that its largest entry lies in [1, 2) (fp16's
+//         exponent range is narrow), then split 11+11+11 bits; entries below 2^-14 of the
+//         largest keep an absolute precision of 2^-25.  The epilogue folds 2^-e into the
+//         scale byte, so the scaling costs nothing per element.
 //
 // One CTA = 1 TMA producer warp, 1 MMA warp (one elected thread issues), and
 // NG epilogue warpgroups of 4 warps; thread t of an epilogue warpgroup owns TMEM
@@ -139,9 +144,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr) {
     d |= (uint64_t)4 << 61;                 // SWIZZLE_64B
     return d;
 }
-// kind::f16 instruction descriptor: D=f32, A=B=bf16, both K-major, N=32, M=128.
-constexpr uint32_t kIdescBf16M128N32 =
-    (1u << 4) | (1u << 7) | (1u << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+// kind::f16 instruction descriptor: D=f32, A and B both bf16 (format code 1) or both fp16 (0),
+// both K-major, N=32, M=128.
+__host__ __device__ constexpr uint32_t idesc_m128n32(bool fp16) {
+    return (1u << 4) | ((fp16 ? 0u : 1u) << 7) | ((fp16 ? 0u : 1u) << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+}
 
 // TMA store of a 2-D box from shared memory (bulk async group of the issuing thread).
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, uint32_t src, int x, int y) {
@@ -182,8 +189,12 @@ struct UmmaSmem {
     static constexpr int kDynBytes = kBytes + 1024;                  // slack for manual alignment
 };
 
-// The fused epilogue math of one 32-channel block held in registers.
-__device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uint4& codes, uint32_t& S) {
+// The fused epilogue math of one 32-channel block held in registers.  acc = y * 2^e
+// (e = the factor image's normalisation exponent; 0 for bf16 images).
+// Common case: the true scale byte S = biased_exp(amax_acc) - 2 - e needs no clamping;
+// then v = acc * 2^(129 - biased_exp(amax_acc)) does not depend on e at all.  Otherwise
+// (block amax below 2^-125, or above fp32's range) the values are first brought back to y.
+__device__ __forceinline__ void encode_block_regs(uint32_t (&acc)[32], int e, uint4& codes, uint32_t& S) {
     float m[4] = {0.f, 0.f, 0.f, 0.f};      // four independent max chains
 #pragma unroll
     for (int c = 0; c < 32; c += 4) {
@@ -192,9 +203,21 @@ __device__ __forceinline__ void encode_block_regs(const uint32_t (&acc)[32], uin
         m[2] = fmaxf(m[2], fabsf(__uint_as_float(acc[c + 2])));
         m[3] = fmaxf(m[3], fabsf(__uint_as_float(acc[c + 3])));
     }
-    const float amax = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
-    S = e8m0_from_amax(amax);
-    const float inv = inv_scale_from_e8m0(S);
+    float amax = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+    const int ea = (int)((__float_as_uint(amax) >> 23) & 0xFFu);
+    const int s_raw = ea - 2 - e;
+    float inv;
+    if (ea >= 2 && s_raw >= 0 && s_raw <= 252) {
+        S = (uint32_t)s_raw;
+        inv = __uint_as_float((uint32_t)(256 - ea) << 23);          // 2^(129 - ea)
+    } else {
+        const float back = __uint_as_float((uint32_t)(127 - e) << 23);   // 2^-e, |e| <= 100
+#pragma unroll
+        for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * back);
+        amax *= back;
+        S = e8m0_from_amax(amax);
+        inv = inv_scale_from_e8m0(S);
+    }
     uint32_t w[4];
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
@@ -237,11 +260,13 @@ struct UmmaProblem {
 // and written the accumulator; frees the stage for the producer and hands the
 // accumulator to the epilogue) -> tempty (4 epilogue warps have read the accumulator).
 // Grid: any size <= number of tiles; CTA b takes tiles b, b + gridDim.x, ...
-template <int NS, int NM, int NG, bool PB, bool WRITE_Y>
+// XF16: X and the factor image are fp16 (else bf16); e_norm: per-set normalisation exponents of
+// the image (all zero for bf16 images).
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y>
 __global__ void __launch_bounds__(128 + 128 * NG, 1)
 quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
-              const uint8_t* __restrict__ b_image, const UmmaProblem prob, uint8_t* __restrict__ q_packed,
-              uint8_t* __restrict__ scales, float* __restrict__ Y) {
+              const uint8_t* __restrict__ b_image, const int* __restrict__ e_norm, const UmmaProblem prob,
+              uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y) {
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
     // A slot must always be served by the same issuer warp and the same epilogue group:
     // only then does program order inside that warp guarantee that a parity wait never
@@ -373,7 +398,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
 #pragma unroll
                     for (int kk = 0; kk < 2; ++kk) {
                         tc_mma_bf16(d_addr, a_desc + (uint64_t)(kk * 2), b_desc[t][kk] + (PB ? slot_off : 0),
-                                    kIdescBf16M128N32, (uint32_t)((t | kk) != 0));
+                                    idesc_m128n32(XF16), (uint32_t)((t | kk) != 0));
                     }
                 }
                 tc_commit(bar_done(s));
@@ -384,6 +409,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
+        const int e_shared = PB ? 0 : __ldg(e_norm);
         for (int n = g; n < my_tiles; n += NG) {
             const int s = n % NS;
             if (!mbar_wait(bar_done(s), (n / NS) & 1, abort_flag)) {
@@ -406,7 +432,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 const bool elected = threadIdx.x == 128;
                 uint4 codes;
                 uint32_t S;
-                encode_block_regs(acc, codes, S);
+                encode_block_regs(acc, __ldg(e_norm + (j < prob.blocks_per_row ? j : 0)), codes, S);
                 if (c == 0) {
                     // the previous group's TMA store must have finished reading the staging tile
                     if (elected) bulk_wait_group_read<0>();
@@ -453,16 +479,18 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     valid = row < prob.n_rows;
                 }
                 if (valid) {
+                    const int e = PB ? __ldg(e_norm + (int)(blk % prob.blocks_per_row)) : e_shared;
                     if (WRITE_Y) {
+                        const float back = __uint_as_float((uint32_t)(127 - e) << 23);    // 2^-e
                         float4* yp = reinterpret_cast<float4*>(Y + blk * 32);
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
-                            yp[i] = make_float4(__uint_as_float(acc[4 * i]), __uint_as_float(acc[4 * i + 1]),
-                                                __uint_as_float(acc[4 * i + 2]), __uint_as_float(acc[4 * i + 3]));
+                            yp[i] = make_float4(__uint_as_float(acc[4 * i]) * back, __uint_as_float(acc[4 * i + 1]) * back,
+                                                __uint_as_float(acc[4 * i + 2]) * back, __uint_as_float(acc[4 * i + 3]) * back);
                     } else {
                         uint4 codes;
                         uint32_t S;
-                        encode_block_regs(acc, codes, S);
+                        encode_block_regs(acc, e, codes, S);
                         st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
                         scales[blk] = (uint8_t)S;
                     }

@@ -20,10 +20,14 @@ struct kroquant_factors {
     int n_sets = 0;
     int device = -1;
     bool identity = false;
-    std::vector<float> G;             // host copy [n_sets][5][2][2]
-    kq::FactorSet* d_G = nullptr;     // device [n_sets]
-    kq::FactorSet* d_Ginv = nullptr;  // device [n_sets], 2x2 inverses
-    uint8_t* d_bimage = nullptr;      // device [n_sets][6 KB]: 3-term bf16 image of K^T, 64B-swizzled
+    bool dense = false;               // created from dense 32x32 blocks: tensor-core path only
+    std::vector<float> G;             // host copy [n_sets][5][2][2] (empty if dense)
+    kq::FactorSet* d_G = nullptr;     // device [n_sets] (null if dense)
+    kq::FactorSet* d_Ginv = nullptr;  // device [n_sets], 2x2 inverses (null if dense)
+    // device [2][n_sets][6 KB]: 3-term images of K^T in the 64B-swizzled operand layout,
+    // first all sets in bf16, then all sets in fp16 (normalised by 2^e_norm)
+    uint8_t* d_bimage = nullptr;
+    int* d_enorm = nullptr;           // device [2][n_sets]: normalisation exponents (bf16: all 0)
 };
 
 namespace {
@@ -81,48 +85,108 @@ int stream_grid(int64_t n_quads) {
     return (int)(want < cap ? want : cap);
 }
 
-// bf16 round-to-nearest-even of a double, returned as the bf16 bit pattern and its value
-uint16_t bf16_of(double v, double* back) {
-    float f = (float)v;
-    uint32_t u;
-    std::memcpy(&u, &f, 4);
-    u += 0x7FFFu + ((u >> 16) & 1u);
-    u &= 0xFFFF0000u;
-    float g;
-    std::memcpy(&g, &u, 4);
-    *back = (double)g;
-    return (uint16_t)(u >> 16);
+// round-to-nearest-even of a double to a 16-bit float format with `mant` explicit significand bits
+// and exponent bias `bias` (bf16: 7, 127; fp16: 10, 15); returns the bit pattern and the value it
+// stands for.  Magnitudes below the format's normal range become subnormals or zero; the callers
+// never pass values that overflow.
+uint16_t round_to_16bit(double v, int mant, int bias, double* back) {
+    *back = 0.0;
+    if (v == 0.0 || !std::isfinite(v)) return 0;
+    const uint16_t sign = v < 0 ? 0x8000u : 0u;
+    const double a = std::fabs(v);
+    int ex;
+    std::frexp(a, &ex);                       // a = m 2^ex, m in [0.5, 1)
+    int e = ex - 1;                           // a = 1.xxx 2^e
+    const int emin = 1 - bias;
+    if (e < emin) e = emin;                   // subnormal range: fixed quantum 2^(emin - mant)
+    const double ulp = std::ldexp(1.0, e - mant);
+    const double q = std::nearbyint(a / ulp); // ties to even (default rounding mode); a / ulp is exact
+    const double r = q * ulp;
+    *back = sign ? -r : r;
+    if (q == 0.0) return sign;
+    int e2;
+    std::frexp(r, &e2);
+    const int er = e2 - 1;                    // may be e + 1 after rounding up
+    uint32_t bits;
+    if (er < emin) {
+        bits = (uint32_t)q;                   // subnormal: the significand itself
+    } else {
+        const uint32_t frac = (uint32_t)std::llround(std::ldexp(r, mant - er)) - (1u << mant);
+        bits = ((uint32_t)(er + bias) << mant) | frac;
+    }
+    return (uint16_t)(sign | bits);
 }
 
-// K^T as three bf16 terms in the 64-byte-swizzled K-major operand layout the MMA reads:
+// Image of K^T as three 16-bit terms in the 64-byte-swizzled K-major operand layout the MMA reads:
 // element (n = c, k = r) of term t at byte  t*2048 + swz(c*64 + 2r),  swz(o) = o ^ (((o >> 7) & 3) << 4).
-void build_b_image(const float* G20, uint8_t* img) {
+// bf16: terms of K itself (e_norm = 0).  fp16: terms of K * 2^e_norm with the largest entry in [1, 2).
+// Returns false if the fp16 normalisation exponent would leave [-100, 100] (or K is all zero).
+bool build_b_image(const double* K /*[32][32] row-major K[r][c]*/, bool fp16, uint8_t* img, int* e_norm) {
     std::memset(img, 0, kq::kBImageBytes);
+    int e = 0;
+    if (fp16) {
+        double kmax = 0.0;
+        for (int i = 0; i < 1024; ++i) kmax = std::fmax(kmax, std::fabs(K[i]));
+        if (!(kmax > 0.0)) return false;
+        int ex;
+        std::frexp(kmax, &ex);                // kmax in [2^(ex-1), 2^ex)
+        e = 1 - ex;
+        if (e < -100 || e > 100) return false;
+    }
+    *e_norm = e;
     for (int r = 0; r < 32; ++r)
         for (int c = 0; c < 32; ++c) {
-            double k = 1.0;
-            for (int f = 0; f < 5; ++f) {
-                const int bit = 4 - f;
-                k *= (double)G20[f * 4 + ((r >> bit) & 1) * 2 + ((c >> bit) & 1)];
-            }
-            double rest = k;
+            double rest = std::ldexp(K[r * 32 + c], e);
             for (int t = 0; t < 3; ++t) {
                 double back;
-                const uint16_t b = bf16_of(rest, &back);
+                const uint16_t b = fp16 ? round_to_16bit(rest, 10, 15, &back) : round_to_16bit(rest, 7, 127, &back);
                 rest -= back;
                 uint32_t off = (uint32_t)(c * 64 + 2 * r);
                 off ^= ((off >> 7) & 3u) << 4;
                 std::memcpy(img + t * kq::kBTermBytes + off, &b, 2);
             }
         }
+    return true;
 }
 
-template <int NS, int NM, int NG, bool PB, bool WRITE_Y>
+// Shared tail of the factor constructors: K = n_sets dense blocks in double.
+kq_status_t finish_factors(kroquant_factors_t* f, const std::vector<double>& K,
+                           const std::vector<kq::FactorSet>* fwd, const std::vector<kq::FactorSet>* inv) {
+    const int n = f->n_sets;
+    std::vector<uint8_t> img((size_t)2 * n * kq::kBImageBytes);
+    std::vector<int> enorm((size_t)2 * n, 0);
+    for (int fmt = 0; fmt < 2; ++fmt)
+        for (int s = 0; s < n; ++s)
+            if (!build_b_image(K.data() + (size_t)s * 1024, fmt == 1,
+                               img.data() + ((size_t)fmt * n + s) * kq::kBImageBytes, &enorm[(size_t)fmt * n + s])) {
+                delete f;
+                return KQ_ERR_FACTORS;
+            }
+    bool ok = cudaGetDevice(&f->device) == cudaSuccess;
+    if (fwd) {
+        ok = ok && cudaMalloc(&f->d_G, sizeof(kq::FactorSet) * n) == cudaSuccess;
+        ok = ok && cudaMalloc(&f->d_Ginv, sizeof(kq::FactorSet) * n) == cudaSuccess;
+        ok = ok && cudaMemcpy(f->d_G, fwd->data(), sizeof(kq::FactorSet) * n, cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(f->d_Ginv, inv->data(), sizeof(kq::FactorSet) * n, cudaMemcpyHostToDevice) == cudaSuccess;
+    }
+    ok = ok && cudaMalloc(&f->d_bimage, img.size()) == cudaSuccess;
+    ok = ok && cudaMalloc(&f->d_enorm, sizeof(int) * enorm.size()) == cudaSuccess;
+    ok = ok && cudaMemcpy(f->d_bimage, img.data(), img.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(f->d_enorm, enorm.data(), sizeof(int) * enorm.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (!ok) {
+        (void)cudaGetLastError();
+        kroquant_factors_destroy(f);
+        return KQ_ERR_CUDA;
+    }
+    return KQ_OK;
+}
+
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y>
 kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
-                        const kq::UmmaProblem& prob,
+                        const int* enorm, const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, int ctas_per_sm, bool pdl, cudaStream_t st) {
     using L = kq::UmmaSmem<NS, PB>;
-    auto kern = kq::quantize_umma<NS, NM, NG, PB, WRITE_Y>;
+    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y>;
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, [&] {
@@ -146,7 +210,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, prob, q, scales, Y) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, enorm, prob, q, scales, Y) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -157,7 +221,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
 // Tensor-core path.  Shared factor set: flat [tokens*d/32][32] view of X.  Per-block
 // factor sets: 2-D view [tokens][d] with one 32-channel column per tile.
 template <bool WRITE_Y>
-kq_status_t run_umma(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, uint8_t* q,
+kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f, uint8_t* q,
                      uint8_t* scales, float* Y, cudaStream_t st) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
@@ -180,7 +244,8 @@ kq_status_t run_umma(const void* X, int64_t tokens, int d, const kroquant_factor
     }
     const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(X), dims, strides, box, estr,
+    if (enc(&tmap, xf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void*>(X), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
@@ -197,31 +262,36 @@ kq_status_t run_umma(const void* X, int64_t tokens, int d, const kroquant_factor
     }
     const int cps = g_umma_ctas_per_sm.load();
     const bool pdl = g_umma_pdl.load() != 0;
-    const uint8_t* b = f->d_bimage;
+    const uint8_t* b = f->d_bimage + (xf16 ? (size_t)f->n_sets * kq::kBImageBytes : 0);
+    const int* en = f->d_enorm + (xf16 ? f->n_sets : 0);
+#define KQ_LAUNCH(NS, NM, NG, PB, XF) \
+    launch_umma<NS, NM, NG, PB, XF, WRITE_Y>(tmap, tmap_q, b, en, prob, q, scales, Y, cps, pdl, st)
+    if (xf16) return pb ? KQ_LAUNCH(4, 1, 1, true, true) : KQ_LAUNCH(4, 2, 1, false, true);
     if (pb) {
         switch (g_umma_cfg.load()) {
             default:
-            case 4: return launch_umma<4, 1, 1, true, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-            case 0: return launch_umma<4, 2, 1, true, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-            case 1: return launch_umma<8, 2, 1, true, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+            case 4: return KQ_LAUNCH(4, 1, 1, true, false);
+            case 0: return KQ_LAUNCH(4, 2, 1, true, false);
+            case 1: return KQ_LAUNCH(8, 2, 1, true, false);
         }
     }
     switch (g_umma_cfg.load()) {
         default:
-        case 0: return launch_umma<2, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 1: return launch_umma<8, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 2: return launch_umma<8, 2, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 3: return launch_umma<2, 1, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 4: return launch_umma<4, 1, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 5: return launch_umma<4, 2, 1, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 6: return launch_umma<16, 2, 2, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
-        case 7: return launch_umma<16, 2, 4, false, WRITE_Y>(tmap, tmap_q, b, prob, q, scales, Y, cps, pdl, st);
+        case 0: return KQ_LAUNCH(2, 2, 1, false, false);
+        case 1: return KQ_LAUNCH(8, 2, 1, false, false);
+        case 2: return KQ_LAUNCH(8, 2, 2, false, false);
+        case 3: return KQ_LAUNCH(2, 1, 1, false, false);
+        case 4: return KQ_LAUNCH(4, 1, 1, false, false);
+        case 5: return KQ_LAUNCH(4, 2, 1, false, false);
+        case 6: return KQ_LAUNCH(16, 2, 2, false, false);
+        case 7: return KQ_LAUNCH(16, 2, 4, false, false);
     }
+#undef KQ_LAUNCH
 }
 
-template <int MODE, bool WRITE_Y>
-kq_status_t run_stream(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, const float* s,
-                       uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
+template <int MODE, bool WRITE_Y, bool XF16>
+kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, const float* s,
+                         uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
     const int64_t n_quads = tokens * (int64_t)(d / 8);
     const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
@@ -234,7 +304,7 @@ kq_status_t run_stream(const void* X, int64_t tokens, int d, const kroquant_fact
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kq::quantize_stream<MODE, WRITE_Y>, reinterpret_cast<const uint4*>(X), n_quads,
+    if (cudaLaunchKernelEx(&cfg, kq::quantize_stream<MODE, WRITE_Y, XF16>, reinterpret_cast<const uint4*>(X), n_quads,
                            d / 32, f ? (const kq::FactorSet*)f->d_G : (const kq::FactorSet*)nullptr,
                            f ? f->n_sets : 0, s, reinterpret_cast<uint32_t*>(q), scales, Y) != cudaSuccess) {
         (void)cudaGetLastError();
@@ -243,6 +313,15 @@ kq_status_t run_stream(const void* X, int64_t tokens, int d, const kroquant_fact
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return KQ_OK;
 }
+
+template <int MODE, bool WRITE_Y>
+kq_status_t run_stream(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f,
+                       const float* s, uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
+    return xf16 ? run_stream_t<MODE, WRITE_Y, true>(X, tokens, d, f, s, q, scales, Y, st)
+                : run_stream_t<MODE, WRITE_Y, false>(X, tokens, d, f, s, q, scales, Y, st);
+}
+
+bool valid_xdtype(kq_xdtype_t t) { return t == KQ_X_BF16 || t == KQ_X_FP16; }
 
 kq_status_t check_factors_for(const kroquant_factors_t* f, int d) {
     if (!f) return KQ_ERR_NULL;
@@ -260,7 +339,8 @@ kq_status_t kroquant_factors_create(const float* G_host, int n_sets, kroquant_fa
     if (n_sets <= 0) return KQ_ERR_FACTORS;
     bool identity = true;
     std::vector<kq::FactorSet> inv(n_sets), fwd(n_sets);
-    for (int s = 0; s < n_sets; ++s)
+    std::vector<double> K((size_t)n_sets * 1024);
+    for (int s = 0; s < n_sets; ++s) {
         for (int k = 0; k < 5; ++k) {
             const float* g = G_host + ((size_t)s * 5 + k) * 4;
             for (int i = 0; i < 4; ++i)
@@ -273,25 +353,25 @@ kq_status_t kroquant_factors_create(const float* G_host, int n_sets, kroquant_fa
             fwd[s].g[k] = make_float4(g[0], g[1], g[2], g[3]);
             inv[s].g[k] = make_float4((float)(e / det), (float)(-b / det), (float)(-c / det), (float)(a / det));
         }
+        // K[r][c] = prod_k G_k[bit_{5-k}(r)][bit_{5-k}(c)], in double
+        const float* G20 = G_host + (size_t)s * 20;
+        for (int r = 0; r < 32; ++r)
+            for (int c = 0; c < 32; ++c) {
+                double v = 1.0;
+                for (int k = 0; k < 5; ++k) {
+                    const int bit = 4 - k;
+                    v *= (double)G20[k * 4 + ((r >> bit) & 1) * 2 + ((c >> bit) & 1)];
+                }
+                K[(size_t)s * 1024 + r * 32 + c] = v;
+            }
+    }
     kroquant_factors_t* f = new (std::nothrow) kroquant_factors_t;
     if (!f) return KQ_ERR_CUDA;
     f->n_sets = n_sets;
     f->identity = identity;
     f->G.assign(G_host, G_host + (size_t)n_sets * 20);
-    std::vector<uint8_t> img((size_t)n_sets * kq::kBImageBytes);
-    for (int s = 0; s < n_sets; ++s) build_b_image(G_host + (size_t)s * 20, img.data() + (size_t)s * kq::kBImageBytes);
-    bool ok = cudaGetDevice(&f->device) == cudaSuccess;
-    ok = ok && cudaMalloc(&f->d_G, sizeof(kq::FactorSet) * n_sets) == cudaSuccess;
-    ok = ok && cudaMalloc(&f->d_Ginv, sizeof(kq::FactorSet) * n_sets) == cudaSuccess;
-    ok = ok && cudaMalloc(&f->d_bimage, img.size()) == cudaSuccess;
-    ok = ok && cudaMemcpy(f->d_G, fwd.data(), sizeof(kq::FactorSet) * n_sets, cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemcpy(f->d_Ginv, inv.data(), sizeof(kq::FactorSet) * n_sets, cudaMemcpyHostToDevice) == cudaSuccess;
-    ok = ok && cudaMemcpy(f->d_bimage, img.data(), img.size(), cudaMemcpyHostToDevice) == cudaSuccess;
-    if (!ok) {
-        (void)cudaGetLastError();
-        kroquant_factors_destroy(f);
-        return KQ_ERR_CUDA;
-    }
+    const kq_status_t rc = finish_factors(f, K, &fwd, &inv);
+    if (rc != KQ_OK) return rc;
     *out = f;
     return KQ_OK;
 }
@@ -312,24 +392,50 @@ kq_status_t kroquant_factors_create_lu(const float* abc_host, int n_sets, kroqua
     return kroquant_factors_create(G.data(), n_sets, out);
 }
 
+kq_status_t kroquant_factors_create_dense(const float* K_host, int n_sets, kroquant_factors_t** out) {
+    if (!K_host || !out) return KQ_ERR_NULL;
+    *out = nullptr;
+    if (n_sets <= 0) return KQ_ERR_FACTORS;
+    std::vector<double> K((size_t)n_sets * 1024);
+    bool identity = true;
+    for (size_t i = 0; i < K.size(); ++i) {
+        if (!std::isfinite(K_host[i])) return KQ_ERR_FACTORS;
+        K[i] = (double)K_host[i];
+        const size_t rc = i % 1024;
+        if (K_host[i] != ((rc / 32 == rc % 32) ? 1.f : 0.f)) identity = false;
+    }
+    kroquant_factors_t* f = new (std::nothrow) kroquant_factors_t;
+    if (!f) return KQ_ERR_CUDA;
+    f->n_sets = n_sets;
+    f->identity = identity;
+    f->dense = true;
+    const kq_status_t rc = finish_factors(f, K, nullptr, nullptr);
+    if (rc != KQ_OK) return rc;
+    *out = f;
+    return KQ_OK;
+}
+
 void kroquant_factors_destroy(kroquant_factors_t* f) {
     if (!f) return;
     if (f->d_G) cudaFree(f->d_G);
     if (f->d_Ginv) cudaFree(f->d_Ginv);
     if (f->d_bimage) cudaFree(f->d_bimage);
+    if (f->d_enorm) cudaFree(f->d_enorm);
     delete f;
 }
 
 kq_status_t kroquant_factors_get(const kroquant_factors_t* f, float* G_host_out) {
     if (!f || !G_host_out) return KQ_ERR_NULL;
+    if (f->dense) return KQ_ERR_UNSUPPORTED;
     std::memcpy(G_host_out, f->G.data(), f->G.size() * sizeof(float));
     return KQ_OK;
 }
 
 int kroquant_factors_n_sets(const kroquant_factors_t* f) { return f ? f->n_sets : 0; }
 
-kq_status_t kroquant_quantize_path(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
-                                   uint8_t* q_packed, uint8_t* scales, kq_path_t path, void* stream) {
+kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                 const kroquant_factors_t* f, uint8_t* q_packed, uint8_t* scales,
+                                 kq_path_t path, void* stream) {
     if (!X || !q_packed || !scales) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
@@ -337,22 +443,30 @@ kq_status_t kroquant_quantize_path(const void* X, int64_t tokens, int d, const k
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
     if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
+    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
+    if (path == KQ_PATH_ALU && f->dense) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool xf16 = x_dtype == KQ_X_FP16;
     if (path == KQ_PATH_AUTO && f->identity)
-        return run_stream<kq::MODE_PLAIN, false>(X, tokens, d, nullptr, nullptr, q_packed, scales, nullptr, st);
+        return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, nullptr, st);
     if (path != KQ_PATH_ALU)
-        return run_umma<false>(X, tokens, d, f, q_packed, scales, nullptr, st);
-    return run_stream<kq::MODE_KRON, false>(X, tokens, d, f, nullptr, q_packed, scales, nullptr, st);
+        return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, nullptr, st);
+    return run_stream<kq::MODE_KRON, false>(X, xf16, tokens, d, f, nullptr, q_packed, scales, nullptr, st);
+}
+
+kq_status_t kroquant_quantize_path(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
+                                   uint8_t* q_packed, uint8_t* scales, kq_path_t path, void* stream) {
+    return kroquant_quantize_ex(X, KQ_X_BF16, tokens, d, f, q_packed, scales, path, stream);
 }
 
 kq_status_t kroquant_quantize(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
                               uint8_t* q_packed, uint8_t* scales, void* stream) {
-    return kroquant_quantize_path(X, tokens, d, f, q_packed, scales, KQ_PATH_AUTO, stream);
+    return kroquant_quantize_ex(X, KQ_X_BF16, tokens, d, f, q_packed, scales, KQ_PATH_AUTO, stream);
 }
 
-kq_status_t kroquant_transform_f32(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
-                                   float* Y, kq_path_t path, void* stream) {
+kq_status_t kroquant_transform_f32_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                      const kroquant_factors_t* f, float* Y, kq_path_t path, void* stream) {
     if (!X || !Y) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
@@ -360,28 +474,38 @@ kq_status_t kroquant_transform_f32(const void* X, int64_t tokens, int d, const k
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(Y)) return KQ_ERR_ALIGN;
     if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
+    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
+    if (path == KQ_PATH_ALU && f->dense) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool xf16 = x_dtype == KQ_X_FP16;
     if (path == KQ_PATH_AUTO && f->identity)
-        return run_stream<kq::MODE_PLAIN, true>(X, tokens, d, nullptr, nullptr, nullptr, nullptr, Y, st);
+        return run_stream<kq::MODE_PLAIN, true>(X, xf16, tokens, d, nullptr, nullptr, nullptr, nullptr, Y, st);
     if (path != KQ_PATH_ALU)
-        return run_umma<true>(X, tokens, d, f, nullptr, nullptr, Y, st);
-    return run_stream<kq::MODE_KRON, true>(X, tokens, d, f, nullptr, nullptr, nullptr, Y, st);
+        return run_umma<true>(X, xf16, tokens, d, f, nullptr, nullptr, Y, st);
+    return run_stream<kq::MODE_KRON, true>(X, xf16, tokens, d, f, nullptr, nullptr, nullptr, Y, st);
 }
 
-kq_status_t kroquant_scale_quantize(const void* X, int64_t tokens, int d, const float* s, uint8_t* q_packed,
-                                    uint8_t* scales, void* stream) {
+kq_status_t kroquant_transform_f32(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
+                                   float* Y, kq_path_t path, void* stream) {
+    return kroquant_transform_f32_ex(X, KQ_X_BF16, tokens, d, f, Y, path, stream);
+}
+
+kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const float* s,
+                                       uint8_t* q_packed, uint8_t* scales, void* stream) {
     if (!X || !s || !q_packed || !scales) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed) || !aligned16(s)) return KQ_ERR_ALIGN;
+    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool xf16 = x_dtype == KQ_X_FP16;
     const int64_t n_quads = tokens * (int64_t)(d / 8);
     const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
     if ((int64_t)grid * 256 < d / 8)      // fewer threads than quad columns: generic kernel
-        return run_stream<kq::MODE_SCALE, false>(X, tokens, d, nullptr, s, q_packed, scales, nullptr, st);
+        return run_stream<kq::MODE_SCALE, false>(X, xf16, tokens, d, nullptr, s, q_packed, scales, nullptr, st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(256);
@@ -391,8 +515,12 @@ kq_status_t kroquant_scale_quantize(const void* X, int64_t tokens, int d, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows, reinterpret_cast<const uint4*>(X), tokens, d / 8, s,
-                           reinterpret_cast<uint32_t*>(q_packed), scales) != cudaSuccess) {
+    const cudaError_t err =
+        xf16 ? cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<true>, reinterpret_cast<const uint4*>(X), tokens,
+                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales)
+             : cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<false>, reinterpret_cast<const uint4*>(X), tokens,
+                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales);
+    if (err != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -400,15 +528,26 @@ kq_status_t kroquant_scale_quantize(const void* X, int64_t tokens, int d, const 
     return KQ_OK;
 }
 
-kq_status_t kroquant_mxfp4_quantize(const void* X, int64_t tokens, int d, uint8_t* q_packed, uint8_t* scales,
-                                    void* stream) {
+kq_status_t kroquant_scale_quantize(const void* X, int64_t tokens, int d, const float* s, uint8_t* q_packed,
+                                    uint8_t* scales, void* stream) {
+    return kroquant_scale_quantize_ex(X, KQ_X_BF16, tokens, d, s, q_packed, scales, stream);
+}
+
+kq_status_t kroquant_mxfp4_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                       uint8_t* q_packed, uint8_t* scales, void* stream) {
     if (!X || !q_packed || !scales) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
+    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
-    return run_stream<kq::MODE_PLAIN, false>(X, tokens, d, nullptr, nullptr, q_packed, scales, nullptr,
-                                             static_cast<cudaStream_t>(stream));
+    return run_stream<kq::MODE_PLAIN, false>(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, nullptr, q_packed, scales,
+                                             nullptr, static_cast<cudaStream_t>(stream));
+}
+
+kq_status_t kroquant_mxfp4_quantize(const void* X, int64_t tokens, int d, uint8_t* q_packed, uint8_t* scales,
+                                    void* stream) {
+    return kroquant_mxfp4_quantize_ex(X, KQ_X_BF16, tokens, d, q_packed, scales, stream);
 }
 
 kq_status_t kroquant_dequantize(const uint8_t* q_packed, const uint8_t* scales, int64_t tokens, int d,
@@ -417,6 +556,7 @@ kq_status_t kroquant_dequantize(const uint8_t* q_packed, const uint8_t* scales, 
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
     if (f && f->n_sets != 1 && f->n_sets != d / 32) return KQ_ERR_FACTORS;
+    if (f && f->dense && !f->identity) return KQ_ERR_UNSUPPORTED;   // no dense inverse on the device
     if (!aligned16(q_packed) || !aligned16(out)) return KQ_ERR_ALIGN;
     if (out_dtype != KQ_OUT_F32 && out_dtype != KQ_OUT_BF16) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
