@@ -43,7 +43,7 @@ typedef enum {
     KQ_ERR_NULL = 1,         /* a required pointer is NULL */
     KQ_ERR_SHAPE = 2,        /* d <= 0, d % 32 != 0, tokens < 0, tokens*d/32 >= 2^31 */
     KQ_ERR_ALIGN = 3,        /* a device pointer is not 16-byte aligned */
-    KQ_ERR_FACTORS = 4,      /* n_sets not in {1, d/32}, non-finite or singular factor */
+    KQ_ERR_FACTORS = 4,      /* n_sets not in {1, d/32}, non-finite or singular factor, handle of another device */
     KQ_ERR_UNSUPPORTED = 5,  /* unknown enum value */
     KQ_ERR_CUDA = 6          /* a CUDA call or launch failed (no device, bad pointer kind, ...) */
 } kq_status_t;

@@ -326,6 +326,9 @@ bool valid_xdtype(kq_xdtype_t t) { return t == KQ_X_BF16 || t == KQ_X_FP16; }
 kq_status_t check_factors_for(const kroquant_factors_t* f, int d) {
     if (!f) return KQ_ERR_NULL;
     if (f->n_sets != 1 && f->n_sets != d / 32) return KQ_ERR_FACTORS;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return KQ_ERR_CUDA; }
+    if (dev != f->device) return KQ_ERR_FACTORS;     // the handle's images live on another device
     return KQ_OK;
 }
 
@@ -555,8 +558,11 @@ kq_status_t kroquant_dequantize(const uint8_t* q_packed, const uint8_t* scales, 
     if (!q_packed || !scales || !out) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
-    if (f && f->n_sets != 1 && f->n_sets != d / 32) return KQ_ERR_FACTORS;
-    if (f && f->dense && !f->identity) return KQ_ERR_UNSUPPORTED;   // no dense inverse on the device
+    if (f) {
+        const kq_status_t frc = check_factors_for(f, d);
+        if (frc != KQ_OK) return frc;
+        if (f->dense && !f->identity) return KQ_ERR_UNSUPPORTED;   // no dense inverse on the device
+    }
     if (!aligned16(q_packed) || !aligned16(out)) return KQ_ERR_ALIGN;
     if (out_dtype != KQ_OUT_F32 && out_dtype != KQ_OUT_BF16) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
