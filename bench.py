@@ -491,8 +491,61 @@ def run_sweep(args):
             del Xs, x0, q, sc
 
 
+# The paper's two latency tables (Section 4.4 and Appendix A): (m, d) and its MI350 / FP16 numbers in
+# microseconds for Q4, Scale, K1, K2 -- context only, another machine.
+PAPER_TABLES = {
+    "power_of_two_d": [((4096, 1024), (9.40, 10.56, 9.96, 14.00)), ((4096, 4096), (22.64, 25.52, 23.88, 27.80)),
+                       ((4096, 16384), (74.44, 75.44, 75.32, 78.52)), ((512, 4096), (7.20, 9.24, 8.12, 10.28)),
+                       ((512, 16384), (13.68, 16.36, 15.36, 19.32))],
+    "production_shapes": [((512, 3072), (6.72, 9.04, 7.64, 8.84)), ((512, 12288), (11.80, 14.68, 13.08, 17.00)),
+                          ((4096, 1152), (10.64, 14.00, 10.68, 14.64)), ((4096, 3072), (18.56, 21.12, 19.28, 23.32)),
+                          ((4096, 3456), (20.60, 24.20, 21.32, 25.36)), ((4096, 4096), (22.08, 25.80, 23.36, 27.28)),
+                          ((4096, 4608), (25.72, 28.40, 26.40, 30.36)), ((4096, 12288), (59.64, 59.12, 59.92, 62.80))],
+}
+
+
+def run_table(args):
+    """The paper's latency tables re-measured on this GPU with FP16 activations: Q4 (bare MXFP4),
+    Scale, K1 (dense 32x32 block handle) and K2 (five-factor handle; here both handles run the same
+    tensor-core kernel on a precomputed operand image).  Back-to-back calls in a CUDA graph over
+    rotating inputs (> 3 x L2).  One JSON line per shape."""
+    import torch
+    from paper_2607_21446_b200 import binding as B
+    B.load_library()
+    stream = torch.cuda.Stream()
+    for table, rows in PAPER_TABLES.items():
+        for (m, d), paper in rows:
+            nbuf = min(28, max(3, int(400e6 // (m * d * 2)) + 1))
+            sp = W.ActivationSpec("table", m, d, seed=4, outlier_channels=max(1, d // 100), outlier_gain=50.0)
+            x0 = torch.from_numpy(W.gen_activations(sp, "fp16").view(np.int16)).cuda().view(torch.float16)
+            Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, nbuf)]
+            q = torch.empty((m, d // 2), dtype=torch.uint8, device="cuda")
+            sc = torch.empty((m, d // 32), dtype=torch.uint8, device="cuda")
+            G = W.gen_factors(4)
+            K = G[0, 0].astype(np.float64)
+            for k in range(1, 5):
+                K = np.kron(K, G[0, k].astype(np.float64))          # input recipe of the dense handle
+            f2, f1 = B.Factors.create(G), B.Factors.create_dense(K.astype(np.float32)[None])
+            sv = torch.from_numpy(W.gen_channel_scales(4, d)).cuda()
+            us = {}
+            for name, fn in (("Q4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)),
+                             ("Scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
+                             ("K1", lambda x: B.kroquant_quantize(x, f1, q, sc, stream=stream)),
+                             ("K2", lambda x: B.kroquant_quantize(x, f2, q, sc, stream=stream))):
+                g = capture(torch, [lambda x=x, fn=fn: fn(x) for x in Xs], stream)
+                ms, _ = time_graph(torch, None, g, stream, max(5, args.steps // 10), 3)
+                us[name] = round(ms * 1e3 / nbuf, 2)
+            print(json.dumps({"table": table, "m": m, "d": d, "dtype": "fp16", "us_b200": us,
+                              "scale_over_k1": round(us["Scale"] / us["K1"], 3),
+                              "scale_over_k2": round(us["Scale"] / us["K2"], 3),
+                              "paper_mi350_us": dict(zip(("Q4", "Scale", "K1", "K2"), paper))}), flush=True)
+            del Xs, x0
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--table", action="store_true",
+                    help="the paper's two latency tables (Q4 / Scale / K1 / K2, FP16) on this GPU")
     ap.add_argument("--sweep", action="store_true",
                     help="tokens x d sweep of KroQuant / Scale / bare MXFP4 (one JSON line per point)")
     ap.add_argument("--single", default=None, metavar="TOKENSxD",
@@ -506,7 +559,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.sweep:
+    if args.table:
+        run_table(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.single:
         run_single(args)

@@ -37,6 +37,12 @@ def lib() -> C.CDLL:
         L.kq_oracle_quantize.argtypes = [vp, i64, i32, vp, i32, vp, vp, vp]
         L.kq_oracle_scale_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.kq_oracle_dequantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, i32]
+        L.kq_oracle_tiled_scale_size.argtypes = [i64, i32]
+        L.kq_oracle_tiled_scale_size.restype = i64
+        L.kq_oracle_tiled_scale_index.argtypes = [i64, i32, i32]
+        L.kq_oracle_tiled_scale_index.restype = i64
+        L.kq_oracle_scales_to_tiled.argtypes = [vp, i64, i32, C.c_uint8, vp]
+        L.kq_oracle_scales_to_tiled.restype = None
         _lib = L
     return _lib
 
@@ -173,4 +179,17 @@ def dequantize(q, scales, G=None, out_bf16: bool = False) -> np.ndarray:
         G = _g(G)
         gp, ns = _p(G), G.shape[0]
     _check(lib().kq_oracle_dequantize(_p(q), _p(scales), t, d, gp, ns, _p(out), int(out_bf16)))
+    return out
+
+
+def tiled_scale_index(r: int, j: int, k_blocks: int) -> int:
+    return int(lib().kq_oracle_tiled_scale_index(r, j, k_blocks))
+
+
+def scales_to_tiled(scales, fill: int = 0) -> np.ndarray:
+    """Row-major scale bytes [rows, k_blocks] -> the 128 x 4 tiled layout block-scaled GEMMs read."""
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    rows, kb = scales.shape
+    out = np.empty(int(lib().kq_oracle_tiled_scale_size(rows, kb)), np.uint8)
+    lib().kq_oracle_scales_to_tiled(_p(scales), rows, kb, fill, _p(out))
     return out

@@ -341,3 +341,30 @@ int kq_oracle_dequantize(const uint8_t *q, const uint8_t *scales, int64_t tokens
     }
     return 0;
 }
+
+/* ---- scale-byte layout for block-scaled tensor-core GEMM consumers ------------------------ */
+/* The W4A4 product of the paper's inference formula (Section 3.4) is a block-scaled MXFP4 GEMM.
+ * Such GEMMs read the E8M0 bytes of an operand [rows][k_blocks] in tiles of 128 rows x 4 k-blocks
+ * (512 bytes each), tiles ordered row-tile-major; inside a tile the byte of (row r, k-block j) sits
+ * at  (r mod 32)*16 + ((r mod 128) div 32)*4 + (j mod 4).  Rows are padded to a multiple of 128 and
+ * k-blocks to a multiple of 4; padding bytes are `fill`.  out must hold
+ * ceil(rows/128)*128 * ceil(k_blocks/4)*4 bytes. */
+int64_t kq_oracle_tiled_scale_size(int64_t rows, int k_blocks)
+{
+    return ((rows + 127) / 128) * 128 * (int64_t)(((k_blocks + 3) / 4) * 4);
+}
+
+int64_t kq_oracle_tiled_scale_index(int64_t r, int j, int k_blocks)
+{
+    int64_t cb = (k_blocks + 3) / 4;
+    return ((r / 128) * cb + j / 4) * 512 + (r % 32) * 16 + ((r % 128) / 32) * 4 + (j % 4);
+}
+
+void kq_oracle_scales_to_tiled(const uint8_t *scales, int64_t rows, int k_blocks, uint8_t fill, uint8_t *out)
+{
+    int64_t n = kq_oracle_tiled_scale_size(rows, k_blocks);
+    for (int64_t i = 0; i < n; ++i) out[i] = fill;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int j = 0; j < k_blocks; ++j)
+            out[kq_oracle_tiled_scale_index(r, j, k_blocks)] = scales[r * k_blocks + j];
+}

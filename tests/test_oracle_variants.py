@@ -70,3 +70,38 @@ def test_scale_and_plain_paths_with_fp16_input():
     assert np.array_equal(co.widen(Xb, "fp16"), x)
     assert np.array_equal(co.scale_transform(Xb, sv, "fp16"),
                           (x.astype(np.float64) * sv.astype(np.float64)[None, :]).astype(np.float32))
+
+
+# ---- tiled scale layout for block-scaled GEMM consumers --------------------------------------
+def test_tiled_scale_layout_hand_indices():
+    # 128 x 4 tiles of 512 bytes; inside a tile: (r % 32) * 16 + (r % 128 // 32) * 4 + j % 4
+    kb = 9                                    # 3 column tiles per row tile
+    assert co.tiled_scale_index(0, 0, kb) == 0
+    assert co.tiled_scale_index(0, 1, kb) == 1
+    assert co.tiled_scale_index(0, 3, kb) == 3
+    assert co.tiled_scale_index(0, 4, kb) == 512             # next column tile
+    assert co.tiled_scale_index(1, 0, kb) == 16
+    assert co.tiled_scale_index(31, 0, kb) == 31 * 16
+    assert co.tiled_scale_index(32, 0, kb) == 4               # second 32-row quarter
+    assert co.tiled_scale_index(96, 2, kb) == 12 + 2
+    assert co.tiled_scale_index(127, 3, kb) == 31 * 16 + 12 + 3 == 511
+    assert co.tiled_scale_index(128, 0, kb) == 3 * 512        # next row tile
+    assert co.tiled_scale_index(130, 8, kb) == 3 * 512 + 2 * 512 + 2 * 16
+
+
+@pytest.mark.parametrize("rows,kb", [(1, 1), (128, 4), (130, 9), (257, 36), (300, 175)])
+def test_tiled_scale_layout_equals_reshape_permute(rows, kb):
+    """Independent statement with library reshapes: pad to [R*128, C*4], split into tiles
+    [R, C, 128, 4], split the 128 rows into [4, 32] and store each tile as [32, 4, 4]."""
+    rng = np.random.default_rng(rows + kb)
+    s = rng.integers(1, 255, size=(rows, kb), dtype=np.uint8)
+    got = co.scales_to_tiled(s, fill=0)
+    R, Cb = (rows + 127) // 128, (kb + 3) // 4
+    p = np.zeros((R * 128, Cb * 4), np.uint8)
+    p[:rows, :kb] = s
+    t = p.reshape(R, 128, Cb, 4).transpose(0, 2, 1, 3)          # [R, C, 128, 4]
+    t = t.reshape(R, Cb, 4, 32, 4).transpose(0, 1, 3, 2, 4)      # [R, C, 32, 4, 4]
+    assert np.array_equal(got, t.reshape(-1))
+    # a bijection on the real entries: every (r, j) lands on a distinct byte
+    idx = {co.tiled_scale_index(r, j, kb) for r in range(min(rows, 140)) for j in range(kb)}
+    assert len(idx) == min(rows, 140) * kb
