@@ -53,6 +53,14 @@ typedef enum { KQ_OUT_F32 = 0, KQ_OUT_BF16 = 1 } kq_dtype_t;
 /* Element type of the activations X.  The entry points without `_ex` take bf16. */
 typedef enum { KQ_X_BF16 = 0, KQ_X_FP16 = 1 } kq_xdtype_t;
 
+/* Where the E8M0 bytes go.  ROWMAJOR: scales[tokens][d/32].  TILED_128X4: the layout block-scaled
+ * tensor-core GEMMs read (the consumer of the paper's W4A4 product, Section 3.4): tiles of 128 rows x
+ * 4 blocks = 512 bytes, row-tile-major; byte of (t, j) at
+ *   ((t/128) * ceil(d/128) + j/4) * 512 + (t%32)*16 + ((t%128)/32)*4 + j%4.
+ * The buffer then holds ceil(tokens/128)*128 * ceil(d/128)*4 bytes; padding bytes are not written.
+ * kroquant_dequantize reads ROWMAJOR only. */
+typedef enum { KQ_SCALES_ROWMAJOR = 0, KQ_SCALES_TILED_128X4 = 1 } kq_scale_layout_t;
+
 /* Which device code applies the transform in kroquant_quantize / kroquant_transform_f32.
  * KQ_PATH_AUTO picks the tensor-core kernel (tcgen05 + TMA) whenever it applies. */
 typedef enum { KQ_PATH_AUTO = 0, KQ_PATH_TENSOR = 1, KQ_PATH_ALU = 2 } kq_path_t;
@@ -97,20 +105,21 @@ kq_status_t kroquant_quantize_path(const void *X, int64_t tokens, int d,
                                    const kroquant_factors_t *f, uint8_t *q_packed,
                                    uint8_t *scales, kq_path_t path, void *stream);
 
-/* The same four operations for activations of either 16-bit type (Section 4.4: the paper's
+/* The same four operations for activations of either 16-bit type and either scale layout (Section 4.4: the paper's
  * kernel benchmarks run on FP16 activations; Appendix D: PixArt-Sigma runs in FP16, SANA and
  * FLUX.1 in BF16).  x_dtype outside the enum gives KQ_ERR_UNSUPPORTED. */
 kq_status_t kroquant_quantize_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
                                  const kroquant_factors_t *f, uint8_t *q_packed, uint8_t *scales,
-                                 kq_path_t path, void *stream);
+                                 kq_scale_layout_t scale_layout, kq_path_t path, void *stream);
 kq_status_t kroquant_transform_f32_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
                                       const kroquant_factors_t *f, float *Y, kq_path_t path,
                                       void *stream);
 kq_status_t kroquant_scale_quantize_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
                                        const float *s, uint8_t *q_packed, uint8_t *scales,
-                                       void *stream);
+                                       kq_scale_layout_t scale_layout, void *stream);
 kq_status_t kroquant_mxfp4_quantize_ex(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
-                                       uint8_t *q_packed, uint8_t *scales, void *stream);
+                                       uint8_t *q_packed, uint8_t *scales,
+                                       kq_scale_layout_t scale_layout, void *stream);
 
 /* Section 3.1 (quantize-then-DEquantize operator Q_b), decode half.
  * f == NULL: out = decoded transformed values  grid[code & 7] * sign * 2^(S-127)

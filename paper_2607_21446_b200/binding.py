@@ -54,10 +54,10 @@ def load_library() -> C.CDLL:
     L.kroquant_factors_create.argtypes = [vp, i32, C.POINTER(vp)]
     L.kroquant_factors_create_lu.argtypes = [vp, i32, C.POINTER(vp)]
     L.kroquant_factors_create_dense.argtypes = [vp, i32, C.POINTER(vp)]
-    L.kroquant_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp]
+    L.kroquant_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, i32, vp]
     L.kroquant_transform_f32_ex.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
-    L.kroquant_scale_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, vp]
-    L.kroquant_mxfp4_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp]
+    L.kroquant_scale_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp]
+    L.kroquant_mxfp4_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
     L.kroquant_factors_destroy.argtypes = [vp]
     L.kroquant_factors_destroy.restype = None
     L.kroquant_factors_get.argtypes = [vp, vp]
@@ -99,6 +99,18 @@ def _ptr(t: Optional[torch.Tensor]):
 
 
 X_DTYPES = {torch.bfloat16: 0, torch.float16: 1}
+SCALE_LAYOUTS = {"rowmajor": 0, "tiled": 1}
+
+
+def tiled_scale_bytes(tokens: int, d: int) -> int:
+    """Size of the scale buffer in the 128 x 4 tiled layout."""
+    return ((tokens + 127) // 128) * 128 * (((d // 32) + 3) // 4) * 4
+
+
+def _scale_buffer(tokens: int, d: int, layout: str, device) -> torch.Tensor:
+    if layout == "tiled":      # padding bytes are never written by the kernels: start from zeros
+        return torch.zeros(tiled_scale_bytes(tokens, d), dtype=torch.uint8, device=device)
+    return torch.empty((tokens, max(d // 32, 0)), dtype=torch.uint8, device=device)
 
 
 def _x_shape(X: torch.Tensor) -> tuple[int, int]:
@@ -164,41 +176,48 @@ class Factors:
 
 
 def kroquant_quantize(X: torch.Tensor, factors: Factors, q_packed: Optional[torch.Tensor] = None,
-                      scales: Optional[torch.Tensor] = None, path: str = "auto", stream=None):
-    """(X bf16 [tokens, d], factors) -> (q_packed uint8 [tokens, d/2], scales uint8 [tokens, d/32])."""
+                      scales: Optional[torch.Tensor] = None, path: str = "auto", stream=None,
+                      scale_layout: str = "rowmajor"):
+    """(X bf16/fp16 [tokens, d], factors) -> (q_packed uint8 [tokens, d/2], scales uint8 [tokens, d/32]
+    or, with scale_layout="tiled", a flat uint8 buffer in the 128 x 4 tiled layout)."""
     tokens, d = _x_shape(X)
     if q_packed is None:
         q_packed = torch.empty((tokens, max(d // 2, 0)), dtype=torch.uint8, device=X.device)
     if scales is None:
-        scales = torch.empty((tokens, max(d // 32, 0)), dtype=torch.uint8, device=X.device)
+        scales = _scale_buffer(tokens, d, scale_layout, X.device)
     _check(load_library().kroquant_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(q_packed),
-                                               _ptr(scales), PATHS[path], C.c_void_p(_stream(stream))),
+                                               _ptr(scales), SCALE_LAYOUTS[scale_layout], PATHS[path],
+                                               C.c_void_p(_stream(stream))),
            "kroquant_quantize")
     return q_packed, scales
 
 
-def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, scales=None, stream=None):
+def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, scales=None, stream=None,
+                            scale_layout: str = "rowmajor"):
     tokens, d = _x_shape(X)
     if s.dtype != torch.float32 or not s.is_cuda or s.numel() != d or not s.is_contiguous():
         raise ValueError("s must be a contiguous CUDA float32 tensor [d]")
     if q_packed is None:
         q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
     if scales is None:
-        scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
+        scales = _scale_buffer(tokens, d, scale_layout, X.device)
     _check(load_library().kroquant_scale_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(s), _ptr(q_packed),
-                                                     _ptr(scales), C.c_void_p(_stream(stream))),
+                                                     _ptr(scales), SCALE_LAYOUTS[scale_layout],
+                                                     C.c_void_p(_stream(stream))),
            "kroquant_scale_quantize")
     return q_packed, scales
 
 
-def kroquant_mxfp4_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=None):
+def kroquant_mxfp4_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=None,
+                            scale_layout: str = "rowmajor"):
     tokens, d = _x_shape(X)
     if q_packed is None:
         q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
     if scales is None:
-        scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
+        scales = _scale_buffer(tokens, d, scale_layout, X.device)
     _check(load_library().kroquant_mxfp4_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(q_packed),
-                                                     _ptr(scales), C.c_void_p(_stream(stream))),
+                                                     _ptr(scales), SCALE_LAYOUTS[scale_layout],
+                                                     C.c_void_p(_stream(stream))),
            "kroquant_mxfp4_quantize")
     return q_packed, scales
 

@@ -80,6 +80,12 @@ __device__ __forceinline__ float absmax8(const float (&y)[8]) {
     return m;
 }
 
+// Position of the scale byte of (row t, block j) in the 128 x 4 tiled layout that block-scaled
+// tensor-core GEMMs read (tiles of 512 bytes, row-tile-major; cb = ceil(blocks_per_row / 4)).
+__device__ __forceinline__ int64_t tiled_scale_index(int64_t t, int j, int cb) {
+    return ((t >> 7) * cb + (j >> 2)) * 512 + (t & 31) * 16 + ((t >> 5) & 3) * 4 + (j & 3);
+}
+
 // streaming (read-once / write-once) global accesses
 __device__ __forceinline__ uint4 ld_stream_16(const void* p) {
     uint4 v;

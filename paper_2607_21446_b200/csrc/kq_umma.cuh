@@ -246,6 +246,7 @@ struct UmmaProblem {
     int64_t n_units;     // PB=false: 128-row tiles ; PB=true: column groups x token tiles
     int n_ttiles;        // PB=true: token tiles (ceil(tokens/128))
     int blocks_per_row;  // d/32
+    int tiled_scales;    // 0: scales[t][d/32] row-major; 1: 128 x 4 tiled layout for GEMM consumers
 };
 
 // NS pipeline slots: slot s = one shared-memory stage + one 32-column TMEM accumulator
@@ -460,7 +461,8 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         uint32_t v;
                         asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(st_scale + 4u * rr + cc) : "memory");
                         if (t < prob.n_rows && jj < prob.blocks_per_row)
-                            scales[t * prob.blocks_per_row + jj] = (uint8_t)v;
+                            scales[prob.tiled_scales ? tiled_scale_index(t, jj, (prob.blocks_per_row + 3) >> 2)
+                                                     : t * prob.blocks_per_row + jj] = (uint8_t)v;
                     }
                 }
             } else {
@@ -492,7 +494,13 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         uint32_t S;
                         encode_block_regs(acc, e, codes, S);
                         st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
-                        scales[blk] = (uint8_t)S;
+                        int64_t si = blk;
+                        if (prob.tiled_scales) {      // flat block index -> (token, block column)
+                            const uint32_t nb = (uint32_t)prob.blocks_per_row;
+                            const uint32_t t = (uint32_t)blk / nb;          // blk < 2^31 is enforced
+                            si = tiled_scale_index(t, (int)((uint32_t)blk - t * nb), (int)((nb + 3) >> 2));
+                        }
+                        scales[si] = (uint8_t)S;
                     }
                 }
             }

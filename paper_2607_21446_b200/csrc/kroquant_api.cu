@@ -222,13 +222,14 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
 // factor sets: 2-D view [tokens][d] with one 32-channel column per tile.
 template <bool WRITE_Y>
 kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f, uint8_t* q,
-                     uint8_t* scales, float* Y, cudaStream_t st) {
+                     uint8_t* scales, bool tiled, float* Y, cudaStream_t st) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
     const bool pb = f->n_sets != 1;
     const int nb = d / 32;
     kq::UmmaProblem prob;
     prob.blocks_per_row = nb;
+    prob.tiled_scales = tiled ? 1 : 0;
     CUtensorMap tmap;
     cuuint64_t dims[2], strides[1];
     if (pb) {
@@ -291,7 +292,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
 
 template <int MODE, bool WRITE_Y, bool XF16>
 kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, const float* s,
-                         uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
+                         uint8_t* q, uint8_t* scales, bool tiled, float* Y, cudaStream_t st) {
     const int64_t n_quads = tokens * (int64_t)(d / 8);
     const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
@@ -306,7 +307,7 @@ kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_fa
     cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
     if (cudaLaunchKernelEx(&cfg, kq::quantize_stream<MODE, WRITE_Y, XF16>, reinterpret_cast<const uint4*>(X), n_quads,
                            d / 32, f ? (const kq::FactorSet*)f->d_G : (const kq::FactorSet*)nullptr,
-                           f ? f->n_sets : 0, s, reinterpret_cast<uint32_t*>(q), scales, Y) != cudaSuccess) {
+                           f ? f->n_sets : 0, s, reinterpret_cast<uint32_t*>(q), scales, Y, tiled ? 1 : 0) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -316,10 +317,12 @@ kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_fa
 
 template <int MODE, bool WRITE_Y>
 kq_status_t run_stream(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f,
-                       const float* s, uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
-    return xf16 ? run_stream_t<MODE, WRITE_Y, true>(X, tokens, d, f, s, q, scales, Y, st)
-                : run_stream_t<MODE, WRITE_Y, false>(X, tokens, d, f, s, q, scales, Y, st);
+                       const float* s, uint8_t* q, uint8_t* scales, bool tiled, float* Y, cudaStream_t st) {
+    return xf16 ? run_stream_t<MODE, WRITE_Y, true>(X, tokens, d, f, s, q, scales, tiled, Y, st)
+                : run_stream_t<MODE, WRITE_Y, false>(X, tokens, d, f, s, q, scales, tiled, Y, st);
 }
+
+bool valid_layout(kq_scale_layout_t l) { return l == KQ_SCALES_ROWMAJOR || l == KQ_SCALES_TILED_128X4; }
 
 bool valid_xdtype(kq_xdtype_t t) { return t == KQ_X_BF16 || t == KQ_X_FP16; }
 
@@ -438,7 +441,7 @@ int kroquant_factors_n_sets(const kroquant_factors_t* f) { return f ? f->n_sets 
 
 kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
                                  const kroquant_factors_t* f, uint8_t* q_packed, uint8_t* scales,
-                                 kq_path_t path, void* stream) {
+                                 kq_scale_layout_t scale_layout, kq_path_t path, void* stream) {
     if (!X || !q_packed || !scales) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
@@ -446,26 +449,27 @@ kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tok
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
     if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
-    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
+    if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
     if (path == KQ_PATH_ALU && f->dense) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
+    const bool tiled = scale_layout == KQ_SCALES_TILED_128X4;
     if (path == KQ_PATH_AUTO && f->identity)
-        return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, nullptr, st);
+        return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, tiled, nullptr, st);
     if (path != KQ_PATH_ALU)
-        return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, nullptr, st);
-    return run_stream<kq::MODE_KRON, false>(X, xf16, tokens, d, f, nullptr, q_packed, scales, nullptr, st);
+        return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, tiled, nullptr, st);
+    return run_stream<kq::MODE_KRON, false>(X, xf16, tokens, d, f, nullptr, q_packed, scales, tiled, nullptr, st);
 }
 
 kq_status_t kroquant_quantize_path(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
                                    uint8_t* q_packed, uint8_t* scales, kq_path_t path, void* stream) {
-    return kroquant_quantize_ex(X, KQ_X_BF16, tokens, d, f, q_packed, scales, path, stream);
+    return kroquant_quantize_ex(X, KQ_X_BF16, tokens, d, f, q_packed, scales, KQ_SCALES_ROWMAJOR, path, stream);
 }
 
 kq_status_t kroquant_quantize(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
                               uint8_t* q_packed, uint8_t* scales, void* stream) {
-    return kroquant_quantize_ex(X, KQ_X_BF16, tokens, d, f, q_packed, scales, KQ_PATH_AUTO, stream);
+    return kroquant_quantize_ex(X, KQ_X_BF16, tokens, d, f, q_packed, scales, KQ_SCALES_ROWMAJOR, KQ_PATH_AUTO, stream);
 }
 
 kq_status_t kroquant_transform_f32_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
@@ -483,10 +487,10 @@ kq_status_t kroquant_transform_f32_ex(const void* X, kq_xdtype_t x_dtype, int64_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
     if (path == KQ_PATH_AUTO && f->identity)
-        return run_stream<kq::MODE_PLAIN, true>(X, xf16, tokens, d, nullptr, nullptr, nullptr, nullptr, Y, st);
+        return run_stream<kq::MODE_PLAIN, true>(X, xf16, tokens, d, nullptr, nullptr, nullptr, nullptr, false, Y, st);
     if (path != KQ_PATH_ALU)
-        return run_umma<true>(X, xf16, tokens, d, f, nullptr, nullptr, Y, st);
-    return run_stream<kq::MODE_KRON, true>(X, xf16, tokens, d, f, nullptr, nullptr, nullptr, Y, st);
+        return run_umma<true>(X, xf16, tokens, d, f, nullptr, nullptr, false, Y, st);
+    return run_stream<kq::MODE_KRON, true>(X, xf16, tokens, d, f, nullptr, nullptr, nullptr, false, Y, st);
 }
 
 kq_status_t kroquant_transform_f32(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
@@ -495,20 +499,22 @@ kq_status_t kroquant_transform_f32(const void* X, int64_t tokens, int d, const k
 }
 
 kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const float* s,
-                                       uint8_t* q_packed, uint8_t* scales, void* stream) {
+                                       uint8_t* q_packed, uint8_t* scales, kq_scale_layout_t scale_layout,
+                                       void* stream) {
     if (!X || !s || !q_packed || !scales) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed) || !aligned16(s)) return KQ_ERR_ALIGN;
-    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
+    if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
+    const int tiled = scale_layout == KQ_SCALES_TILED_128X4 ? 1 : 0;
     const int64_t n_quads = tokens * (int64_t)(d / 8);
     const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
     if ((int64_t)grid * 256 < d / 8)      // fewer threads than quad columns: generic kernel
-        return run_stream<kq::MODE_SCALE, false>(X, xf16, tokens, d, nullptr, s, q_packed, scales, nullptr, st);
+        return run_stream<kq::MODE_SCALE, false>(X, xf16, tokens, d, nullptr, s, q_packed, scales, tiled != 0, nullptr, st);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(256);
@@ -520,9 +526,9 @@ kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
     const cudaError_t err =
         xf16 ? cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<true>, reinterpret_cast<const uint4*>(X), tokens,
-                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales)
+                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales, tiled)
              : cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<false>, reinterpret_cast<const uint4*>(X), tokens,
-                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales);
+                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales, tiled);
     if (err != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
@@ -533,24 +539,26 @@ kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
 
 kq_status_t kroquant_scale_quantize(const void* X, int64_t tokens, int d, const float* s, uint8_t* q_packed,
                                     uint8_t* scales, void* stream) {
-    return kroquant_scale_quantize_ex(X, KQ_X_BF16, tokens, d, s, q_packed, scales, stream);
+    return kroquant_scale_quantize_ex(X, KQ_X_BF16, tokens, d, s, q_packed, scales, KQ_SCALES_ROWMAJOR, stream);
 }
 
 kq_status_t kroquant_mxfp4_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
-                                       uint8_t* q_packed, uint8_t* scales, void* stream) {
+                                       uint8_t* q_packed, uint8_t* scales, kq_scale_layout_t scale_layout,
+                                       void* stream) {
     if (!X || !q_packed || !scales) return KQ_ERR_NULL;
     kq_status_t rc = check_shape(tokens, d);
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
-    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
+    if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     return run_stream<kq::MODE_PLAIN, false>(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, nullptr, q_packed, scales,
-                                             nullptr, static_cast<cudaStream_t>(stream));
+                                             scale_layout == KQ_SCALES_TILED_128X4, nullptr,
+                                             static_cast<cudaStream_t>(stream));
 }
 
 kq_status_t kroquant_mxfp4_quantize(const void* X, int64_t tokens, int d, uint8_t* q_packed, uint8_t* scales,
                                     void* stream) {
-    return kroquant_mxfp4_quantize_ex(X, KQ_X_BF16, tokens, d, q_packed, scales, stream);
+    return kroquant_mxfp4_quantize_ex(X, KQ_X_BF16, tokens, d, q_packed, scales, KQ_SCALES_ROWMAJOR, stream);
 }
 
 kq_status_t kroquant_dequantize(const uint8_t* q_packed, const uint8_t* scales, int64_t tokens, int d,
