@@ -37,6 +37,8 @@ def lib() -> C.CDLL:
         L.kq_oracle_quantize.argtypes = [vp, i64, i32, vp, i32, vp, vp, vp]
         L.kq_oracle_scale_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.kq_oracle_dequantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, i32]
+        L.kq_oracle_round_y_to_16bit.argtypes = [vp, i64, i32, vp]
+        L.kq_oracle_round_y_to_16bit.restype = None
         L.kq_oracle_tiled_scale_size.argtypes = [i64, i32]
         L.kq_oracle_tiled_scale_size.restype = i64
         L.kq_oracle_tiled_scale_index.argtypes = [i64, i32, i32]
@@ -192,4 +194,12 @@ def scales_to_tiled(scales, fill: int = 0) -> np.ndarray:
     rows, kb = scales.shape
     out = np.empty(int(lib().kq_oracle_tiled_scale_size(rows, kb)), np.uint8)
     lib().kq_oracle_scales_to_tiled(_p(scales), rows, kb, fill, _p(out))
+    return out
+
+
+def round_y_to_16bit(Y, out_dtype: str = "bf16") -> np.ndarray:
+    """The transformed activations in 16 bits (uint16 patterns): float y rounded to nearest even."""
+    Y = np.ascontiguousarray(Y, dtype=np.float32)
+    out = np.empty(Y.shape, np.uint16)
+    lib().kq_oracle_round_y_to_16bit(_p(Y), Y.size, X_DTYPES[out_dtype], _p(out))
     return out

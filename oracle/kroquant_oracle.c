@@ -342,6 +342,36 @@ int kq_oracle_dequantize(const uint8_t *q, const uint8_t *scales, int64_t tokens
     return 0;
 }
 
+/* ---- 16-bit copy of the transformed activations ------------------------------------------- */
+/* The low-rank branch of the inference formula (Section 3.4: A T L R; Appendix D: "activations
+ * forwarded to the low-rank branch are kept at 16-bit") consumes A T in the activations' own 16-bit
+ * type: the float pre-rounding value y rounded once more, to nearest even.  out_dtype: 0 = bf16,
+ * 1 = fp16 (values beyond 65504 become infinity). */
+static uint16_t float_to_fp16_bits_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    double a = fabs((double)f);
+    if (isnan(f)) return (uint16_t)(sign | 0x7E00u);
+    if (a >= 65520.0) return (uint16_t)(sign | 0x7C00u);          /* rounds to infinity */
+    if (a == 0.0) return sign;
+    int e;
+    frexp(a, &e);                                                  /* a = m 2^e, m in [0.5, 1) */
+    int ex = e - 1;
+    if (ex < -14) ex = -14;                                        /* subnormal quantum 2^-24 */
+    double q = nearbyint(ldexp(a, 10 - ex));                       /* ties to even */
+    if (ex == -14 && q < 1024.0) return (uint16_t)(sign | (uint16_t)q);
+    if (q >= 2048.0) { q /= 2.0; ex += 1; }
+    return (uint16_t)(sign | (uint16_t)((ex + 15) << 10) | (uint16_t)((int)q - 1024));
+}
+
+void kq_oracle_round_y_to_16bit(const float *Y, int64_t n, int out_dtype, uint16_t *out)
+{
+    for (int64_t i = 0; i < n; ++i)
+        out[i] = out_dtype ? float_to_fp16_bits_rne(Y[i]) : float_to_bf16_bits_rne(Y[i]);
+}
+
 /* ---- scale-byte layout for block-scaled tensor-core GEMM consumers ------------------------ */
 /* The W4A4 product of the paper's inference formula (Section 3.4) is a block-scaled MXFP4 GEMM.
  * Such GEMMs read the E8M0 bytes of an operand [rows][k_blocks] in tiles of 128 rows x 4 k-blocks

@@ -105,3 +105,24 @@ def test_tiled_scale_layout_equals_reshape_permute(rows, kb):
     # a bijection on the real entries: every (r, j) lands on a distinct byte
     idx = {co.tiled_scale_index(r, j, kb) for r in range(min(rows, 140)) for j in range(kb)}
     assert len(idx) == min(rows, 140) * kb
+
+
+# ---- 16-bit copy of the transformed activations ---------------------------------------------------
+def test_rounding_y_to_16_bits_matches_library_casts():
+    import torch
+    rng = np.random.default_rng(3)
+    y = np.concatenate([
+        (rng.standard_normal(20000) * np.exp(rng.uniform(-12, 8, 20000))).astype(np.float32),
+        np.array([0.0, -0.0, 65504.0, 65519.9, 65520.0, -70000.0, 2.0 ** -24, 2.0 ** -25, 1.5 * 2.0 ** -25,
+                  2.0 ** -14, 1.00048828125, 1.0009765625, 1.00146484375], np.float32)])
+    # every float that is exactly half-way between two fp16 / bf16 neighbours around 1..2
+    ties16 = (1.0 + (np.arange(0, 2048, 2) + 1) / 2048.0).astype(np.float32)
+    tiesb = (1.0 + (np.arange(0, 256, 2) + 1) / 256.0).astype(np.float32)
+    y = np.concatenate([y, ties16, tiesb, -ties16])
+    got16 = co.round_y_to_16bit(y, "fp16")
+    with np.errstate(over="ignore"):
+        ref16 = y.astype(np.float16).view(np.uint16)                 # NumPy: round to nearest even
+    assert np.array_equal(got16, ref16)
+    gotb = co.round_y_to_16bit(y, "bf16")
+    refb = torch.from_numpy(y.copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(gotb, refb)
