@@ -121,6 +121,15 @@ kq_status_t kroquant_mxfp4_quantize_ex(const void *X, kq_xdtype_t x_dtype, int64
                                        uint8_t *q_packed, uint8_t *scales,
                                        kq_scale_layout_t scale_layout, void *stream);
 
+/* Section 3.4 (inference formula  O = Q(A T) Q(W~ - L R)^T + A T L R): one pass over X that
+ * writes both operands of the layer's two branches: the MXFP4 codes and scales of A T, and A T
+ * itself in X's own 16-bit type (AT_out: DEVICE [tokens][d], each value the float pre-rounding value
+ * rounded to nearest even; fp16 overflows to infinity beyond 65504).  Tensor-core path; identity
+ * factors are not short-cut.  Adds 2 bytes per element of HBM writes. */
+kq_status_t kroquant_quantize_dual(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                   const kroquant_factors_t *f, uint8_t *q_packed, uint8_t *scales,
+                                   kq_scale_layout_t scale_layout, void *AT_out, void *stream);
+
 /* Section 3.1 (quantize-then-DEquantize operator Q_b), decode half.
  * f == NULL: out = decoded transformed values  grid[code & 7] * sign * 2^(S-127)
  * (what a W4A4 GEMM consumes).  With factors: additionally multiplied by

@@ -22,7 +22,7 @@ PATHS = {"auto": 0, "tensor": 1, "alu": 2}
 EXPORTS = [
     "kroquant_factors_create", "kroquant_factors_create_lu", "kroquant_factors_create_dense",
     "kroquant_factors_destroy", "kroquant_quantize_ex", "kroquant_transform_f32_ex",
-    "kroquant_scale_quantize_ex", "kroquant_mxfp4_quantize_ex",
+    "kroquant_scale_quantize_ex", "kroquant_mxfp4_quantize_ex", "kroquant_quantize_dual",
     "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize",
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
@@ -56,6 +56,7 @@ def load_library() -> C.CDLL:
     L.kroquant_factors_create_dense.argtypes = [vp, i32, C.POINTER(vp)]
     L.kroquant_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, i32, vp]
     L.kroquant_transform_f32_ex.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
+    L.kroquant_quantize_dual.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp]
     L.kroquant_scale_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp]
     L.kroquant_mxfp4_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
     L.kroquant_factors_destroy.argtypes = [vp]
@@ -190,6 +191,22 @@ def kroquant_quantize(X: torch.Tensor, factors: Factors, q_packed: Optional[torc
                                                C.c_void_p(_stream(stream))),
            "kroquant_quantize")
     return q_packed, scales
+
+
+def kroquant_quantize_dual(X: torch.Tensor, factors: Factors, q_packed=None, scales=None, AT=None, stream=None,
+                           scale_layout: str = "rowmajor"):
+    """One pass: MXFP4(X T) and X T itself in X's dtype -> (q_packed, scales, AT)."""
+    tokens, d = _x_shape(X)
+    if q_packed is None:
+        q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
+    if scales is None:
+        scales = _scale_buffer(tokens, d, scale_layout, X.device)
+    if AT is None:
+        AT = torch.empty_like(X)
+    _check(load_library().kroquant_quantize_dual(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(q_packed),
+                                                 _ptr(scales), SCALE_LAYOUTS[scale_layout], _ptr(AT),
+                                                 C.c_void_p(_stream(stream))), "kroquant_quantize_dual")
+    return q_packed, scales, AT
 
 
 def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, scales=None, stream=None,

@@ -31,6 +31,7 @@
 // its TMEM before returning.
 #pragma once
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include "kq_common.cuh"
 
 namespace kq {
@@ -189,6 +190,31 @@ struct UmmaSmem {
     static constexpr int kDynBytes = kBytes + 1024;                  // slack for manual alignment
 };
 
+// Optional second output: the block's 32 transformed values y = acc * 2^-e rounded to X's own
+// 16-bit type (round-to-nearest-even), 64 contiguous bytes -- what the 16-bit low-rank branch of
+// the quantized layer consumes (paper Section 3.4).
+template <bool XF16>
+__device__ __forceinline__ void store_block_16bit(const uint32_t (&acc)[32], int e, uint4* dst) {
+    const float back = __uint_as_float((uint32_t)(127 - e) << 23);      // 2^-e
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float a = __uint_as_float(acc[8 * v + 2 * i]) * back;
+            const float b = __uint_as_float(acc[8 * v + 2 * i + 1]) * back;
+            if (XF16) {
+                const __half2 h = __floats2half2_rn(a, b);
+                w[i] = *reinterpret_cast<const uint32_t*>(&h);
+            } else {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                w[i] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+        }
+        dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 // The fused epilogue math of one 32-channel block held in registers.  acc = y * 2^e
 // (e = the factor image's normalisation exponent; 0 for bf16 images).
 // Common case: the true scale byte S = biased_exp(amax_acc) - 2 - e needs no clamping;
@@ -267,7 +293,8 @@ template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y>
 __global__ void __launch_bounds__(128 + 128 * NG, 1)
 quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
               const uint8_t* __restrict__ b_image, const int* __restrict__ e_norm, const UmmaProblem prob,
-              uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y) {
+              uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y,
+              uint4* __restrict__ at_out) {
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
     // A slot must always be served by the same issuer warp and the same epilogue group:
     // only then does program order inside that warp guarantee that a parity wait never
@@ -433,7 +460,11 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 const bool elected = threadIdx.x == 128;
                 uint4 codes;
                 uint32_t S;
-                encode_block_regs(acc, __ldg(e_norm + (j < prob.blocks_per_row ? j : 0)), codes, S);
+                const int e_j = __ldg(e_norm + (j < prob.blocks_per_row ? j : 0));
+                if (at_out != nullptr && j < prob.blocks_per_row &&
+                    (int64_t)tt * kTileRows + r < prob.n_rows)
+                    store_block_16bit<XF16>(acc, e_j, at_out + (((int64_t)tt * kTileRows + r) * prob.blocks_per_row + j) * 4);
+                encode_block_regs(acc, e_j, codes, S);
                 if (c == 0) {
                     // the previous group's TMA store must have finished reading the staging tile
                     if (elected) bulk_wait_group_read<0>();
@@ -492,6 +523,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     } else {
                         uint4 codes;
                         uint32_t S;
+                        if (at_out != nullptr) store_block_16bit<XF16>(acc, e, at_out + blk * 4);
                         encode_block_regs(acc, e, codes, S);
                         st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
                         int64_t si = blk;

@@ -184,7 +184,8 @@ kq_status_t finish_factors(kroquant_factors_t* f, const std::vector<double>& K,
 template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y>
 kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
                         const int* enorm, const kq::UmmaProblem& prob,
-                        uint8_t* q, uint8_t* scales, float* Y, int ctas_per_sm, bool pdl, cudaStream_t st) {
+                        uint8_t* q, uint8_t* scales, float* Y, void* at_out, int ctas_per_sm, bool pdl,
+                        cudaStream_t st) {
     using L = kq::UmmaSmem<NS, PB>;
     auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y>;
     static std::once_flag once;
@@ -210,7 +211,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, enorm, prob, q, scales, Y) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, enorm, prob, q, scales, Y, reinterpret_cast<uint4*>(at_out)) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -222,7 +223,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
 // factor sets: 2-D view [tokens][d] with one 32-channel column per tile.
 template <bool WRITE_Y>
 kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f, uint8_t* q,
-                     uint8_t* scales, bool tiled, float* Y, cudaStream_t st) {
+                     uint8_t* scales, bool tiled, float* Y, void* at_out, cudaStream_t st) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
     const bool pb = f->n_sets != 1;
@@ -266,7 +267,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     const uint8_t* b = f->d_bimage + (xf16 ? (size_t)f->n_sets * kq::kBImageBytes : 0);
     const int* en = f->d_enorm + (xf16 ? f->n_sets : 0);
 #define KQ_LAUNCH(NS, NM, NG, PB, XF) \
-    launch_umma<NS, NM, NG, PB, XF, WRITE_Y>(tmap, tmap_q, b, en, prob, q, scales, Y, cps, pdl, st)
+    launch_umma<NS, NM, NG, PB, XF, WRITE_Y>(tmap, tmap_q, b, en, prob, q, scales, Y, at_out, cps, pdl, st)
     if (xf16) return pb ? KQ_LAUNCH(4, 1, 1, true, true) : KQ_LAUNCH(4, 2, 1, false, true);
     if (pb) {
         switch (g_umma_cfg.load()) {
@@ -458,8 +459,23 @@ kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tok
     if (path == KQ_PATH_AUTO && f->identity)
         return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, tiled, nullptr, st);
     if (path != KQ_PATH_ALU)
-        return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, tiled, nullptr, st);
+        return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, tiled, nullptr, nullptr, st);
     return run_stream<kq::MODE_KRON, false>(X, xf16, tokens, d, f, nullptr, q_packed, scales, tiled, nullptr, st);
+}
+
+kq_status_t kroquant_quantize_dual(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                   const kroquant_factors_t* f, uint8_t* q_packed, uint8_t* scales,
+                                   kq_scale_layout_t scale_layout, void* AT_out, void* stream) {
+    if (!X || !q_packed || !scales || !AT_out) return KQ_ERR_NULL;
+    kq_status_t rc = check_shape(tokens, d);
+    if (rc != KQ_OK) return rc;
+    rc = check_factors_for(f, d);
+    if (rc != KQ_OK) return rc;
+    if (!aligned16(X) || !aligned16(q_packed) || !aligned16(AT_out)) return KQ_ERR_ALIGN;
+    if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
+    if (tokens == 0) return KQ_OK;
+    return run_umma<false>(X, x_dtype == KQ_X_FP16, tokens, d, f, q_packed, scales,
+                           scale_layout == KQ_SCALES_TILED_128X4, nullptr, AT_out, static_cast<cudaStream_t>(stream));
 }
 
 kq_status_t kroquant_quantize_path(const void* X, int64_t tokens, int d, const kroquant_factors_t* f,
@@ -489,7 +505,7 @@ kq_status_t kroquant_transform_f32_ex(const void* X, kq_xdtype_t x_dtype, int64_
     if (path == KQ_PATH_AUTO && f->identity)
         return run_stream<kq::MODE_PLAIN, true>(X, xf16, tokens, d, nullptr, nullptr, nullptr, nullptr, false, Y, st);
     if (path != KQ_PATH_ALU)
-        return run_umma<true>(X, xf16, tokens, d, f, nullptr, nullptr, false, Y, st);
+        return run_umma<true>(X, xf16, tokens, d, f, nullptr, nullptr, false, Y, nullptr, st);
     return run_stream<kq::MODE_KRON, true>(X, xf16, tokens, d, f, nullptr, nullptr, nullptr, false, Y, st);
 }
 
