@@ -333,20 +333,24 @@ def run_ours(args):
     hq = [torch.empty(c["q"].shape, dtype=torch.uint8).pin_memory() for c in calls[:2]]
     hs = [torch.empty(c["s"].shape, dtype=torch.uint8).pin_memory() for c in calls[:2]]
 
+    pipe = B.HostPipeline(device)      # upload / kernel / download of neighbouring calls overlap
+
     def e2e_step():
-        with torch.cuda.stream(stream):
-            for c in calls:
-                k = c["shape_idx"]
-                B.quantize_from_host(hx[k], c["factors"], c["X"], c["q"], c["s"], hq[k], hs[k], stream=stream)
+        for c in calls:
+            k = c["shape_idx"]
+            pipe.submit(hx[k], c["factors"], c["X"], c["q"], c["s"], hq[k], hs[k])
     # (the device copies of X are overwritten by identical data: calls[0:2] hold the unrolled tensors;
     #  the other 26 device buffers receive the same host tensor, which changes no timing-relevant property)
+    torch.cuda.synchronize()
     e2e_step()
+    pipe.synchronize()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         e2e_step()
+    pipe.synchronize()
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
     if dist is not None:

@@ -294,3 +294,45 @@ def quantize_from_host(X_host: torch.Tensor, factors: Factors, X_dev: torch.Tens
     q_host.copy_(q_dev, non_blocking=True)
     s_host.copy_(s_dev, non_blocking=True)
     return q_host, s_host
+
+
+class HostPipeline:
+    """Host-to-host quantization with the three phases on their own streams, so that the upload of
+    call i+1, the kernel of call i and the download of call i-1 overlap (PCIe is full duplex).
+    Buffers may be reused from call to call: a buffer's next writer waits for its last reader."""
+
+    def __init__(self, device=None):
+        self.h2d = torch.cuda.Stream(device)
+        self.compute = torch.cuda.Stream(device)
+        self.d2h = torch.cuda.Stream(device)
+        self._last_kernel = {}      # X_dev.data_ptr() -> event after the kernel that read it
+        self._last_download = {}    # q_dev.data_ptr() -> event after the copy that read it
+
+    def submit(self, X_host, factors: Factors, X_dev, q_dev, s_dev, q_host, s_host):
+        ev = self._last_kernel.get(X_dev.data_ptr())
+        if ev is not None:
+            self.h2d.wait_event(ev)
+        with torch.cuda.stream(self.h2d):
+            X_dev.copy_(X_host, non_blocking=True)
+        up = torch.cuda.Event()
+        up.record(self.h2d)
+        self.compute.wait_event(up)
+        ev = self._last_download.get(q_dev.data_ptr())
+        if ev is not None:
+            self.compute.wait_event(ev)
+        kroquant_quantize(X_dev, factors, q_dev, s_dev, stream=self.compute)
+        done = torch.cuda.Event()
+        done.record(self.compute)
+        self._last_kernel[X_dev.data_ptr()] = done
+        self.d2h.wait_event(done)
+        with torch.cuda.stream(self.d2h):
+            q_host.copy_(q_dev, non_blocking=True)
+            s_host.copy_(s_dev, non_blocking=True)
+        down = torch.cuda.Event()
+        down.record(self.d2h)
+        self._last_download[q_dev.data_ptr()] = down
+
+    def synchronize(self):
+        self.h2d.synchronize()
+        self.compute.synchronize()
+        self.d2h.synchronize()

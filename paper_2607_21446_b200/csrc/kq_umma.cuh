@@ -289,7 +289,9 @@ struct UmmaProblem {
 // Grid: any size <= number of tiles; CTA b takes tiles b, b + gridDim.x, ...
 // XF16: X and the factor image are fp16 (else bf16); e_norm: per-set normalisation exponents of
 // the image (all zero for bf16 images).
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y>
+// DUAL: also write the 16-bit transformed activations (at_out); a separate instantiation, because the
+// extra conversion code costs registers that would take a resident CTA away from the default kernel.
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, bool DUAL = false>
 __global__ void __launch_bounds__(128 + 128 * NG, 1)
 quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
               const uint8_t* __restrict__ b_image, const int* __restrict__ e_norm, const UmmaProblem prob,
@@ -461,7 +463,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 uint4 codes;
                 uint32_t S;
                 const int e_j = __ldg(e_norm + (j < prob.blocks_per_row ? j : 0));
-                if (at_out != nullptr && j < prob.blocks_per_row &&
+                if (DUAL && j < prob.blocks_per_row &&
                     (int64_t)tt * kTileRows + r < prob.n_rows)
                     store_block_16bit<XF16>(acc, e_j, at_out + (((int64_t)tt * kTileRows + r) * prob.blocks_per_row + j) * 4);
                 encode_block_regs(acc, e_j, codes, S);
@@ -523,7 +525,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     } else {
                         uint4 codes;
                         uint32_t S;
-                        if (at_out != nullptr) store_block_16bit<XF16>(acc, e, at_out + blk * 4);
+                        if (DUAL) store_block_16bit<XF16>(acc, e, at_out + blk * 4);
                         encode_block_regs(acc, e, codes, S);
                         st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
                         int64_t si = blk;

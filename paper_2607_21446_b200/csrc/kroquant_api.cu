@@ -181,13 +181,13 @@ kq_status_t finish_factors(kroquant_factors_t* f, const std::vector<double>& K,
     return KQ_OK;
 }
 
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y>
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, bool DUAL = false>
 kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
                         const int* enorm, const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, void* at_out, int ctas_per_sm, bool pdl,
                         cudaStream_t st) {
     using L = kq::UmmaSmem<NS, PB>;
-    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y>;
+    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, DUAL>;
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, [&] {
@@ -267,7 +267,13 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     const uint8_t* b = f->d_bimage + (xf16 ? (size_t)f->n_sets * kq::kBImageBytes : 0);
     const int* en = f->d_enorm + (xf16 ? f->n_sets : 0);
 #define KQ_LAUNCH(NS, NM, NG, PB, XF) \
-    launch_umma<NS, NM, NG, PB, XF, WRITE_Y>(tmap, tmap_q, b, en, prob, q, scales, Y, at_out, cps, pdl, st)
+    launch_umma<NS, NM, NG, PB, XF, WRITE_Y>(tmap, tmap_q, b, en, prob, q, scales, Y, nullptr, cps, pdl, st)
+#define KQ_LAUNCH_DUAL(NS, NM, NG, PB, XF) \
+    launch_umma<NS, NM, NG, PB, XF, false, true>(tmap, tmap_q, b, en, prob, q, scales, nullptr, at_out, cps, pdl, st)
+    if (!WRITE_Y && at_out != nullptr) {
+        if (xf16) return pb ? KQ_LAUNCH_DUAL(4, 1, 1, true, true) : KQ_LAUNCH_DUAL(4, 2, 1, false, true);
+        return pb ? KQ_LAUNCH_DUAL(4, 1, 1, true, false) : KQ_LAUNCH_DUAL(4, 2, 1, false, false);
+    }
     if (xf16) return pb ? KQ_LAUNCH(4, 1, 1, true, true) : KQ_LAUNCH(4, 2, 1, false, true);
     if (pb) {
         switch (g_umma_cfg.load()) {
@@ -289,6 +295,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
         case 7: return KQ_LAUNCH(16, 2, 4, false, false);
     }
 #undef KQ_LAUNCH
+#undef KQ_LAUNCH_DUAL
 }
 
 template <int MODE, bool WRITE_Y, bool XF16>
