@@ -69,13 +69,13 @@ __device__ __forceinline__ uint32_t encode8(const float (&y)[8], float amax_bloc
 // latency-bandwidth product asks for).
 constexpr int kStreamUnroll = 4;
 
-template <int MODE, bool WRITE_Y, bool XF16>
+template <int MODE, bool WRITE_Y, bool XF16, bool TILED>
 __global__ void __launch_bounds__(256)
 quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row,
                 const FactorSet* __restrict__ factors, int n_sets,
                 const float* __restrict__ chan_scale,
                 uint32_t* __restrict__ q_packed, uint8_t* __restrict__ scales,
-                float* __restrict__ Y, int tiled_scales) {
+                float* __restrict__ Y) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;   // multiple of 32: quads stay lane-aligned
@@ -138,7 +138,7 @@ quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row
                     st_stream_4(q_packed + q, codes);
                     if (quad == 0) {
                         int64_t si = blk;
-                        if (tiled_scales) si = tiled_scale_index(blk / blocks_per_row, j, (blocks_per_row + 3) >> 2);
+                        if (TILED) si = tiled_scale_index(blk / blocks_per_row, j, (blocks_per_row + 3) >> 2);
                         scales[si] = (uint8_t)S;
                     }
                 }
@@ -153,11 +153,11 @@ quantize_stream(const uint4* __restrict__ X, int64_t n_quads, int blocks_per_row
 // per item.  Requires gridDim.x * blockDim.x >= d/8.  The four lanes of a quad always
 // work on the same row, so the amax shuffles use a per-quad mask (trip counts may differ
 // between quads of one warp).
-template <bool XF16>
+template <bool XF16, bool TILED>
 __global__ void __launch_bounds__(256)
 scale_quantize_rows(const uint4* __restrict__ X, int64_t tokens, int quads_per_row,
                     const float* __restrict__ chan_scale, uint32_t* __restrict__ q_packed,
-                    uint8_t* __restrict__ scales, int tiled_scales) {
+                    uint8_t* __restrict__ scales) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t n_threads = (int64_t)gridDim.x * blockDim.x;
@@ -193,7 +193,7 @@ scale_quantize_rows(const uint4* __restrict__ X, int64_t tokens, int quads_per_r
             const int64_t q = rr * quads_per_row + p;
             st_stream_4(q_packed + q, codes);
             if (quad == 0)
-                scales[tiled_scales ? tiled_scale_index(rr, p >> 2, (quads_per_row + 15) >> 4) : (q >> 2)] = (uint8_t)S;
+                scales[TILED ? tiled_scale_index(rr, p >> 2, (quads_per_row + 15) >> 4) : (q >> 2)] = (uint8_t)S;
         }
     }
 }

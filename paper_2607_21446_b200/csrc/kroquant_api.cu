@@ -298,9 +298,9 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
 #undef KQ_LAUNCH_DUAL
 }
 
-template <int MODE, bool WRITE_Y, bool XF16>
+template <int MODE, bool WRITE_Y, bool XF16, bool TILED>
 kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_factors_t* f, const float* s,
-                         uint8_t* q, uint8_t* scales, bool tiled, float* Y, cudaStream_t st) {
+                         uint8_t* q, uint8_t* scales, float* Y, cudaStream_t st) {
     const int64_t n_quads = tokens * (int64_t)(d / 8);
     const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
@@ -313,9 +313,9 @@ kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_fa
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kq::quantize_stream<MODE, WRITE_Y, XF16>, reinterpret_cast<const uint4*>(X), n_quads,
-                           d / 32, f ? (const kq::FactorSet*)f->d_G : (const kq::FactorSet*)nullptr,
-                           f ? f->n_sets : 0, s, reinterpret_cast<uint32_t*>(q), scales, Y, tiled ? 1 : 0) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kq::quantize_stream<MODE, WRITE_Y, XF16, TILED>, reinterpret_cast<const uint4*>(X),
+                           n_quads, d / 32, f ? (const kq::FactorSet*)f->d_G : (const kq::FactorSet*)nullptr,
+                           f ? f->n_sets : 0, s, reinterpret_cast<uint32_t*>(q), scales, Y) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -326,8 +326,11 @@ kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_fa
 template <int MODE, bool WRITE_Y>
 kq_status_t run_stream(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f,
                        const float* s, uint8_t* q, uint8_t* scales, bool tiled, float* Y, cudaStream_t st) {
-    return xf16 ? run_stream_t<MODE, WRITE_Y, true>(X, tokens, d, f, s, q, scales, tiled, Y, st)
-                : run_stream_t<MODE, WRITE_Y, false>(X, tokens, d, f, s, q, scales, tiled, Y, st);
+    if (tiled && !WRITE_Y)
+        return xf16 ? run_stream_t<MODE, false, true, true>(X, tokens, d, f, s, q, scales, Y, st)
+                    : run_stream_t<MODE, false, false, true>(X, tokens, d, f, s, q, scales, Y, st);
+    return xf16 ? run_stream_t<MODE, WRITE_Y, true, false>(X, tokens, d, f, s, q, scales, Y, st)
+                : run_stream_t<MODE, WRITE_Y, false, false>(X, tokens, d, f, s, q, scales, Y, st);
 }
 
 bool valid_layout(kq_scale_layout_t l) { return l == KQ_SCALES_ROWMAJOR || l == KQ_SCALES_TILED_128X4; }
@@ -547,11 +550,15 @@ kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
-    const cudaError_t err =
-        xf16 ? cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<true>, reinterpret_cast<const uint4*>(X), tokens,
-                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales, tiled)
-             : cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<false>, reinterpret_cast<const uint4*>(X), tokens,
-                                  d / 8, s, reinterpret_cast<uint32_t*>(q_packed), scales, tiled);
+    const uint4* x4 = reinterpret_cast<const uint4*>(X);
+    uint32_t* q32 = reinterpret_cast<uint32_t*>(q_packed);
+    cudaError_t err;
+    if (xf16)
+        err = tiled ? cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<true, true>, x4, tokens, d / 8, s, q32, scales)
+                    : cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<true, false>, x4, tokens, d / 8, s, q32, scales);
+    else
+        err = tiled ? cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<false, true>, x4, tokens, d / 8, s, q32, scales)
+                    : cudaLaunchKernelEx(&cfg, kq::scale_quantize_rows<false, false>, x4, tokens, d / 8, s, q32, scales);
     if (err != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
