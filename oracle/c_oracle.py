@@ -37,6 +37,7 @@ def lib() -> C.CDLL:
         L.kq_oracle_quantize.argtypes = [vp, i64, i32, vp, i32, vp, vp, vp]
         L.kq_oracle_scale_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.kq_oracle_dequantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, i32]
+        L.kq_oracle_hadamard_transform_x.argtypes = [vp, i32, i64, i32, vp]
         L.kq_oracle_round_y_to_16bit.argtypes = [vp, i64, i32, vp]
         L.kq_oracle_round_y_to_16bit.restype = None
         L.kq_oracle_tiled_scale_size.argtypes = [i64, i32]
@@ -203,3 +204,18 @@ def round_y_to_16bit(Y, out_dtype: str = "bf16") -> np.ndarray:
     out = np.empty(Y.shape, np.uint16)
     lib().kq_oracle_round_y_to_16bit(_p(Y), Y.size, X_DTYPES[out_dtype], _p(out))
     return out
+
+
+def hadamard_transform(X, x_dtype: str = "bf16") -> np.ndarray:
+    """float32( x H_d / sqrt(d) ) over the full row (d a power of two)."""
+    X = _x(X)
+    Y = np.empty(X.shape, np.float32)
+    if lib().kq_oracle_hadamard_transform_x(_p(X), X_DTYPES[x_dtype], X.shape[0], X.shape[1], _p(Y)) != 0:
+        raise ValueError("oracle: d must be a power of two >= 32")
+    return Y
+
+
+def hadamard_quantize(X, x_dtype: str = "bf16"):
+    Y = hadamard_transform(X, x_dtype)
+    q, s = mx_encode(Y)
+    return q, s, Y

@@ -342,6 +342,29 @@ int kq_oracle_dequantize(const uint8_t *q, const uint8_t *scales, int64_t tokens
     return 0;
 }
 
+/* ---- full-d Walsh-Hadamard baseline (Section 4.4 "FWHT") --------------------------------------- */
+/* The paper's FWHT comparison applies the normalised Hadamard matrix of the full hidden size
+ * (Section 1: "a fixed orthogonal and symmetric matrix with normalized +-1 entries"; Section 3.2:
+ * H_n is the Kronecker product of log2 n copies of (1/sqrt 2) [[1,1],[1,-1]]) and needs d to be a
+ * power of two (Section 4.4).  Definition written out: H[r][c] = (-1)^popcount(r & c) / sqrt(d),
+ * y_c = float( sum_r x_r H[r][c] ), sums in double, ascending r.  O(d^2) per row. */
+int kq_oracle_hadamard_transform_x(const uint16_t *X, int x_dtype, int64_t tokens, int d, float *Y)
+{
+    if (d < KQ_BLOCK || (d & (d - 1)) || tokens < 0) return -1;
+    double norm = 1.0 / sqrt((double)d);
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < tokens; ++t)
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int r = 0; r < d; ++r) {
+                double x = (double)load_x(X, t * d + r, x_dtype);
+                acc += (__builtin_popcount((unsigned)(r & c)) & 1) ? -x : x;
+            }
+            Y[t * d + c] = (float)(acc * norm);
+        }
+    return 0;
+}
+
 /* ---- 16-bit copy of the transformed activations ------------------------------------------- */
 /* The low-rank branch of the inference formula (Section 3.4: A T L R; Appendix D: "activations
  * forwarded to the low-rank branch are kept at 16-bit") consumes A T in the activations' own 16-bit

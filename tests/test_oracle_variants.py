@@ -126,3 +126,35 @@ def test_rounding_y_to_16_bits_matches_library_casts():
     gotb = co.round_y_to_16bit(y, "bf16")
     refb = torch.from_numpy(y.copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(gotb, refb)
+
+
+# ---- full-d Hadamard baseline -------------------------------------------------------------------------
+@pytest.mark.parametrize("d", [32, 64, 256, 1024])
+def test_hadamard_transform_against_scipy(d):
+    from scipy.linalg import hadamard
+    Xb = W.gen_activations(W.ActivationSpec("h", 5, d, seed=d, outlier_channels=2, outlier_gain=50.0))
+    x = W.bf16_bits_to_f32(Xb).astype(np.float64)
+    Y = co.hadamard_transform(Xb)
+    ref = x @ (hadamard(d).astype(np.float64) / np.sqrt(d))            # Sylvester construction, library
+    assert np.allclose(Y, ref, rtol=2e-7, atol=2e-7 * np.abs(ref).max())
+    # orthogonal and symmetric: applying it twice gives x back
+    back = Y.astype(np.float64) @ (hadamard(d) / np.sqrt(d))
+    assert np.allclose(back, x, atol=1e-5 * np.abs(x).max())
+    # d = 32 coincides with the block transform at the paper's Hadamard initialisation
+    if d == 32:
+        G = co.lu_to_factors(W.hadamard_lu_params(1))
+        assert np.allclose(Y, co.transform(Xb, G), rtol=1e-6, atol=1e-6 * np.abs(Y).max())
+    with pytest.raises(ValueError):
+        co.hadamard_transform(np.zeros((1, 96), np.uint16))
+
+
+def test_hadamard_constant_row_and_single_spike():
+    d = 128
+    ones = W.f32_to_bf16_bits(np.ones((1, d), np.float32))
+    y = co.hadamard_transform(ones)[0]
+    assert y[0] == np.float32(np.sqrt(d)) and not y[1:].any()
+    spike = np.zeros((1, d), np.float32)
+    spike[0, 5] = 3.0
+    y = co.hadamard_transform(W.f32_to_bf16_bits(spike))[0]
+    signs = np.array([(-1.0) ** bin(5 & c).count("1") for c in range(d)])
+    assert np.array_equal(y, (3.0 * signs / np.sqrt(d)).astype(np.float32))
