@@ -496,11 +496,11 @@ def run_sweep(args):
 
 
 # The paper's two latency tables (Section 4.4 and Appendix A): (m, d) and its MI350 / FP16 numbers in
-# microseconds for Q4, Scale, K1, K2 -- context only, another machine.
+# microseconds for Q4, Scale, K1, K2 (and FWHT where given) -- context only, another machine.
 PAPER_TABLES = {
-    "power_of_two_d": [((4096, 1024), (9.40, 10.56, 9.96, 14.00)), ((4096, 4096), (22.64, 25.52, 23.88, 27.80)),
-                       ((4096, 16384), (74.44, 75.44, 75.32, 78.52)), ((512, 4096), (7.20, 9.24, 8.12, 10.28)),
-                       ((512, 16384), (13.68, 16.36, 15.36, 19.32))],
+    "power_of_two_d": [((4096, 1024), (9.40, 10.56, 9.96, 14.00, 18.16)), ((4096, 4096), (22.64, 25.52, 23.88, 27.80, 68.04)),
+                       ((4096, 16384), (74.44, 75.44, 75.32, 78.52, 186.04)), ((512, 4096), (7.20, 9.24, 8.12, 10.28, 14.40)),
+                       ((512, 16384), (13.68, 16.36, 15.36, 19.32, 33.96))],
     "production_shapes": [((512, 3072), (6.72, 9.04, 7.64, 8.84)), ((512, 12288), (11.80, 14.68, 13.08, 17.00)),
                           ((4096, 1152), (10.64, 14.00, 10.68, 14.64)), ((4096, 3072), (18.56, 21.12, 19.28, 23.32)),
                           ((4096, 3456), (20.60, 24.20, 21.32, 25.36)), ((4096, 4096), (22.08, 25.80, 23.36, 27.28)),
@@ -532,17 +532,21 @@ def run_table(args):
             f2, f1 = B.Factors.create(G), B.Factors.create_dense(K.astype(np.float32)[None])
             sv = torch.from_numpy(W.gen_channel_scales(4, d)).cuda()
             us = {}
-            for name, fn in (("Q4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)),
-                             ("Scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
-                             ("K1", lambda x: B.kroquant_quantize(x, f1, q, sc, stream=stream)),
-                             ("K2", lambda x: B.kroquant_quantize(x, f2, q, sc, stream=stream))):
+            kernels = [("Q4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)),
+                       ("Scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
+                       ("K1", lambda x: B.kroquant_quantize(x, f1, q, sc, stream=stream)),
+                       ("K2", lambda x: B.kroquant_quantize(x, f2, q, sc, stream=stream))]
+            if d & (d - 1) == 0:
+                kernels.append(("FWHT", lambda x: B.kroquant_fwht_quantize(x, q, sc, stream=stream)))
+            for name, fn in kernels:
                 g = capture(torch, [lambda x=x, fn=fn: fn(x) for x in Xs], stream)
                 ms, _ = time_graph(torch, None, g, stream, max(5, args.steps // 10), 3)
                 us[name] = round(ms * 1e3 / nbuf, 2)
             print(json.dumps({"table": table, "m": m, "d": d, "dtype": "fp16", "us_b200": us,
                               "scale_over_k1": round(us["Scale"] / us["K1"], 3),
                               "scale_over_k2": round(us["Scale"] / us["K2"], 3),
-                              "paper_mi350_us": dict(zip(("Q4", "Scale", "K1", "K2"), paper))}), flush=True)
+                              "fwht_over_k2": round(us["FWHT"] / us["K2"], 3) if "FWHT" in us else None,
+                              "paper_mi350_us": dict(zip(("Q4", "Scale", "K1", "K2", "FWHT"), paper))}), flush=True)
             del Xs, x0
 
 

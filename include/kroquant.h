@@ -149,6 +149,15 @@ kq_status_t kroquant_scale_quantize(const void *X, int64_t tokens, int d, const 
 kq_status_t kroquant_mxfp4_quantize(const void *X, int64_t tokens, int d, uint8_t *q_packed,
                                     uint8_t *scales, void *stream);
 
+/* Section 4.4 "FWHT": the full-d comparison transform  y = x H_d / sqrt(d)  (normalised
+ * Walsh-Hadamard over the whole row; d a power of two, 32 <= d <= 16384, else KQ_ERR_SHAPE) followed
+ * by the same MXFP4 encoder; row-major scales.  The _transform_f32 form exports the pre-rounding
+ * values (DEVICE float [tokens][d]). */
+kq_status_t kroquant_fwht_quantize(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                   uint8_t *q_packed, uint8_t *scales, void *stream);
+kq_status_t kroquant_fwht_transform_f32(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                        float *Y, void *stream);
+
 /* Debug/parity export of the pre-rounding values: Y[tokens][d] (DEVICE float) =
  * X T, produced by the same device code as kroquant_quantize_path up to the
  * encoder. */

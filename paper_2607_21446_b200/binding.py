@@ -23,6 +23,7 @@ EXPORTS = [
     "kroquant_factors_create", "kroquant_factors_create_lu", "kroquant_factors_create_dense",
     "kroquant_factors_destroy", "kroquant_quantize_ex", "kroquant_transform_f32_ex",
     "kroquant_scale_quantize_ex", "kroquant_mxfp4_quantize_ex", "kroquant_quantize_dual",
+    "kroquant_fwht_quantize", "kroquant_fwht_transform_f32",
     "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize",
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
@@ -57,6 +58,8 @@ def load_library() -> C.CDLL:
     L.kroquant_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, i32, vp]
     L.kroquant_transform_f32_ex.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
     L.kroquant_quantize_dual.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp]
+    L.kroquant_fwht_quantize.argtypes = [vp, i32, i64, i32, vp, vp, vp]
+    L.kroquant_fwht_transform_f32.argtypes = [vp, i32, i64, i32, vp, vp]
     L.kroquant_scale_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp]
     L.kroquant_mxfp4_quantize_ex.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
     L.kroquant_factors_destroy.argtypes = [vp]
@@ -207,6 +210,27 @@ def kroquant_quantize_dual(X: torch.Tensor, factors: Factors, q_packed=None, sca
                                                  _ptr(scales), SCALE_LAYOUTS[scale_layout], _ptr(AT),
                                                  C.c_void_p(_stream(stream))), "kroquant_quantize_dual")
     return q_packed, scales, AT
+
+
+def kroquant_fwht_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=None):
+    """Full-d Walsh-Hadamard comparison quantizer (d a power of two, 32..16384)."""
+    tokens, d = _x_shape(X)
+    if q_packed is None:
+        q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
+    if scales is None:
+        scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
+    _check(load_library().kroquant_fwht_quantize(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(q_packed), _ptr(scales),
+                                                 C.c_void_p(_stream(stream))), "kroquant_fwht_quantize")
+    return q_packed, scales
+
+
+def kroquant_fwht_transform_f32(X: torch.Tensor, Y=None, stream=None):
+    tokens, d = _x_shape(X)
+    if Y is None:
+        Y = torch.empty((tokens, d), dtype=torch.float32, device=X.device)
+    _check(load_library().kroquant_fwht_transform_f32(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(Y),
+                                                      C.c_void_p(_stream(stream))), "kroquant_fwht_transform_f32")
+    return Y
 
 
 def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, scales=None, stream=None,

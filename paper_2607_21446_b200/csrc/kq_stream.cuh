@@ -9,6 +9,7 @@
 //                                       factor by factor (Section 3.2 / 3.5)
 //   transform_stream        the butterfly alone, float output (parity export)
 //   dequantize_stream       decode (+ optional inverse butterfly, Section 3.2)
+//   fwht_quantize           full-d Walsh-Hadamard + encoder (the paper's FWHT comparison)
 #pragma once
 #include "kq_common.cuh"
 
@@ -194,6 +195,116 @@ scale_quantize_rows(const uint4* __restrict__ X, int64_t tokens, int quads_per_r
             st_stream_4(q_packed + q, codes);
             if (quad == 0)
                 scales[TILED ? tiled_scale_index(rr, p >> 2, (quads_per_row + 15) >> 4) : (q >> 2)] = (uint8_t)S;
+        }
+    }
+}
+
+// Full-d fast Walsh-Hadamard transform + MXFP4 (the paper's "FWHT" comparison, Section 4.4):
+// y = x H_d / sqrt(d), H_d[r][c] = (-1)^popcount(r & c), d a power of two, 32 <= d <= 16384.
+// Thread t of a row owns channels 8t..8t+7 (and, for d = 16384, d/2 + 8t.. as a second group):
+// index bits 0-2 are butterflied in registers, bits 3-7 by warp shuffles, the bits above by
+// exchanging the eight values through shared memory once per bit.  A CTA holds
+// blockDim.x / (threads per row) rows at a time.  Unlike the block-diagonal transforms this needs
+// log2(d) passes over the row; it is a comparison kernel, not tuned beyond coalesced I/O.
+template <bool XF16, bool WRITE_Y>
+__global__ void __launch_bounds__(1024)
+fwht_quantize(const uint4* __restrict__ X, int64_t tokens, int d, float norm,
+              uint32_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y) {
+    __shared__ float xch[1024 * 8];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const bool two_groups = d > 8192;                     // 16 elements per thread
+    const int tpr = two_groups ? 1024 : d / 8;            // threads per row
+    const int rows_per_cta = blockDim.x / tpr;
+    const int t = threadIdx.x % tpr;                      // thread inside the row
+    const int row_in_cta = threadIdx.x / tpr;
+    const int quads_per_row = d / 8;
+    const int n_groups = two_groups ? 2 : 1;
+    int log_tpr = 0;
+    while ((1 << log_tpr) < tpr) ++log_tpr;
+    const int64_t n_row_groups = (tokens + rows_per_cta - 1) / rows_per_cta;
+    for (int64_t rg = blockIdx.x; rg < n_row_groups; rg += gridDim.x) {
+        const int64_t row = rg * rows_per_cta + row_in_cta;
+        const bool live = row < tokens;
+        float v[2][8];
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            if (g < n_groups) {
+                const uint4 raw = live ? ld_stream_16(X + row * quads_per_row + g * (quads_per_row / 2) + t)
+                                       : make_uint4(0u, 0u, 0u, 0u);
+                widen8_any<XF16>(raw, v[g]);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            if (g >= n_groups) continue;
+            // index bits 0..2: inside the thread
+#pragma unroll
+            for (int b = 0; b < 3; ++b)
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (!(i & (1 << b))) {
+                        const float a = v[g][i], c = v[g][i | (1 << b)];
+                        v[g][i] = a + c;
+                        v[g][i | (1 << b)] = a - c;
+                    }
+            // index bits 3..7: across lanes (only those inside the row when a row has < 32 threads)
+            const int lane_bits = log_tpr < 5 ? log_tpr : 5;
+            for (int b = 0; b < lane_bits; ++b) {
+                const bool upper = (t >> b) & 1;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float o = __shfl_xor_sync(0xFFFFFFFFu, v[g][i], 1 << b);
+                    v[g][i] = upper ? o - v[g][i] : v[g][i] + o;
+                }
+            }
+            // index bits 8 and up: across warps, through shared memory
+            for (int b = 5; b < log_tpr; ++b) {
+                __syncthreads();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) xch[i * 1024 + threadIdx.x] = v[g][i];
+                __syncthreads();
+                const bool upper = (t >> b) & 1;
+                const int partner = threadIdx.x ^ (1 << b);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float o = xch[i * 1024 + partner];
+                    v[g][i] = upper ? o - v[g][i] : v[g][i] + o;
+                }
+            }
+        }
+        if (two_groups) {                                   // top index bit: between the two groups
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float a = v[0][i], c = v[1][i];
+                v[0][i] = a + c;
+                v[1][i] = a - c;
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < 2; ++g) {
+            if (g >= n_groups) continue;
+            float y[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) y[i] = v[g][i] * norm;
+            const int64_t q = row * quads_per_row + g * (quads_per_row / 2) + t;
+            if (WRITE_Y) {
+                if (live) {
+                    float4* yp = reinterpret_cast<float4*>(Y) + 2 * q;
+                    yp[0] = make_float4(y[0], y[1], y[2], y[3]);
+                    yp[1] = make_float4(y[4], y[5], y[6], y[7]);
+                }
+            } else {
+                float amax = absmax8(y);
+                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+                uint32_t S;
+                const uint32_t codes = encode8(y, amax, S);
+                if (live) {
+                    st_stream_4(q_packed + q, codes);
+                    if ((t & 3) == 0) scales[q >> 2] = (uint8_t)S;
+                }
+            }
         }
     }
 }

@@ -591,6 +591,59 @@ kq_status_t kroquant_mxfp4_quantize(const void* X, int64_t tokens, int d, uint8_
     return kroquant_mxfp4_quantize_ex(X, KQ_X_BF16, tokens, d, q_packed, scales, KQ_SCALES_ROWMAJOR, stream);
 }
 
+static kq_status_t run_fwht(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, uint8_t* q_packed,
+                            uint8_t* scales, float* Y, void* stream) {
+    if (!X || (!Y && (!q_packed || !scales))) return KQ_ERR_NULL;
+    if (tokens < 0 || d < 32 || d > 16384 || (d & (d - 1))) return KQ_ERR_SHAPE;
+    if (!aligned16(X) || (Y ? !aligned16(Y) : !aligned16(q_packed))) return KQ_ERR_ALIGN;
+    if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
+    if (tokens == 0) return KQ_OK;
+    const int sms = sm_count();
+    if (sms <= 0) return KQ_ERR_CUDA;
+    const int tpr = d > 8192 ? 1024 : d / 8;
+    const int threads = tpr < 256 ? 256 : tpr;
+    const int rows_per_cta = threads / tpr;
+    const int64_t groups = (tokens + rows_per_cta - 1) / rows_per_cta;
+    const int64_t cap = (int64_t)sms * (2048 / threads);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(groups < cap ? groups : cap));
+    cfg.blockDim = dim3(threads);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
+    const float norm = (float)(1.0 / std::sqrt((double)d));
+    const uint4* x4 = reinterpret_cast<const uint4*>(X);
+    uint32_t* q32 = reinterpret_cast<uint32_t*>(q_packed);
+    const bool xf16 = x_dtype == KQ_X_FP16;
+    cudaError_t err;
+    if (Y)
+        err = xf16 ? cudaLaunchKernelEx(&cfg, kq::fwht_quantize<true, true>, x4, tokens, d, norm, q32, scales, Y)
+                   : cudaLaunchKernelEx(&cfg, kq::fwht_quantize<false, true>, x4, tokens, d, norm, q32, scales, Y);
+    else
+        err = xf16 ? cudaLaunchKernelEx(&cfg, kq::fwht_quantize<true, false>, x4, tokens, d, norm, q32, scales, Y)
+                   : cudaLaunchKernelEx(&cfg, kq::fwht_quantize<false, false>, x4, tokens, d, norm, q32, scales, Y);
+    if (err != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KQ_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
+}
+
+kq_status_t kroquant_fwht_quantize(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, uint8_t* q_packed,
+                                   uint8_t* scales, void* stream) {
+    return run_fwht(X, x_dtype, tokens, d, q_packed, scales, nullptr, stream);
+}
+
+kq_status_t kroquant_fwht_transform_f32(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, float* Y,
+                                        void* stream) {
+    if (!Y) return KQ_ERR_NULL;
+    return run_fwht(X, x_dtype, tokens, d, nullptr, nullptr, Y, stream);
+}
+
 kq_status_t kroquant_dequantize(const uint8_t* q_packed, const uint8_t* scales, int64_t tokens, int d,
                                 const kroquant_factors_t* f, void* out, kq_dtype_t out_dtype, void* stream) {
     if (!q_packed || !scales || !out) return KQ_ERR_NULL;

@@ -149,3 +149,28 @@ def test_pixart_shaped_fp16_full_size(B):
     qo, so, Y = co.quantize(Xb, G, "fp16")
     print(P.check_values(Yg.cpu().numpy(), Y, "fp16"),
           P.check_codes(q.cpu().numpy(), s.cpu().numpy(), qo, so, Y, exact=False, x_dtype="fp16"))
+
+
+# ---- full-d Walsh-Hadamard comparison kernel -------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+@pytest.mark.parametrize("tokens,d", [(1, 32), (70, 64), (33, 256), (130, 1024), (37, 4096), (9, 8192), (5, 16384)])
+def test_fwht_quantize(B, dtype, tokens, d):
+    Xb = W.gen_activations(spec(tokens, d, seed=d + tokens), dtype)
+    X = dev(Xb, dtype)
+    q, s = B.kroquant_fwht_quantize(X)
+    Yg = B.kroquant_fwht_transform_f32(X)
+    qo, so, Y = co.hadamard_quantize(Xb, dtype)
+    print(d, P.check_values(Yg.cpu().numpy(), Y, dtype))
+    P.check_codes(q.cpu().numpy(), s.cpu().numpy(), qo, so, Y, exact=False, x_dtype=dtype)
+
+
+def test_fwht_rejects_other_sizes(B):
+    import ctypes as C
+    L = B.load_library()
+    X = torch.zeros((4, 96), dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros((4, 48), dtype=torch.uint8, device="cuda")
+    s = torch.zeros((4, 3), dtype=torch.uint8, device="cuda")
+    args = lambda d: (C.c_void_p(X.data_ptr()), 0, 4, d, C.c_void_p(q.data_ptr()), C.c_void_p(s.data_ptr()), None)
+    assert L.kroquant_fwht_quantize(*args(96)) == 2          # not a power of two
+    assert L.kroquant_fwht_quantize(*args(16)) == 2
+    assert L.kroquant_fwht_quantize(*args(32768)) == 2
