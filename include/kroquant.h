@@ -57,7 +57,8 @@ typedef enum { KQ_X_BF16 = 0, KQ_X_FP16 = 1 } kq_xdtype_t;
  * tensor-core GEMMs read (the consumer of the paper's W4A4 product, Section 3.4): tiles of 128 rows x
  * 4 blocks = 512 bytes, row-tile-major; byte of (t, j) at
  *   ((t/128) * ceil(d/128) + j/4) * 512 + (t%32)*16 + ((t%128)/32)*4 + j%4.
- * The buffer then holds ceil(tokens/128)*128 * ceil(d/128)*4 bytes; padding bytes are not written.
+ * The buffer then holds ceil(tokens/128)*128 * ceil(d/128)*4 bytes (16-byte aligned for per-block
+ * factor sets); padding bytes are left untouched or written as 0.
  * kroquant_dequantize reads ROWMAJOR only. */
 typedef enum { KQ_SCALES_ROWMAJOR = 0, KQ_SCALES_TILED_128X4 = 1 } kq_scale_layout_t;
 

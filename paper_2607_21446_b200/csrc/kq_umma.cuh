@@ -266,7 +266,7 @@ __device__ __forceinline__ void encode_block_regs(uint32_t (&acc)[32], int e, ui
 //     d/2) and scale bytes (128 x 4) are staged in shared memory and written once per
 //     group, because 16-byte and 1-byte pieces scattered at a row pitch cost one L2 write
 //     transaction each (measured: they halve the kernel's throughput).
-constexpr int kPbCols = 4;
+constexpr int kPbCols = 4;   // = the column count of the consumer's 128 x 4 scale tile
 struct UmmaProblem {
     int64_t n_rows;      // PB=false: tokens*d/32 ; PB=true: tokens
     int64_t n_units;     // PB=false: 128-row tiles ; PB=true: column groups x token tiles
@@ -476,7 +476,13 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
                              ::"r"(st_codes + 64u * r + 16u * (uint32_t)(c ^ ((r >> 1) & 3))),
                                "r"(codes.x), "r"(codes.y), "r"(codes.z), "r"(codes.w) : "memory");
-                asm volatile("st.shared.u8 [%0], %1;" ::"r"(st_scale + 4u * r + c), "r"(S) : "memory");
+                // scale byte: staged row-major [r][c], or directly in the order of the consumer's 128 x 4
+                // tile (a unit IS one such tile): (r % 32) * 16 + (r / 32) * 4 + c.  A column beyond d/32
+                // (ragged last group) stages 0.
+                const uint32_t S_st = j < prob.blocks_per_row ? S : 0u;
+                const uint32_t s_off = prob.tiled_scales ? (uint32_t)((r & 31) * 16 + (r >> 5) * 4 + c)
+                                                         : (uint32_t)(4 * r + c);
+                asm volatile("st.shared.u8 [%0], %1;" ::"r"(st_scale + s_off), "r"(S_st) : "memory");
                 if (c == kPbCols - 1) {
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     named_barrier_sync(1, 128);
@@ -484,18 +490,28 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         tma_store_2d(&tmap_q, st_codes, 16 * kPbCols * jg, tt * kTileRows);   // clips ragged edges
                         bulk_commit_group();
                     }
-                    // scale bytes: lane l writes byte (l & 3) of row 8i + (l >> 2): 8 rows x 4 bytes per store
+                    if (prob.tiled_scales) {
+                        // the unit's 512 scale bytes are one contiguous tile of the output: one warp, 16 B per lane
+                        if (quarter == 0) {
+                            uint4 v;
+                            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                         : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(st_scale + 16u * lane) : "memory");
+                            const int64_t tile = (int64_t)tt * ((prob.blocks_per_row + kPbCols - 1) / kPbCols) + jg;
+                            reinterpret_cast<uint4*>(scales + tile * 512)[lane] = v;
+                        }
+                    } else {
+                        // row-major: lane l writes byte (l & 3) of row 8i + (l >> 2): 8 rows x 4 bytes per store
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int rr = quarter * 32 + i * 8 + (lane >> 2);
-                        const int cc = lane & 3;
-                        const int64_t t = (int64_t)tt * kTileRows + rr;
-                        const int jj = jg * kPbCols + cc;
-                        uint32_t v;
-                        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(st_scale + 4u * rr + cc) : "memory");
-                        if (t < prob.n_rows && jj < prob.blocks_per_row)
-                            scales[prob.tiled_scales ? tiled_scale_index(t, jj, (prob.blocks_per_row + 3) >> 2)
-                                                     : t * prob.blocks_per_row + jj] = (uint8_t)v;
+                        for (int i = 0; i < 4; ++i) {
+                            const int rr = quarter * 32 + i * 8 + (lane >> 2);
+                            const int cc = lane & 3;
+                            const int64_t t = (int64_t)tt * kTileRows + rr;
+                            const int jj = jg * kPbCols + cc;
+                            uint32_t v;
+                            asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(st_scale + 4u * rr + cc) : "memory");
+                            if (t < prob.n_rows && jj < prob.blocks_per_row)
+                                scales[t * prob.blocks_per_row + jj] = (uint8_t)v;
+                        }
                     }
                 }
             } else {
