@@ -167,6 +167,22 @@ def gen_dense_blocks(seed: int, n_sets: int = 1) -> np.ndarray:
     return out
 
 
+def gen_weights(seed: int, o: int, d: int) -> np.ndarray:
+    """bf16 bit patterns of a synthetic linear-layer weight ``W[o, d]``: N(0, 1/d) entries with a
+    log-normal per-input-channel gain (sigma 0.5), the kind of channel imbalance smoothing and
+    rotations are meant to even out.  Used by the calibration workload only."""
+    rng = np.random.default_rng(seed + 3000)
+    w = rng.standard_normal((o, d), dtype=np.float32) / np.float32(math.sqrt(d))
+    gain = np.exp(rng.normal(0.0, 0.5, size=d)).astype(np.float32)
+    return f32_to_bf16_bits(w * gain[None, :])
+
+
+def calib_spec(rows: int, d: int, seed: int = 5) -> ActivationSpec:
+    """Calibration activations: the rows of all samples stacked, 1 % outlier channels x 50."""
+    return ActivationSpec(f"calib-{rows}x{d}", rows, d, seed,
+                          outlier_channels=max(1, round(0.01 * d)), outlier_gain=50.0)
+
+
 def tiny_spec() -> ActivationSpec:
     return ActivationSpec("tiny", 256, 1152, seed=0, outlier_channels=12,
                           outlier_gain=50.0, spike_rows=4, spike_gain=8.0)
