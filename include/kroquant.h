@@ -177,6 +177,55 @@ kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes,
  * launches with programmatic stream serialization.  Process-wide. */
 kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl);
 
+/* ---- Layer-wise calibration of the transform (Section 3.3; set-up of Appendix D) ----
+ *
+ * Minimises, over the parameters theta = (a_k, b_k, c_k), k = 1..5, of every factor set,
+ *     L = L_out + lambda_A L_A + lambda_W L_W,
+ *     L_out = ||Q(A T) Q(W T^-T)^T - A W^T||_F^2 / (M o),
+ *     L_A = ||Q(A T) - A T||_F^2 / (M d),   L_W = ||Q(W T^-T) - W T^-T||_F^2 / (o d),
+ * with Adam (beta1 0.9, beta2 0.999, eps 1e-8, bias correction) from the Hadamard
+ * initialisation (a, b, c) = (1/sqrt 2, 1/sqrt 2, 1).  Q is MXFP4 quantise-then-dequantise;
+ * in the backward pass it has the identity Jacobian (straight-through), and in L_A and L_W the
+ * quantised tensor is a constant target, so dL_A/d(AT) = 2 (AT - Q(AT)) / (M d).
+ *
+ * A [M][d] and W [o][d] are DEVICE bf16, row-major, 16-byte aligned, owned by the caller and
+ * must stay valid and unchanged for the life of the object.  M is the number of calibration
+ * rows (all samples stacked), a multiple of 8; o and d are multiples of 32; n_sets is 1 (one
+ * factor set for the layer) or d/32 (one per block).  create allocates all work space
+ * (about 14 M d + 10 M o bytes), forms A W^T, evaluates the three terms at the initialisation and
+ * sets lambda_A = L_out/L_A, lambda_W = L_out/L_W there; it synchronizes `stream`.  The object is
+ * tied to the device that was current at creation.  All three contractions of a step run on the
+ * tensor cores in bf16 with fp32 accumulation (exact products for the forward one); the output
+ * error is rounded to bf16 once before the two backward contractions. */
+typedef struct kroquant_calib kroquant_calib_t;
+
+kq_status_t kroquant_calib_create(const void *A, const void *W, int64_t M, int o, int d, int n_sets,
+                                  void *stream, kroquant_calib_t **out);
+void kroquant_calib_destroy(kroquant_calib_t *c);
+
+/* theta_host: [n_sets][5][3] floats (a, b, c).  set also clears the optimiser state and the step count. */
+kq_status_t kroquant_calib_set_theta(kroquant_calib_t *c, const float *theta_host);
+kq_status_t kroquant_calib_get_theta(const kroquant_calib_t *c, float *theta_host_out);
+/* lam_host: {lambda_A, lambda_W}. */
+kq_status_t kroquant_calib_set_lambdas(kroquant_calib_t *c, const float *lam_host);
+kq_status_t kroquant_calib_get_lambdas(const kroquant_calib_t *c, float *lam_host_out);
+/* The factors G_k = L_k U_k of the current parameters, [n_sets][5][2][2] floats, ready for
+ * kroquant_factors_create. */
+kq_status_t kroquant_calib_get_factors(const kroquant_calib_t *c, float *G_host_out);
+
+/* Evaluate at the current parameters without changing them: losses_host_out[3] = {L_out, L_A, L_W}
+ * (doubles), grad_host_out [n_sets][5][3] floats = dL/dtheta (may be NULL: forward pass only).
+ * Synchronizes `stream`. */
+kq_status_t kroquant_calib_loss_grad(kroquant_calib_t *c, double *losses_host_out, float *grad_host_out,
+                                     void *stream);
+
+/* `steps` Adam steps (1 <= steps <= 4096) with learning rate lr.  history_host_out, if not NULL,
+ * receives [steps + 1][3] doubles: the three terms before each step and, in the last row, at the
+ * final parameters (one more forward pass).  Asynchronous on `stream` if history_host_out is NULL,
+ * otherwise synchronizes it. */
+kq_status_t kroquant_calib_run(kroquant_calib_t *c, int steps, float lr, double *history_host_out,
+                               void *stream);
+
 /* Number of kernels this library has launched in the calling process (all streams). */
 int64_t kroquant_launch_count(void);
 

@@ -29,6 +29,9 @@ EXPORTS = [
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
     "kroquant_debug_set_umma_config", "kroquant_launch_count", "kroquant_last_device_error",
     "kroquant_status_string",
+    "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
+    "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
+    "kroquant_calib_loss_grad", "kroquant_calib_run",
 ]
 
 
@@ -79,6 +82,13 @@ def load_library() -> C.CDLL:
     L.kroquant_last_device_error.argtypes = [vp, C.POINTER(i32)]
     L.kroquant_status_string.argtypes = [i32]
     L.kroquant_status_string.restype = C.c_char_p
+    L.kroquant_calib_create.argtypes = [vp, vp, i64, i32, i32, i32, vp, C.POINTER(vp)]
+    L.kroquant_calib_destroy.argtypes = [vp]
+    L.kroquant_calib_destroy.restype = None
+    for name in ("set_theta", "get_theta", "set_lambdas", "get_lambdas", "get_factors"):
+        getattr(L, "kroquant_calib_" + name).argtypes = [vp, vp]
+    L.kroquant_calib_loss_grad.argtypes = [vp, vp, vp, vp]
+    L.kroquant_calib_run.argtypes = [vp, i32, C.c_float, vp, vp]
     _lib = L
     return L
 
@@ -360,3 +370,79 @@ class HostPipeline:
         self.h2d.synchronize()
         self.compute.synchronize()
         self.d2h.synchronize()
+
+
+class Calibrator:
+    """Handle of a kroquant_calib_t: layer-wise calibration of the transform (Section 3.3).
+
+    A [M, d] and W [o, d] are contiguous CUDA bfloat16 tensors; they are kept alive by this object.
+    """
+
+    def __init__(self, A: torch.Tensor, W: torch.Tensor, n_sets: int = 1, stream=None):
+        for t in (A, W):
+            if t.dim() != 2 or t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+                raise ValueError("A and W must be contiguous 2-D CUDA bfloat16 tensors")
+        if A.shape[1] != W.shape[1]:
+            raise ValueError("A [M, d] and W [o, d] must share d")
+        self.A, self.W, self.n_sets = A, W, n_sets
+        self.M, self.d, self.o = A.shape[0], A.shape[1], W.shape[0]
+        out = C.c_void_p()
+        _check(load_library().kroquant_calib_create(_ptr(A), _ptr(W), self.M, self.o, self.d, n_sets,
+                                                    _stream(stream), C.byref(out)), "kroquant_calib_create")
+        self._h = out
+
+    def destroy(self) -> None:
+        if getattr(self, "_h", None):
+            load_library().kroquant_calib_destroy(self._h)
+            self._h = None
+
+    __del__ = destroy
+
+    def _get(self, name: str, shape) -> np.ndarray:
+        out = np.empty(shape, np.float32)
+        _check(getattr(load_library(), "kroquant_calib_get_" + name)(self._h, out.ctypes.data_as(C.c_void_p)),
+               "kroquant_calib_get_" + name)
+        return out
+
+    @property
+    def theta(self) -> np.ndarray:
+        return self._get("theta", (self.n_sets, 5, 3))
+
+    @theta.setter
+    def theta(self, value) -> None:
+        v = np.ascontiguousarray(value, dtype=np.float32)
+        if v.shape != (self.n_sets, 5, 3):
+            raise ValueError("theta must have shape [n_sets, 5, 3]")
+        _check(load_library().kroquant_calib_set_theta(self._h, v.ctypes.data_as(C.c_void_p)), "kroquant_calib_set_theta")
+
+    @property
+    def lambdas(self) -> np.ndarray:
+        return self._get("lambdas", (2,))
+
+    @lambdas.setter
+    def lambdas(self, value) -> None:
+        v = np.ascontiguousarray(value, dtype=np.float32)
+        if v.shape != (2,):
+            raise ValueError("lambdas = (lambda_A, lambda_W)")
+        _check(load_library().kroquant_calib_set_lambdas(self._h, v.ctypes.data_as(C.c_void_p)),
+               "kroquant_calib_set_lambdas")
+
+    def factors(self) -> np.ndarray:
+        """G [n_sets, 5, 2, 2] of the current parameters (input of Factors.create)."""
+        return self._get("factors", (self.n_sets, 5, 2, 2))
+
+    def loss_grad(self, grad: bool = True, stream=None):
+        """-> (losses float64 [3] = (L_out, L_A, L_W), dL/dtheta float32 [n_sets, 5, 3] or None)."""
+        losses = np.empty(3, np.float64)
+        g = np.empty((self.n_sets, 5, 3), np.float32) if grad else None
+        _check(load_library().kroquant_calib_loss_grad(self._h, losses.ctypes.data_as(C.c_void_p),
+                                                       g.ctypes.data_as(C.c_void_p) if grad else None,
+                                                       _stream(stream)), "kroquant_calib_loss_grad")
+        return losses, g
+
+    def run(self, steps: int, lr: float = 1e-2, history: bool = True, stream=None):
+        """`steps` Adam steps; -> history float64 [steps + 1, 3] (or None, asynchronous)."""
+        h = np.empty((steps + 1, 3), np.float64) if history else None
+        _check(load_library().kroquant_calib_run(self._h, steps, lr, h.ctypes.data_as(C.c_void_p) if history else None,
+                                                 _stream(stream)), "kroquant_calib_run")
+        return h

@@ -1,0 +1,308 @@
+// CUDA-core kernels of the calibration loop (paper Section 3.3; optimiser set-up of Appendix D).
+//
+//   calib_build_blocks  theta (a,b,c per factor) -> K = G1 (x) .. (x) G5 and P = K^-T, dense 32x32
+//   calib_fakequant     V = X_j B_j per 32-channel block, Vq = Q(V) as bf16, R = V - Vq, sum R^2
+//   transpose_bf16      [R][C] -> [C][R]
+//   calib_block_grad    partial sums of X_j^T G_j over chunks of rows
+//   calib_param_step    block gradients -> d/d(a,b,c) through the Kronecker and LU structure, Adam
+//   calib_lambdas       lambda_A = L_out/L_A, lambda_W = L_out/L_W at the initialisation
+//
+// The three big contractions in between are the tensor-core GEMM of kq_gemm.cuh.
+#pragma once
+#include <cuda_bf16.h>
+#include "kq_common.cuh"
+
+namespace kq {
+
+// ---- theta -> dense blocks -----------------------------------------------------------------
+// One CTA of 1024 threads per factor set; thread (r, c).  G_k = [[a, b], [a c, b c - 1/a]]
+// (Section 3.2, L_k U_k multiplied out); H_k = G_k^-T = [[1/a - b c, a c], [b, -a]] (det G_k = -1).
+// K[r][c] = prod_k G_k[bit(r)][bit(c)] with G_1 on the most significant index bit.
+__global__ void __launch_bounds__(1024)
+calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, float* __restrict__ Pout) {
+    const int s = blockIdx.x;
+    const int r = threadIdx.x >> 5, c = threadIdx.x & 31;
+    double k = 1.0, p = 1.0;
+#pragma unroll
+    for (int f = 0; f < 5; ++f) {
+        const double a = theta[(s * 5 + f) * 3 + 0], b = theta[(s * 5 + f) * 3 + 1], cc = theta[(s * 5 + f) * 3 + 2];
+        const int rb = (r >> (4 - f)) & 1, cb = (c >> (4 - f)) & 1;
+        const double g = rb == 0 ? (cb == 0 ? a : b) : (cb == 0 ? a * cc : b * cc - 1.0 / a);
+        const double h = rb == 0 ? (cb == 0 ? 1.0 / a - b * cc : a * cc) : (cb == 0 ? b : -a);
+        k *= g;
+        p *= h;
+    }
+    Kout[s * 1024 + threadIdx.x] = (float)k;
+    Pout[s * 1024 + threadIdx.x] = (float)p;
+}
+
+// ---- transform + fake quantisation ---------------------------------------------------------
+// grid (row groups, d/32); 128 threads; thread = one row of block column j.  The block matrix
+// sits in shared memory and is read as warp-wide broadcasts.  Q is the MXFP4 encoder of the
+// quantizer kernels followed by its decoder; Vq is exact in bf16.
+__device__ __forceinline__ float e2m1_nibble_value(uint32_t code) {
+    const uint32_t m = code & 7u;
+    const float mag = m < 2u ? 0.5f * (float)m : (float)(2u + (m & 1u)) * (float)(1u << ((m >> 1) - 1u)) * 0.5f;
+    return (code & 8u) ? -mag : mag;
+}
+
+__global__ void __launch_bounds__(128)
+calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int n_sets, int64_t rows, int d,
+                __nv_bfloat16* __restrict__ Vq, float* __restrict__ Res, double* __restrict__ sumsq) {
+    __shared__ __align__(16) float Bs[32][32];
+    __shared__ double red[4];
+    const int j = blockIdx.y;
+    const float* Bj = B + (size_t)(n_sets == 1 ? 0 : j) * 1024;
+    for (int i = threadIdx.x; i < 1024; i += 128) Bs[i >> 5][i & 31] = Bj[i];
+    __syncthreads();
+    double sq = 0.0;
+    for (int64_t row = (int64_t)blockIdx.x * 128 + threadIdx.x; row < rows; row += (int64_t)gridDim.x * 128) {
+        const uint4* xp = reinterpret_cast<const uint4*>(X + row * d + j * 32);
+        float x[32];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            float t[8];
+            widen8(ld_stream_16(xp + q), t);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[8 * q + i] = t[i];
+        }
+        float v[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) v[c] = 0.f;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4) {
+                const float4 b = *reinterpret_cast<const float4*>(&Bs[r][4 * c4]);
+                v[4 * c4 + 0] = fmaf(x[r], b.x, v[4 * c4 + 0]);
+                v[4 * c4 + 1] = fmaf(x[r], b.y, v[4 * c4 + 1]);
+                v[4 * c4 + 2] = fmaf(x[r], b.z, v[4 * c4 + 2]);
+                v[4 * c4 + 3] = fmaf(x[r], b.w, v[4 * c4 + 3]);
+            }
+        }
+        float amax = 0.f;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) amax = fmaxf(amax, fabsf(v[c]));
+        const uint32_t S = e8m0_from_amax(amax);
+        const float inv = inv_scale_from_e8m0(S), sc = scale_from_e8m0(S);
+        uint4* qp = reinterpret_cast<uint4*>(Vq + row * d + j * 32);
+        float4* rp = reinterpret_cast<float4*>(Res + row * d + j * 32);
+        float sq_row = 0.f;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const uint32_t codes = e2m1x8(v[8 * g] * inv, v[8 * g + 1] * inv, v[8 * g + 2] * inv, v[8 * g + 3] * inv,
+                                          v[8 * g + 4] * inv, v[8 * g + 5] * inv, v[8 * g + 6] * inv, v[8 * g + 7] * inv);
+            float qv[8], rr[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                qv[i] = e2m1_nibble_value(codes >> (4 * i)) * sc;
+                rr[i] = v[8 * g + i] - qv[i];
+                sq_row = fmaf(rr[i], rr[i], sq_row);
+            }
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(qv[2 * i], qv[2 * i + 1]);
+                w[i] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            qp[g] = make_uint4(w[0], w[1], w[2], w[3]);
+            rp[2 * g] = make_float4(rr[0], rr[1], rr[2], rr[3]);
+            rp[2 * g + 1] = make_float4(rr[4], rr[5], rr[6], rr[7]);
+        }
+        sq += (double)sq_row;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const double t = red[0] + red[1] + red[2] + red[3];
+        if (t != 0.0) atomicAdd(sumsq, t);
+    }
+}
+
+// ---- bf16 transpose: in [R][C] -> out [C][R]; 64 x 64 tiles, 256 threads ---------------------
+__global__ void __launch_bounds__(256)
+transpose_bf16(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, int64_t R, int64_t C) {
+    __shared__ uint16_t tile[64][66];
+    const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+    for (int i = ty; i < 64; i += 4)
+        if (r0 + i < R && c0 + tx < C) tile[i][tx] = in[(r0 + i) * C + c0 + tx];
+    __syncthreads();
+    for (int i = ty; i < 64; i += 4)
+        if (c0 + i < C && r0 + tx < R) out[(c0 + i) * R + r0 + tx] = tile[tx][i];
+}
+
+// ---- block gradients: part[chunk][j][32][32] = sum over the chunk's rows of x_j^T g_j ---------
+// grid (chunks, d/32); 256 threads = 4 row groups x 64; a thread owns a 4 x 4 patch of the
+// 32 x 32 result for its row group; tiles of 64 rows are staged in shared memory as fp32.
+constexpr int kGradTileRows = 64;
+__global__ void __launch_bounds__(256)
+calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, int64_t rows, int d,
+                 int64_t rows_per_chunk, float* __restrict__ part) {
+    __shared__ __align__(16) float xs[kGradTileRows][32];
+    __shared__ __align__(16) float gs[kGradTileRows][32];
+    const int j = blockIdx.y;
+    const int64_t r_begin = (int64_t)blockIdx.x * rows_per_chunk;
+    const int64_t r_end = r_begin + rows_per_chunk < rows ? r_begin + rows_per_chunk : rows;
+    const int grp = threadIdx.x >> 6;
+    const int r4 = ((threadIdx.x & 63) >> 3) * 4, c4 = (threadIdx.x & 7) * 4;
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    for (int64_t t0 = r_begin; t0 < r_end; t0 += kGradTileRows) {
+        // stage: thread -> (row = tid / 4, 8 channels = (tid % 4) * 8)
+        {
+            const int lr = threadIdx.x >> 2, ch = (threadIdx.x & 3) * 8;
+            const int64_t row = t0 + lr;
+            float xv[8];
+            float4 g0, g1;
+            if (row < r_end) {
+                widen8(ld_stream_16(X + row * d + j * 32 + ch), xv);
+                const float4* gp = reinterpret_cast<const float4*>(G + row * d + j * 32 + ch);
+                g0 = __ldg(gp);
+                g1 = __ldg(gp + 1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) xv[i] = 0.f;
+                g0 = g1 = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            *reinterpret_cast<float4*>(&xs[lr][ch]) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+            *reinterpret_cast<float4*>(&xs[lr][ch + 4]) = make_float4(xv[4], xv[5], xv[6], xv[7]);
+            *reinterpret_cast<float4*>(&gs[lr][ch]) = g0;
+            *reinterpret_cast<float4*>(&gs[lr][ch + 4]) = g1;
+        }
+        __syncthreads();
+#pragma unroll 4
+        for (int i = 0; i < kGradTileRows / 4; ++i) {
+            const int lr = grp * (kGradTileRows / 4) + i;
+            const float4 xa = *reinterpret_cast<const float4*>(&xs[lr][r4]);
+            const float4 ga = *reinterpret_cast<const float4*>(&gs[lr][c4]);
+            const float xv[4] = {xa.x, xa.y, xa.z, xa.w};
+            const float gv[4] = {ga.x, ga.y, ga.z, ga.w};
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(xv[a], gv[b], acc[a][b]);
+        }
+        __syncthreads();
+    }
+    // sum the four row groups through shared memory (reuse xs/gs: 2 x 8 KB = 4 x 1024 floats)
+    float* red = &xs[0][0];            // xs and gs are adjacent only by luck; use them separately
+    float* red2 = &gs[0][0];
+    float* mine = grp < 2 ? red + grp * 1024 : red2 + (grp - 2) * 1024;
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) mine[(r4 + a) * 32 + c4 + b] = acc[a][b];
+    __syncthreads();
+    float* dst = part + ((size_t)blockIdx.x * gridDim.y + j) * 1024;
+    for (int i = threadIdx.x; i < 1024; i += 256)
+        dst[i] = (red[i] + red[1024 + i]) + (red2[i] + red2[1024 + i]);
+}
+
+// ---- block gradients -> parameter gradients -> Adam -------------------------------------------
+// One CTA of 1024 threads per factor set; thread (R, C) first sums its entry of dK and dP over
+// the row chunks (and over all block columns when the set is shared).  For B = F_1 (x) .. (x) F_5,
+// d/dF_k[r][c] = sum over (R, C) with bit_k(R) = r, bit_k(C) = c of dB[R][C] * prod_{l != k} F_l[..].
+// Then d/d(a, b, c) by the closed-form derivatives of G_k and H_k = G_k^-T, and one Adam step
+// (beta1 0.9, beta2 0.999, eps 1e-8, bias correction) when do_update != 0.
+struct CalibStepArgs {
+    const float* partK; int chunksK;
+    const float* partP; int chunksP;
+    int nb, n_sets;
+    float* theta; float* adam_m; float* adam_v; float* grad_out;
+    float lr; int t; int do_update;
+};
+
+__global__ void __launch_bounds__(1024)
+calib_param_step(const CalibStepArgs a) {
+    __shared__ double bucket[2][5][2][2];
+    __shared__ double Gs[5][2][2], Hs[5][2][2];
+    __shared__ double th[5][3];          // the parameters as they were when the step began
+    const int s = blockIdx.x;
+    const int R = threadIdx.x >> 5, C = threadIdx.x & 31;
+    if (threadIdx.x < 40) (&bucket[0][0][0][0])[threadIdx.x] = 0.0;
+    if (threadIdx.x < 5) {
+        const int f = threadIdx.x;
+        const double aa = a.theta[(s * 5 + f) * 3 + 0], bb = a.theta[(s * 5 + f) * 3 + 1], cc = a.theta[(s * 5 + f) * 3 + 2];
+        th[f][0] = aa; th[f][1] = bb; th[f][2] = cc;
+        Gs[f][0][0] = aa; Gs[f][0][1] = bb; Gs[f][1][0] = aa * cc; Gs[f][1][1] = bb * cc - 1.0 / aa;
+        Hs[f][0][0] = 1.0 / aa - bb * cc; Hs[f][0][1] = aa * cc; Hs[f][1][0] = bb; Hs[f][1][1] = -aa;
+    }
+    double dk = 0.0, dp = 0.0;
+    const int j_begin = a.n_sets == 1 ? 0 : s, j_end = a.n_sets == 1 ? a.nb : s + 1;
+    for (int j = j_begin; j < j_end; ++j) {
+        for (int ch = 0; ch < a.chunksK; ++ch) dk += (double)a.partK[((size_t)ch * a.nb + j) * 1024 + threadIdx.x];
+        for (int ch = 0; ch < a.chunksP; ++ch) dp += (double)a.partP[((size_t)ch * a.nb + j) * 1024 + threadIdx.x];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+        double wg = 1.0, wh = 1.0;
+#pragma unroll
+        for (int l = 0; l < 5; ++l) {
+            if (l == k) continue;
+            const int rb = (R >> (4 - l)) & 1, cb = (C >> (4 - l)) & 1;
+            wg *= Gs[l][rb][cb];
+            wh *= Hs[l][rb][cb];
+        }
+        const int rk = (R >> (4 - k)) & 1, ck = (C >> (4 - k)) & 1;
+        // warp-level pre-reduction: within a warp R is fixed and C varies, so lanes with equal ck share a bucket
+        double vg = dk * wg, vh = dp * wh;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const double og = __shfl_xor_sync(0xFFFFFFFFu, vg, o), oh = __shfl_xor_sync(0xFFFFFFFFu, vh, o);
+            // lanes whose partner has the same bit k of C merge; the bit that distinguishes the two
+            // buckets is lane bit (4 - k): skip the exchange across it
+            if (o != (16 >> k)) { vg += og; vh += oh; }
+        }
+        // after the loop, lanes 0 and (16 >> k) hold the sums of the two ck classes
+        if (C == 0 || C == (16 >> k)) {
+            atomicAdd(&bucket[0][k][rk][ck], vg);
+            atomicAdd(&bucket[1][k][rk][ck], vh);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < 15) {
+        const int k = threadIdx.x / 3, which = threadIdx.x % 3;
+        const double aa = th[k][0], bb = th[k][1], cc = th[k][2];
+        const double (*dG)[2] = bucket[0][k];
+        const double (*dH)[2] = bucket[1][k];
+        double g;
+        if (which == 0)        // d/da: dG/da = [[1,0],[c,1/a^2]], dH/da = [[-1/a^2, c],[0,-1]]
+            g = dG[0][0] + cc * dG[1][0] + dG[1][1] / (aa * aa) - dH[0][0] / (aa * aa) + cc * dH[0][1] - dH[1][1];
+        else if (which == 1)   // d/db: dG/db = [[0,1],[0,c]], dH/db = [[-c,0],[1,0]]
+            g = dG[0][1] + cc * dG[1][1] - cc * dH[0][0] + dH[1][0];
+        else                   // d/dc: dG/dc = [[0,0],[a,b]], dH/dc = [[-b,a],[0,0]]
+            g = aa * dG[1][0] + bb * dG[1][1] - bb * dH[0][0] + aa * dH[0][1];
+        const int idx = (s * 5 + k) * 3 + which;
+        if (a.grad_out) a.grad_out[idx] = (float)g;
+        if (a.do_update) {
+            const double b1 = 0.9, b2 = 0.999, eps = 1e-8;
+            const double m = b1 * (double)a.adam_m[idx] + (1.0 - b1) * g;
+            const double v = b2 * (double)a.adam_v[idx] + (1.0 - b2) * g * g;
+            a.adam_m[idx] = (float)m;
+            a.adam_v[idx] = (float)v;
+            const double mhat = m / (1.0 - pow(b1, (double)a.t));
+            const double vhat = v / (1.0 - pow(b2, (double)a.t));
+            const double th = (which == 0 ? aa : which == 1 ? bb : cc) - (double)a.lr * mhat / (sqrt(vhat) + eps);
+            a.theta[idx] = (float)th;
+        }
+    }
+}
+
+// lambdas from the three loss sums at the initialisation: losses are sums of squares still to be
+// divided by their element counts (n_out, n_a, n_w)
+__global__ void calib_lambdas(const double* __restrict__ sums, double n_out, double n_a, double n_w, float* __restrict__ lam) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        const double lo = sums[0] / n_out, la = sums[1] / n_a, lw = sums[2] / n_w;
+        lam[0] = la > 0.0 ? (float)(lo / la) : 0.f;
+        lam[1] = lw > 0.0 ? (float)(lo / lw) : 0.f;
+    }
+}
+
+}  // namespace kq

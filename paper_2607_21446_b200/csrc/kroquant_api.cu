@@ -720,3 +720,5 @@ const char* kroquant_status_string(kq_status_t s) {
 }
 
 }  // extern "C"
+
+#include "kroquant_calib_api.cuh"

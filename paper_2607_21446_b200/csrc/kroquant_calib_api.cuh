@@ -1,0 +1,335 @@
+// Host side of the calibration loop (declarations and contract: include/kroquant.h).
+// Included at the end of kroquant_api.cu: one translation unit, one device error word.
+#pragma once
+#include "kq_calib.cuh"
+#include "kq_gemm.cuh"
+
+struct kroquant_calib {
+    int device = -1;
+    int64_t M = 0;
+    int o = 0, d = 0, nb = 0, n_sets = 0;
+    const uint16_t* A = nullptr;       // caller-owned
+    const uint16_t* W = nullptr;
+    uint8_t* pool = nullptr;           // one allocation; everything below points into it
+    float *theta = nullptr, *adam_m = nullptr, *adam_v = nullptr, *grad = nullptr, *lam = nullptr;
+    float *Kd = nullptr, *Pd = nullptr;
+    __nv_bfloat16 *Yq = nullptr, *YqT = nullptr, *Zq = nullptr, *ZqT = nullptr, *dO = nullptr, *dOT = nullptr;
+    float *ResY = nullptr, *ResZ = nullptr, *R = nullptr, *dY = nullptr, *dZ = nullptr;
+    float *partK = nullptr, *partP = nullptr;
+    int chunksK = 0, chunksP = 0;
+    int64_t rpcK = 0, rpcP = 0;
+    double* sums = nullptr;            // [3] sums of squares of the evaluation in flight
+    double* hist = nullptr;            // [kHistCap][3]
+    int t = 0;                         // Adam steps taken
+    CUtensorMap tm_A_a, tm_W_b, tm_Yq_a, tm_Zq_b, tm_dO_a, tm_ZqT_b, tm_dOT_a, tm_YqT_b;
+};
+
+namespace {
+
+constexpr int kHistCap = 4097;
+
+// [rows][K] bf16 row-major as a GEMM operand: box = 64 K-elements (128 bytes) x box_rows rows
+bool make_operand_map(CUtensorMap* tm, const void* ptr, int64_t rows, int64_t K, int box_rows) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kq::kGemmBK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, int M, int N, int K, const float* aux,
+                        int64_t ld_aux, const float* coef_ptr, float coef_mul, float out_scale, float* out_f32,
+                        __nv_bfloat16* out_bf16, int64_t ld_out, double* sumsq, cudaStream_t st) {
+    static std::atomic<int> attr_done{0};
+    if (!attr_done.load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kq::gemm_nt_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kGemmDynBytes) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return KQ_ERR_CUDA;
+        }
+        attr_done.store(1, std::memory_order_release);
+    }
+    kq::GemmProblem p;
+    p.M = M; p.N = N; p.K = K;
+    p.tiles_m = (M + kq::kGemmBM - 1) / kq::kGemmBM;
+    p.tiles_n = (N + kq::kGemmBN - 1) / kq::kGemmBN;
+    p.k_blocks = (K + kq::kGemmBK - 1) / kq::kGemmBK;
+    p.aux = aux; p.ld_aux = ld_aux; p.coef_ptr = coef_ptr; p.coef_mul = coef_mul; p.out_scale = out_scale;
+    p.out_f32 = out_f32; p.out_bf16 = out_bf16; p.ld_out = ld_out; p.sumsq = sumsq;
+    const int sms = sm_count();
+    if (sms <= 0) return KQ_ERR_CUDA;
+    const int tiles = p.tiles_m * p.tiles_n;
+    const int grid = tiles < sms ? tiles : sms;
+    kq::gemm_nt_umma<<<grid, kq::kGemmThreads, kq::kGemmDynBytes, st>>>(ta, tb, p);
+    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
+}
+
+bool launched() {
+    if (cudaGetLastError() != cudaSuccess) return false;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return true;
+}
+
+// One evaluation at the current parameters.  backward: also the gradient; update: Adam step.
+// hist_row >= 0: copy the three sums of squares to that history row.
+kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr, int hist_row, cudaStream_t st) {
+    const int64_t M = c->M;
+    const int o = c->o, d = c->d, nb = c->nb;
+    const int sms = sm_count();
+    if (sms <= 0) return KQ_ERR_CUDA;
+    kq::calib_build_blocks<<<c->n_sets, 1024, 0, st>>>(c->theta, c->Kd, c->Pd);
+    if (!launched()) return KQ_ERR_CUDA;
+    if (cudaMemsetAsync(c->sums, 0, 3 * sizeof(double), st) != cudaSuccess) return KQ_ERR_CUDA;
+    auto fq_grid = [&](int64_t rows) {
+        int64_t gx = (rows + 127) / 128;
+        const int64_t cap = ((int64_t)sms * 16 + nb - 1) / nb;        // about 16 CTAs of 128 threads per SM
+        if (gx > cap) gx = cap;
+        if (gx < 1) gx = 1;
+        return dim3((unsigned)gx, (unsigned)nb);
+    };
+    kq::calib_fakequant<<<fq_grid(M), 128, 0, st>>>(c->A, c->Kd, c->n_sets, M, d, c->Yq, c->ResY, c->sums + 1);
+    if (!launched()) return KQ_ERR_CUDA;
+    kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, c->ResZ, c->sums + 2);
+    if (!launched()) return KQ_ERR_CUDA;
+    // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o))
+    kq_status_t rc = launch_gemm(c->tm_Yq_a, c->tm_Zq_b, (int)M, o, d, c->R, o, nullptr, -1.0f,
+                                 (float)(2.0 / ((double)M * o)), nullptr, backward ? c->dO : nullptr, o, c->sums, st);
+    if (rc != KQ_OK) return rc;
+    if (hist_row >= 0 &&
+        cudaMemcpyAsync(c->hist + 3 * hist_row, c->sums, 3 * sizeof(double), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return KQ_ERR_CUDA;
+    if (!backward) return KQ_OK;
+    auto tr = [&](const __nv_bfloat16* in, __nv_bfloat16* out, int64_t R, int64_t C) {
+        kq::transpose_bf16<<<dim3((unsigned)((C + 63) / 64), (unsigned)((R + 63) / 64)), 256, 0, st>>>(
+            reinterpret_cast<const uint16_t*>(in), reinterpret_cast<uint16_t*>(out), R, C);
+        return launched();
+    };
+    if (!tr(c->Yq, c->YqT, M, d) || !tr(c->Zq, c->ZqT, o, d) || !tr(c->dO, c->dOT, M, o)) return KQ_ERR_CUDA;
+    // dY = dO Zq + lambda_A 2 (Y - Yq) / (M d);  dZ = dO^T Yq + lambda_W 2 (Z - Zq) / (o d)
+    rc = launch_gemm(c->tm_dO_a, c->tm_ZqT_b, (int)M, d, o, c->ResY, d, c->lam, (float)(2.0 / ((double)M * d)), 1.0f,
+                     c->dY, nullptr, d, nullptr, st);
+    if (rc != KQ_OK) return rc;
+    rc = launch_gemm(c->tm_dOT_a, c->tm_YqT_b, o, d, (int)M, c->ResZ, d, c->lam + 1, (float)(2.0 / ((double)o * d)), 1.0f,
+                     c->dZ, nullptr, d, nullptr, st);
+    if (rc != KQ_OK) return rc;
+    kq::calib_block_grad<<<dim3((unsigned)c->chunksK, (unsigned)nb), 256, 0, st>>>(c->A, c->dY, M, d, c->rpcK, c->partK);
+    if (!launched()) return KQ_ERR_CUDA;
+    kq::calib_block_grad<<<dim3((unsigned)c->chunksP, (unsigned)nb), 256, 0, st>>>(c->W, c->dZ, o, d, c->rpcP, c->partP);
+    if (!launched()) return KQ_ERR_CUDA;
+    kq::CalibStepArgs a;
+    a.partK = c->partK; a.chunksK = c->chunksK; a.partP = c->partP; a.chunksP = c->chunksP;
+    a.nb = nb; a.n_sets = c->n_sets;
+    a.theta = c->theta; a.adam_m = c->adam_m; a.adam_v = c->adam_v; a.grad_out = c->grad;
+    a.lr = lr; a.t = c->t + 1; a.do_update = update ? 1 : 0;
+    kq::calib_param_step<<<c->n_sets, 1024, 0, st>>>(a);
+    if (!launched()) return KQ_ERR_CUDA;
+    if (update) c->t += 1;
+    return KQ_OK;
+}
+
+void chunking(int64_t rows, int nb, int sms, int* chunks, int64_t* rpc) {
+    int64_t want = ((int64_t)sms * 8 + nb - 1) / nb;             // about 8 CTAs per SM in total
+    if (want < 1) want = 1;
+    if (want > 64) want = 64;
+    int64_t r = (rows + want - 1) / want;
+    r = (r + kq::kGradTileRows - 1) / kq::kGradTileRows * kq::kGradTileRows;
+    if (r < kq::kGradTileRows) r = kq::kGradTileRows;
+    *rpc = r;
+    *chunks = (int)((rows + r - 1) / r);
+}
+
+kq_status_t calib_check(const kroquant_calib_t* c) {
+    if (!c) return KQ_ERR_NULL;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KQ_ERR_CUDA;
+    if (dev != c->device) return KQ_ERR_UNSUPPORTED;
+    return KQ_OK;
+}
+
+void hadamard_theta(std::vector<float>& th, int n_sets) {
+    th.resize((size_t)n_sets * 15);
+    const float h = (float)std::sqrt(0.5);
+    for (int i = 0; i < n_sets * 5; ++i) { th[3 * i] = h; th[3 * i + 1] = h; th[3 * i + 2] = 1.0f; }
+}
+
+}  // namespace
+
+extern "C" {
+
+kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o, int d, int n_sets, void* stream,
+                                  kroquant_calib_t** out) {
+    if (!A || !W || !out) return KQ_ERR_NULL;
+    *out = nullptr;
+    if (M <= 0 || o <= 0 || d <= 0 || M % 8 || o % 32 || d % 32 || M > (1 << 30)) return KQ_ERR_SHAPE;
+    if (n_sets != 1 && n_sets != d / 32) return KQ_ERR_FACTORS;
+    if (!aligned16(A) || !aligned16(W)) return KQ_ERR_ALIGN;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    kroquant_calib_t* c = new (std::nothrow) kroquant_calib_t();
+    if (!c) return KQ_ERR_CUDA;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return KQ_ERR_CUDA; }
+    const int sms = sm_count();
+    if (sms <= 0) { delete c; return KQ_ERR_CUDA; }
+    c->M = M; c->o = o; c->d = d; c->nb = d / 32; c->n_sets = n_sets;
+    c->A = static_cast<const uint16_t*>(A);
+    c->W = static_cast<const uint16_t*>(W);
+    chunking(M, c->nb, sms, &c->chunksK, &c->rpcK);
+    chunking(o, c->nb, sms, &c->chunksP, &c->rpcP);
+
+    // carve one allocation; every piece 256-byte aligned
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t at = off; off += (bytes + 255) & ~(size_t)255; return at; };
+    const size_t Md = (size_t)M * d, od = (size_t)o * d, Mo = (size_t)M * o, np = (size_t)n_sets * 15;
+    const size_t o_theta = take(np * 4), o_m = take(np * 4), o_v = take(np * 4), o_grad = take(np * 4), o_lam = take(8);
+    const size_t o_K = take((size_t)n_sets * 4096), o_P = take((size_t)n_sets * 4096);
+    const size_t o_Yq = take(Md * 2), o_YqT = take(Md * 2), o_Zq = take(od * 2), o_ZqT = take(od * 2);
+    const size_t o_dO = take(Mo * 2), o_dOT = take(Mo * 2);
+    const size_t o_ResY = take(Md * 4), o_ResZ = take(od * 4), o_R = take(Mo * 4), o_dY = take(Md * 4), o_dZ = take(od * 4);
+    const size_t o_pK = take((size_t)c->chunksK * c->nb * 4096), o_pP = take((size_t)c->chunksP * c->nb * 4096);
+    const size_t o_sums = take(3 * 8), o_hist = take((size_t)kHistCap * 3 * 8);
+    if (cudaMalloc(&c->pool, off) != cudaSuccess) { (void)cudaGetLastError(); delete c; return KQ_ERR_CUDA; }
+    uint8_t* b = c->pool;
+    c->theta = (float*)(b + o_theta); c->adam_m = (float*)(b + o_m); c->adam_v = (float*)(b + o_v);
+    c->grad = (float*)(b + o_grad); c->lam = (float*)(b + o_lam);
+    c->Kd = (float*)(b + o_K); c->Pd = (float*)(b + o_P);
+    c->Yq = (__nv_bfloat16*)(b + o_Yq); c->YqT = (__nv_bfloat16*)(b + o_YqT);
+    c->Zq = (__nv_bfloat16*)(b + o_Zq); c->ZqT = (__nv_bfloat16*)(b + o_ZqT);
+    c->dO = (__nv_bfloat16*)(b + o_dO); c->dOT = (__nv_bfloat16*)(b + o_dOT);
+    c->ResY = (float*)(b + o_ResY); c->ResZ = (float*)(b + o_ResZ); c->R = (float*)(b + o_R);
+    c->dY = (float*)(b + o_dY); c->dZ = (float*)(b + o_dZ);
+    c->partK = (float*)(b + o_pK); c->partP = (float*)(b + o_pP);
+    c->sums = (double*)(b + o_sums); c->hist = (double*)(b + o_hist);
+
+    bool ok = make_operand_map(&c->tm_A_a, c->A, M, d, kq::kGemmBM) && make_operand_map(&c->tm_W_b, c->W, o, d, kq::kGemmBN) &&
+              make_operand_map(&c->tm_Yq_a, c->Yq, M, d, kq::kGemmBM) && make_operand_map(&c->tm_Zq_b, c->Zq, o, d, kq::kGemmBN) &&
+              make_operand_map(&c->tm_dO_a, c->dO, M, o, kq::kGemmBM) && make_operand_map(&c->tm_ZqT_b, c->ZqT, d, o, kq::kGemmBN) &&
+              make_operand_map(&c->tm_dOT_a, c->dOT, o, M, kq::kGemmBM) && make_operand_map(&c->tm_YqT_b, c->YqT, d, M, kq::kGemmBN);
+    kq_status_t rc = ok ? KQ_OK : KQ_ERR_CUDA;
+    std::vector<float> th;
+    hadamard_theta(th, n_sets);
+    if (rc == KQ_OK && (cudaMemsetAsync(c->pool, 0, o_K, st) != cudaSuccess ||      // theta, m, v, grad, lambdas
+                        cudaMemcpyAsync(c->theta, th.data(), np * 4, cudaMemcpyHostToDevice, st) != cudaSuccess))
+        rc = KQ_ERR_CUDA;
+    // R = A W^T
+    if (rc == KQ_OK)
+        rc = launch_gemm(c->tm_A_a, c->tm_W_b, (int)M, o, d, nullptr, 0, nullptr, 1.0f, 1.0f, c->R, nullptr, o, nullptr, st);
+    // the three terms at the initialisation -> lambdas
+    if (rc == KQ_OK) rc = calib_eval(c, false, false, 0.f, 0, st);
+    if (rc == KQ_OK) {
+        kq::calib_lambdas<<<1, 32, 0, st>>>(c->sums, (double)M * o, (double)M * d, (double)o * d, c->lam);
+        if (!launched()) rc = KQ_ERR_CUDA;
+    }
+    if (rc == KQ_OK && cudaStreamSynchronize(st) != cudaSuccess) { (void)cudaGetLastError(); rc = KQ_ERR_CUDA; }
+    if (rc != KQ_OK) { kroquant_calib_destroy(c); return rc; }
+    *out = c;
+    return KQ_OK;
+}
+
+void kroquant_calib_destroy(kroquant_calib_t* c) {
+    if (!c) return;
+    if (c->pool) (void)cudaFree(c->pool);
+    delete c;
+}
+
+kq_status_t kroquant_calib_set_theta(kroquant_calib_t* c, const float* theta_host) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (!theta_host) return KQ_ERR_NULL;
+    const size_t np = (size_t)c->n_sets * 15;
+    for (size_t i = 0; i < np; i += 3)
+        if (!(std::fabs(theta_host[i]) > 0.f) || !std::isfinite(theta_host[i]) || !std::isfinite(theta_host[i + 1]) ||
+            !std::isfinite(theta_host[i + 2]))
+            return KQ_ERR_FACTORS;                       // a = 0 has no LU form
+    if (cudaMemcpy(c->theta, theta_host, np * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(c->adam_m, 0, np * 4) != cudaSuccess || cudaMemset(c->adam_v, 0, np * 4) != cudaSuccess)
+        return KQ_ERR_CUDA;
+    c->t = 0;
+    return KQ_OK;
+}
+
+kq_status_t kroquant_calib_get_theta(const kroquant_calib_t* c, float* theta_host_out) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (!theta_host_out) return KQ_ERR_NULL;
+    return cudaMemcpy(theta_host_out, c->theta, (size_t)c->n_sets * 60, cudaMemcpyDeviceToHost) == cudaSuccess ? KQ_OK
+                                                                                                                 : KQ_ERR_CUDA;
+}
+
+kq_status_t kroquant_calib_set_lambdas(kroquant_calib_t* c, const float* lam_host) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (!lam_host) return KQ_ERR_NULL;
+    return cudaMemcpy(c->lam, lam_host, 8, cudaMemcpyHostToDevice) == cudaSuccess ? KQ_OK : KQ_ERR_CUDA;
+}
+
+kq_status_t kroquant_calib_get_lambdas(const kroquant_calib_t* c, float* lam_host_out) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (!lam_host_out) return KQ_ERR_NULL;
+    return cudaMemcpy(lam_host_out, c->lam, 8, cudaMemcpyDeviceToHost) == cudaSuccess ? KQ_OK : KQ_ERR_CUDA;
+}
+
+kq_status_t kroquant_calib_get_factors(const kroquant_calib_t* c, float* G_host_out) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (!G_host_out) return KQ_ERR_NULL;
+    std::vector<float> th((size_t)c->n_sets * 15);
+    if (cudaMemcpy(th.data(), c->theta, th.size() * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return KQ_ERR_CUDA;
+    for (int i = 0; i < c->n_sets * 5; ++i) {
+        const double a = th[3 * i], b = th[3 * i + 1], cc = th[3 * i + 2];
+        G_host_out[4 * i + 0] = (float)a;
+        G_host_out[4 * i + 1] = (float)b;
+        G_host_out[4 * i + 2] = (float)(cc * a);
+        G_host_out[4 * i + 3] = (float)(cc * b - 1.0 / a);
+    }
+    return KQ_OK;
+}
+
+kq_status_t kroquant_calib_loss_grad(kroquant_calib_t* c, double* losses_host_out, float* grad_host_out, void* stream) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (!losses_host_out) return KQ_ERR_NULL;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    rc = calib_eval(c, grad_host_out != nullptr, false, 0.f, -1, st);
+    if (rc != KQ_OK) return rc;
+    double s[3];
+    if (cudaMemcpyAsync(s, c->sums, sizeof(s), cudaMemcpyDeviceToHost, st) != cudaSuccess) return KQ_ERR_CUDA;
+    if (grad_host_out &&
+        cudaMemcpyAsync(grad_host_out, c->grad, (size_t)c->n_sets * 60, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return KQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) { (void)cudaGetLastError(); return KQ_ERR_CUDA; }
+    losses_host_out[0] = s[0] / ((double)c->M * c->o);
+    losses_host_out[1] = s[1] / ((double)c->M * c->d);
+    losses_host_out[2] = s[2] / ((double)c->o * c->d);
+    return KQ_OK;
+}
+
+kq_status_t kroquant_calib_run(kroquant_calib_t* c, int steps, float lr, double* history_host_out, void* stream) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (steps < 1 || steps > kHistCap - 1 || !(lr > 0.f)) return KQ_ERR_SHAPE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    for (int i = 0; i < steps; ++i) {
+        rc = calib_eval(c, true, true, lr, i, st);
+        if (rc != KQ_OK) return rc;
+    }
+    if (!history_host_out) return KQ_OK;
+    rc = calib_eval(c, false, false, 0.f, steps, st);
+    if (rc != KQ_OK) return rc;
+    if (cudaMemcpyAsync(history_host_out, c->hist, (size_t)(steps + 1) * 24, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KQ_ERR_CUDA;
+    }
+    const double n[3] = {(double)c->M * c->o, (double)c->M * c->d, (double)c->o * c->d};
+    for (int i = 0; i <= steps; ++i)
+        for (int k = 0; k < 3; ++k) history_host_out[3 * i + k] /= n[k];
+    return KQ_OK;
+}
+
+}  // extern "C"
