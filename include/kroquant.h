@@ -226,6 +226,20 @@ kq_status_t kroquant_calib_loss_grad(kroquant_calib_t *c, double *losses_host_ou
 kq_status_t kroquant_calib_run(kroquant_calib_t *c, int steps, float lr, double *history_host_out,
                                void *stream);
 
+/* Backward of the block transform with respect to the blocks (the reduction inside a calibration
+ * step, Section 3.3, offered on its own for callers that run their own optimisation loop):
+ *     out[s] = sum over rows t, and over block columns j served by set s, of  x_{t,j}^T g_{t,j},
+ * x_{t,j} the 32 channels of block j of row t of X (DEVICE bf16 [rows][d]) and g_{t,j} the same
+ * slice of G (DEVICE fp32 [rows][d], the gradient with respect to X T).  n_sets is 1 or d/32;
+ * out is DEVICE fp32 [n_sets][32][32].  The kernel first writes partial sums per chunk of rows
+ * into `scratch` (DEVICE, 16-byte aligned, at least kroquant_block_grad_scratch_bytes(rows, d)
+ * bytes, contents irrelevant before and after), then reduces them in a fixed order, so the result
+ * is deterministic.  Errors: KQ_ERR_NULL, KQ_ERR_SHAPE (d % 32, rows < 0, scratch too small),
+ * KQ_ERR_FACTORS (n_sets), KQ_ERR_ALIGN, KQ_ERR_CUDA.  rows == 0 writes zeros. */
+int64_t kroquant_block_grad_scratch_bytes(int64_t rows, int d);
+kq_status_t kroquant_block_grad(const void *X, const float *G, int64_t rows, int d, int n_sets,
+                                void *scratch, int64_t scratch_bytes, float *out, void *stream);
+
 /* Number of kernels this library has launched in the calling process (all streams). */
 int64_t kroquant_launch_count(void);
 

@@ -32,6 +32,7 @@ EXPORTS = [
     "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
     "kroquant_calib_loss_grad", "kroquant_calib_run",
+    "kroquant_block_grad_scratch_bytes", "kroquant_block_grad",
 ]
 
 
@@ -89,6 +90,9 @@ def load_library() -> C.CDLL:
         getattr(L, "kroquant_calib_" + name).argtypes = [vp, vp]
     L.kroquant_calib_loss_grad.argtypes = [vp, vp, vp, vp]
     L.kroquant_calib_run.argtypes = [vp, i32, C.c_float, vp, vp]
+    L.kroquant_block_grad_scratch_bytes.argtypes = [i64, i32]
+    L.kroquant_block_grad_scratch_bytes.restype = i64
+    L.kroquant_block_grad.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, vp]
     _lib = L
     return L
 
@@ -370,6 +374,24 @@ class HostPipeline:
         self.h2d.synchronize()
         self.compute.synchronize()
         self.d2h.synchronize()
+
+
+def kroquant_block_grad(X: torch.Tensor, G: torch.Tensor, n_sets: int = 1, out: Optional[torch.Tensor] = None,
+                        stream=None) -> torch.Tensor:
+    """out[s] = sum of x_j^T g_j over rows (and over block columns for a shared set): float32
+    [n_sets, 32, 32].  X: CUDA bfloat16 [rows, d]; G: CUDA float32 [rows, d].  The scratch buffer the
+    kernel needs is allocated here (torch) and passed down."""
+    rows, d = _x_shape(X)
+    if X.dtype != torch.bfloat16 or G.dtype != torch.float32 or G.shape != X.shape or not G.is_contiguous():
+        raise ValueError("X bfloat16 [rows, d] and G float32 [rows, d], both contiguous")
+    L = load_library()
+    if out is None:
+        out = torch.empty((n_sets, 32, 32), dtype=torch.float32, device=X.device)
+    nbytes = max(int(L.kroquant_block_grad_scratch_bytes(rows, d)), 16)
+    scratch = torch.empty(nbytes, dtype=torch.uint8, device=X.device)
+    _check(L.kroquant_block_grad(_ptr(X), _ptr(G), rows, d, n_sets, _ptr(scratch), nbytes, _ptr(out), _stream(stream)),
+           "kroquant_block_grad")
+    return out
 
 
 class Calibrator:

@@ -4,6 +4,7 @@
 //   calib_fakequant     V = X_j B_j per 32-channel block, Vq = Q(V) as bf16, R = V - Vq, sum R^2
 //   transpose_bf16      [R][C] -> [C][R]
 //   calib_block_grad    partial sums of X_j^T G_j over chunks of rows
+//   calib_reduce_parts  sum of the partial blocks
 //   calib_param_step    block gradients -> d/d(a,b,c) through the Kronecker and LU structure, Adam
 //   calib_lambdas       lambda_A = L_out/L_A, lambda_W = L_out/L_W at the initialisation
 //
@@ -204,16 +205,37 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
         dst[i] = (red[i] + red[1024 + i]) + (red2[i] + red2[1024 + i]);
 }
 
+// ---- sum of partial blocks: out[j][e] = sum_p part[p][j][e], e < 1024 --------------------------
+// grid (32, J), 1024 threads: CTA x owns 32 consecutive entries; warp w adds the partials
+// p = w, w + 32, ... in double, then the 32 warps are combined in a fixed order (deterministic).
+// A shared factor set is the case J = 1 with the (chunk, block column) pairs flattened into P.
+__global__ void __launch_bounds__(1024)
+calib_reduce_parts(const float* __restrict__ part, int P, float* __restrict__ out) {
+    __shared__ double sm[32][33];
+    const int J = gridDim.y, jj = blockIdx.y;
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int e = blockIdx.x * 32 + lane;
+    double acc = 0.0;
+    for (int p = w; p < P; p += 32) acc += (double)__ldg(part + ((size_t)p * J + jj) * 1024 + e);
+    sm[w][lane] = acc;
+    __syncthreads();
+    if (w == 0) {
+        double t = 0.0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) t += sm[i][lane];
+        out[(size_t)jj * 1024 + e] = (float)t;
+    }
+}
+
 // ---- block gradients -> parameter gradients -> Adam -------------------------------------------
-// One CTA of 1024 threads per factor set; thread (R, C) first sums its entry of dK and dP over
-// the row chunks (and over all block columns when the set is shared).  For B = F_1 (x) .. (x) F_5,
+// One CTA of 1024 threads per factor set; thread (R, C) holds its entry of dK and dP (already
+// summed over rows, and over block columns when the set is shared).  For B = F_1 (x) .. (x) F_5,
 // d/dF_k[r][c] = sum over (R, C) with bit_k(R) = r, bit_k(C) = c of dB[R][C] * prod_{l != k} F_l[..].
 // Then d/d(a, b, c) by the closed-form derivatives of G_k and H_k = G_k^-T, and one Adam step
 // (beta1 0.9, beta2 0.999, eps 1e-8, bias correction) when do_update != 0.
 struct CalibStepArgs {
-    const float* partK; int chunksK;
-    const float* partP; int chunksP;
-    int nb, n_sets;
+    const float* dK;           // [n_sets][32][32]
+    const float* dP;           // [n_sets][32][32]
     float* theta; float* adam_m; float* adam_v; float* grad_out;
     float lr; int t; int do_update;
 };
@@ -233,12 +255,8 @@ calib_param_step(const CalibStepArgs a) {
         Gs[f][0][0] = aa; Gs[f][0][1] = bb; Gs[f][1][0] = aa * cc; Gs[f][1][1] = bb * cc - 1.0 / aa;
         Hs[f][0][0] = 1.0 / aa - bb * cc; Hs[f][0][1] = aa * cc; Hs[f][1][0] = bb; Hs[f][1][1] = -aa;
     }
-    double dk = 0.0, dp = 0.0;
-    const int j_begin = a.n_sets == 1 ? 0 : s, j_end = a.n_sets == 1 ? a.nb : s + 1;
-    for (int j = j_begin; j < j_end; ++j) {
-        for (int ch = 0; ch < a.chunksK; ++ch) dk += (double)a.partK[((size_t)ch * a.nb + j) * 1024 + threadIdx.x];
-        for (int ch = 0; ch < a.chunksP; ++ch) dp += (double)a.partP[((size_t)ch * a.nb + j) * 1024 + threadIdx.x];
-    }
+    const double dk = (double)a.dK[(size_t)s * 1024 + threadIdx.x];
+    const double dp = (double)a.dP[(size_t)s * 1024 + threadIdx.x];
     __syncthreads();
 #pragma unroll
     for (int k = 0; k < 5; ++k) {

@@ -15,7 +15,8 @@ struct kroquant_calib {
     float *Kd = nullptr, *Pd = nullptr;
     __nv_bfloat16 *Yq = nullptr, *YqT = nullptr, *Zq = nullptr, *ZqT = nullptr, *dO = nullptr, *dOT = nullptr;
     float *ResY = nullptr, *ResZ = nullptr, *R = nullptr, *dY = nullptr, *dZ = nullptr;
-    float *partK = nullptr, *partP = nullptr;
+    float *partK = nullptr, *partP = nullptr;     // partial block sums [chunks][nb][32][32]
+    float *dK = nullptr, *dP = nullptr;           // reduced block gradients [n_sets][32][32]
     int chunksK = 0, chunksP = 0;
     int64_t rpcK = 0, rpcP = 0;
     double* sums = nullptr;            // [3] sums of squares of the evaluation in flight
@@ -76,6 +77,32 @@ bool launched() {
     return true;
 }
 
+void chunking(int64_t rows, int nb, int sms, int* chunks, int64_t* rpc) {
+    int64_t want = ((int64_t)sms * 8 + nb - 1) / nb;             // about 8 CTAs per SM in total
+    if (want < 1) want = 1;
+    if (want > 64) want = 64;
+    int64_t r = (rows + want - 1) / want;
+    r = (r + kq::kGradTileRows - 1) / kq::kGradTileRows * kq::kGradTileRows;
+    if (r < kq::kGradTileRows) r = kq::kGradTileRows;
+    *rpc = r;
+    *chunks = (int)((rows + r - 1) / r);
+}
+
+// out[s] = sum over rows (and over block columns for a shared set) of x_j^T g_j: partial sums per
+// chunk of rows into `part` ([chunks][nb][32][32] floats), then one deterministic reduction.
+kq_status_t run_block_grad(const uint16_t* X, const float* G, int64_t rows, int d, int n_sets, int chunks, int64_t rpc,
+                           float* part, float* out, cudaStream_t st) {
+    const int nb = d / 32;
+    kq::calib_block_grad<<<dim3((unsigned)chunks, (unsigned)nb), 256, 0, st>>>(X, G, rows, d, rpc, part);
+    if (!launched()) return KQ_ERR_CUDA;
+    if (n_sets == 1)
+        kq::calib_reduce_parts<<<dim3(32, 1), 1024, 0, st>>>(part, chunks * nb, out);
+    else
+        kq::calib_reduce_parts<<<dim3(32, (unsigned)nb), 1024, 0, st>>>(part, chunks, out);
+    if (!launched()) return KQ_ERR_CUDA;
+    return KQ_OK;
+}
+
 // One evaluation at the current parameters.  backward: also the gradient; update: Adam step.
 // hist_row >= 0: copy the three sums of squares to that history row.
 kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr, int hist_row, cudaStream_t st) {
@@ -118,30 +145,18 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
     rc = launch_gemm(c->tm_dOT_a, c->tm_YqT_b, o, d, (int)M, c->ResZ, d, c->lam + 1, (float)(2.0 / ((double)o * d)), 1.0f,
                      c->dZ, nullptr, d, nullptr, st);
     if (rc != KQ_OK) return rc;
-    kq::calib_block_grad<<<dim3((unsigned)c->chunksK, (unsigned)nb), 256, 0, st>>>(c->A, c->dY, M, d, c->rpcK, c->partK);
-    if (!launched()) return KQ_ERR_CUDA;
-    kq::calib_block_grad<<<dim3((unsigned)c->chunksP, (unsigned)nb), 256, 0, st>>>(c->W, c->dZ, o, d, c->rpcP, c->partP);
-    if (!launched()) return KQ_ERR_CUDA;
+    rc = run_block_grad(c->A, c->dY, M, d, c->n_sets, c->chunksK, c->rpcK, c->partK, c->dK, st);
+    if (rc != KQ_OK) return rc;
+    rc = run_block_grad(c->W, c->dZ, o, d, c->n_sets, c->chunksP, c->rpcP, c->partP, c->dP, st);
+    if (rc != KQ_OK) return rc;
     kq::CalibStepArgs a;
-    a.partK = c->partK; a.chunksK = c->chunksK; a.partP = c->partP; a.chunksP = c->chunksP;
-    a.nb = nb; a.n_sets = c->n_sets;
+    a.dK = c->dK; a.dP = c->dP;
     a.theta = c->theta; a.adam_m = c->adam_m; a.adam_v = c->adam_v; a.grad_out = c->grad;
     a.lr = lr; a.t = c->t + 1; a.do_update = update ? 1 : 0;
     kq::calib_param_step<<<c->n_sets, 1024, 0, st>>>(a);
     if (!launched()) return KQ_ERR_CUDA;
     if (update) c->t += 1;
     return KQ_OK;
-}
-
-void chunking(int64_t rows, int nb, int sms, int* chunks, int64_t* rpc) {
-    int64_t want = ((int64_t)sms * 8 + nb - 1) / nb;             // about 8 CTAs per SM in total
-    if (want < 1) want = 1;
-    if (want > 64) want = 64;
-    int64_t r = (rows + want - 1) / want;
-    r = (r + kq::kGradTileRows - 1) / kq::kGradTileRows * kq::kGradTileRows;
-    if (r < kq::kGradTileRows) r = kq::kGradTileRows;
-    *rpc = r;
-    *chunks = (int)((rows + r - 1) / r);
 }
 
 kq_status_t calib_check(const kroquant_calib_t* c) {
@@ -161,6 +176,36 @@ void hadamard_theta(std::vector<float>& th, int n_sets) {
 }  // namespace
 
 extern "C" {
+
+int64_t kroquant_block_grad_scratch_bytes(int64_t rows, int d) {
+    if (rows < 0 || d <= 0 || d % 32) return -1;
+    const int sms = sm_count();
+    if (sms <= 0) return -1;
+    int chunks;
+    int64_t rpc;
+    chunking(rows > 0 ? rows : 1, d / 32, sms, &chunks, &rpc);
+    return (int64_t)chunks * (d / 32) * 4096;
+}
+
+kq_status_t kroquant_block_grad(const void* X, const float* G, int64_t rows, int d, int n_sets, void* scratch,
+                                int64_t scratch_bytes, float* out, void* stream) {
+    if (!out) return KQ_ERR_NULL;
+    if (rows < 0 || d <= 0 || d % 32) return KQ_ERR_SHAPE;
+    if (n_sets != 1 && n_sets != d / 32) return KQ_ERR_FACTORS;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (rows == 0)
+        return cudaMemsetAsync(out, 0, (size_t)n_sets * 4096, st) == cudaSuccess ? KQ_OK : KQ_ERR_CUDA;
+    if (!X || !G || !scratch) return KQ_ERR_NULL;
+    if (!aligned16(X) || !aligned16(G) || !aligned16(scratch) || !aligned16(out)) return KQ_ERR_ALIGN;
+    const int sms = sm_count();
+    if (sms <= 0) return KQ_ERR_CUDA;
+    int chunks;
+    int64_t rpc;
+    chunking(rows, d / 32, sms, &chunks, &rpc);
+    if (scratch_bytes < (int64_t)chunks * (d / 32) * 4096) return KQ_ERR_SHAPE;
+    return run_block_grad(static_cast<const uint16_t*>(X), G, rows, d, n_sets, chunks, rpc, static_cast<float*>(scratch),
+                          out, st);
+}
 
 kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o, int d, int n_sets, void* stream,
                                   kroquant_calib_t** out) {
@@ -191,6 +236,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     const size_t o_dO = take(Mo * 2), o_dOT = take(Mo * 2);
     const size_t o_ResY = take(Md * 4), o_ResZ = take(od * 4), o_R = take(Mo * 4), o_dY = take(Md * 4), o_dZ = take(od * 4);
     const size_t o_pK = take((size_t)c->chunksK * c->nb * 4096), o_pP = take((size_t)c->chunksP * c->nb * 4096);
+    const size_t o_dK = take((size_t)n_sets * 4096), o_dP = take((size_t)n_sets * 4096);
     const size_t o_sums = take(3 * 8), o_hist = take((size_t)kHistCap * 3 * 8);
     if (cudaMalloc(&c->pool, off) != cudaSuccess) { (void)cudaGetLastError(); delete c; return KQ_ERR_CUDA; }
     uint8_t* b = c->pool;
@@ -203,6 +249,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     c->ResY = (float*)(b + o_ResY); c->ResZ = (float*)(b + o_ResZ); c->R = (float*)(b + o_R);
     c->dY = (float*)(b + o_dY); c->dZ = (float*)(b + o_dZ);
     c->partK = (float*)(b + o_pK); c->partP = (float*)(b + o_pP);
+    c->dK = (float*)(b + o_dK); c->dP = (float*)(b + o_dP);
     c->sums = (double*)(b + o_sums); c->hist = (double*)(b + o_hist);
 
     bool ok = make_operand_map(&c->tm_A_a, c->A, M, d, kq::kGemmBM) && make_operand_map(&c->tm_W_b, c->W, o, d, kq::kGemmBN) &&

@@ -163,6 +163,25 @@ def test_calibrated_factors_feed_the_quantizer():
     cal.destroy()
 
 
+@pytest.mark.parametrize("rows,d", [(1000, 256), (64, 96), (8, 32), (4104, 1152)])
+@pytest.mark.parametrize("shared", [True, False])
+def test_block_grad_against_the_oracle(rows, d, shared):
+    rng = np.random.default_rng(rows + d)
+    X_bits = wl.gen_activations(wl.calib_spec(rows, d, 81))
+    X = wl.bf16_bits_to_f32(X_bits).astype(np.float64)
+    Gm = rng.standard_normal((rows, d)).astype(np.float32)
+    n_sets = 1 if shared else d // 32
+    dev = torch.device("cuda:0")
+    X_t = torch.from_numpy(X_bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    out = kb.kroquant_block_grad(X_t, torch.from_numpy(Gm).to(dev), n_sets).cpu().numpy()
+    ref = co._block_grads(X, Gm.astype(np.float64), n_sets)
+    # fp32 products and partial sums: error of a sum of n terms ~ sqrt(n) 2^-24 of its absolute sum
+    bound = 1e-5 * (np.abs(X).T @ np.abs(Gm).astype(np.float64)).max()
+    assert np.abs(out - ref).max() <= bound
+    again = kb.kroquant_block_grad(X_t, torch.from_numpy(Gm).to(dev), n_sets).cpu().numpy()
+    assert np.array_equal(out, again)                   # fixed summation order
+
+
 def test_argument_checks():
     A, W, A_t, W_t = _case(256, 64, 128, 71)
     with pytest.raises(kb.KroQuantError):
