@@ -240,6 +240,30 @@ int64_t kroquant_block_grad_scratch_bytes(int64_t rows, int d);
 kq_status_t kroquant_block_grad(const void *X, const float *G, int64_t rows, int d, int n_sets,
                                 void *scratch, int64_t scratch_bytes, float *out, void *stream);
 
+/* kroquant_block_grad for callers that have no device memory to give.  (The paper has no
+ * counterpart: this is a property of the library interface, not of the method.)
+ *
+ * Who needs it: a host program that talks to this library through the plain C ABI and owns no
+ * allocator; an inference or training process in which a framework claimed the device memory up
+ * front, so that an allocation made behind its back fails or fragments its pool; a latency-bound
+ * loop that cannot afford the device-wide synchronisation an allocation implies.  Such a caller
+ * cannot supply the scratch buffer kroquant_block_grad asks for, so this entry point keeps one
+ * inside the library: a fixed 8 MiB device array (2048 partial 32 x 32 blocks) that every GPU
+ * loading the library holds until the process ends.
+ *
+ * Same arguments, result and error codes as kroquant_block_grad minus the scratch pair; X, G and
+ * out are still the caller's.  The call allocates and frees nothing.  A problem whose partial
+ * sums do not fit - more than 2048 of them; on a 148-SM GPU every d <= 32768 fits whatever the
+ * row count, and no d > 65536 does - is refused with KQ_ERR_UNSUPPORTED and nothing is launched.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call before any stream capture begins.  All calls share the one array.  Nothing
+ * in it needs clearing: each call overwrites every partial block it later reads, and never reads
+ * what an earlier call left.  For the same reason two calls that overlap on the GPU (different
+ * streams, or different host threads without ordering) race on it and both results are
+ * undefined: order them on one stream or with events. */
+kq_status_t kroquant_block_grad_static(const void *X, const float *G, int64_t rows, int d, int n_sets,
+                                       float *out, void *stream);
+
 /* Number of kernels this library has launched in the calling process (all streams). */
 int64_t kroquant_launch_count(void);
 

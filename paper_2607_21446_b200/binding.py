@@ -32,7 +32,7 @@ EXPORTS = [
     "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
     "kroquant_calib_loss_grad", "kroquant_calib_run",
-    "kroquant_block_grad_scratch_bytes", "kroquant_block_grad",
+    "kroquant_block_grad_scratch_bytes", "kroquant_block_grad", "kroquant_block_grad_static",
 ]
 
 
@@ -93,6 +93,7 @@ def load_library() -> C.CDLL:
     L.kroquant_block_grad_scratch_bytes.argtypes = [i64, i32]
     L.kroquant_block_grad_scratch_bytes.restype = i64
     L.kroquant_block_grad.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, vp]
+    L.kroquant_block_grad_static.argtypes = [vp, vp, i64, i32, i32, vp, vp]
     _lib = L
     return L
 
@@ -392,6 +393,19 @@ def kroquant_block_grad(X: torch.Tensor, G: torch.Tensor, n_sets: int = 1, out: 
     _check(L.kroquant_block_grad(_ptr(X), _ptr(G), rows, d, n_sets, _ptr(scratch), nbytes, _ptr(out), _stream(stream)),
            "kroquant_block_grad")
     return out
+
+
+def kroquant_block_grad_static(X: torch.Tensor, G: torch.Tensor, n_sets: int, out: torch.Tensor, stream=None) -> None:
+    """kroquant_block_grad without a scratch buffer: the library's built-in one is used, so nothing is
+    allocated here or below (``out``, float32 [n_sets, 32, 32], must be supplied).  For callers whose
+    device memory is spoken for; see the header for the size limit and the sharing rules."""
+    rows, d = _x_shape(X)
+    if X.dtype != torch.bfloat16 or G.dtype != torch.float32 or G.shape != X.shape or not G.is_contiguous():
+        raise ValueError("X bfloat16 [rows, d] and G float32 [rows, d], both contiguous")
+    if out.dtype != torch.float32 or tuple(out.shape) != (n_sets, 32, 32) or not out.is_contiguous() or not out.is_cuda:
+        raise ValueError("out must be a contiguous CUDA float32 tensor [n_sets, 32, 32]")
+    _check(load_library().kroquant_block_grad_static(_ptr(X), _ptr(G), rows, d, n_sets, _ptr(out), _stream(stream)),
+           "kroquant_block_grad_static")
 
 
 class Calibrator:

@@ -722,3 +722,59 @@ const char* kroquant_status_string(kq_status_t s) {
 }  // extern "C"
 
 #include "kroquant_calib_api.cuh"
+
+// ---- block gradient without any allocation -------------------------------------------------
+// Same kernels as kroquant_block_grad; the partial sums go to a buffer that is part of the
+// library image instead of one the caller has to find memory for.  Every GPU that loads the
+// library carries these 8 MiB until the process exits.
+namespace {
+
+constexpr int64_t kStaticGradBlocks = 2048;                       // partial 32 x 32 blocks
+static __device__ __align__(256) float g_block_grad_scratch[kStaticGradBlocks * 1024];   // 8 MiB
+
+// In host code the array's name is only a handle for the runtime, not something a kernel can
+// dereference: the device address has to be asked for, per device, with that device current.
+std::mutex g_static_grad_mutex;
+float* g_static_grad_ptr[64] = {nullptr};
+
+kq_status_t static_grad_scratch(float** ptr_out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_grad_mutex);
+    if (!g_static_grad_ptr[dev]) {
+        float* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_block_grad_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return KQ_ERR_CUDA;
+        }
+        g_static_grad_ptr[dev] = p;
+    }
+    *ptr_out = g_static_grad_ptr[dev];
+    return KQ_OK;
+}
+
+}  // namespace
+
+extern "C" kq_status_t kroquant_block_grad_static(const void* X, const float* G, int64_t rows, int d, int n_sets,
+                                                  float* out, void* stream) {
+    if (!out) return KQ_ERR_NULL;
+    if (rows < 0 || d <= 0 || d % 32) return KQ_ERR_SHAPE;
+    if (n_sets != 1 && n_sets != d / 32) return KQ_ERR_FACTORS;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (rows == 0)
+        return cudaMemsetAsync(out, 0, (size_t)n_sets * 4096, st) == cudaSuccess ? KQ_OK : KQ_ERR_CUDA;
+    if (!X || !G) return KQ_ERR_NULL;
+    if (!aligned16(X) || !aligned16(G) || !aligned16(out)) return KQ_ERR_ALIGN;
+    const int sms = sm_count();
+    if (sms <= 0) return KQ_ERR_CUDA;
+    int chunks;
+    int64_t rpc;
+    chunking(rows, d / 32, sms, &chunks, &rpc);
+    if ((int64_t)chunks * (d / 32) > kStaticGradBlocks) return KQ_ERR_UNSUPPORTED;   // larger than the built-in buffer
+    float* scratch = nullptr;
+    const kq_status_t rc = static_grad_scratch(&scratch);
+    if (rc != KQ_OK) return rc;
+    // every partial block that the reduction reads is written first by this call: nothing in
+    // the buffer has to start at zero, and what an earlier call left there is never read
+    return run_block_grad(static_cast<const uint16_t*>(X), G, rows, d, n_sets, chunks, rpc, scratch, out, st);
+}
