@@ -1,8 +1,7 @@
 // CUDA-core kernels of the calibration loop (paper Section 3.3; optimiser set-up of Appendix D).
 //
 //   calib_build_blocks  theta (a,b,c per factor) -> K = G1 (x) .. (x) G5 and P = K^-T, dense 32x32
-//   calib_fakequant     V = X_j B_j per 32-channel block, Vq = Q(V) as bf16, R = V - Vq, sum R^2
-//   transpose_bf16      [R][C] -> [C][R]
+//   calib_fakequant     V = X_j B_j per 32-channel block, Vq = Q(V) as bf16 (and transposed), R = V - Vq, sum R^2
 //   calib_block_grad    partial sums of X_j^T G_j over chunks of rows
 //   calib_reduce_parts  sum of the partial blocks
 //   calib_param_step    block gradients -> d/d(a,b,c) through the Kronecker and LU structure, Adam
@@ -38,101 +37,134 @@ calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, fl
 }
 
 // ---- transform + fake quantisation ---------------------------------------------------------
-// grid (row groups, d/32); 128 threads; thread = one row of block column j.  The block matrix
-// sits in shared memory and is read as warp-wide broadcasts.  Q is the MXFP4 encoder of the
-// quantizer kernels followed by its decoder; Vq is exact in bf16.
+// V = X_j B_j on the tensor cores (mma.sync m16n8k16, bf16 inputs, fp32 accumulate): B_j is split
+// into three bf16 terms held in registers for the life of the CTA, so every product is exact and
+// only the accumulation rounds (the same device as in the quantizer kernels).  grid (row groups,
+// d/32); 4 warps; a warp owns 16 rows per iteration, the CTA 64.  Q is the MXFP4 encoder of the
+// quantizer kernels followed by its decoder; Vq is exact in bf16.  Outputs: Vq [rows][d],
+// its transpose VqT [d][rows] (staged through shared memory, 16-byte segments), R = V - Vq,
+// and the sum of R^2.
 __device__ __forceinline__ float e2m1_nibble_value(uint32_t code) {
     const uint32_t m = code & 7u;
     const float mag = m < 2u ? 0.5f * (float)m : (float)(2u + (m & 1u)) * (float)(1u << ((m >> 1) - 1u)) * 0.5f;
     return (code & 8u) ? -mag : mag;
 }
+__device__ __forceinline__ void split3_bf16(float x, uint32_t (&t)[3]) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(h0);
+    const __nv_bfloat16 h1 = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 h2 = __float2bfloat16_rn(r1 - __bfloat162float(h1));
+    t[0] = __bfloat16_as_ushort(h0); t[1] = __bfloat16_as_ushort(h1); t[2] = __bfloat16_as_ushort(h2);
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
+constexpr int kFqRows = 64;
 __global__ void __launch_bounds__(128)
 calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int n_sets, int64_t rows, int d,
-                __nv_bfloat16* __restrict__ Vq, float* __restrict__ Res, double* __restrict__ sumsq) {
-    __shared__ __align__(16) float Bs[32][32];
+                __nv_bfloat16* __restrict__ Vq, __nv_bfloat16* __restrict__ VqT, float* __restrict__ Res,
+                double* __restrict__ sumsq) {
+    __shared__ __align__(16) uint16_t tt[32][kFqRows + 8];
     __shared__ double red[4];
     const int j = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, q = lane & 3;
     const float* Bj = B + (size_t)(n_sets == 1 ? 0 : j) * 1024;
-    for (int i = threadIdx.x; i < 1024; i += 128) Bs[i >> 5][i & 31] = Bj[i];
-    __syncthreads();
+    // B fragments: n-tile t (columns 8t..8t+7), k-step s (rows 16s..16s+15 of B), half h (k + 8)
+    uint32_t bf[3][4][2][2];
+#pragma unroll
+    for (int t = 0; t < 4; ++t)
+#pragma unroll
+        for (int s = 0; s < 2; ++s)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int k0 = 16 * s + 2 * q + 8 * h, n = 8 * t + g;
+                uint32_t lo[3], hi[3];
+                split3_bf16(__ldg(Bj + k0 * 32 + n), lo);
+                split3_bf16(__ldg(Bj + (k0 + 1) * 32 + n), hi);
+#pragma unroll
+                for (int m = 0; m < 3; ++m) bf[m][t][s][h] = lo[m] | (hi[m] << 16);
+            }
     double sq = 0.0;
-    for (int64_t row = (int64_t)blockIdx.x * 128 + threadIdx.x; row < rows; row += (int64_t)gridDim.x * 128) {
-        const uint4* xp = reinterpret_cast<const uint4*>(X + row * d + j * 32);
-        float x[32];
+    for (int64_t row0 = (int64_t)blockIdx.x * kFqRows; row0 < rows; row0 += (int64_t)gridDim.x * kFqRows) {
+        const int64_t r_lo = row0 + warp * 16 + g, r_hi = r_lo + 8;
+        uint32_t a[2][4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            float t[8];
-            widen8(ld_stream_16(xp + q), t);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[8 * q + i] = t[i];
+        for (int s = 0; s < 2; ++s) {
+            const uint16_t* plo = X + r_lo * d + j * 32 + 16 * s + 2 * q;
+            const uint16_t* phi = X + r_hi * d + j * 32 + 16 * s + 2 * q;
+            a[s][0] = r_lo < rows ? __ldg(reinterpret_cast<const uint32_t*>(plo)) : 0u;
+            a[s][1] = r_hi < rows ? __ldg(reinterpret_cast<const uint32_t*>(phi)) : 0u;
+            a[s][2] = r_lo < rows ? __ldg(reinterpret_cast<const uint32_t*>(plo + 8)) : 0u;
+            a[s][3] = r_hi < rows ? __ldg(reinterpret_cast<const uint32_t*>(phi + 8)) : 0u;
         }
-        float v[32];
+        float acc[4][4];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) v[c] = 0.f;
+        for (int t = 0; t < 4; ++t)
 #pragma unroll
-        for (int r = 0; r < 32; ++r) {
+            for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
 #pragma unroll
-            for (int c4 = 0; c4 < 8; ++c4) {
-                const float4 b = *reinterpret_cast<const float4*>(&Bs[r][4 * c4]);
-                v[4 * c4 + 0] = fmaf(x[r], b.x, v[4 * c4 + 0]);
-                v[4 * c4 + 1] = fmaf(x[r], b.y, v[4 * c4 + 1]);
-                v[4 * c4 + 2] = fmaf(x[r], b.z, v[4 * c4 + 2]);
-                v[4 * c4 + 3] = fmaf(x[r], b.w, v[4 * c4 + 3]);
+        for (int m = 2; m >= 0; --m)           // smallest term first
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int s = 0; s < 2; ++s) mma_bf16_16816(acc[t], a[s], bf[m][t][s][0], bf[m][t][s][1]);
+        float sq_it = 0.f;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            // this thread's 8 values of row (g + 8 half): columns 8t + 2q, 8t + 2q + 1
+            float v[8];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) { v[2 * t] = acc[t][2 * half]; v[2 * t + 1] = acc[t][2 * half + 1]; }
+            float amax = absmax8(v);
+            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+            const uint32_t S = e8m0_from_amax(amax);
+            const float inv = inv_scale_from_e8m0(S), sc = scale_from_e8m0(S);
+            const uint32_t codes = e2m1x8(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv,
+                                          v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
+            const int64_t row = half ? r_hi : r_lo;
+            const int rpos = warp * 16 + g + 8 * half;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const float q0 = e2m1_nibble_value(codes >> (8 * t)) * sc;
+                const float q1 = e2m1_nibble_value(codes >> (8 * t + 4)) * sc;
+                const float e0 = v[2 * t] - q0, e1 = v[2 * t + 1] - q1;
+                sq_it = fmaf(e0, e0, fmaf(e1, e1, sq_it));
+                const __nv_bfloat162 hq = __floats2bfloat162_rn(q0, q1);
+                const uint32_t packed = *reinterpret_cast<const uint32_t*>(&hq);
+                const int col = 8 * t + 2 * q;
+                tt[col][rpos] = (uint16_t)(packed & 0xFFFFu);
+                tt[col + 1][rpos] = (uint16_t)(packed >> 16);
+                if (row < rows) {
+                    *reinterpret_cast<uint32_t*>(Vq + row * d + j * 32 + col) = packed;
+                    *reinterpret_cast<float2*>(Res + row * d + j * 32 + col) = make_float2(e0, e1);
+                }
             }
         }
-        float amax = 0.f;
+        sq += (double)sq_it;
+        __syncthreads();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) amax = fmaxf(amax, fabsf(v[c]));
-        const uint32_t S = e8m0_from_amax(amax);
-        const float inv = inv_scale_from_e8m0(S), sc = scale_from_e8m0(S);
-        uint4* qp = reinterpret_cast<uint4*>(Vq + row * d + j * 32);
-        float4* rp = reinterpret_cast<float4*>(Res + row * d + j * 32);
-        float sq_row = 0.f;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const uint32_t codes = e2m1x8(v[8 * g] * inv, v[8 * g + 1] * inv, v[8 * g + 2] * inv, v[8 * g + 3] * inv,
-                                          v[8 * g + 4] * inv, v[8 * g + 5] * inv, v[8 * g + 6] * inv, v[8 * g + 7] * inv);
-            float qv[8], rr[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                qv[i] = e2m1_nibble_value(codes >> (4 * i)) * sc;
-                rr[i] = v[8 * g + i] - qv[i];
-                sq_row = fmaf(rr[i], rr[i], sq_row);
-            }
-            uint32_t w[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const __nv_bfloat162 h = __floats2bfloat162_rn(qv[2 * i], qv[2 * i + 1]);
-                w[i] = *reinterpret_cast<const uint32_t*>(&h);
-            }
-            qp[g] = make_uint4(w[0], w[1], w[2], w[3]);
-            rp[2 * g] = make_float4(rr[0], rr[1], rr[2], rr[3]);
-            rp[2 * g + 1] = make_float4(rr[4], rr[5], rr[6], rr[7]);
+        for (int i = 0; i < 2; ++i) {
+            const int seg = threadIdx.x + 128 * i;
+            const int col = seg >> 3, rs = (seg & 7) * 8;
+            if (row0 + rs < rows)          // rows is a multiple of 8: a segment is all valid or all past the end
+                *reinterpret_cast<uint4*>(VqT + (int64_t)(j * 32 + col) * rows + row0 + rs) =
+                    *reinterpret_cast<const uint4*>(&tt[col][rs]);
         }
-        sq += (double)sq_row;
+        __syncthreads();
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+    if (lane == 0) red[warp] = sq;
     __syncthreads();
     if (threadIdx.x == 0) {
         const double t = red[0] + red[1] + red[2] + red[3];
         if (t != 0.0) atomicAdd(sumsq, t);
     }
-}
-
-// ---- bf16 transpose: in [R][C] -> out [C][R]; 64 x 64 tiles, 256 threads ---------------------
-__global__ void __launch_bounds__(256)
-transpose_bf16(const uint16_t* __restrict__ in, uint16_t* __restrict__ out, int64_t R, int64_t C) {
-    __shared__ uint16_t tile[64][66];
-    const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
-    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
-    for (int i = ty; i < 64; i += 4)
-        if (r0 + i < R && c0 + tx < C) tile[i][tx] = in[(r0 + i) * C + c0 + tx];
-    __syncthreads();
-    for (int i = ty; i < 64; i += 4)
-        if (c0 + i < C && r0 + tx < R) out[(c0 + i) * R + r0 + tx] = tile[tx][i];
 }
 
 // ---- block gradients: part[chunk][j][32][32] = sum over the chunk's rows of x_j^T g_j ---------

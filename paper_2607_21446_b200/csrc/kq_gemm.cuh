@@ -1,7 +1,7 @@
 // bf16 x bf16 -> fp32 "NT" GEMM for sm_100a, used by the calibration loop (paper Section 3.3):
 //     C[M][N] = A[M][K] * B[N][K]^T,     A and B row-major with K contiguous,
 // with a fused epilogue   v = acc + coef * aux[row][col];  [sum += v^2];  out = v (fp32)
-// or out = bf16(out_scale * v).  The three contractions of one calibration step
+// or out = bf16(out_scale * v) (optionally also its transpose).  The three contractions of one calibration step
 // (Q(AT) Q(WT^-T)^T - A W^T, dO Q(WT^-T), dO^T Q(AT)) all have this form.
 //
 // One persistent CTA per SM: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
@@ -49,6 +49,8 @@ struct GemmProblem {
     float* out_f32;            // [M][ld_out] or null
     __nv_bfloat16* out_bf16;   // [M][ld_out] or null
     int64_t ld_out;
+    __nv_bfloat16* out_bf16_t; // transposed copy of the bf16 output, [N][ld_out_t], or null
+    int64_t ld_out_t;
     double* sumsq;             // += sum of v^2 over the whole matrix, or null
 };
 
@@ -237,6 +239,12 @@ gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
                             w[h] = *reinterpret_cast<const uint32_t*>(&b);
                         }
                         op[q] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    if (p.out_bf16_t) {
+                        // lanes hold consecutive rows: each store instruction writes 64 contiguous bytes
+                        __nv_bfloat16* tp = p.out_bf16_t + (int64_t)col * p.ld_out_t + row;
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) tp[(int64_t)q * p.ld_out_t] = __float2bfloat16_rn(v[q] * p.out_scale);
                     }
                 }
                 }

@@ -44,7 +44,8 @@ bool make_operand_map(CUtensorMap* tm, const void* ptr, int64_t rows, int64_t K,
 
 kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, int M, int N, int K, const float* aux,
                         int64_t ld_aux, const float* coef_ptr, float coef_mul, float out_scale, float* out_f32,
-                        __nv_bfloat16* out_bf16, int64_t ld_out, double* sumsq, cudaStream_t st) {
+                        __nv_bfloat16* out_bf16, int64_t ld_out, double* sumsq, cudaStream_t st,
+                        __nv_bfloat16* out_bf16_t = nullptr, int64_t ld_out_t = 0) {
     static std::atomic<int> attr_done{0};
     if (!attr_done.load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kq::gemm_nt_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kGemmDynBytes) !=
@@ -61,6 +62,7 @@ kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, int M, int
     p.k_blocks = (K + kq::kGemmBK - 1) / kq::kGemmBK;
     p.aux = aux; p.ld_aux = ld_aux; p.coef_ptr = coef_ptr; p.coef_mul = coef_mul; p.out_scale = out_scale;
     p.out_f32 = out_f32; p.out_bf16 = out_bf16; p.ld_out = ld_out; p.sumsq = sumsq;
+    p.out_bf16_t = out_bf16_t; p.ld_out_t = ld_out_t;
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
     const int tiles = p.tiles_m * p.tiles_n;
@@ -114,30 +116,25 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
     if (!launched()) return KQ_ERR_CUDA;
     if (cudaMemsetAsync(c->sums, 0, 3 * sizeof(double), st) != cudaSuccess) return KQ_ERR_CUDA;
     auto fq_grid = [&](int64_t rows) {
-        int64_t gx = (rows + 127) / 128;
+        int64_t gx = (rows + kq::kFqRows - 1) / kq::kFqRows;
         const int64_t cap = ((int64_t)sms * 16 + nb - 1) / nb;        // about 16 CTAs of 128 threads per SM
         if (gx > cap) gx = cap;
         if (gx < 1) gx = 1;
         return dim3((unsigned)gx, (unsigned)nb);
     };
-    kq::calib_fakequant<<<fq_grid(M), 128, 0, st>>>(c->A, c->Kd, c->n_sets, M, d, c->Yq, c->ResY, c->sums + 1);
+    kq::calib_fakequant<<<fq_grid(M), 128, 0, st>>>(c->A, c->Kd, c->n_sets, M, d, c->Yq, c->YqT, c->ResY, c->sums + 1);
     if (!launched()) return KQ_ERR_CUDA;
-    kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, c->ResZ, c->sums + 2);
+    kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, c->ZqT, c->ResZ, c->sums + 2);
     if (!launched()) return KQ_ERR_CUDA;
     // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o))
     kq_status_t rc = launch_gemm(c->tm_Yq_a, c->tm_Zq_b, (int)M, o, d, c->R, o, nullptr, -1.0f,
-                                 (float)(2.0 / ((double)M * o)), nullptr, backward ? c->dO : nullptr, o, c->sums, st);
+                                 (float)(2.0 / ((double)M * o)), nullptr, backward ? c->dO : nullptr, o, c->sums, st,
+                                 backward ? c->dOT : nullptr, M);
     if (rc != KQ_OK) return rc;
     if (hist_row >= 0 &&
         cudaMemcpyAsync(c->hist + 3 * hist_row, c->sums, 3 * sizeof(double), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return KQ_ERR_CUDA;
     if (!backward) return KQ_OK;
-    auto tr = [&](const __nv_bfloat16* in, __nv_bfloat16* out, int64_t R, int64_t C) {
-        kq::transpose_bf16<<<dim3((unsigned)((C + 63) / 64), (unsigned)((R + 63) / 64)), 256, 0, st>>>(
-            reinterpret_cast<const uint16_t*>(in), reinterpret_cast<uint16_t*>(out), R, C);
-        return launched();
-    };
-    if (!tr(c->Yq, c->YqT, M, d) || !tr(c->Zq, c->ZqT, o, d) || !tr(c->dO, c->dOT, M, o)) return KQ_ERR_CUDA;
     // dY = dO Zq + lambda_A 2 (Y - Yq) / (M d);  dZ = dO^T Yq + lambda_W 2 (Z - Zq) / (o d)
     rc = launch_gemm(c->tm_dO_a, c->tm_ZqT_b, (int)M, d, o, c->ResY, d, c->lam, (float)(2.0 / ((double)M * d)), 1.0f,
                      c->dY, nullptr, d, nullptr, st);
