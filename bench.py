@@ -546,6 +546,91 @@ def run_table(args):
             del Xs, x0
 
 
+def run_calib(args):
+    """Calibration loop (Section 3.3): `--steps` Adam steps on a synthetic layer, timed with CUDA
+    events on the launching stream after `--warmup` steps.  One JSON line: ms per step, the rate of
+    the three contractions of a step (3 x 2 M o d flop) against the measured bf16 tensor peak, the
+    objective before/after, and the float64 oracle timed on a row sample of the same layer."""
+    import torch
+    from paper_2607_21446_b200 import binding as B
+    B.load_library()
+    M, o, d = (int(v) for v in args.calib.lower().split("x"))
+    n_sets = d // 32 if args.per_block else 1
+    A_bits = W.gen_activations(W.calib_spec(M, d))
+    W_bits = W.gen_weights(5, o, d)
+    dev = torch.device("cuda:0")
+    A_t = torch.from_numpy(A_bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    W_t = torch.from_numpy(W_bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    stream = torch.cuda.current_stream()
+    launches0 = B.kroquant_launch_count()
+    cal = B.Calibrator(A_t, W_t, n_sets)
+    lam = cal.lambdas.astype(np.float64)
+    l_first, _ = cal.loss_grad(grad=False)
+    cal.run(max(args.warmup, 3), history=False)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    t_wait = time.time()
+    while sampler.count() < 2 and time.time() - t_wait < 3.0:
+        cal.run(1, history=False)
+        torch.cuda.synchronize()
+    l0 = B.kroquant_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    cal.run(args.steps, history=False)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    launches = B.kroquant_launch_count() - l0
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1) / args.steps
+    l_last, _ = cal.loss_grad(grad=False)
+    flop = 3 * 2.0 * M * o * d
+    peak_tf, kind = 1590.0, "fallback"
+    pth = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pth):
+        with open(pth) as f:
+            mp = json.load(f)
+        if "bf16_tflops" in mp:
+            peak_tf, kind = float(mp["bf16_tflops"]), "measured"
+    # CPU oracle on a bounded sample: the first rows of A with the full W (cost is linear in rows)
+    from oracle import calib_oracle as co
+    rows_s = min(M, max(64, int(5.0e11 // (6.0 * o * d)) // 8 * 8))      # about 10 s of CPU work
+    A_s = W.bf16_bits_to_f32(A_bits[:rows_s]).astype(np.float64)
+    W_s = W.bf16_bits_to_f32(W_bits).astype(np.float64)
+    th = co.hadamard_theta(n_sets)
+    t0 = time.time()
+    _, terms_s, g_s = co.loss_and_grad(A_s, W_s, th, lam[0], lam[1])
+    cpu_s = time.time() - t0
+    # parity of the sample on the GPU: same rows, same parameters, same lambdas
+    cal_s = B.Calibrator(A_t[:rows_s].contiguous(), W_t, n_sets)
+    cal_s.lambdas = lam.astype(np.float32)
+    terms_g, g_g = cal_s.loss_grad()
+    parity = {"rows": rows_s,
+              "loss_rel_err": float(np.max(np.abs(terms_g - terms_s) / np.abs(terms_s))),
+              "grad_err_over_max": float(np.abs(g_g - g_s).max() / np.abs(g_s).max())}
+    cal_s.destroy()
+    tot = lambda l: float(l[0] + lam[0] * l[1] + lam[1] * l[2])
+    print(json.dumps({
+        "metric": "calibration_step_time", "value": round(ms, 4), "unit": "ms", "higher_is_better": False,
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "dtype": "bf16 operands, fp32 accumulate",
+        "data": "synthetic", "config": {"workload": f"calibration M={M} o={o} d={d} n_sets={n_sets}",
+                                        "l2": "operands and work space exceed L2"},
+        "gpu_launches": int(launches), "launches_per_step": launches / args.steps,
+        "roofline": {"bound": "tensor", "achieved": round(flop / ms / 1e9, 1), "peak": peak_tf, "unit": "TFLOP/s",
+                     "frac": round(flop / ms / 1e9 / peak_tf, 4), "traffic": None,
+                     "note": f"3 contractions x 2 M o d flop / step time, of {kind} bf16 peak; the step also "
+                             "runs the fake-quant, block-gradient and optimiser kernels"},
+        "objective": {"lambda_A": lam[0], "lambda_W": lam[1], "at_init": [float(v) for v in l_first],
+                      "after": [float(v) for v in l_last], "total_at_init": tot(l_first), "total_after": tot(l_last),
+                      "adam_steps_taken": int(args.steps + max(args.warmup, 3))},
+        "cpu_baseline": {"value": round(cpu_s * 1e3 * M / rows_s, 1), "unit": "ms", "cores": os.cpu_count(),
+                         "kind": "oracle", "sample": f"one loss+gradient evaluation on the first {rows_s} of {M} rows "
+                                                     f"({cpu_s:.2f} s), scaled linearly in rows"},
+        "parity": parity, "clocks": clocks, "device_error": B.kroquant_last_device_error(),
+    }), flush=True)
+    cal.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", action="store_true",
@@ -557,6 +642,8 @@ def main():
     ap.add_argument("--kernel", default="kroquant", choices=["kroquant", "scale", "plain"])
     ap.add_argument("--calls", type=int, default=8)
     ap.add_argument("--per-block", action="store_true", help="with --single: one factor set per 32-channel block")
+    ap.add_argument("--calib", default=None, metavar="MxOxD",
+                    help="calibration loop on a synthetic layer, e.g. 16384x3072x3072 (with --per-block: one set per block)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
@@ -569,6 +656,8 @@ def main():
         run_sweep(args)
     elif args.single:
         run_single(args)
+    elif args.calib:
+        run_calib(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -44,10 +44,11 @@ calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, fl
 // quantizer kernels followed by its decoder; Vq is exact in bf16.  Outputs: Vq [rows][d],
 // its transpose VqT [d][rows] (staged through shared memory, 16-byte segments), R = V - Vq,
 // and the sum of R^2.
-__device__ __forceinline__ float e2m1_nibble_value(uint32_t code) {
-    const uint32_t m = code & 7u;
-    const float mag = m < 2u ? 0.5f * (float)m : (float)(2u + (m & 1u)) * (float)(1u << ((m >> 1) - 1u)) * 0.5f;
-    return (code & 8u) ? -mag : mag;
+// two E2M1 codes (one byte, even element in the low nibble) -> two floats, by the hardware convert
+__device__ __forceinline__ float2 e2m1x2_to_float2(uint32_t byte) {
+    uint32_t h2;
+    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(byte));
+    return __half22float2(*reinterpret_cast<const __half2*>(&h2));
 }
 __device__ __forceinline__ void split3_bf16(float x, uint32_t (&t)[3]) {
     const __nv_bfloat16 h0 = __float2bfloat16_rn(x);
@@ -89,9 +90,9 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
                 for (int m = 0; m < 3; ++m) bf[m][t][s][h] = lo[m] | (hi[m] << 16);
             }
     double sq = 0.0;
-    for (int64_t row0 = (int64_t)blockIdx.x * kFqRows; row0 < rows; row0 += (int64_t)gridDim.x * kFqRows) {
+    // A fragments of the 16 rows this warp owns in the 64-row group starting at row0
+    auto load_a = [&](int64_t row0, uint32_t (&a)[2][4]) {
         const int64_t r_lo = row0 + warp * 16 + g, r_hi = r_lo + 8;
-        uint32_t a[2][4];
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
             const uint16_t* plo = X + r_lo * d + j * 32 + 16 * s + 2 * q;
@@ -101,6 +102,18 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
             a[s][2] = r_lo < rows ? __ldg(reinterpret_cast<const uint32_t*>(plo + 8)) : 0u;
             a[s][3] = r_hi < rows ? __ldg(reinterpret_cast<const uint32_t*>(phi + 8)) : 0u;
         }
+    };
+    const int64_t stride = (int64_t)gridDim.x * kFqRows;
+    uint32_t a_next[2][4];
+    load_a((int64_t)blockIdx.x * kFqRows, a_next);
+    for (int64_t row0 = (int64_t)blockIdx.x * kFqRows; row0 < rows; row0 += stride) {
+        const int64_t r_lo = row0 + warp * 16 + g, r_hi = r_lo + 8;
+        uint32_t a[2][4];
+#pragma unroll
+        for (int s = 0; s < 2; ++s)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[s][i] = a_next[s][i];
+        if (row0 + stride < rows) load_a(row0 + stride, a_next);      // in flight during this group's math and stores
         float acc[4][4];
 #pragma unroll
         for (int t = 0; t < 4; ++t)
@@ -130,8 +143,8 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
             const int rpos = warp * 16 + g + 8 * half;
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
-                const float q0 = e2m1_nibble_value(codes >> (8 * t)) * sc;
-                const float q1 = e2m1_nibble_value(codes >> (8 * t + 4)) * sc;
+                const float2 dq = e2m1x2_to_float2((codes >> (8 * t)) & 0xFFu);
+                const float q0 = dq.x * sc, q1 = dq.y * sc;
                 const float e0 = v[2 * t] - q0, e1 = v[2 * t + 1] - q1;
                 sq_it = fmaf(e0, e0, fmaf(e1, e1, sq_it));
                 const __nv_bfloat162 hq = __floats2bfloat162_rn(q0, q1);
@@ -168,8 +181,10 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
 }
 
 // ---- block gradients: part[chunk][j][32][32] = sum over the chunk's rows of x_j^T g_j ---------
-// grid (chunks, d/32); 256 threads = 4 row groups x 64; a thread owns a 4 x 4 patch of the
-// 32 x 32 result for its row group; tiles of 64 rows are staged in shared memory as fp32.
+// grid (chunks, d/32); 256 threads = 4 row groups x 64 patches; a thread owns a 4 x 4 patch of the
+// 32 x 32 result for its row group; tiles of 64 rows are staged in shared memory as fp32 while the
+// next tile's global loads are already in flight.  (8 x 8 patches halve the shared-memory reads
+// per FMA but cost so many registers that the kernel ran slower.)
 constexpr int kGradTileRows = 64;
 __global__ void __launch_bounds__(256)
 calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, int64_t rows, int d,
@@ -179,36 +194,42 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
     const int j = blockIdx.y;
     const int64_t r_begin = (int64_t)blockIdx.x * rows_per_chunk;
     const int64_t r_end = r_begin + rows_per_chunk < rows ? r_begin + rows_per_chunk : rows;
-    const int grp = threadIdx.x >> 6;
+    const int grp = threadIdx.x >> 6;                         // 4 row groups of 16 rows per tile
     const int r4 = ((threadIdx.x & 63) >> 3) * 4, c4 = (threadIdx.x & 7) * 4;
     float acc[4][4];
 #pragma unroll
     for (int a = 0; a < 4; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    // global -> registers for the tile after the one being multiplied: thread -> (row = tid / 4,
+    // 8 channels = (tid % 4) * 8)
+    const int lr_st = threadIdx.x >> 2, ch_st = (threadIdx.x & 3) * 8;
+    uint4 px = make_uint4(0u, 0u, 0u, 0u);
+    float4 pg0 = make_float4(0.f, 0.f, 0.f, 0.f), pg1 = pg0;
+    auto fetch = [&](int64_t t0) {
+        const int64_t row = t0 + lr_st;
+        if (row < r_end) {
+            px = ld_stream_16(X + row * d + j * 32 + ch_st);
+            const float4* gp = reinterpret_cast<const float4*>(G + row * d + j * 32 + ch_st);
+            pg0 = __ldg(gp);
+            pg1 = __ldg(gp + 1);
+        } else {
+            px = make_uint4(0u, 0u, 0u, 0u);
+            pg0 = pg1 = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    if (r_begin < r_end) fetch(r_begin);
     for (int64_t t0 = r_begin; t0 < r_end; t0 += kGradTileRows) {
-        // stage: thread -> (row = tid / 4, 8 channels = (tid % 4) * 8)
         {
-            const int lr = threadIdx.x >> 2, ch = (threadIdx.x & 3) * 8;
-            const int64_t row = t0 + lr;
             float xv[8];
-            float4 g0, g1;
-            if (row < r_end) {
-                widen8(ld_stream_16(X + row * d + j * 32 + ch), xv);
-                const float4* gp = reinterpret_cast<const float4*>(G + row * d + j * 32 + ch);
-                g0 = __ldg(gp);
-                g1 = __ldg(gp + 1);
-            } else {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) xv[i] = 0.f;
-                g0 = g1 = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            *reinterpret_cast<float4*>(&xs[lr][ch]) = make_float4(xv[0], xv[1], xv[2], xv[3]);
-            *reinterpret_cast<float4*>(&xs[lr][ch + 4]) = make_float4(xv[4], xv[5], xv[6], xv[7]);
-            *reinterpret_cast<float4*>(&gs[lr][ch]) = g0;
-            *reinterpret_cast<float4*>(&gs[lr][ch + 4]) = g1;
+            widen8(px, xv);
+            *reinterpret_cast<float4*>(&xs[lr_st][ch_st]) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+            *reinterpret_cast<float4*>(&xs[lr_st][ch_st + 4]) = make_float4(xv[4], xv[5], xv[6], xv[7]);
+            *reinterpret_cast<float4*>(&gs[lr_st][ch_st]) = pg0;
+            *reinterpret_cast<float4*>(&gs[lr_st][ch_st + 4]) = pg1;
         }
         __syncthreads();
+        if (t0 + kGradTileRows < r_end) fetch(t0 + kGradTileRows);       // lands while this tile is multiplied
 #pragma unroll 4
         for (int i = 0; i < kGradTileRows / 4; ++i) {
             const int lr = grp * (kGradTileRows / 4) + i;
@@ -223,8 +244,8 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
         }
         __syncthreads();
     }
-    // sum the four row groups through shared memory (reuse xs/gs: 2 x 8 KB = 4 x 1024 floats)
-    float* red = &xs[0][0];            // xs and gs are adjacent only by luck; use them separately
+    // sum the four row groups through the staging memory (2 x 8 KB = 4 x 1024 floats)
+    float* red = &xs[0][0];
     float* red2 = &gs[0][0];
     float* mine = grp < 2 ? red + grp * 1024 : red2 + (grp - 2) * 1024;
 #pragma unroll
@@ -232,9 +253,15 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
 #pragma unroll
         for (int b = 0; b < 4; ++b) mine[(r4 + a) * 32 + c4 + b] = acc[a][b];
     __syncthreads();
+    float tot[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int e = threadIdx.x + 256 * i;
+        tot[i] = (red[e] + red[1024 + e]) + (red2[e] + red2[1024 + e]);
+    }
     float* dst = part + ((size_t)blockIdx.x * gridDim.y + j) * 1024;
-    for (int i = threadIdx.x; i < 1024; i += 256)
-        dst[i] = (red[i] + red[1024 + i]) + (red2[i] + red2[1024 + i]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) dst[threadIdx.x + 256 * i] = tot[i];
 }
 
 // ---- sum of partial blocks: out[j][e] = sum_p part[p][j][e], e < 1024 --------------------------

@@ -5,7 +5,7 @@
 // (Q(AT) Q(WT^-T)^T - A W^T, dO Q(WT^-T), dO^T Q(AT)) all have this form.
 //
 // One persistent CTA per SM: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
-// warps 2..5 = epilogue.  Tile 128 x 256, K step 64 (one 128-byte swizzle atom), four
+// warps 2..9 = epilogue (two warps per TMEM lane quarter, each taking half of the columns).  Tile 128 x 256, K step 64 (one 128-byte swizzle atom), four
 // stages of 48 KB, two 256-column fp32 accumulators in TMEM so that the epilogue of
 // tile i overlaps the main loop of tile i + 1.  The products are exact whenever the
 // operands are MXFP4 values (they are bf16-representable); only the fp32 accumulation
@@ -23,7 +23,7 @@ constexpr int kGemmABytes = kGemmBM * kGemmBK * 2;            // 16 KB
 constexpr int kGemmBBytes = kGemmBN * kGemmBK * 2;            // 32 KB
 constexpr int kGemmStageBytes = kGemmABytes + kGemmBBytes;    // 48 KB
 constexpr int kGemmGroupM = 16;                               // tile rasterisation: 16 row tiles per group
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 320;                             // producer, issuer, 8 epilogue warps
 // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2]
 constexpr int kGemmBarOff = kGemmStages * kGemmStageBytes;
 constexpr int kGemmNumBars = 2 * kGemmStages + 4;
@@ -105,7 +105,7 @@ gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kGemmStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull(a), 1); mbar_init(bar_tempty(a), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull(a), 1); mbar_init(bar_tempty(a), 8); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -179,8 +179,9 @@ gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
             }
         }
     } else {
-        // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+        // ---------------- epilogue: warps 2..9, TMEM lane quarter = warp % 4 ----------------
         const int quarter = warp & 3;
+        const int chalf = (warp - 2) >> 2;                  // which half of the tile's columns
         const float coef = p.coef_mul * (p.coef_ptr ? __ldg(p.coef_ptr) : 1.0f);
         double sq = 0.0;
         for (int i = 0; i < my_tiles; ++i) {
@@ -195,7 +196,7 @@ gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
             const int64_t row = (int64_t)tm * kGemmBM + quarter * 32 + lane;
             const bool row_ok = row < p.M;
             float sq_tile = 0.f;
-            for (int c = 0; c < kGemmBN / 32; ++c) {
+            for (int c = chalf * (kGemmBN / 64); c < (chalf + 1) * (kGemmBN / 64); ++c) {
                 const int col = tn * kGemmBN + c * 32;
                 if (col >= p.N) break;                      // warp-uniform; N is a multiple of 32
                 uint32_t r[32];
