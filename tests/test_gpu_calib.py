@@ -3,8 +3,8 @@
 Tolerances (derived in the design notes): the forward contraction has exact products and fp32
 accumulation, the transform is fp32 FMA, so the three loss terms agree to ~1e-5 relative; codes that
 sit on a rounding boundary may flip, which moves L_out by O(1/(M d)) relative.  The output error is
-rounded to bf16 (2^-9 relative per element, independent signs) before the two backward contractions,
-which bounds the gradient error by a few 1e-3 of its largest component.
+rounded to bf16 (2^-9 relative per element, independent signs) before the two backward contractions;
+over the o M terms of a block-gradient entry that averages down to ~1e-5 of the largest component.
 """
 import numpy as np
 import pytest
@@ -16,8 +16,8 @@ from paper_2607_21446_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-LOSS_RTOL = 2e-4
-GRAD_TOL = 5e-3          # of max |g|
+LOSS_RTOL = 1e-4         # measured 2e-7 ... 3e-5 (largest at the Hadamard start, where values sit on ties)
+GRAD_TOL = 5e-4          # of max |g|; measured 2e-6 ... 9e-5
 
 
 def _case(M, o, d, seed):
