@@ -554,6 +554,7 @@ def run_calib(args):
     import torch
     from paper_2607_21446_b200 import binding as B
     B.load_library()
+    B.set_gemm_pair(not args.gemm_single)
     M, o, d = (int(v) for v in args.calib.lower().split("x"))
     n_sets = d // 32 if args.per_block else 1
     A_bits = W.gen_activations(W.calib_spec(M, d))
@@ -614,6 +615,7 @@ def run_calib(args):
         "metric": "calibration_step_time", "value": round(ms, 4), "unit": "ms", "higher_is_better": False,
         "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "dtype": "bf16 operands, fp32 accumulate",
         "data": "synthetic", "config": {"workload": f"calibration M={M} o={o} d={d} n_sets={n_sets}",
+                                        "gemm": "one CTA, 128x256 tiles" if args.gemm_single else "CTA pairs, 256x256 tiles",
                                         "l2": "operands and work space exceed L2"},
         "gpu_launches": int(launches), "launches_per_step": launches / args.steps,
         "roofline": {"bound": "tensor", "achieved": round(flop / ms / 1e9, 1), "peak": peak_tf, "unit": "TFLOP/s",
@@ -644,6 +646,8 @@ def main():
     ap.add_argument("--per-block", action="store_true", help="with --single: one factor set per 32-channel block")
     ap.add_argument("--calib", default=None, metavar="MxOxD",
                     help="calibration loop on a synthetic layer, e.g. 16384x3072x3072 (with --per-block: one set per block)")
+    ap.add_argument("--gemm-single", action="store_true",
+                    help="with --calib: one-CTA 128x256 GEMM tiles instead of CTA pairs on 256x256 tiles")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)

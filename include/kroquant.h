@@ -199,6 +199,11 @@ kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_
  * error is rounded to bf16 once before the two backward contractions. */
 typedef struct kroquant_calib kroquant_calib_t;
 
+/* Test and tuning knob: which tensor-core GEMM the calibration calls launch from now on.
+ * 1 (default): pairs of CTAs on 256 x 256 tiles (tcgen05 cta_group::2); 0: one CTA per 128 x 256
+ * tile.  Both compute the same contractions; results differ only in fp32 summation order. */
+kq_status_t kroquant_debug_set_gemm_pair(int on);
+
 kq_status_t kroquant_calib_create(const void *A, const void *W, int64_t M, int o, int d, int n_sets,
                                   void *stream, kroquant_calib_t **out);
 void kroquant_calib_destroy(kroquant_calib_t *c);

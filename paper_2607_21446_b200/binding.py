@@ -33,6 +33,7 @@ EXPORTS = [
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
     "kroquant_calib_loss_grad", "kroquant_calib_run",
     "kroquant_block_grad_scratch_bytes", "kroquant_block_grad", "kroquant_block_grad_static",
+    "kroquant_debug_set_gemm_pair",
 ]
 
 
@@ -94,6 +95,7 @@ def load_library() -> C.CDLL:
     L.kroquant_block_grad_scratch_bytes.restype = i64
     L.kroquant_block_grad.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, vp]
     L.kroquant_block_grad_static.argtypes = [vp, vp, i64, i32, i32, vp, vp]
+    L.kroquant_debug_set_gemm_pair.argtypes = [i32]
     _lib = L
     return L
 
@@ -406,6 +408,11 @@ def kroquant_block_grad_static(X: torch.Tensor, G: torch.Tensor, n_sets: int, ou
         raise ValueError("out must be a contiguous CUDA float32 tensor [n_sets, 32, 32]")
     _check(load_library().kroquant_block_grad_static(_ptr(X), _ptr(G), rows, d, n_sets, _ptr(out), _stream(stream)),
            "kroquant_block_grad_static")
+
+
+def set_gemm_pair(on: bool) -> None:
+    """Choose the calibration GEMM: pairs of CTAs on 256 x 256 tiles (default) or one CTA per tile."""
+    _check(load_library().kroquant_debug_set_gemm_pair(1 if on else 0), "kroquant_debug_set_gemm_pair")
 
 
 class Calibrator:

@@ -82,6 +82,54 @@ __device__ __forceinline__ void gemm_tile_coords(int t, const GemmProblem& p, in
     tn = r / m_count;
 }
 
+// Epilogue of one row x 32 columns held in registers: v = acc + coef * aux; [sum v^2]; stores.
+__device__ __forceinline__ void gemm_epilogue_chunk(const GemmProblem& p, const uint32_t (&r)[32], int64_t row, int col,
+                                                    float coef, float& sq_tile) {
+    float v[32];
+    if (p.aux) {
+        const float4* ap = reinterpret_cast<const float4*>(p.aux + row * p.ld_aux + col);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 a = __ldg(ap + q);
+            v[4 * q + 0] = fmaf(coef, a.x, __uint_as_float(r[4 * q + 0]));
+            v[4 * q + 1] = fmaf(coef, a.y, __uint_as_float(r[4 * q + 1]));
+            v[4 * q + 2] = fmaf(coef, a.z, __uint_as_float(r[4 * q + 2]));
+            v[4 * q + 3] = fmaf(coef, a.w, __uint_as_float(r[4 * q + 3]));
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
+    }
+    if (p.sumsq) {
+#pragma unroll
+        for (int q = 0; q < 32; ++q) sq_tile = fmaf(v[q], v[q], sq_tile);
+    }
+    if (p.out_f32) {
+        float4* op = reinterpret_cast<float4*>(p.out_f32 + row * p.ld_out + col);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    }
+    if (p.out_bf16) {
+        uint4* op = reinterpret_cast<uint4*>(p.out_bf16 + row * p.ld_out + col);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * q + 2 * h] * p.out_scale, v[8 * q + 2 * h + 1] * p.out_scale);
+                w[h] = *reinterpret_cast<const uint32_t*>(&b);
+            }
+            op[q] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        if (p.out_bf16_t) {
+            // lanes hold consecutive rows: each store instruction writes 64 contiguous bytes
+            __nv_bfloat16* tp = p.out_bf16_t + (int64_t)col * p.ld_out_t + row;
+#pragma unroll
+            for (int q = 0; q < 32; ++q) tp[(int64_t)q * p.ld_out_t] = __float2bfloat16_rn(v[q] * p.out_scale);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
              const GemmProblem p) {
@@ -203,52 +251,7 @@ gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
                 tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kGemmBN + c * 32), r);
                 // rows past M are computed on zero-filled operands and dropped; the warp reconverges
                 // below before the next (warp-wide) TMEM load
-                if (row_ok) {
-                float v[32];
-                if (p.aux) {
-                    const float4* ap = reinterpret_cast<const float4*>(p.aux + row * p.ld_aux + col);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 a = __ldg(ap + q);
-                        v[4 * q + 0] = fmaf(coef, a.x, __uint_as_float(r[4 * q + 0]));
-                        v[4 * q + 1] = fmaf(coef, a.y, __uint_as_float(r[4 * q + 1]));
-                        v[4 * q + 2] = fmaf(coef, a.z, __uint_as_float(r[4 * q + 2]));
-                        v[4 * q + 3] = fmaf(coef, a.w, __uint_as_float(r[4 * q + 3]));
-                    }
-                } else {
-#pragma unroll
-                    for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
-                }
-                if (p.sumsq) {
-#pragma unroll
-                    for (int q = 0; q < 32; ++q) sq_tile = fmaf(v[q], v[q], sq_tile);
-                }
-                if (p.out_f32) {
-                    float4* op = reinterpret_cast<float4*>(p.out_f32 + row * p.ld_out + col);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-                }
-                if (p.out_bf16) {
-                    uint4* op = reinterpret_cast<uint4*>(p.out_bf16 + row * p.ld_out + col);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            const __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * q + 2 * h] * p.out_scale,
-                                                                           v[8 * q + 2 * h + 1] * p.out_scale);
-                            w[h] = *reinterpret_cast<const uint32_t*>(&b);
-                        }
-                        op[q] = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                    if (p.out_bf16_t) {
-                        // lanes hold consecutive rows: each store instruction writes 64 contiguous bytes
-                        __nv_bfloat16* tp = p.out_bf16_t + (int64_t)col * p.ld_out_t + row;
-#pragma unroll
-                        for (int q = 0; q < 32; ++q) tp[(int64_t)q * p.ld_out_t] = __float2bfloat16_rn(v[q] * p.out_scale);
-                    }
-                }
-                }
+                if (row_ok) gemm_epilogue_chunk(p, r, row, col, coef, sq_tile);
                 __syncwarp();
             }
             sq += (double)sq_tile;

@@ -1,0 +1,235 @@
+// Two-SM variant of the calibration GEMM (kq_gemm.cuh): a cluster of two CTAs works on one
+// 256 x 256 tile with tcgen05.mma.cta_group::2.  CTA r of the pair holds rows 128r..128r+127 of
+// the A tile and rows 128r..128r+127 of the B tile (half of the N extent) in its own shared memory
+// and the accumulators of its 128 output rows in its own TMEM; the instruction, issued by CTA 0
+// only, reads both CTAs' shared memory.  Per 128 x 256 x 16 of work an SM now reads 8 KB of
+// operands instead of 12 KB, which takes the shared-memory path out of the critical position
+// it has in the one-CTA kernel, and a stage shrinks to 32 KB, so six stages fit.
+//
+// Synchronisation (all barriers sit at the same offsets in both CTAs):
+//   full[s]   waited on by CTA 0's issuer; CTA 0's producer arms it with the bytes of BOTH CTAs'
+//             loads, and both producers direct their TMA completions to CTA 0's barrier;
+//   empty[s]  one per CTA, each waited on by that CTA's producer; released for both CTAs by one
+//             multicast tcgen05.commit of the issuer;
+//   tfull[a]  one per CTA, waited on by that CTA's epilogue; signalled by a multicast commit;
+//   tempty[a] CTA 0's only: the 8 epilogue warps of each CTA arrive on it (CTA 1 remotely).
+// No load uses cluster multicast.  Every wait is bounded; both CTAs meet at a cluster barrier
+// before they free TMEM and exit, so neither touches the other's shared memory after it is gone.
+#pragma once
+#include "kq_gemm.cuh"
+
+namespace kq {
+
+constexpr int kGemm2BM = 256;                                  // rows of the pair's tile
+constexpr int kGemm2Stages = 6;
+constexpr int kGemm2ABytes = 128 * kGemmBK * 2;                // 16 KB: this CTA's half of A
+constexpr int kGemm2BBytes = 128 * kGemmBK * 2;                // 16 KB: this CTA's half of B
+constexpr int kGemm2StageBytes = kGemm2ABytes + kGemm2BBytes;  // 32 KB
+constexpr int kGemm2BarOff = kGemm2Stages * kGemm2StageBytes;
+constexpr int kGemm2NumBars = 2 * kGemm2Stages + 4;
+constexpr int kGemm2TmemSlotOff = kGemm2BarOff + 8 * kGemm2NumBars;
+constexpr int kGemm2AbortOff = kGemm2TmemSlotOff + 4;
+constexpr int kGemm2DynBytes = kGemm2AbortOff + 4 + 1024;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank) {
+    uint32_t out;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(addr), "r"(rank));
+    return out;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of this CTA's box into its own shared memory; the completion goes to `bar_cluster`,
+// which may be the partner's barrier.  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar_cluster) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+                 " [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrive on the barrier at this offset in both CTAs of the pair once all MMAs issued so far are done
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// kind::f16, D = f32, A = B = bf16, both K-major, M = 256 (pair), N = 256
+__host__ __device__ constexpr uint32_t idesc_m256n256_bf16() {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+}
+
+// p.tiles_m counts 256-row tiles here.  gridDim.x = 2 x (number of pairs); cluster size 2.
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_nt_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const GemmProblem p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;            // the same offset in both CTAs
+    uint8_t* base_ptr = smem_raw + (base - raw);
+    const uint32_t bar0 = base + kGemm2BarOff;
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar0 + 8u * (kGemm2Stages + s); };
+    auto bar_tfull = [&](int a) { return bar0 + 8u * (2 * kGemm2Stages + a); };
+    auto bar_tempty = [&](int a) { return bar0 + 8u * (2 * kGemm2Stages + 2 + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kGemm2TmemSlotOff);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + kGemm2AbortOff);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                 // 0 = leader (issues the MMAs)
+    const int pair = (int)(blockIdx.x >> 1), n_pairs = (int)(gridDim.x >> 1);
+    const int n_tiles = p.tiles_m * p.tiles_n;
+    const int my_tiles = pair < n_tiles ? (n_tiles - pair + n_pairs - 1) / n_pairs : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kGemm2Stages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull(a), 1); mbar_init(bar_tempty(a), 16); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+    }
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + (uint32_t)kGemm2TmemSlotOff), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    // the partner's barriers must be initialised before anything is sent to them
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    int issued = 0;            // producer thread: pipeline iterations whose loads were issued
+    if (warp == 0) {
+        // ---------------- TMA producer (both CTAs) ----------------
+        if (lane == 0) {
+            int it = 0;
+            for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
+                int tm, tn;
+                gemm_tile_coords(pair + i * n_pairs, p, tm, tn);
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % kGemm2Stages;
+                    if (it >= kGemm2Stages && !mbar_wait(bar_empty(s), ((it / kGemm2Stages) - 1) & 1, abort_flag)) {
+                        if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_GEMM_PRODUCER); *abort_flag = 1; }
+                        break;
+                    }
+                    const uint32_t dst = base + s * kGemm2StageBytes;
+                    const uint32_t leader_full = mapa_shared(bar_full(s), 0);
+                    if (rank == 0) mbar_expect_tx(bar_full(s), 2 * kGemm2StageBytes);   // both CTAs' bytes
+                    tma_load_2d_pair(dst, &tmap_a, kb * kGemmBK, tm * kGemm2BM + (int)rank * 128, leader_full);
+                    tma_load_2d_pair(dst + kGemm2ABytes, &tmap_b, kb * kGemmBK, tn * kGemmBN + (int)rank * 128, leader_full);
+                    issued = it + 1;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        if (lane == 0 && rank == 0) {
+            const uint64_t a_desc0 = smem_desc_sw128(base);
+            const uint64_t b_desc0 = smem_desc_sw128(base + kGemm2ABytes);
+            int it = 0;
+            bool ok = true;
+            for (int i = 0; ok && i < my_tiles; ++i) {
+                const int acc = i & 1;
+                if (i >= 2 && !mbar_wait(bar_tempty(acc), ((i >> 1) - 1) & 1, abort_flag)) {
+                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_GEMM_MMA); *abort_flag = 1; }
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_addr = tmem_base + (uint32_t)(acc * kGemmBN);
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % kGemm2Stages;
+                    if (!mbar_wait(bar_full(s), (it / kGemm2Stages) & 1, abort_flag)) {
+                        if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_GEMM_MMA); *abort_flag = 1; }
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t off = (uint64_t)((s * kGemm2StageBytes) >> 4);
+#pragma unroll
+                    for (int k = 0; k < kGemmBK / 16; ++k)
+                        tc_mma_bf16_pair(d_addr, a_desc0 + off + (uint64_t)(2 * k), b_desc0 + off + (uint64_t)(2 * k),
+                                         idesc_m256n256_bf16(), (uint32_t)((kb | k) != 0));
+                    tc_commit_pair(bar_empty(s));
+                }
+                if (ok) tc_commit_pair(bar_tfull(acc));
+            }
+        }
+    } else {
+        // ---------------- epilogue: warps 2..9 of both CTAs, each CTA its own 128 rows ----------------
+        const int quarter = warp & 3;
+        const int chalf = (warp - 2) >> 2;
+        const float coef = p.coef_mul * (p.coef_ptr ? __ldg(p.coef_ptr) : 1.0f);
+        double sq = 0.0;
+        for (int i = 0; i < my_tiles; ++i) {
+            const int acc = i & 1;
+            int tm, tn;
+            gemm_tile_coords(pair + i * n_pairs, p, tm, tn);
+            if (!mbar_wait(bar_tfull(acc), (i >> 1) & 1, abort_flag)) {
+                if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_GEMM_EPILOGUE); *abort_flag = 1; }
+                break;
+            }
+            tc_fence_after();
+            const int64_t row = (int64_t)tm * kGemm2BM + (int)rank * 128 + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+            float sq_tile = 0.f;
+            for (int c = chalf * (kGemmBN / 64); c < (chalf + 1) * (kGemmBN / 64); ++c) {
+                const int col = tn * kGemmBN + c * 32;
+                if (col >= p.N) break;
+                uint32_t r[32];
+                tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kGemmBN + c * 32), r);
+                if (row_ok) gemm_epilogue_chunk(p, r, row, col, coef, sq_tile);
+                __syncwarp();
+            }
+            sq += (double)sq_tile;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(bar_tempty(acc), 0));
+        }
+        if (p.sumsq) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
+            if (lane == 0 && sq != 0.0) atomicAdd(p.sumsq, sq);
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0 && rank == 0) {
+        // abort path only: the leader's full barriers see every load of the pair complete; wait for the
+        // ones this CTA armed before the shared memory goes away
+        int never = 0;
+        for (int m = (issued > kGemm2Stages ? issued - kGemm2Stages : 0); m < issued; ++m)
+            if (!mbar_wait(bar_full(m % kGemm2Stages), (m / kGemm2Stages) & 1, &never))
+                atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_GEMM_DRAIN);
+    }
+    __syncthreads();
+    cluster_sync_all();          // the partner is done with this CTA's shared memory and barriers
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace kq

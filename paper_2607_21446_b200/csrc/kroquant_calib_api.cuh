@@ -3,6 +3,7 @@
 #pragma once
 #include "kq_calib.cuh"
 #include "kq_gemm.cuh"
+#include "kq_gemm2.cuh"
 
 struct kroquant_calib {
     int device = -1;
@@ -22,7 +23,10 @@ struct kroquant_calib {
     double* sums = nullptr;            // [3] sums of squares of the evaluation in flight
     double* hist = nullptr;            // [kHistCap][3]
     int t = 0;                         // Adam steps taken
+    // GEMM operands: "_a" = 128-row boxes (A operand, and both operands of the paired kernel),
+    // "_b" = 256-row boxes (B operand of the one-CTA kernel)
     CUtensorMap tm_A_a, tm_W_b, tm_Yq_a, tm_Zq_b, tm_dO_a, tm_ZqT_b, tm_dOT_a, tm_YqT_b;
+    CUtensorMap tm_W_a, tm_Zq_a, tm_ZqT_a, tm_YqT_a;
 };
 
 namespace {
@@ -42,22 +46,29 @@ bool make_operand_map(CUtensorMap* tm, const void* ptr, int64_t rows, int64_t K,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, int M, int N, int K, const float* aux,
-                        int64_t ld_aux, const float* coef_ptr, float coef_mul, float out_scale, float* out_f32,
-                        __nv_bfloat16* out_bf16, int64_t ld_out, double* sumsq, cudaStream_t st,
+std::atomic<int> g_gemm_pair{1};       // 1: two-CTA 256 x 256 tiles (default); 0: one-CTA 128 x 256 tiles
+
+// tb = B operand map with 256-row boxes (one-CTA kernel), tb2 = the same tensor with 128-row boxes
+kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, int M, int N, int K,
+                        const float* aux, int64_t ld_aux, const float* coef_ptr, float coef_mul, float out_scale,
+                        float* out_f32, __nv_bfloat16* out_bf16, int64_t ld_out, double* sumsq, cudaStream_t st,
                         __nv_bfloat16* out_bf16_t = nullptr, int64_t ld_out_t = 0) {
     static std::atomic<int> attr_done{0};
     if (!attr_done.load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kq::gemm_nt_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kGemmDynBytes) !=
-            cudaSuccess) {
+                cudaSuccess ||
+            cudaFuncSetAttribute(kq::gemm_nt_umma_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kGemm2DynBytes) !=
+                cudaSuccess) {
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
         }
         attr_done.store(1, std::memory_order_release);
     }
+    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0;
+    const int bm = pair ? kq::kGemm2BM : kq::kGemmBM;
     kq::GemmProblem p;
     p.M = M; p.N = N; p.K = K;
-    p.tiles_m = (M + kq::kGemmBM - 1) / kq::kGemmBM;
+    p.tiles_m = (M + bm - 1) / bm;
     p.tiles_n = (N + kq::kGemmBN - 1) / kq::kGemmBN;
     p.k_blocks = (K + kq::kGemmBK - 1) / kq::kGemmBK;
     p.aux = aux; p.ld_aux = ld_aux; p.coef_ptr = coef_ptr; p.coef_mul = coef_mul; p.out_scale = out_scale;
@@ -66,9 +77,29 @@ kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, int M, int
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
     const int tiles = p.tiles_m * p.tiles_n;
-    const int grid = tiles < sms ? tiles : sms;
-    kq::gemm_nt_umma<<<grid, kq::kGemmThreads, kq::kGemmDynBytes, st>>>(ta, tb, p);
-    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    if (pair) {
+        const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * pairs));
+        cfg.blockDim = dim3(kq::kGemmThreads);
+        cfg.dynamicSmemBytes = kq::kGemm2DynBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kq::gemm_nt_umma_pair, ta, tb2, p) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KQ_ERR_CUDA;
+        }
+    } else {
+        const int grid = tiles < sms ? tiles : sms;
+        kq::gemm_nt_umma<<<grid, kq::kGemmThreads, kq::kGemmDynBytes, st>>>(ta, tb, p);
+        if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return KQ_OK;
 }
@@ -127,7 +158,7 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
     kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, c->ZqT, c->ResZ, c->sums + 2);
     if (!launched()) return KQ_ERR_CUDA;
     // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o))
-    kq_status_t rc = launch_gemm(c->tm_Yq_a, c->tm_Zq_b, (int)M, o, d, c->R, o, nullptr, -1.0f,
+    kq_status_t rc = launch_gemm(c->tm_Yq_a, c->tm_Zq_b, c->tm_Zq_a, (int)M, o, d, c->R, o, nullptr, -1.0f,
                                  (float)(2.0 / ((double)M * o)), nullptr, backward ? c->dO : nullptr, o, c->sums, st,
                                  backward ? c->dOT : nullptr, M);
     if (rc != KQ_OK) return rc;
@@ -136,10 +167,10 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
         return KQ_ERR_CUDA;
     if (!backward) return KQ_OK;
     // dY = dO Zq + lambda_A 2 (Y - Yq) / (M d);  dZ = dO^T Yq + lambda_W 2 (Z - Zq) / (o d)
-    rc = launch_gemm(c->tm_dO_a, c->tm_ZqT_b, (int)M, d, o, c->ResY, d, c->lam, (float)(2.0 / ((double)M * d)), 1.0f,
+    rc = launch_gemm(c->tm_dO_a, c->tm_ZqT_b, c->tm_ZqT_a, (int)M, d, o, c->ResY, d, c->lam, (float)(2.0 / ((double)M * d)), 1.0f,
                      c->dY, nullptr, d, nullptr, st);
     if (rc != KQ_OK) return rc;
-    rc = launch_gemm(c->tm_dOT_a, c->tm_YqT_b, o, d, (int)M, c->ResZ, d, c->lam + 1, (float)(2.0 / ((double)o * d)), 1.0f,
+    rc = launch_gemm(c->tm_dOT_a, c->tm_YqT_b, c->tm_YqT_a, o, d, (int)M, c->ResZ, d, c->lam + 1, (float)(2.0 / ((double)o * d)), 1.0f,
                      c->dZ, nullptr, d, nullptr, st);
     if (rc != KQ_OK) return rc;
     rc = run_block_grad(c->A, c->dY, M, d, c->n_sets, c->chunksK, c->rpcK, c->partK, c->dK, st);
@@ -204,6 +235,11 @@ kq_status_t kroquant_block_grad(const void* X, const float* G, int64_t rows, int
                           out, st);
 }
 
+kq_status_t kroquant_debug_set_gemm_pair(int on) {
+    g_gemm_pair.store(on ? 1 : 0, std::memory_order_relaxed);
+    return KQ_OK;
+}
+
 kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o, int d, int n_sets, void* stream,
                                   kroquant_calib_t** out) {
     if (!A || !W || !out) return KQ_ERR_NULL;
@@ -252,7 +288,9 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     bool ok = make_operand_map(&c->tm_A_a, c->A, M, d, kq::kGemmBM) && make_operand_map(&c->tm_W_b, c->W, o, d, kq::kGemmBN) &&
               make_operand_map(&c->tm_Yq_a, c->Yq, M, d, kq::kGemmBM) && make_operand_map(&c->tm_Zq_b, c->Zq, o, d, kq::kGemmBN) &&
               make_operand_map(&c->tm_dO_a, c->dO, M, o, kq::kGemmBM) && make_operand_map(&c->tm_ZqT_b, c->ZqT, d, o, kq::kGemmBN) &&
-              make_operand_map(&c->tm_dOT_a, c->dOT, o, M, kq::kGemmBM) && make_operand_map(&c->tm_YqT_b, c->YqT, d, M, kq::kGemmBN);
+              make_operand_map(&c->tm_dOT_a, c->dOT, o, M, kq::kGemmBM) && make_operand_map(&c->tm_YqT_b, c->YqT, d, M, kq::kGemmBN) &&
+              make_operand_map(&c->tm_W_a, c->W, o, d, 128) && make_operand_map(&c->tm_Zq_a, c->Zq, o, d, 128) &&
+              make_operand_map(&c->tm_ZqT_a, c->ZqT, d, o, 128) && make_operand_map(&c->tm_YqT_a, c->YqT, d, M, 128);
     kq_status_t rc = ok ? KQ_OK : KQ_ERR_CUDA;
     std::vector<float> th;
     hadamard_theta(th, n_sets);
@@ -261,7 +299,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
         rc = KQ_ERR_CUDA;
     // R = A W^T
     if (rc == KQ_OK)
-        rc = launch_gemm(c->tm_A_a, c->tm_W_b, (int)M, o, d, nullptr, 0, nullptr, 1.0f, 1.0f, c->R, nullptr, o, nullptr, st);
+        rc = launch_gemm(c->tm_A_a, c->tm_W_b, c->tm_W_a, (int)M, o, d, nullptr, 0, nullptr, 1.0f, 1.0f, c->R, nullptr, o, nullptr, st);
     // the three terms at the initialisation -> lambdas
     if (rc == KQ_OK) rc = calib_eval(c, false, false, 0.f, 0, st);
     if (rc == KQ_OK) {

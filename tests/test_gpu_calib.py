@@ -20,6 +20,15 @@ LOSS_RTOL = 1e-4         # measured 2e-7 ... 3e-5 (largest at the Hadamard start
 GRAD_TOL = 5e-4          # of max |g|; measured 2e-6 ... 9e-5
 
 
+@pytest.fixture(autouse=True, params=["pair", "single"])
+def gemm_variant(request):
+    """Every test runs with both tensor-core GEMM kernels: CTA pairs on 256 x 256 tiles (the default)
+    and one CTA per 128 x 256 tile."""
+    kb.set_gemm_pair(request.param == "pair")
+    yield request.param
+    kb.set_gemm_pair(True)
+
+
 def _case(M, o, d, seed):
     A_bits = wl.gen_activations(wl.calib_spec(M, d, seed))
     W_bits = wl.gen_weights(seed, o, d)
