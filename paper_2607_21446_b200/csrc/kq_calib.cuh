@@ -181,87 +181,117 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
 }
 
 // ---- block gradients: part[chunk][j][32][32] = sum over the chunk's rows of x_j^T g_j ---------
-// grid (chunks, d/32); 256 threads = 4 row groups x 64 patches; a thread owns a 4 x 4 patch of the
-// 32 x 32 result for its row group; tiles of 64 rows are staged in shared memory as fp32 while the
-// next tile's global loads are already in flight.  (8 x 8 patches halve the shared-memory reads
-// per FMA but cost so many registers that the kernel ran slower.)
+// grid (chunks, d/32); 4 warps.  Tiles of 64 rows are staged in shared memory as bf16: X as it is,
+// G (fp32) split into three bf16 terms that add up to it exactly, so the tensor-core products
+// (mma.sync m16n8k16, fp32 accumulate) are exact.  Both operands are stored row-major [row][channel]
+// and fetched with transposing ldmatrix, which yields x^T as the "A" fragments (m = channel of X,
+// k = row) and g as the "B" fragments (k = row, n = channel of G).  Warp w multiplies rows
+// 16w..16w+15 of every tile into its own 32 x 32 accumulator; the four are summed at the end.
 constexpr int kGradTileRows = 64;
-__global__ void __launch_bounds__(256)
+constexpr int kGradPitch = 40;                 // bf16 elements per staged row: 80 bytes, conflict-free ldmatrix
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
+}
+__global__ void __launch_bounds__(128)
 calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, int64_t rows, int d,
                  int64_t rows_per_chunk, float* __restrict__ part) {
-    __shared__ __align__(16) float xs[kGradTileRows][32];
-    __shared__ __align__(16) float gs[kGradTileRows][32];
+    __shared__ __align__(16) uint16_t xs[kGradTileRows][kGradPitch];
+    __shared__ __align__(16) uint16_t gs[3][kGradTileRows][kGradPitch];
+    __shared__ __align__(16) float red[4][1024];
     const int j = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t r_begin = (int64_t)blockIdx.x * rows_per_chunk;
     const int64_t r_end = r_begin + rows_per_chunk < rows ? r_begin + rows_per_chunk : rows;
-    const int grp = threadIdx.x >> 6;                         // 4 row groups of 16 rows per tile
-    const int r4 = ((threadIdx.x & 63) >> 3) * 4, c4 = (threadIdx.x & 7) * 4;
-    float acc[4][4];
+    float acc[2][4][4];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 2; ++a)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
-    // global -> registers for the tile after the one being multiplied: thread -> (row = tid / 4,
-    // 8 channels = (tid % 4) * 8)
-    const int lr_st = threadIdx.x >> 2, ch_st = (threadIdx.x & 3) * 8;
-    uint4 px = make_uint4(0u, 0u, 0u, 0u);
-    float4 pg0 = make_float4(0.f, 0.f, 0.f, 0.f), pg1 = pg0;
+        for (int b = 0; b < 4; ++b)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
+    // staging roles: X tile = 64 rows x 4 segments of 8 channels (2 per thread);
+    // G tile = 64 rows x 8 segments of 4 channels (4 per thread)
+    uint4 px[2];
+    float4 pg[4];
     auto fetch = [&](int64_t t0) {
-        const int64_t row = t0 + lr_st;
-        if (row < r_end) {
-            px = ld_stream_16(X + row * d + j * 32 + ch_st);
-            const float4* gp = reinterpret_cast<const float4*>(G + row * d + j * 32 + ch_st);
-            pg0 = __ldg(gp);
-            pg1 = __ldg(gp + 1);
-        } else {
-            px = make_uint4(0u, 0u, 0u, 0u);
-            pg0 = pg1 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int seg = threadIdx.x + 128 * i;
+            const int64_t row = t0 + (seg >> 2);
+            px[i] = row < r_end ? ld_stream_16(X + row * d + j * 32 + (seg & 3) * 8) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int seg = threadIdx.x + 128 * i;
+            const int64_t row = t0 + (seg >> 3);
+            pg[i] = row < r_end ? __ldg(reinterpret_cast<const float4*>(G + row * d + j * 32 + (seg & 7) * 4))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     };
     if (r_begin < r_end) fetch(r_begin);
+    const uint32_t xs_base = (uint32_t)__cvta_generic_to_shared(&xs[0][0]);
+    const uint32_t gs_base = (uint32_t)__cvta_generic_to_shared(&gs[0][0][0]);
+    // ldmatrix lane addresses inside this warp's 16 rows (see the header comment)
+    const int mid = lane >> 3, l7 = lane & 7;
+    const uint32_t a_off = (uint32_t)(((16 * warp + (mid >> 1) * 8 + l7) * kGradPitch + (mid & 1) * 8) * 2);
+    const uint32_t b_off = (uint32_t)(((16 * warp + (mid & 1) * 8 + l7) * kGradPitch + (mid >> 1) * 8) * 2);
     for (int64_t t0 = r_begin; t0 < r_end; t0 += kGradTileRows) {
-        {
-            float xv[8];
-            widen8(px, xv);
-            *reinterpret_cast<float4*>(&xs[lr_st][ch_st]) = make_float4(xv[0], xv[1], xv[2], xv[3]);
-            *reinterpret_cast<float4*>(&xs[lr_st][ch_st + 4]) = make_float4(xv[4], xv[5], xv[6], xv[7]);
-            *reinterpret_cast<float4*>(&gs[lr_st][ch_st]) = pg0;
-            *reinterpret_cast<float4*>(&gs[lr_st][ch_st + 4]) = pg1;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int seg = threadIdx.x + 128 * i;
+            *reinterpret_cast<uint4*>(&xs[seg >> 2][(seg & 3) * 8]) = px[i];
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int seg = threadIdx.x + 128 * i;
+            const float gv[4] = {pg[i].x, pg[i].y, pg[i].z, pg[i].w};
+            uint32_t t[4][3];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) split3_bf16(gv[e], t[e]);
+#pragma unroll
+            for (int m = 0; m < 3; ++m)
+                *reinterpret_cast<uint2*>(&gs[m][seg >> 3][(seg & 7) * 4]) =
+                    make_uint2(t[0][m] | (t[1][m] << 16), t[2][m] | (t[3][m] << 16));
         }
         __syncthreads();
         if (t0 + kGradTileRows < r_end) fetch(t0 + kGradTileRows);       // lands while this tile is multiplied
-#pragma unroll 4
-        for (int i = 0; i < kGradTileRows / 4; ++i) {
-            const int lr = grp * (kGradTileRows / 4) + i;
-            const float4 xa = *reinterpret_cast<const float4*>(&xs[lr][r4]);
-            const float4 ga = *reinterpret_cast<const float4*>(&gs[lr][c4]);
-            const float xv[4] = {xa.x, xa.y, xa.z, xa.w};
-            const float gv[4] = {ga.x, ga.y, ga.z, ga.w};
+        uint32_t af[2][4];
+        ldmatrix_x4_trans(af[0], xs_base + a_off);                       // channels 0..15 of X
+        ldmatrix_x4_trans(af[1], xs_base + a_off + 32);                  // channels 16..31
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
+        for (int m = 2; m >= 0; --m) {                                   // smallest term first
+            uint32_t bfr[2][4];
+            const uint32_t gm = gs_base + (uint32_t)(m * kGradTileRows * kGradPitch * 2) + b_off;
+            ldmatrix_x4_trans(bfr[0], gm);                               // channels 0..15 of G: n-tiles 0, 1
+            ldmatrix_x4_trans(bfr[1], gm + 32);                          // channels 16..31: n-tiles 2, 3
 #pragma unroll
-                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(xv[a], gv[b], acc[a][b]);
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt)
+                    mma_bf16_16816(acc[mt][nt], af[mt], bfr[nt >> 1][(nt & 1) * 2], bfr[nt >> 1][(nt & 1) * 2 + 1]);
         }
         __syncthreads();
     }
-    // sum the four row groups through the staging memory (2 x 8 KB = 4 x 1024 floats)
-    float* red = &xs[0][0];
-    float* red2 = &gs[0][0];
-    float* mine = grp < 2 ? red + grp * 1024 : red2 + (grp - 2) * 1024;
+    // accumulator fragment: c0, c1 = (m = g, n = 2q, 2q + 1); c2, c3 = (m = g + 8, same n)
+    {
+        const int g = lane >> 2, q = lane & 3;
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+        for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-        for (int b = 0; b < 4; ++b) mine[(r4 + a) * 32 + c4 + b] = acc[a][b];
-    __syncthreads();
-    float tot[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int e = threadIdx.x + 256 * i;
-        tot[i] = (red[e] + red[1024 + e]) + (red2[e] + red2[1024 + e]);
+            for (int nt = 0; nt < 4; ++nt) {
+                const int m0 = 16 * mt + g, n0 = 8 * nt + 2 * q;
+                *reinterpret_cast<float2*>(&red[warp][m0 * 32 + n0]) = make_float2(acc[mt][nt][0], acc[mt][nt][1]);
+                *reinterpret_cast<float2*>(&red[warp][(m0 + 8) * 32 + n0]) = make_float2(acc[mt][nt][2], acc[mt][nt][3]);
+            }
     }
+    __syncthreads();
     float* dst = part + ((size_t)blockIdx.x * gridDim.y + j) * 1024;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) dst[threadIdx.x + 256 * i] = tot[i];
+    for (int i = 0; i < 8; ++i) {
+        const int e = threadIdx.x + 128 * i;
+        dst[e] = (red[0][e] + red[1][e]) + (red[2][e] + red[3][e]);
+    }
 }
 
 // ---- sum of partial blocks: out[j][e] = sum_p part[p][j][e], e < 1024 --------------------------
