@@ -192,7 +192,7 @@ kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_
  * must stay valid and unchanged for the life of the object.  M is the number of calibration
  * rows (all samples stacked), a multiple of 8; o and d are multiples of 32; n_sets is 1 (one
  * factor set for the layer) or d/32 (one per block).  create allocates all work space
- * (about 14 M d + 10 M o bytes), forms A W^T, evaluates the three terms at the initialisation and
+ * (about 12 M d + 8 M o bytes), forms A W^T, evaluates the three terms at the initialisation and
  * sets lambda_A = L_out/L_A, lambda_W = L_out/L_W there; it synchronizes `stream`.  The object is
  * tied to the device that was current at creation.  All three contractions of a step run on the
  * tensor cores in bf16 with fp32 accumulation (exact products for the forward one); the output
@@ -217,6 +217,11 @@ kq_status_t kroquant_calib_get_lambdas(const kroquant_calib_t *c, float *lam_hos
 /* The factors G_k = L_k U_k of the current parameters, [n_sets][5][2][2] floats, ready for
  * kroquant_factors_create. */
 kq_status_t kroquant_calib_get_factors(const kroquant_calib_t *c, float *G_host_out);
+/* The factors of the weight-side transform T^-T (Section 3.3: the layer runs Q(A T) Q(W T^-T)^T):
+ * (G_1 (x) ... (x) G_5)^-T = G_1^-T (x) ... (x) G_5^-T, so it is again a Kronecker set,
+ * H_k = G_k^-T = [[1/a - b c, a c], [b, -a]]; [n_sets][5][2][2] floats, ready for
+ * kroquant_factors_create, with which kroquant_quantize(W, ...) yields Q(W T^-T) offline. */
+kq_status_t kroquant_calib_get_weight_factors(const kroquant_calib_t *c, float *H_host_out);
 
 /* Evaluate at the current parameters without changing them: losses_host_out[3] = {L_out, L_A, L_W}
  * (doubles), grad_host_out [n_sets][5][3] floats = dL/dtheta (may be NULL: forward pass only).

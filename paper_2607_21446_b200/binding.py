@@ -33,7 +33,7 @@ EXPORTS = [
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
     "kroquant_calib_loss_grad", "kroquant_calib_run",
     "kroquant_block_grad_scratch_bytes", "kroquant_block_grad", "kroquant_block_grad_static",
-    "kroquant_debug_set_gemm_pair",
+    "kroquant_debug_set_gemm_pair", "kroquant_calib_get_weight_factors",
 ]
 
 
@@ -87,7 +87,7 @@ def load_library() -> C.CDLL:
     L.kroquant_calib_create.argtypes = [vp, vp, i64, i32, i32, i32, vp, C.POINTER(vp)]
     L.kroquant_calib_destroy.argtypes = [vp]
     L.kroquant_calib_destroy.restype = None
-    for name in ("set_theta", "get_theta", "set_lambdas", "get_lambdas", "get_factors"):
+    for name in ("set_theta", "get_theta", "set_lambdas", "get_lambdas", "get_factors", "get_weight_factors"):
         getattr(L, "kroquant_calib_" + name).argtypes = [vp, vp]
     L.kroquant_calib_loss_grad.argtypes = [vp, vp, vp, vp]
     L.kroquant_calib_run.argtypes = [vp, i32, C.c_float, vp, vp]
@@ -473,6 +473,10 @@ class Calibrator:
     def factors(self) -> np.ndarray:
         """G [n_sets, 5, 2, 2] of the current parameters (input of Factors.create)."""
         return self._get("factors", (self.n_sets, 5, 2, 2))
+
+    def weight_factors(self) -> np.ndarray:
+        """H [n_sets, 5, 2, 2] with H_k = G_k^-T: the Kronecker set of T^-T, for quantizing W offline."""
+        return self._get("weight_factors", (self.n_sets, 5, 2, 2))
 
     def loss_grad(self, grad: bool = True, stream=None):
         """-> (losses float64 [3] = (L_out, L_A, L_W), dL/dtheta float32 [n_sets, 5, 3] or None)."""

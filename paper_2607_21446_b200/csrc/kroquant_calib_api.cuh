@@ -372,6 +372,22 @@ kq_status_t kroquant_calib_get_factors(const kroquant_calib_t* c, float* G_host_
     return KQ_OK;
 }
 
+kq_status_t kroquant_calib_get_weight_factors(const kroquant_calib_t* c, float* H_host_out) {
+    kq_status_t rc = calib_check(c);
+    if (rc != KQ_OK) return rc;
+    if (!H_host_out) return KQ_ERR_NULL;
+    std::vector<float> th((size_t)c->n_sets * 15);
+    if (cudaMemcpy(th.data(), c->theta, th.size() * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return KQ_ERR_CUDA;
+    for (int i = 0; i < c->n_sets * 5; ++i) {
+        const double a = th[3 * i], b = th[3 * i + 1], cc = th[3 * i + 2];
+        H_host_out[4 * i + 0] = (float)(1.0 / a - b * cc);
+        H_host_out[4 * i + 1] = (float)(a * cc);
+        H_host_out[4 * i + 2] = (float)b;
+        H_host_out[4 * i + 3] = (float)(-a);
+    }
+    return KQ_OK;
+}
+
 kq_status_t kroquant_calib_loss_grad(kroquant_calib_t* c, double* losses_host_out, float* grad_host_out, void* stream) {
     kq_status_t rc = calib_check(c);
     if (rc != KQ_OK) return rc;

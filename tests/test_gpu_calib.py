@@ -191,6 +191,47 @@ def test_block_grad_against_the_oracle(rows, d, shared):
     assert np.array_equal(out, again)                   # fixed summation order
 
 
+@pytest.mark.parametrize("shared", [True, False])
+def test_calibrated_layer_through_the_quantizer_and_the_block_scaled_gemm(shared):
+    """End of the pipeline (Section 3.3 objective, Section 3.4 inference form): calibrate, hand the
+    activation factors and the weight factors (T^-T is again a Kronecker set) to the quantizer,
+    multiply the two MXFP4 operands with the library's block-scaled tensor-core GEMM, and find the
+    output error the calibrator reported."""
+    F = torch.nn.functional
+    if not hasattr(F, "scaled_mm"):
+        pytest.skip("torch.nn.functional.scaled_mm not available")
+    M, o, d, seed = 512, 256, 512, 77
+    A, W, A_t, W_t = _case(M, o, d, seed)
+    n_sets = 1 if shared else d // 32
+    cal = kb.Calibrator(A_t, W_t, n_sets)
+    hist = cal.run(10, lr=1e-2)
+    theta = cal.theta.astype(np.float64)
+    G, H = cal.factors(), cal.weight_factors()
+    K_ref, P_ref = co.blocks_of(theta)
+    for s_ in range(n_sets):
+        assert np.allclose(co.kron5(G[s_].astype(np.float64)), K_ref[s_], rtol=1e-5, atol=1e-6)
+        assert np.allclose(co.kron5(H[s_].astype(np.float64)), P_ref[s_], rtol=1e-5, atol=1e-6)
+    fa, fw = kb.Factors.create(G), kb.Factors.create(H)
+    qa, sa = kb.kroquant_quantize(A_t, fa, scale_layout="tiled")
+    qw, sw = kb.kroquant_quantize(W_t, fw, scale_layout="tiled")
+    out = F.scaled_mm(qa.view(torch.float4_e2m1fn_x2), qw.view(torch.float4_e2m1fn_x2).t(),
+                      sa.view(torch.float8_e8m0fnu), F.ScalingType.BlockWise1x32,
+                      sw.view(torch.float8_e8m0fnu), F.ScalingType.BlockWise1x32,
+                      swizzle_a=F.SwizzleType.SWIZZLE_32_4_4, swizzle_b=F.SwizzleType.SWIZZLE_32_4_4,
+                      output_dtype=torch.bfloat16).double().cpu().numpy()
+    # the oracle's forward pass with the float32 factors the quantizer was given
+    f = co.forward(A, W, theta)
+    ref = f["Yq"] @ f["Zq"].T
+    # bf16 output of the library GEMM (2^-9 relative); a few codes may differ (float32 factors)
+    assert np.abs(out - ref).max() <= 6e-3 * np.abs(ref).max()
+    L_out = np.sum((out - A @ W.T) ** 2) / (M * o)
+    assert np.isclose(L_out, hist[-1, 0], rtol=2e-2)
+    assert np.isclose(f["L_out"], hist[-1, 0], rtol=LOSS_RTOL)
+    fa.destroy()
+    fw.destroy()
+    cal.destroy()
+
+
 def test_argument_checks():
     A, W, A_t, W_t = _case(256, 64, 128, 71)
     with pytest.raises(kb.KroQuantError):
