@@ -633,6 +633,69 @@ def run_calib(args):
     cal.destroy()
 
 
+def run_gemm_fp4(args):
+    """W4A4 consumer GEMM (Section 3.4) on synthetic operands: this library's block-scaled FP4 kernel, the
+    library GEMM behind torch.nn.functional.scaled_mm, and cuBLAS bf16 on the unquantized operands, timed
+    with CUDA events after warm-up; one JSON line."""
+    import torch
+    from paper_2607_21446_b200 import binding as B
+    B.load_library()
+    M, N, K = (int(v) for v in args.gemm_fp4.lower().split("x"))
+    g = torch.Generator(device="cuda")
+    g.manual_seed(0)
+    A = torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
+    Wt = (torch.randn(N, K, device="cuda", generator=g) / K ** 0.5).to(torch.bfloat16)
+    qa, sa = B.kroquant_mxfp4_quantize(A, scale_layout="tiled")
+    qw, sw = B.kroquant_mxfp4_quantize(Wt, scale_layout="tiled")
+    out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    F = torch.nn.functional
+
+    def timed(fn):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps * 1e3
+
+    l0 = B.kroquant_launch_count()
+    us_own = timed(lambda: B.kroquant_gemm_mxfp4(qa, sa, qw, sw, out=out))
+    launches = B.kroquant_launch_count() - l0
+    us_lib = None
+    if hasattr(F, "scaled_mm"):
+        us_lib = timed(lambda: F.scaled_mm(
+            qa.view(torch.float4_e2m1fn_x2), qw.view(torch.float4_e2m1fn_x2).t(),
+            sa.view(torch.float8_e8m0fnu), F.ScalingType.BlockWise1x32, sw.view(torch.float8_e8m0fnu),
+            F.ScalingType.BlockWise1x32, swizzle_a=F.SwizzleType.SWIZZLE_32_4_4,
+            swizzle_b=F.SwizzleType.SWIZZLE_32_4_4, output_dtype=torch.bfloat16))
+    us_bf16 = timed(lambda: torch.matmul(A, Wt.t()))
+    flop = 2.0 * M * N * K
+    peak_bf16, kind = 1590.0, "fallback"
+    pth = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pth):
+        with open(pth) as f:
+            mp = json.load(f)
+        if "bf16_tflops" in mp:
+            peak_bf16, kind = float(mp["bf16_tflops"]), "measured"
+    peak = 4.0 * peak_bf16          # nominal fp4 : bf16 ratio of the dense peaks (9 : 2.25)
+    print(json.dumps({
+        "metric": "w4a4_gemm_time", "value": round(us_own, 2), "unit": "us", "higher_is_better": False, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "dtype": "e2m1 x e2m1 with e8m0 block scales, fp32 accumulate",
+        "data": "synthetic", "config": {"workload": f"W4A4 GEMM M={M} N={N} K={K}, bf16 output"},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "achieved": round(flop / us_own / 1e6, 1), "peak": round(peak, 1), "unit": "TFLOP/s",
+                     "frac": round(flop / us_own / 1e6 / peak, 4), "traffic": None,
+                     "note": f"peak = {kind} bf16 peak x 4 (nominal fp4 : bf16 ratio)"},
+        "library_fp4_us": None if us_lib is None else round(us_lib, 2),
+        "library_fp4_tflops": None if us_lib is None else round(flop / us_lib / 1e6, 1),
+        "cublas_bf16_us": round(us_bf16, 2), "cublas_bf16_tflops": round(flop / us_bf16 / 1e6, 1),
+        "device_error": B.kroquant_last_device_error()}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", action="store_true",
@@ -646,6 +709,8 @@ def main():
     ap.add_argument("--per-block", action="store_true", help="with --single: one factor set per 32-channel block")
     ap.add_argument("--calib", default=None, metavar="MxOxD",
                     help="calibration loop on a synthetic layer, e.g. 16384x3072x3072 (with --per-block: one set per block)")
+    ap.add_argument("--gemm-fp4", default=None, metavar="MxNxK",
+                    help="W4A4 consumer GEMM, e.g. 4608x3072x3072: own FP4 kernel vs library FP4 vs cuBLAS bf16")
     ap.add_argument("--gemm-single", action="store_true",
                     help="with --calib: one-CTA 128x256 GEMM tiles instead of CTA pairs on 256x256 tiles")
     ap.add_argument("--gpus", type=int, default=1)
@@ -662,6 +727,8 @@ def main():
         run_single(args)
     elif args.calib:
         run_calib(args)
+    elif args.gemm_fp4:
+        run_gemm_fp4(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -177,6 +177,21 @@ kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes,
  * launches with programmatic stream serialization.  Process-wide. */
 kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl);
 
+/* The W4A4 product of the quantized layer (Section 3.4: O = Q(A T) Q(W~)^T + A T L R):
+ *     out[m][n] = sum_k a[m][k] 2^(sa[m][k/32] - 127) * b[n][k] 2^(sb[n][k/32] - 127)  (+ add[m][n])
+ * on the block-scaled FP4 tensor-core path (fp32 accumulation).  a_codes [M][K/2] and b_codes
+ * [N][K/2] are packed E2M1 codes and a_scales, b_scales E8M0 bytes in KQ_SCALES_TILED_128X4 layout
+ * (sizes ceil(rows/128)*128 * ceil(K/128)*4), i.e. exactly what the quantizer entry points write;
+ * padding bytes of the scale buffers must not be 0xFF (the quantizers leave them untouched: start
+ * from zeros).  add (optional, DEVICE bf16 [M][N]) is added to the result: the low-rank branch.
+ * out: DEVICE [M][N], bf16 or fp32 per out_dtype.  K % 32 == 0, N % 32 == 0; all pointers 16-byte
+ * aligned; every product of the sum is exact, only the fp32 accumulation rounds.  Asynchronous on
+ * `stream`, allocates nothing.  Errors: KQ_ERR_NULL, KQ_ERR_SHAPE, KQ_ERR_ALIGN,
+ * KQ_ERR_UNSUPPORTED (out_dtype), KQ_ERR_CUDA. */
+kq_status_t kroquant_gemm_mxfp4(const uint8_t *a_codes, const uint8_t *a_scales, const uint8_t *b_codes,
+                                const uint8_t *b_scales, int64_t M, int N, int K, const void *add_bf16,
+                                void *out, kq_dtype_t out_dtype, void *stream);
+
 /* ---- Layer-wise calibration of the transform (Section 3.3; set-up of Appendix D) ----
  *
  * Minimises, over the parameters theta = (a_k, b_k, c_k), k = 1..5, of every factor set,

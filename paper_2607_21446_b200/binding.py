@@ -33,7 +33,7 @@ EXPORTS = [
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
     "kroquant_calib_loss_grad", "kroquant_calib_run",
     "kroquant_block_grad_scratch_bytes", "kroquant_block_grad", "kroquant_block_grad_static",
-    "kroquant_debug_set_gemm_pair", "kroquant_calib_get_weight_factors",
+    "kroquant_debug_set_gemm_pair", "kroquant_calib_get_weight_factors", "kroquant_gemm_mxfp4",
 ]
 
 
@@ -96,6 +96,7 @@ def load_library() -> C.CDLL:
     L.kroquant_block_grad.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, vp]
     L.kroquant_block_grad_static.argtypes = [vp, vp, i64, i32, i32, vp, vp]
     L.kroquant_debug_set_gemm_pair.argtypes = [i32]
+    L.kroquant_gemm_mxfp4.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, vp]
     _lib = L
     return L
 
@@ -408,6 +409,34 @@ def kroquant_block_grad_static(X: torch.Tensor, G: torch.Tensor, n_sets: int, ou
         raise ValueError("out must be a contiguous CUDA float32 tensor [n_sets, 32, 32]")
     _check(load_library().kroquant_block_grad_static(_ptr(X), _ptr(G), rows, d, n_sets, _ptr(out), _stream(stream)),
            "kroquant_block_grad_static")
+
+
+def kroquant_gemm_mxfp4(a_codes: torch.Tensor, a_scales: torch.Tensor, b_codes: torch.Tensor, b_scales: torch.Tensor,
+                        add: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                        out_dtype=torch.bfloat16, stream=None) -> torch.Tensor:
+    """out[M, N] = (codes, tiled scales of A [M, K]) x (codes, tiled scales of B [N, K])^T (+ add): the W4A4
+    product on the block-scaled FP4 tensor-core path.  Inputs are what the quantizer calls return with
+    ``scale_layout="tiled"``."""
+    for t in (a_codes, a_scales, b_codes, b_scales):
+        if t.dtype != torch.uint8 or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("codes and scales must be contiguous CUDA uint8 tensors")
+    M, half = a_codes.shape
+    N = b_codes.shape[0]
+    if b_codes.shape[1] != half:
+        raise ValueError("A and B must share K")
+    K = 2 * half
+    if a_scales.numel() != tiled_scale_bytes(M, K) or b_scales.numel() != tiled_scale_bytes(N, K):
+        raise ValueError("scales must be in the tiled layout (tiled_scale_bytes(rows, K) bytes)")
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=a_codes.device)
+    if out.dtype not in (torch.bfloat16, torch.float32) or tuple(out.shape) != (M, N) or not out.is_contiguous():
+        raise ValueError("out must be a contiguous bfloat16 or float32 tensor [M, N]")
+    if add is not None and (add.dtype != torch.bfloat16 or tuple(add.shape) != (M, N) or not add.is_contiguous()):
+        raise ValueError("add must be a contiguous bfloat16 tensor [M, N]")
+    _check(load_library().kroquant_gemm_mxfp4(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), M, N, K,
+                                              _ptr(add), _ptr(out), 1 if out.dtype == torch.bfloat16 else 0,
+                                              _stream(stream)), "kroquant_gemm_mxfp4")
+    return out
 
 
 def set_gemm_pair(on: bool) -> None:

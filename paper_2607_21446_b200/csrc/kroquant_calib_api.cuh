@@ -4,6 +4,7 @@
 #include "kq_calib.cuh"
 #include "kq_gemm.cuh"
 #include "kq_gemm2.cuh"
+#include "kq_gemm_fp4.cuh"
 
 struct kroquant_calib {
     int device = -1;
@@ -233,6 +234,59 @@ kq_status_t kroquant_block_grad(const void* X, const float* G, int64_t rows, int
     if (scratch_bytes < (int64_t)chunks * (d / 32) * 4096) return KQ_ERR_SHAPE;
     return run_block_grad(static_cast<const uint16_t*>(X), G, rows, d, n_sets, chunks, rpc, static_cast<float*>(scratch),
                           out, st);
+}
+
+kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
+                                const uint8_t* b_scales, int64_t M, int N, int K, const void* add_bf16, void* out,
+                                kq_dtype_t out_dtype, void* stream) {
+    if (!a_codes || !a_scales || !b_codes || !b_scales || !out) return KQ_ERR_NULL;
+    if (M < 0 || N <= 0 || K <= 0 || K % 32 || N % 32 || M > (1 << 30)) return KQ_ERR_SHAPE;
+    if (out_dtype != KQ_OUT_F32 && out_dtype != KQ_OUT_BF16) return KQ_ERR_UNSUPPORTED;
+    if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) || !aligned16(out) ||
+        (add_bf16 && !aligned16(add_bf16)))
+        return KQ_ERR_ALIGN;
+    if (M == 0) return KQ_OK;
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return KQ_ERR_CUDA;
+    static std::atomic<int> attr_done{0};
+    if (!attr_done.load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kq::gemm_mxfp4_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kF4DynBytes) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return KQ_ERR_CUDA;
+        }
+        attr_done.store(1, std::memory_order_release);
+    }
+    CUtensorMap ta, tb;
+    const cuuint32_t estr[2] = {1, 1};
+    const cuuint32_t box[2] = {(cuuint32_t)kq::kF4BKBytes, 128};
+    const cuuint64_t adims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)M}, bdims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)N};
+    const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+    if (enc(&ta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(a_codes), adims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+        enc(&tb, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(b_codes), bdims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return KQ_ERR_CUDA;
+    kq::Fp4GemmProblem p;
+    p.M = (int)M; p.N = N; p.K = K;
+    p.tiles_m = (int)((M + kq::kF4BM - 1) / kq::kF4BM);
+    p.tiles_n = (N + kq::kF4BN - 1) / kq::kF4BN;
+    p.k_blocks = (K + kq::kF4BKElems - 1) / kq::kF4BKElems;
+    p.sfa = a_scales; p.sfb = b_scales;
+    p.add = static_cast<const __nv_bfloat16*>(add_bf16); p.ld_add = N;
+    p.out_bf16 = out_dtype == KQ_OUT_BF16 ? static_cast<__nv_bfloat16*>(out) : nullptr;
+    p.out_f32 = out_dtype == KQ_OUT_F32 ? static_cast<float*>(out) : nullptr;
+    p.ld_out = N;
+    const int sms = sm_count();
+    if (sms <= 0) return KQ_ERR_CUDA;
+    const int tiles = p.tiles_m * p.tiles_n;
+    kq::gemm_mxfp4_umma<<<tiles < sms ? tiles : sms, kq::kGemmThreads, kq::kF4DynBytes,
+                          reinterpret_cast<cudaStream_t>(stream)>>>(ta, tb, p);
+    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return KQ_OK;
 }
 
 kq_status_t kroquant_debug_set_gemm_pair(int on) {

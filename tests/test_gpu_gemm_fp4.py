@@ -1,0 +1,145 @@
+"""kroquant_gemm_mxfp4: the W4A4 product of the quantized layer (Section 3.4) on the block-scaled FP4
+tensor-core path, fed by the quantizer's own outputs (packed codes + tiled scale bytes).
+
+Every product a*b*2^(sa+sb) is exact in fp32, so the only error is the order of the fp32 accumulation:
+the tolerance is 1e-6 of sum |a||b| per output (measured: 0 on most shapes, 2e-8 at K = 3072).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import c_oracle as co
+from oracle import calib_oracle as cal
+from paper_2607_21446_b200 import binding as kb
+from paper_2607_21446_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-6
+
+
+def _operand(rows, K, seed, spread=True):
+    """bf16 tensor whose 32-blocks have scales spread over 2^-3 .. 2^3 (so that scale bytes differ)."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    x = torch.randn(rows, K, device="cuda", generator=g)
+    if spread:
+        e = torch.randint(-3, 4, (rows, K // 32), device="cuda", generator=g).float()
+        x = x * torch.exp2(e).repeat_interleave(32, 1)
+    return x.to(torch.bfloat16).contiguous()
+
+
+def _decoded(x_bf16):
+    """-> (codes, tiled scales) from the GPU quantizer and the oracle's decode of the same operand."""
+    q_t, s_t = kb.kroquant_mxfp4_quantize(x_bf16, scale_layout="tiled")
+    q_r, s_r = kb.kroquant_mxfp4_quantize(x_bf16)
+    assert torch.equal(q_t, q_r)
+    dec = co.dequantize(q_r.cpu().numpy(), s_r.cpu().numpy()).astype(np.float64)
+    return q_t, s_t, dec
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (1, 32, 32), (130, 96, 288), (257, 160, 1152), (300, 512, 5600),
+                                   (1000, 1056, 2240)])
+def test_against_the_decoded_float64_product(M, N, K):
+    A, W = _operand(M, K, 1), _operand(N, K, 2)
+    qa, sa, Ad = _decoded(A)
+    qw, sw, Wd = _decoded(W)
+    ref = Ad @ Wd.T
+    bound = np.abs(Ad) @ np.abs(Wd).T
+    out = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, out_dtype=torch.float32)
+    torch.cuda.synchronize()
+    o = out.double().cpu().numpy()
+    assert np.all(np.isfinite(o))
+    assert np.all(np.abs(o - ref) <= TOL * bound + 1e-300)
+    assert kb.kroquant_last_device_error() == 0
+    # bf16 output = the fp32 result rounded once
+    out16 = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, out_dtype=torch.bfloat16)
+    assert torch.equal(out16, out.to(torch.bfloat16))
+
+
+def test_low_rank_branch_is_added_before_the_single_rounding():
+    M, N, K = 384, 256, 512
+    A, W = _operand(M, K, 3), _operand(N, K, 4)
+    qa, sa, Ad = _decoded(A)
+    qw, sw, Wd = _decoded(W)
+    add = _operand(M, N, 5, spread=False)
+    out = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, add=add, out_dtype=torch.float32)
+    ref = Ad @ Wd.T + add.double().cpu().numpy()
+    bound = np.abs(Ad) @ np.abs(Wd).T + np.abs(add.double().cpu().numpy())
+    assert np.all(np.abs(out.double().cpu().numpy() - ref) <= TOL * bound)
+
+
+def test_same_result_as_the_library_block_scaled_gemm():
+    F = torch.nn.functional
+    if not hasattr(F, "scaled_mm"):
+        pytest.skip("torch.nn.functional.scaled_mm not available")
+    M, N, K = 512, 384, 1152
+    A, W = _operand(M, K, 6), _operand(N, K, 7)
+    qa, sa, _ = _decoded(A)
+    qw, sw, _ = _decoded(W)
+    lib = F.scaled_mm(qa.view(torch.float4_e2m1fn_x2), qw.view(torch.float4_e2m1fn_x2).t(),
+                      sa.view(torch.float8_e8m0fnu), F.ScalingType.BlockWise1x32,
+                      sw.view(torch.float8_e8m0fnu), F.ScalingType.BlockWise1x32,
+                      swizzle_a=F.SwizzleType.SWIZZLE_32_4_4, swizzle_b=F.SwizzleType.SWIZZLE_32_4_4,
+                      output_dtype=torch.bfloat16)
+    ours = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, out_dtype=torch.bfloat16)
+    # both round an (almost) identical fp32 sum to bf16: at most one bf16 step apart, and rarely
+    diff = (ours.float() - lib.float()).abs()
+    assert float((diff > 0).float().mean()) < 1e-3
+    assert float((diff / lib.float().abs().clamp_min(1e-30)).max()) <= 2.0 ** -7
+
+
+@pytest.mark.parametrize("per_block", [False, True])
+def test_quantized_layer_from_activations_to_output(per_block):
+    """The inference form of Section 3.4 with this library's own kernels end to end: KroQuant quantizer on
+    the activations (factors G), the same quantizer on the weights with the Kronecker set of T^-T, then the
+    FP4 GEMM; compared with the oracle's Q(A T) Q(W T^-T)^T."""
+    M, o, d, seed = 640, 384, 1152, 9
+    n_sets = d // 32 if per_block else 1
+    A_bits = wl.gen_activations(wl.calib_spec(M, d, seed))
+    W_bits = wl.gen_weights(seed, o, d)
+    theta = wl.gen_lu_params(seed, n_sets).astype(np.float64)
+    G = cal.lu_factors(theta).astype(np.float32)
+    H = np.stack([[np.linalg.inv(G[s, k].astype(np.float64)).T for k in range(5)] for s in range(n_sets)]).astype(np.float32)
+    dev = torch.device("cuda:0")
+    A_t = torch.from_numpy(A_bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    W_t = torch.from_numpy(W_bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    fa, fw = kb.Factors.create(G), kb.Factors.create(H)
+    qa, sa = kb.kroquant_quantize(A_t, fa, scale_layout="tiled")
+    qw, sw = kb.kroquant_quantize(W_t, fw, scale_layout="tiled")
+    out = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, out_dtype=torch.float32).double().cpu().numpy()
+    # (1) the GEMM on the codes the GPU quantizer produced: exact up to the accumulation order
+    qa_r, sa_r = kb.kroquant_quantize(A_t, fa)
+    qw_r, sw_r = kb.kroquant_quantize(W_t, fw)
+    assert torch.equal(qa_r, qa) and torch.equal(qw_r, qw)
+    Ad = co.dequantize(qa_r.cpu().numpy(), sa_r.cpu().numpy()).astype(np.float64)
+    Wd = co.dequantize(qw_r.cpu().numpy(), sw_r.cpu().numpy()).astype(np.float64)
+    assert np.all(np.abs(out - Ad @ Wd.T) <= TOL * (np.abs(Ad) @ np.abs(Wd).T))
+    # (2) the whole chain against the oracle's own quantizer: a code within 1e-5 of a rounding boundary
+    # may differ (parity rule of the quantizer); each such code moves one output row or column by one grid
+    # step of one element (large for an outlier channel), so the comparison is in the Frobenius norm
+    qa_o, sa_o, _ = co.quantize(A_bits, G)
+    qw_o, sw_o, _ = co.quantize(W_bits, H)
+    ref = co.dequantize(qa_o, sa_o).astype(np.float64) @ co.dequantize(qw_o, sw_o).astype(np.float64).T
+    assert np.linalg.norm(out - ref) <= 5e-3 * np.linalg.norm(ref)
+    assert (qa.cpu().numpy() != qa_o).mean() <= 1e-4 and (qw.cpu().numpy() != qw_o).mean() <= 1e-4
+    fa.destroy()
+    fw.destroy()
+
+
+def test_argument_checks():
+    A, W = _operand(128, 128, 1), _operand(128, 128, 2)
+    qa, sa, _ = _decoded(A)
+    qw, sw, _ = _decoded(W)
+    L = kb.load_library()
+    import ctypes as C
+    out = torch.empty((128, 128), dtype=torch.float32, device="cuda")
+    p = lambda t: C.c_void_p(t.data_ptr())
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert L.kroquant_gemm_mxfp4(p(qa), p(sa), p(qw), p(sw), 128, 128, 100, None, p(out), 0, st) == 2      # K % 32
+    assert L.kroquant_gemm_mxfp4(p(qa), p(sa), p(qw), p(sw), 128, 100, 128, None, p(out), 0, st) == 2      # N % 32
+    assert L.kroquant_gemm_mxfp4(p(qa), None, p(qw), p(sw), 128, 128, 128, None, p(out), 0, st) == 1       # null
+    assert L.kroquant_gemm_mxfp4(p(qa), p(sa), p(qw), p(sw), 128, 128, 128, None, p(out), 7, st) == 5      # dtype
+    assert L.kroquant_gemm_mxfp4(p(qa), p(sa), p(qw), p(sw), 0, 128, 128, None, p(out), 0, st) == 0        # empty
+    with pytest.raises(ValueError):
+        kb.kroquant_gemm_mxfp4(qa, sa[:100], qw, sw)
