@@ -214,9 +214,10 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t *a_codes, const uint8_t *a_scales,
  * error is rounded to bf16 once before the two backward contractions. */
 typedef struct kroquant_calib kroquant_calib_t;
 
-/* Test and tuning knob: which tensor-core GEMM the calibration calls launch from now on.
- * 1 (default): pairs of CTAs on 256 x 256 tiles (tcgen05 cta_group::2); 0: one CTA per 128 x 256
- * tile.  Both compute the same contractions; results differ only in fp32 summation order. */
+/* Test and tuning knob: which tensor-core GEMM kernels the calibration calls and kroquant_gemm_mxfp4
+ * launch from now on.  1 (default): pairs of CTAs on 256 x 256 tiles (tcgen05 cta_group::2); 0: one
+ * CTA per tile (128 x 256 bf16, 128 x 128 FP4).  Both compute the same contractions; results differ
+ * only in fp32 summation order. */
 kq_status_t kroquant_debug_set_gemm_pair(int on);
 
 kq_status_t kroquant_calib_create(const void *A, const void *W, int64_t M, int o, int d, int n_sets,

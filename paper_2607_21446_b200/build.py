@@ -13,7 +13,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libkroquant.so")
 SOURCES = [os.path.join(CSRC, "kroquant_api.cu")]
-HEADERS = [os.path.join(CSRC, n) for n in ("kq_common.cuh", "kq_stream.cuh", "kq_umma.cuh", "kq_gemm.cuh", "kq_gemm2.cuh", "kq_gemm_fp4.cuh", "kq_calib.cuh",
+HEADERS = [os.path.join(CSRC, n) for n in ("kq_common.cuh", "kq_stream.cuh", "kq_umma.cuh", "kq_gemm.cuh", "kq_gemm2.cuh", "kq_gemm_fp4.cuh", "kq_gemm_fp4_pair.cuh", "kq_calib.cuh",
                                                "kroquant_calib_api.cuh")] + [
     os.path.join(os.path.dirname(PKG), "include", "kroquant.h")]
 

@@ -5,6 +5,7 @@
 #include "kq_gemm.cuh"
 #include "kq_gemm2.cuh"
 #include "kq_gemm_fp4.cuh"
+#include "kq_gemm_fp4_pair.cuh"
 
 struct kroquant_calib {
     int device = -1;
@@ -251,7 +252,9 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
     static std::atomic<int> attr_done{0};
     if (!attr_done.load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kq::gemm_mxfp4_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kF4DynBytes) !=
-            cudaSuccess) {
+                cudaSuccess ||
+            cudaFuncSetAttribute(kq::gemm_mxfp4_umma_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kq::kF4PDynBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
         }
@@ -269,11 +272,14 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
+    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0;
+    const int bm = pair ? 256 : kq::kF4BM, bn = pair ? 256 : kq::kF4BN;
     kq::Fp4GemmProblem p;
     p.M = (int)M; p.N = N; p.K = K;
-    p.tiles_m = (int)((M + kq::kF4BM - 1) / kq::kF4BM);
-    p.tiles_n = (N + kq::kF4BN - 1) / kq::kF4BN;
-    p.k_blocks = (K + kq::kF4BKElems - 1) / kq::kF4BKElems;
+    p.tiles_m = (int)((M + bm - 1) / bm);
+    p.tiles_n = (N + bn - 1) / bn;
+    const int k_tiles = (K + kq::kF4BKElems - 1) / kq::kF4BKElems;       // 128-element scale tiles along K
+    p.k_blocks = pair ? (K + 255) / 256 : k_tiles;                        // pipeline stages per output tile
     p.sfa = a_scales; p.sfb = b_scales;
     p.add = static_cast<const __nv_bfloat16*>(add_bf16); p.ld_add = N;
     p.out_bf16 = out_dtype == KQ_OUT_BF16 ? static_cast<__nv_bfloat16*>(out) : nullptr;
@@ -282,9 +288,52 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
     const int tiles = p.tiles_m * p.tiles_n;
-    kq::gemm_mxfp4_umma<<<tiles < sms ? tiles : sms, kq::kGemmThreads, kq::kF4DynBytes,
-                          reinterpret_cast<cudaStream_t>(stream)>>>(ta, tb, p);
-    if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (pair) {
+        // the tiled scale buffers as [row tiles][k tiles][128 x 32-bit]
+        CUtensorMap tsa, tsb;
+        const cuuint32_t estr3[3] = {1, 1, 1};
+        const cuuint64_t sstr[2] = {512, (cuuint64_t)k_tiles * 512};
+        const cuuint64_t sadims[3] = {128, (cuuint64_t)k_tiles, (cuuint64_t)((M + 127) / 128)};
+        const cuuint64_t sbdims[3] = {128, (cuuint64_t)k_tiles, (cuuint64_t)((N + 127) / 128)};
+        const cuuint32_t sabox[3] = {128, 2, 1}, sbbox[3] = {128, 2, 2};
+        // codes with 128-byte boxes (one 128-byte swizzle atom per row) for this kernel
+        const cuuint32_t box2[2] = {(cuuint32_t)kq::kF4PKBytes, 128};
+        if (enc(&ta, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(a_codes), adims, strides, box2, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            enc(&tb, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(b_codes), bdims, strides, box2, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return KQ_ERR_CUDA;
+        if (enc(&tsa, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t*>(a_scales), sadims, sstr, sabox, estr3,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+            enc(&tsb, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<uint8_t*>(b_scales), sbdims, sstr, sbbox, estr3,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return KQ_ERR_CUDA;
+        const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * pairs));
+        cfg.blockDim = dim3(kq::kGemmThreads);
+        cfg.dynamicSmemBytes = kq::kF4PDynBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kq::gemm_mxfp4_umma_pair, ta, tb, tsa, tsb, p) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KQ_ERR_CUDA;
+        }
+    } else {
+        kq::gemm_mxfp4_umma<<<tiles < sms ? tiles : sms, kq::kGemmThreads, kq::kF4DynBytes, st>>>(ta, tb, p);
+        if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+    }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return KQ_OK;
 }

@@ -18,6 +18,14 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-6
 
 
+@pytest.fixture(autouse=True, params=["pair", "single"])
+def gemm_variant(request):
+    """Every test runs with both kernels: CTA pairs on 256 x 256 tiles (default) and one CTA per 128 x 128 tile."""
+    kb.set_gemm_pair(request.param == "pair")
+    yield request.param
+    kb.set_gemm_pair(True)
+
+
 def _operand(rows, K, seed, spread=True):
     """bf16 tensor whose 32-blocks have scales spread over 2^-3 .. 2^3 (so that scale bytes differ)."""
     g = torch.Generator(device="cuda")
