@@ -42,6 +42,28 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
                  " [%0], [%1, {%2, %3, %4}], [%5];"
                  ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar_cluster) : "memory");
 }
+// TMEM load without the completion wait (several can be in flight), the wait, and a no-op that makes
+// every later use of the registers depend on a statement placed after the wait
+__device__ __forceinline__ void tc_ld_32x32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void pin_after_wait(uint32_t (&r)[32]) {
+    asm volatile(""
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
+}
 __device__ __forceinline__ void tc_cp_sf_pair(uint32_t tmem_dst, uint64_t sdesc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(tmem_dst), "l"(sdesc) : "memory");
 }
@@ -189,23 +211,26 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             tc_fence_after();
             const int64_t row = (int64_t)tm * 256 + (int)rank * 128 + quarter * 32 + lane;
             const bool row_ok = row < p.M;
-            // four chunks of 32 columns per warp; the accumulator goes back to the issuer right after the
-            // last TMEM load, the last chunk is converted and stored from registers after that
-#pragma unroll 1
+            // this warp's 32 lanes x 128 columns go to registers in one sweep, and the accumulator goes back
+            // to the issuer at once; conversion and stores run from registers while the next tile's MMAs
+            // already write TMEM
+            uint32_t r[4][32];
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc)
+                tc_ld_32x32_nowait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((chalf * 4 + cc) * 32), r[cc]);
+            tc_wait_ld();
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) pin_after_wait(r[cc]);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(bar_tempty, 0));
+#pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
-                const int c = chalf * 4 + cc;
-                const int col = tn * 256 + c * 32;
-                uint32_t r[32];
-                tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(c * 32), r);
-                if (cc == 3) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(mapa_shared(bar_tempty, 0));
-                }
+                const int col = tn * 256 + (chalf * 4 + cc) * 32;
                 if (row_ok && col < p.N) {
                     float v[32];
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[q]);
+                    for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[cc][q]);
                     if (p.add) {
                         const uint4* ap = reinterpret_cast<const uint4*>(p.add + row * p.ld_add + col);
 #pragma unroll
@@ -235,8 +260,8 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                         }
                     }
                 }
-                __syncwarp();
             }
+            __syncwarp();
         }
     }
 
