@@ -696,6 +696,56 @@ def run_gemm_fp4(args):
         "device_error": B.kroquant_last_device_error()}), flush=True)
 
 
+def run_layer(args):
+    """The quantized linear layer of Section 3.4, one call per step (quantizer + W4A4 GEMM), against the
+    bf16 GEMM it replaces; inputs and outputs rotate over buffers that exceed L2.  One JSON line."""
+    import torch
+    from paper_2607_21446_b200 import binding as B
+    B.load_library()
+    t, o, d = (int(v) for v in args.layer.lower().split("x"))
+    nbuf = max(2, int(300e6 // (t * (d + o) * 2)) + 1)
+    sp = W.ActivationSpec("layer", t, d, seed=3, outlier_channels=max(1, d // 200), outlier_gain=100.0)
+    x0 = torch.from_numpy(W.gen_activations(sp).view(np.int16)).cuda().view(torch.bfloat16)
+    Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, nbuf)]
+    outs = [torch.empty((t, o), dtype=torch.bfloat16, device="cuda") for _ in range(nbuf)]
+    Wt = torch.from_numpy(W.gen_weights(3, o, d).view(np.int16)).cuda().view(torch.bfloat16)
+    G = W.gen_factors(3, n_sets=d // 32 if args.per_block else 1)
+    H = np.stack([[np.linalg.inv(G[s_, k].astype(np.float64)).T for k in range(5)] for s_ in range(G.shape[0])]).astype(np.float32)
+    layer = B.LinearW4A4.from_weights(Wt, G, H)
+    q = torch.empty((t, d // 2), dtype=torch.uint8, device="cuda")
+    sc = torch.zeros(B.tiled_scale_bytes(t, d), dtype=torch.uint8, device="cuda")
+
+    def timed(fn):
+        for i in range(max(args.warmup, 3)):
+            fn(i % nbuf)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            fn(i % nbuf)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps * 1e3
+
+    l0 = B.kroquant_launch_count()
+    us_layer = timed(lambda i: layer(Xs[i], out=outs[i]))
+    launches = B.kroquant_launch_count() - l0
+    us_quant = timed(lambda i: B.kroquant_quantize(Xs[i], layer.factors, q, sc, scale_layout="tiled"))
+    us_gemm = timed(lambda i: B.kroquant_gemm_mxfp4(q, sc, layer.w_codes, layer.w_scales, out=outs[i]))
+    us_bf16 = timed(lambda i: torch.matmul(Xs[i], Wt.t(), out=outs[i]))
+    flop = 2.0 * t * o * d
+    print(json.dumps({
+        "metric": "quantized_linear_layer_time", "value": round(us_layer, 2), "unit": "us", "higher_is_better": False,
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "data": "synthetic",
+        "dtype": "bf16 activations -> MXFP4 x MXFP4, fp32 accumulate, bf16 output",
+        "config": {"workload": f"linear layer tokens={t} d={d} o={o}, n_sets={G.shape[0]}",
+                   "l2": f"{nbuf} rotating input/output buffer pairs ({nbuf * t * (d + o) * 2 / 1e6:.0f} MB)"},
+        "gpu_launches": int(launches), "launches_per_step": launches / (args.steps + max(args.warmup, 3)),
+        "quantizer_us": round(us_quant, 2), "w4a4_gemm_us": round(us_gemm, 2), "cublas_bf16_gemm_us": round(us_bf16, 2),
+        "speedup_vs_bf16_gemm": round(us_bf16 / us_layer, 3), "effective_tflops": round(flop / us_layer / 1e6, 1),
+        "device_error": B.kroquant_last_device_error()}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", action="store_true",
@@ -709,6 +759,8 @@ def main():
     ap.add_argument("--per-block", action="store_true", help="with --single: one factor set per 32-channel block")
     ap.add_argument("--calib", default=None, metavar="MxOxD",
                     help="calibration loop on a synthetic layer, e.g. 16384x3072x3072 (with --per-block: one set per block)")
+    ap.add_argument("--layer", default=None, metavar="TOKENSxOxD",
+                    help="quantized linear layer (quantizer + W4A4 GEMM) vs the bf16 GEMM, e.g. 4608x3072x3072")
     ap.add_argument("--gemm-fp4", default=None, metavar="MxNxK",
                     help="W4A4 consumer GEMM, e.g. 4608x3072x3072: own FP4 kernel vs library FP4 vs cuBLAS bf16")
     ap.add_argument("--gemm-single", action="store_true",
@@ -729,6 +781,8 @@ def main():
         run_calib(args)
     elif args.gemm_fp4:
         run_gemm_fp4(args)
+    elif args.layer:
+        run_layer(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -192,6 +192,21 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t *a_codes, const uint8_t *a_scales,
                                 const uint8_t *b_scales, int64_t M, int N, int K, const void *add_bf16,
                                 void *out, kq_dtype_t out_dtype, void *stream);
 
+/* The quantized linear layer of Section 3.4 in one call:
+ *     out = Q(X T) Q(W~)^T (+ add),   Q(X T) by kroquant_quantize_ex (tensor path, tiled scales),
+ *                                     the product by kroquant_gemm_mxfp4,
+ * two launches on `stream`, no allocation, no synchronization.  X: DEVICE [tokens][d] (x_dtype);
+ * f: the activation-side factors; w_codes [o][d/2], w_scales (tiled, for o rows): the weights
+ * quantized offline (e.g. by kroquant_quantize with the factors of kroquant_calib_get_weight_factors);
+ * q_work [tokens][d/2] and s_work (tiled size for tokens rows; its padding bytes must not be 0xFF:
+ * clear it once) receive Q(X T) and can be reused by the next call on the same stream; add: optional
+ * DEVICE bf16 [tokens][o]; out: DEVICE [tokens][o] bf16 or fp32.  o % 32 == 0.  Error codes of the
+ * two calls. */
+kq_status_t kroquant_linear_w4a4(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                 const kroquant_factors_t *f, const uint8_t *w_codes,
+                                 const uint8_t *w_scales, int o, uint8_t *q_work, uint8_t *s_work,
+                                 const void *add_bf16, void *out, kq_dtype_t out_dtype, void *stream);
+
 /* ---- Layer-wise calibration of the transform (Section 3.3; set-up of Appendix D) ----
  *
  * Minimises, over the parameters theta = (a_k, b_k, c_k), k = 1..5, of every factor set,

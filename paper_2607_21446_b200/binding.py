@@ -34,6 +34,7 @@ EXPORTS = [
     "kroquant_calib_loss_grad", "kroquant_calib_run",
     "kroquant_block_grad_scratch_bytes", "kroquant_block_grad", "kroquant_block_grad_static",
     "kroquant_debug_set_gemm_pair", "kroquant_calib_get_weight_factors", "kroquant_gemm_mxfp4",
+    "kroquant_linear_w4a4",
 ]
 
 
@@ -97,6 +98,7 @@ def load_library() -> C.CDLL:
     L.kroquant_block_grad_static.argtypes = [vp, vp, i64, i32, i32, vp, vp]
     L.kroquant_debug_set_gemm_pair.argtypes = [i32]
     L.kroquant_gemm_mxfp4.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, vp]
+    L.kroquant_linear_w4a4.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, i32, vp]
     _lib = L
     return L
 
@@ -437,6 +439,43 @@ def kroquant_gemm_mxfp4(a_codes: torch.Tensor, a_scales: torch.Tensor, b_codes: 
                                               _ptr(add), _ptr(out), 1 if out.dtype == torch.bfloat16 else 0,
                                               _stream(stream)), "kroquant_gemm_mxfp4")
     return out
+
+
+class LinearW4A4:
+    """The quantized linear layer of Section 3.4: holds the activation factors, the offline-quantized
+    weights (codes + tiled scales) and the work buffers for Q(X T); ``__call__`` runs quantizer + FP4 GEMM
+    (two launches, nothing allocated after the first call for a given number of tokens)."""
+
+    def __init__(self, factors: "Factors", w_codes: torch.Tensor, w_scales: torch.Tensor):
+        self.factors, self.w_codes, self.w_scales = factors, w_codes, w_scales
+        self.o, self.d = w_codes.shape[0], 2 * w_codes.shape[1]
+        self._work = {}
+
+    @classmethod
+    def from_weights(cls, W: torch.Tensor, G_act, G_weight) -> "LinearW4A4":
+        """W: CUDA bf16 [o, d]; G_act / G_weight: factor sets [n_sets, 5, 2, 2] of T and T^-T."""
+        fw = Factors.create(G_weight)
+        q, s = kroquant_quantize(W, fw, scale_layout="tiled")
+        torch.cuda.current_stream().synchronize()
+        fw.destroy()
+        return cls(Factors.create(G_act), q, s)
+
+    def __call__(self, X: torch.Tensor, add: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                 out_dtype=torch.bfloat16, stream=None) -> torch.Tensor:
+        tokens, d = _x_shape(X)
+        if d != self.d:
+            raise ValueError("X [tokens, d] does not match the weights")
+        if tokens not in self._work:
+            self._work[tokens] = (torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device),
+                                  torch.zeros(tiled_scale_bytes(tokens, d), dtype=torch.uint8, device=X.device))
+        q, s = self._work[tokens]
+        if out is None:
+            out = torch.empty((tokens, self.o), dtype=out_dtype, device=X.device)
+        _check(load_library().kroquant_linear_w4a4(
+            _ptr(X), X_DTYPES[X.dtype], tokens, d, self.factors._h, _ptr(self.w_codes), _ptr(self.w_scales), self.o,
+            _ptr(q), _ptr(s), _ptr(add), _ptr(out), 1 if out.dtype == torch.bfloat16 else 0, _stream(stream)),
+            "kroquant_linear_w4a4")
+        return out
 
 
 def set_gemm_pair(on: bool) -> None:

@@ -338,6 +338,18 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
     return KQ_OK;
 }
 
+kq_status_t kroquant_linear_w4a4(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const kroquant_factors_t* f,
+                                 const uint8_t* w_codes, const uint8_t* w_scales, int o, uint8_t* q_work, uint8_t* s_work,
+                                 const void* add_bf16, void* out, kq_dtype_t out_dtype, void* stream) {
+    if (!w_codes || !w_scales || !out) return KQ_ERR_NULL;
+    if (o <= 0 || o % 32) return KQ_ERR_SHAPE;
+    if (out_dtype != KQ_OUT_F32 && out_dtype != KQ_OUT_BF16) return KQ_ERR_UNSUPPORTED;
+    const kq_status_t rc =
+        kroquant_quantize_ex(X, x_dtype, tokens, d, f, q_work, s_work, KQ_SCALES_TILED_128X4, KQ_PATH_AUTO, stream);
+    if (rc != KQ_OK) return rc;
+    return kroquant_gemm_mxfp4(q_work, s_work, w_codes, w_scales, tokens, o, d, add_bf16, out, out_dtype, stream);
+}
+
 kq_status_t kroquant_debug_set_gemm_pair(int on) {
     g_gemm_pair.store(on ? 1 : 0, std::memory_order_relaxed);
     return KQ_OK;

@@ -135,6 +135,25 @@ def test_quantized_layer_from_activations_to_output(per_block):
     fw.destroy()
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+def test_linear_layer_call_equals_the_two_separate_calls(dtype):
+    M, o, d, seed = 300, 256, 1152, 13
+    A_bits = wl.gen_activations(wl.calib_spec(M, d, seed), "fp16" if dtype == torch.float16 else "bf16")
+    A_t = torch.from_numpy(A_bits.view(np.int16)).cuda().view(dtype)
+    W_t = torch.from_numpy(wl.gen_weights(seed, o, d).view(np.int16)).cuda().view(torch.bfloat16)
+    theta = wl.gen_lu_params(seed, 1).astype(np.float64)
+    G = cal.lu_factors(theta).astype(np.float32)
+    H = np.stack([[np.linalg.inv(G[0, k].astype(np.float64)).T for k in range(5)]]).astype(np.float32)
+    layer = kb.LinearW4A4.from_weights(W_t, G, H)
+    add = _operand(M, o, 14, spread=False)
+    out = layer(A_t, add=add)
+    out_again = layer(A_t, add=add)          # work buffers reused
+    qa, sa = kb.kroquant_quantize(A_t, layer.factors, scale_layout="tiled")
+    ref = kb.kroquant_gemm_mxfp4(qa, sa, layer.w_codes, layer.w_scales, add=add)
+    assert torch.equal(out, ref) and torch.equal(out_again, ref)
+    assert kb.kroquant_last_device_error() == 0
+
+
 def test_argument_checks():
     A, W = _operand(128, 128, 1), _operand(128, 128, 2)
     qa, sa, _ = _decoded(A)
