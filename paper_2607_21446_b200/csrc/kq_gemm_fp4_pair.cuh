@@ -9,10 +9,13 @@
 // column).  TMEM per CTA: one 256-column accumulator plus 24 columns of scales per stage - there is
 // no room for a second accumulator, so the epilogue hands the accumulator back as soon as its last
 // TMEM load has completed and converts and stores from registers afterwards.
-// Synchronisation as in kq_gemm2.cuh: both CTAs' loads complete on CTA 0's full barrier; CTA 0
-// issues the scale copies (tcgen05.cp.cta_group::2 copies in both CTAs, each from its own shared
-// memory) and the MMAs, and releases stages and accumulators in both CTAs with multicast commits;
-// all 16 epilogue warps arrive on CTA 0's accumulator-empty barrier.  No multicast loads.
+// Synchronisation as in kq_gemm2.cuh: both CTAs' loads complete on CTA 0's full barrier.  In CTA 0 one
+// warp issues the scale copies of a stage (tcgen05.cp.cta_group::2 copies in both CTAs, each from its
+// own shared memory) and commits them to the stage's sfready barrier; another warp waits for that and
+// issues the four MMAs - an issue costs its thread about 60 cycles, and eleven of them per 512-cycle
+// stage in one thread kept the tensor core waiting.  Multicast commits release stages and signal
+// the accumulator in both CTAs; all 16 epilogue warps arrive on CTA 0's accumulator-empty barrier.
+// No multicast loads.
 #pragma once
 #include "kq_gemm2.cuh"
 #include "kq_gemm_fp4.cuh"
@@ -30,7 +33,8 @@ constexpr int kF4PSfbOff = kF4PSfaOff + 1024;            // 2 KB: scales of all 
 constexpr int kF4PLoadBytes = kF4PSfbOff + 2048;         // 35 KB loaded per CTA and stage
 constexpr int kF4PStageBytes = kF4PLoadBytes;            // 35 KB = 35 x 1024
 constexpr int kF4PBarOff = kF4PStages * kF4PStageBytes;
-constexpr int kF4PNumBars = 2 * kF4PStages + 2;          // full[S], empty[S], tfull, tempty
+constexpr int kF4PNumBars = 3 * kF4PStages + 2;          // full[S], empty[S], sfready[S], tfull, tempty
+constexpr int kF4PThreads = 352;                          // producer, MMA issuer, 8 epilogue warps, scale-copy warp
 constexpr int kF4PTmemSlotOff = kF4PBarOff + 8 * kF4PNumBars;
 constexpr int kF4PAbortOff = kF4PTmemSlotOff + 4;
 constexpr int kF4PDynBytes = kF4PAbortOff + 4 + 1024;
@@ -83,7 +87,7 @@ __device__ __forceinline__ void tc_mma_mxf4_pair(uint32_t tmem_d, uint64_t desc_
 // p.tiles_m, p.tiles_n count 256 x 256 tiles; p.k_blocks counts stages of 256 elements.  tmap_sfa /
 // tmap_sfb: the tiled scale buffers viewed as [row tiles][k tiles][128 x 32-bit]; boxes of 2 k tiles
 // x 1 and 2 row tiles (k tiles past the end read as zero: scale 2^-127 on all-zero codes).
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __launch_bounds__(kF4PThreads, 1)
 gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                      const __grid_constant__ CUtensorMap tmap_sfa, const __grid_constant__ CUtensorMap tmap_sfb,
                      const Fp4GemmProblem p) {
@@ -94,8 +98,9 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const uint32_t bar0 = base + kF4PBarOff;
     auto bar_full = [&](int s) { return bar0 + 8u * s; };
     auto bar_empty = [&](int s) { return bar0 + 8u * (kF4PStages + s); };
-    const uint32_t bar_tfull = bar0 + 8u * (2 * kF4PStages);
-    const uint32_t bar_tempty = bar0 + 8u * (2 * kF4PStages + 1);
+    auto bar_sfready = [&](int s) { return bar0 + 8u * (2 * kF4PStages + s); };
+    const uint32_t bar_tfull = bar0 + 8u * (3 * kF4PStages);
+    const uint32_t bar_tempty = bar0 + 8u * (3 * kF4PStages + 1);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + kF4PTmemSlotOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + kF4PAbortOff);
 
@@ -107,7 +112,7 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const int my_tiles = pair < n_tiles ? (n_tiles - pair + n_pairs - 1) / n_pairs : 0;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kF4PStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int s = 0; s < kF4PStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); mbar_init(bar_sfready(s), 1); }
         mbar_init(bar_tfull, 1);
         mbar_init(bar_tempty, 16);
         *abort_flag = 0;
@@ -156,12 +161,10 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             }
         }
     } else if (warp == 1) {
-        // ---------------- scale copies and MMAs (leader CTA only) ----------------
+        // ---------------- MMA issuer (leader CTA only) ----------------
         if (lane == 0 && rank == 0) {
             const uint64_t a_desc0 = smem_desc_sw128(base);
             const uint64_t b_desc0 = smem_desc_sw128(base + kF4PABytes);
-            const uint64_t sfa_desc0 = smem_desc_sf(base + kF4PSfaOff);
-            const uint64_t sfb_desc0 = smem_desc_sf(base + kF4PSfbOff);
             int it = 0;
             bool ok = true;
             for (int i = 0; ok && i < my_tiles; ++i) {
@@ -172,7 +175,8 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 tc_fence_after();
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % kF4PStages;
-                    if (!mbar_wait(bar_full(s), (it / kF4PStages) & 1, abort_flag)) {
+                    // sfready[s]: the stage's codes have landed in both CTAs and its scales are in TMEM
+                    if (!mbar_wait(bar_sfready(s), (it / kF4PStages) & 1, abort_flag)) {
                         if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_GEMM_MMA); *abort_flag = 1; }
                         ok = false;
                         break;
@@ -181,12 +185,6 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     const uint64_t off = (uint64_t)((s * kF4PStageBytes) >> 4);
                     const uint32_t t_sfa = tmem_base + (uint32_t)(kF4PSfCol0 + 24 * s);
                     const uint32_t t_sfb = t_sfa + 8;
-#pragma unroll
-                    for (int y = 0; y < 2; ++y) {          // k tile y of the stage: elements 128 y .. 128 y + 127
-                        tc_cp_sf_pair(t_sfa + 4 * y, sfa_desc0 + off + (uint64_t)((512 * y) >> 4));
-                        tc_cp_sf_pair(t_sfb + 8 * y, sfb_desc0 + off + (uint64_t)((512 * y) >> 4));               // B rows 0..127
-                        tc_cp_sf_pair(t_sfb + 8 * y + 4, sfb_desc0 + off + (uint64_t)((512 * (2 + y)) >> 4));   // B rows 128..255
-                    }
 #pragma unroll
                     for (int k = 0; k < 4; ++k)            // 64 elements = 32 bytes of K per instruction
                         tc_mma_mxf4_pair(tmem_base, a_desc0 + off + (uint64_t)(2 * k), b_desc0 + off + (uint64_t)(2 * k),
@@ -197,7 +195,34 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 if (ok) tc_commit_pair(bar_tfull);
             }
         }
-    } else {
+    } else if (warp == 10) {
+        // ---------------- scale tiles: shared memory -> TMEM of both CTAs (leader CTA only) ----------------
+        if (lane == 0 && rank == 0) {
+            const uint64_t sfa_desc0 = smem_desc_sf(base + kF4PSfaOff);
+            const uint64_t sfb_desc0 = smem_desc_sf(base + kF4PSfbOff);
+            const int total = my_tiles * p.k_blocks;
+            for (int it = 0; it < total; ++it) {
+                const int s = it % kF4PStages;
+                // full[s] of this round also means the MMAs that read the slot's previous scales are done
+                if (!mbar_wait(bar_full(s), (it / kF4PStages) & 1, abort_flag)) {
+                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_GEMM_MMA); *abort_flag = 1; }
+                    break;
+                }
+                tc_fence_after();
+                const uint64_t off = (uint64_t)((s * kF4PStageBytes) >> 4);
+                const uint32_t t_sfa = tmem_base + (uint32_t)(kF4PSfCol0 + 24 * s);
+                const uint32_t t_sfb = t_sfa + 8;
+#pragma unroll
+                for (int y = 0; y < 2; ++y) {          // k tile y of the stage: elements 128 y .. 128 y + 127
+                    tc_cp_sf_pair(t_sfa + 4 * y, sfa_desc0 + off + (uint64_t)((512 * y) >> 4));
+                    tc_cp_sf_pair(t_sfb + 8 * y, sfb_desc0 + off + (uint64_t)((512 * y) >> 4));               // B rows 0..127
+                    tc_cp_sf_pair(t_sfb + 8 * y + 4, sfb_desc0 + off + (uint64_t)((512 * (2 + y)) >> 4));   // B rows 128..255
+                }
+                asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             ::"r"(bar_sfready(s)) : "memory");
+            }
+        }
+    } else if (warp < 10) {
         // ---------------- epilogue: warps 2..9 of both CTAs; warp = lane quarter x column half ----------------
         const int quarter = warp & 3;
         const int chalf = (warp - 2) >> 2;

@@ -316,7 +316,7 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
         const int pairs = tiles < sms / 2 ? tiles : sms / 2;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(2 * pairs));
-        cfg.blockDim = dim3(kq::kGemmThreads);
+        cfg.blockDim = dim3(kq::kF4PThreads);
         cfg.dynamicSmemBytes = kq::kF4PDynBytes;
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
