@@ -68,6 +68,11 @@ __device__ __forceinline__ void pin_after_wait(uint32_t (&r)[32]) {
           "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
         :: "memory");
 }
+// 32-byte store (one full sector per lane); the address must be 32-byte aligned
+__device__ __forceinline__ void st_global_32(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
 __device__ __forceinline__ void tc_cp_sf_pair(uint32_t tmem_dst, uint64_t sdesc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(tmem_dst), "l"(sdesc) : "memory");
 }
@@ -226,6 +231,8 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         // ---------------- epilogue: warps 2..9 of both CTAs; warp = lane quarter x column half ----------------
         const int quarter = warp & 3;
         const int chalf = (warp - 2) >> 2;
+        // full-sector (32-byte) stores when the output base allows it; row pitches and column offsets always do
+        const bool wide = ((reinterpret_cast<uintptr_t>(p.out_bf16) | reinterpret_cast<uintptr_t>(p.out_f32)) & 31u) == 0;
         for (int i = 0; i < my_tiles; ++i) {
             int tm, tn;
             fp4_tile_coords(pair + i * n_pairs, p, tm, tn);
@@ -267,21 +274,38 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                         }
                     }
                     if (p.out_f32) {
-                        float4* op = reinterpret_cast<float4*>(p.out_f32 + row * p.ld_out + col);
+                        float* op = p.out_f32 + row * p.ld_out + col;
+                        if (wide) {
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                            for (int q = 0; q < 4; ++q) {
+                                uint32_t w[8];
+#pragma unroll
+                                for (int h = 0; h < 8; ++h) w[h] = __float_as_uint(v[8 * q + h]);
+                                st_global_32(op + 8 * q, w);
+                            }
+                        } else {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                reinterpret_cast<float4*>(op)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                        }
                     }
                     if (p.out_bf16) {
-                        uint4* op = reinterpret_cast<uint4*>(p.out_bf16 + row * p.ld_out + col);
+                        __nv_bfloat16* op = p.out_bf16 + row * p.ld_out + col;
+                        uint32_t w[16];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            uint32_t w[4];
+                        for (int h = 0; h < 16; ++h) {
+                            const __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * h], v[2 * h + 1]);
+                            w[h] = *reinterpret_cast<const uint32_t*>(&b);
+                        }
+                        if (wide) {
+                            const uint32_t lo[8] = {w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]};
+                            const uint32_t hi[8] = {w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]};
+                            st_global_32(op, lo);
+                            st_global_32(op + 16, hi);
+                        } else {
 #pragma unroll
-                            for (int h = 0; h < 4; ++h) {
-                                const __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * q + 2 * h], v[8 * q + 2 * h + 1]);
-                                w[h] = *reinterpret_cast<const uint32_t*>(&b);
-                            }
-                            op[q] = make_uint4(w[0], w[1], w[2], w[3]);
+                            for (int q = 0; q < 4; ++q)
+                                reinterpret_cast<uint4*>(op)[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
                         }
                     }
                 }

@@ -65,6 +65,23 @@ def test_against_the_decoded_float64_product(M, N, K):
     assert torch.equal(out16, out.to(torch.bfloat16))
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_output_base_that_is_only_16_byte_aligned(dtype):
+    """The epilogue uses 32-byte stores when the output base allows it and 16-byte stores otherwise."""
+    M, N, K = 200, 288, 256
+    A, W = _operand(M, K, 21), _operand(N, K, 22)
+    qa, sa, _ = _decoded(A)
+    qw, sw, _ = _decoded(W)
+    ref = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, out_dtype=dtype)
+    shift = 16 // ref.element_size()
+    flat = torch.zeros(M * N + shift, dtype=dtype, device="cuda")
+    out = flat[shift:].view(M, N)
+    assert out.data_ptr() % 32 == 16
+    kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, out=out)
+    assert torch.equal(out, ref)
+    assert float(flat[:shift].abs().max()) == 0.0
+
+
 def test_low_rank_branch_is_added_before_the_single_rounding():
     M, N, K = 384, 256, 512
     A, W = _operand(M, K, 3), _operand(N, K, 4)
