@@ -82,6 +82,12 @@ __device__ __forceinline__ void gemm_tile_coords(int t, const GemmProblem& p, in
     tn = r / m_count;
 }
 
+// 32-byte store (one full sector per lane); the address must be 32-byte aligned
+__device__ __forceinline__ void st_global_32(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
+
 // Epilogue of one row x 32 columns held in registers: v = acc + coef * aux; [sum v^2]; stores.
 __device__ __forceinline__ void gemm_epilogue_chunk(const GemmProblem& p, const uint32_t (&r)[32], int64_t row, int col,
                                                     float coef, float& sq_tile) {
@@ -104,22 +110,41 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmProblem& p, const 
 #pragma unroll
         for (int q = 0; q < 32; ++q) sq_tile = fmaf(v[q], v[q], sq_tile);
     }
+    // full-sector stores when the output base allows it (row pitches and column offsets always do:
+    // N is a multiple of 32)
     if (p.out_f32) {
-        float4* op = reinterpret_cast<float4*>(p.out_f32 + row * p.ld_out + col);
+        float* op = p.out_f32 + row * p.ld_out + col;
+        if ((reinterpret_cast<uintptr_t>(p.out_f32) & 31u) == 0) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            for (int q = 0; q < 4; ++q) {
+                uint32_t w[8];
+#pragma unroll
+                for (int h = 0; h < 8; ++h) w[h] = __float_as_uint(v[8 * q + h]);
+                st_global_32(op + 8 * q, w);
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                reinterpret_cast<float4*>(op)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        }
     }
     if (p.out_bf16) {
-        uint4* op = reinterpret_cast<uint4*>(p.out_bf16 + row * p.ld_out + col);
+        __nv_bfloat16* op = p.out_bf16 + row * p.ld_out + col;
+        uint32_t w[16];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            uint32_t w[4];
+        for (int h = 0; h < 16; ++h) {
+            const __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * h] * p.out_scale, v[2 * h + 1] * p.out_scale);
+            w[h] = *reinterpret_cast<const uint32_t*>(&b);
+        }
+        if ((reinterpret_cast<uintptr_t>(p.out_bf16) & 31u) == 0) {
+            const uint32_t lo[8] = {w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]};
+            const uint32_t hi[8] = {w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]};
+            st_global_32(op, lo);
+            st_global_32(op + 16, hi);
+        } else {
 #pragma unroll
-            for (int h = 0; h < 4; ++h) {
-                const __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * q + 2 * h] * p.out_scale, v[8 * q + 2 * h + 1] * p.out_scale);
-                w[h] = *reinterpret_cast<const uint32_t*>(&b);
-            }
-            op[q] = make_uint4(w[0], w[1], w[2], w[3]);
+            for (int q = 0; q < 4; ++q)
+                reinterpret_cast<uint4*>(op)[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
         }
         if (p.out_bf16_t) {
             // lanes hold consecutive rows: each store instruction writes 64 contiguous bytes
