@@ -88,19 +88,35 @@ __device__ __forceinline__ void st_global_32(void* p, const uint32_t (&w)[8]) {
                  ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
 
+// 32-byte read-only load; the address must be 32-byte aligned
+__device__ __forceinline__ void ld_global_nc_32(const void* p, uint32_t (&w)[8]) {
+    asm volatile("ld.global.nc.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "l"(p));
+}
+
 // Epilogue of one row x 32 columns held in registers: v = acc + coef * aux; [sum v^2]; stores.
 __device__ __forceinline__ void gemm_epilogue_chunk(const GemmProblem& p, const uint32_t (&r)[32], int64_t row, int col,
                                                     float coef, float& sq_tile) {
     float v[32];
     if (p.aux) {
-        const float4* ap = reinterpret_cast<const float4*>(p.aux + row * p.ld_aux + col);
+        const float* ap = p.aux + row * p.ld_aux + col;
+        if ((reinterpret_cast<uintptr_t>(p.aux) & 31u) == 0) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const float4 a = __ldg(ap + q);
-            v[4 * q + 0] = fmaf(coef, a.x, __uint_as_float(r[4 * q + 0]));
-            v[4 * q + 1] = fmaf(coef, a.y, __uint_as_float(r[4 * q + 1]));
-            v[4 * q + 2] = fmaf(coef, a.z, __uint_as_float(r[4 * q + 2]));
-            v[4 * q + 3] = fmaf(coef, a.w, __uint_as_float(r[4 * q + 3]));
+            for (int q = 0; q < 4; ++q) {
+                uint32_t a[8];
+                ld_global_nc_32(ap + 8 * q, a);
+#pragma unroll
+                for (int h = 0; h < 8; ++h) v[8 * q + h] = fmaf(coef, __uint_as_float(a[h]), __uint_as_float(r[8 * q + h]));
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const float4 a = __ldg(reinterpret_cast<const float4*>(ap) + q);
+                v[4 * q + 0] = fmaf(coef, a.x, __uint_as_float(r[4 * q + 0]));
+                v[4 * q + 1] = fmaf(coef, a.y, __uint_as_float(r[4 * q + 1]));
+                v[4 * q + 2] = fmaf(coef, a.z, __uint_as_float(r[4 * q + 2]));
+                v[4 * q + 3] = fmaf(coef, a.w, __uint_as_float(r[4 * q + 3]));
+            }
         }
     } else {
 #pragma unroll
