@@ -196,22 +196,29 @@ struct UmmaSmem {
 template <bool XF16>
 __device__ __forceinline__ void store_block_16bit(const uint32_t (&acc)[32], int e, uint4* dst) {
     const float back = __uint_as_float((uint32_t)(127 - e) << 23);      // 2^-e
+    uint32_t w[16];
 #pragma unroll
-    for (int v = 0; v < 4; ++v) {
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float a = __uint_as_float(acc[8 * v + 2 * i]) * back;
-            const float b = __uint_as_float(acc[8 * v + 2 * i + 1]) * back;
-            if (XF16) {
-                const __half2 h = __floats2half2_rn(a, b);
-                w[i] = *reinterpret_cast<const uint32_t*>(&h);
-            } else {
-                const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-                w[i] = *reinterpret_cast<const uint32_t*>(&h);
-            }
+    for (int i = 0; i < 16; ++i) {
+        const float a = __uint_as_float(acc[2 * i]) * back;
+        const float b = __uint_as_float(acc[2 * i + 1]) * back;
+        if (XF16) {
+            const __half2 h = __floats2half2_rn(a, b);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+        } else {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
         }
-        dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    // the 64 bytes of a block are 64-byte aligned relative to the buffer: two full-sector stores when the
+    // buffer itself is 32-byte aligned, four 16-byte stores otherwise
+    if ((reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     ::"l"(dst + 2), "r"(w[8]), "r"(w[9]), "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15]) : "memory");
+    } else {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) dst[v] = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
     }
 }
 
@@ -533,11 +540,24 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     const int e = PB ? __ldg(e_norm + (int)(blk % prob.blocks_per_row)) : e_shared;
                     if (WRITE_Y) {
                         const float back = __uint_as_float((uint32_t)(127 - e) << 23);    // 2^-e
-                        float4* yp = reinterpret_cast<float4*>(Y + blk * 32);
+                        float* yp = Y + blk * 32;
+                        if ((reinterpret_cast<uintptr_t>(yp) & 31u) == 0) {         // full-sector stores
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            yp[i] = make_float4(__uint_as_float(acc[4 * i]) * back, __uint_as_float(acc[4 * i + 1]) * back,
+                            for (int i = 0; i < 4; ++i) {
+                                uint32_t w[8];
+#pragma unroll
+                                for (int h = 0; h < 8; ++h) w[h] = __float_as_uint(__uint_as_float(acc[8 * i + h]) * back);
+                                asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                             ::"l"(yp + 8 * i), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]),
+                                               "r"(w[6]), "r"(w[7]) : "memory");
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                reinterpret_cast<float4*>(yp)[i] =
+                                    make_float4(__uint_as_float(acc[4 * i]) * back, __uint_as_float(acc[4 * i + 1]) * back,
                                                 __uint_as_float(acc[4 * i + 2]) * back, __uint_as_float(acc[4 * i + 3]) * back);
+                        }
                     } else {
                         uint4 codes;
                         uint32_t S;
