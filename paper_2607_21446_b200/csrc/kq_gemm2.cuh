@@ -13,7 +13,7 @@
 //             multicast tcgen05.commit of the issuer;
 //   tfull[a]  one per CTA, waited on by that CTA's epilogue; signalled by a multicast commit;
 //   tempty[a] CTA 0's only: the 8 epilogue warps of each CTA arrive on it (CTA 1 remotely).
-// No load uses cluster multicast.  Every wait is bounded; both CTAs meet at a cluster barrier
+// Each CTA fetches its own operand halves with plain per-CTA TMA copies.  Every wait is bounded; both CTAs meet at a cluster barrier
 // before they free TMEM and exit, so neither touches the other's shared memory after it is gone.
 #pragma once
 #include "kq_gemm.cuh"
@@ -46,7 +46,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA load of this CTA's box into its own shared memory; the completion goes to `bar_cluster`,
-// which may be the partner's barrier.  No multicast.
+// which may be the partner's barrier.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tmap, int x, int y, uint32_t bar_cluster) {
     asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
                  " [%0], [%1, {%2, %3}], [%4];"

@@ -15,7 +15,7 @@
 // issues the four MMAs - an issue costs its thread about 60 cycles, and eleven of them per 512-cycle
 // stage in one thread kept the tensor core waiting.  Multicast commits release stages and signal
 // the accumulator in both CTAs; all 16 epilogue warps arrive on CTA 0's accumulator-empty barrier.
-// No multicast loads.
+// Each CTA fetches its own data with plain per-CTA TMA copies.
 #pragma once
 #include "kq_gemm2.cuh"
 #include "kq_gemm_fp4.cuh"
