@@ -43,6 +43,10 @@ struct Fp4GemmProblem {
     __nv_bfloat16* out_bf16;           // [M][ld_out] or null
     float* out_f32;                    // [M][ld_out] or null
     int64_t ld_out;
+    // pair kernel only: when use_epi != 0 the epilogue of the bf16 GEMM (kq_gemm.cuh: v = acc + coef * aux,
+    // sum of v^2, scaled bf16 output and its transpose) runs instead of add / out above
+    int use_epi;
+    GemmProblem epi;
 };
 
 // 32 rows x 16 bytes, rows 16 bytes apart (no swizzle): source descriptor of the scale-tile copy

@@ -228,6 +228,8 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const int chalf = (warp - 2) >> 2;
         // full-sector (32-byte) stores when the output base allows it; row pitches and column offsets always do
         const bool wide = ((reinterpret_cast<uintptr_t>(p.out_bf16) | reinterpret_cast<uintptr_t>(p.out_f32)) & 31u) == 0;
+        const float epi_coef = p.use_epi ? p.epi.coef_mul * (p.epi.coef_ptr ? __ldg(p.epi.coef_ptr) : 1.0f) : 0.f;
+        double sq = 0.0;
         for (int i = 0; i < my_tiles; ++i) {
             int tm, tn;
             fp4_tile_coords(pair + i * n_pairs, p, tm, tn);
@@ -251,10 +253,13 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(bar_tempty, 0));
+            float sq_tile = 0.f;
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
                 const int col = tn * 256 + (chalf * 4 + cc) * 32;
-                if (row_ok && col < p.N) {
+                if (p.use_epi) {
+                    if (row_ok && col < p.N) gemm_epilogue_chunk(p.epi, r[cc], row, col, epi_coef, sq_tile);
+                } else if (row_ok && col < p.N) {
                     float v[32];
 #pragma unroll
                     for (int q = 0; q < 32; ++q) v[q] = __uint_as_float(r[cc][q]);
@@ -305,7 +310,13 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     }
                 }
             }
+            sq += (double)sq_tile;
             __syncwarp();
+        }
+        if (p.use_epi && p.epi.sumsq) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);
+            if (lane == 0 && sq != 0.0) atomicAdd(p.epi.sumsq, sq);
         }
     }
 

@@ -20,6 +20,8 @@ struct kroquant_calib {
     float *ResY = nullptr, *ResZ = nullptr, *R = nullptr, *dY = nullptr, *dZ = nullptr;
     float *partK = nullptr, *partP = nullptr;     // partial block sums [chunks][nb][32][32]
     float *dK = nullptr, *dP = nullptr;           // reduced block gradients [n_sets][32][32]
+    // Q(AT) and Q(WT^-T) once more as packed codes + tiled scale bytes: operands of the FP4 forward GEMM
+    uint8_t *qY = nullptr, *sY = nullptr, *qZ = nullptr, *sZ = nullptr;
     int chunksK = 0, chunksP = 0;
     int64_t rpcK = 0, rpcP = 0;
     double* sums = nullptr;            // [3] sums of squares of the evaluation in flight
@@ -30,6 +32,10 @@ struct kroquant_calib {
     CUtensorMap tm_A_a, tm_W_b, tm_Yq_a, tm_Zq_b, tm_dO_a, tm_ZqT_b, tm_dOT_a, tm_YqT_b;
     CUtensorMap tm_W_a, tm_Zq_a, tm_ZqT_a, tm_YqT_a;
 };
+
+kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
+                            const uint8_t* b_scales, int64_t M, int N, int K, const void* add_bf16, void* out,
+                            kq_dtype_t out_dtype, const kq::GemmProblem* epi, void* stream);
 
 namespace {
 
@@ -159,10 +165,28 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
     if (!launched()) return KQ_ERR_CUDA;
     kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, c->ZqT, c->ResZ, c->sums + 2);
     if (!launched()) return KQ_ERR_CUDA;
-    // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o))
-    kq_status_t rc = launch_gemm(c->tm_Yq_a, c->tm_Zq_b, c->tm_Zq_a, (int)M, o, d, c->R, o, nullptr, -1.0f,
-                                 (float)(2.0 / ((double)M * o)), nullptr, backward ? c->dO : nullptr, o, c->sums, st,
-                                 backward ? c->dOT : nullptr, M);
+    // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o)) and its transpose.  Yq and Zq are MXFP4 values,
+    // so with the paired kernels the product runs on the FP4 tensor-core path: re-encoding Yq, Zq with the
+    // bare MXFP4 encoder returns their codes and scales exactly (the encoder is idempotent on its own output)
+    kq_status_t rc;
+    if (g_gemm_pair.load(std::memory_order_relaxed) != 0) {
+        rc = run_stream<kq::MODE_PLAIN, false>(c->Yq, false, M, d, nullptr, nullptr, c->qY, c->sY, true, nullptr, st);
+        if (rc != KQ_OK) return rc;
+        rc = run_stream<kq::MODE_PLAIN, false>(c->Zq, false, o, d, nullptr, nullptr, c->qZ, c->sZ, true, nullptr, st);
+        if (rc != KQ_OK) return rc;
+        kq::GemmProblem e{};
+        e.M = (int)M; e.N = o; e.K = d;
+        e.aux = c->R; e.ld_aux = o; e.coef_ptr = nullptr; e.coef_mul = -1.0f;
+        e.out_scale = (float)(2.0 / ((double)M * o));
+        e.out_f32 = nullptr; e.out_bf16 = backward ? c->dO : nullptr; e.ld_out = o;
+        e.out_bf16_t = backward ? c->dOT : nullptr; e.ld_out_t = M;
+        e.sumsq = c->sums;
+        rc = launch_gemm_fp4(c->qY, c->sY, c->qZ, c->sZ, M, o, d, nullptr, nullptr, KQ_OUT_BF16, &e, st);
+    } else {
+        rc = launch_gemm(c->tm_Yq_a, c->tm_Zq_b, c->tm_Zq_a, (int)M, o, d, c->R, o, nullptr, -1.0f,
+                         (float)(2.0 / ((double)M * o)), nullptr, backward ? c->dO : nullptr, o, c->sums, st,
+                         backward ? c->dOT : nullptr, M);
+    }
     if (rc != KQ_OK) return rc;
     if (hist_row >= 0 &&
         cudaMemcpyAsync(c->hist + 3 * hist_row, c->sums, 3 * sizeof(double), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
@@ -240,10 +264,19 @@ kq_status_t kroquant_block_grad(const void* X, const float* G, int64_t rows, int
 kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
                                 const uint8_t* b_scales, int64_t M, int N, int K, const void* add_bf16, void* out,
                                 kq_dtype_t out_dtype, void* stream) {
-    if (!a_codes || !a_scales || !b_codes || !b_scales || !out) return KQ_ERR_NULL;
+    return launch_gemm_fp4(a_codes, a_scales, b_codes, b_scales, M, N, K, add_bf16, out, out_dtype, nullptr, stream);
+}
+
+}  // extern "C"
+
+// epi != null (paired kernel only): run the bf16 GEMM's fused epilogue described by *epi instead of add / out
+kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
+                            const uint8_t* b_scales, int64_t M, int N, int K, const void* add_bf16, void* out,
+                            kq_dtype_t out_dtype, const kq::GemmProblem* epi, void* stream) {
+    if (!a_codes || !a_scales || !b_codes || !b_scales || (!out && !epi)) return KQ_ERR_NULL;
     if (M < 0 || N <= 0 || K <= 0 || K % 32 || N % 32 || M > (1 << 30)) return KQ_ERR_SHAPE;
     if (out_dtype != KQ_OUT_F32 && out_dtype != KQ_OUT_BF16) return KQ_ERR_UNSUPPORTED;
-    if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) || !aligned16(out) ||
+    if (!aligned16(a_codes) || !aligned16(a_scales) || !aligned16(b_codes) || !aligned16(b_scales) || (out && !aligned16(out)) ||
         (add_bf16 && !aligned16(add_bf16)))
         return KQ_ERR_ALIGN;
     if (M == 0) return KQ_OK;
@@ -272,7 +305,7 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
-    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0;
+    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0 || epi != nullptr;
     const int bm = pair ? 256 : kq::kF4BM, bn = pair ? 256 : kq::kF4BN;
     kq::Fp4GemmProblem p;
     p.M = (int)M; p.N = N; p.K = K;
@@ -285,6 +318,8 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
     p.out_bf16 = out_dtype == KQ_OUT_BF16 ? static_cast<__nv_bfloat16*>(out) : nullptr;
     p.out_f32 = out_dtype == KQ_OUT_F32 ? static_cast<float*>(out) : nullptr;
     p.ld_out = N;
+    p.use_epi = epi ? 1 : 0;
+    if (epi) p.epi = *epi; else p.epi = kq::GemmProblem{};
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
     const int tiles = p.tiles_m * p.tiles_n;
@@ -338,6 +373,8 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t* a_codes, const uint8_t* a_scales,
     return KQ_OK;
 }
 
+extern "C" {
+
 kq_status_t kroquant_linear_w4a4(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const kroquant_factors_t* f,
                                  const uint8_t* w_codes, const uint8_t* w_scales, int o, uint8_t* q_work, uint8_t* s_work,
                                  const void* add_bf16, void* out, kq_dtype_t out_dtype, void* stream) {
@@ -385,6 +422,9 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     const size_t o_ResY = take(Md * 4), o_ResZ = take(od * 4), o_R = take(Mo * 4), o_dY = take(Md * 4), o_dZ = take(od * 4);
     const size_t o_pK = take((size_t)c->chunksK * c->nb * 4096), o_pP = take((size_t)c->chunksP * c->nb * 4096);
     const size_t o_dK = take((size_t)n_sets * 4096), o_dP = take((size_t)n_sets * 4096);
+    const size_t kt = (size_t)((d + 127) / 128) * 512;                       // scale bytes per 128-row tile
+    const size_t sY_bytes = (size_t)((M + 127) / 128) * kt, sZ_bytes = (size_t)((o + 127) / 128) * kt;
+    const size_t o_qY = take(Md / 2), o_sY = take(sY_bytes), o_qZ = take(od / 2), o_sZ = take(sZ_bytes);
     const size_t o_sums = take(3 * 8), o_hist = take((size_t)kHistCap * 3 * 8);
     if (cudaMalloc(&c->pool, off) != cudaSuccess) { (void)cudaGetLastError(); delete c; return KQ_ERR_CUDA; }
     uint8_t* b = c->pool;
@@ -398,6 +438,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     c->dY = (float*)(b + o_dY); c->dZ = (float*)(b + o_dZ);
     c->partK = (float*)(b + o_pK); c->partP = (float*)(b + o_pP);
     c->dK = (float*)(b + o_dK); c->dP = (float*)(b + o_dP);
+    c->qY = b + o_qY; c->sY = b + o_sY; c->qZ = b + o_qZ; c->sZ = b + o_sZ;
     c->sums = (double*)(b + o_sums); c->hist = (double*)(b + o_hist);
 
     bool ok = make_operand_map(&c->tm_A_a, c->A, M, d, kq::kGemmBM) && make_operand_map(&c->tm_W_b, c->W, o, d, kq::kGemmBN) &&
@@ -409,6 +450,9 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     kq_status_t rc = ok ? KQ_OK : KQ_ERR_CUDA;
     std::vector<float> th;
     hadamard_theta(th, n_sets);
+    if (rc == KQ_OK && (cudaMemsetAsync(c->sY, 0, sY_bytes, st) != cudaSuccess ||    // padding bytes stay zero
+                        cudaMemsetAsync(c->sZ, 0, sZ_bytes, st) != cudaSuccess))
+        rc = KQ_ERR_CUDA;
     if (rc == KQ_OK && (cudaMemsetAsync(c->pool, 0, o_K, st) != cudaSuccess ||      // theta, m, v, grad, lambdas
                         cudaMemcpyAsync(c->theta, th.data(), np * 4, cudaMemcpyHostToDevice, st) != cudaSuccess))
         rc = KQ_ERR_CUDA;
