@@ -42,8 +42,8 @@ calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, fl
 // only the accumulation rounds (the same device as in the quantizer kernels).  grid (row groups,
 // d/32); 4 warps; a warp owns 16 rows per iteration, the CTA 64.  Q is the MXFP4 encoder of the
 // quantizer kernels followed by its decoder; Vq is exact in bf16.  Outputs: Vq [rows][d],
-// its transpose VqT [d][rows] (staged through shared memory, 16-byte segments), R = V - Vq,
-// and the sum of R^2.
+// optionally its transpose VqT [d][rows] (staged through shared memory, 16-byte segments; only the
+// one-CTA GEMM needs it, the paired GEMM reads Vq in either orientation), R = V - Vq, and the sum of R^2.
 // two E2M1 codes (one byte, even element in the low nibble) -> two floats, by the hardware convert
 __device__ __forceinline__ float2 e2m1x2_to_float2(uint32_t byte) {
     uint32_t h2;
@@ -150,8 +150,10 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
                 const __nv_bfloat162 hq = __floats2bfloat162_rn(q0, q1);
                 const uint32_t packed = *reinterpret_cast<const uint32_t*>(&hq);
                 const int col = 8 * t + 2 * q;
-                tt[col][rpos] = (uint16_t)(packed & 0xFFFFu);
-                tt[col + 1][rpos] = (uint16_t)(packed >> 16);
+                if (VqT) {
+                    tt[col][rpos] = (uint16_t)(packed & 0xFFFFu);
+                    tt[col + 1][rpos] = (uint16_t)(packed >> 16);
+                }
                 if (row < rows) {
                     *reinterpret_cast<uint32_t*>(Vq + row * d + j * 32 + col) = packed;
                     *reinterpret_cast<float2*>(Res + row * d + j * 32 + col) = make_float2(e0, e1);
@@ -159,16 +161,18 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
             }
         }
         sq += (double)sq_it;
-        __syncthreads();
+        if (VqT) {                         // kernel argument: the same for every thread
+            __syncthreads();
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const int seg = threadIdx.x + 128 * i;
-            const int col = seg >> 3, rs = (seg & 7) * 8;
-            if (row0 + rs < rows)          // rows is a multiple of 8: a segment is all valid or all past the end
-                *reinterpret_cast<uint4*>(VqT + (int64_t)(j * 32 + col) * rows + row0 + rs) =
-                    *reinterpret_cast<const uint4*>(&tt[col][rs]);
+            for (int i = 0; i < 2; ++i) {
+                const int seg = threadIdx.x + 128 * i;
+                const int col = seg >> 3, rs = (seg & 7) * 8;
+                if (row0 + rs < rows)      // rows is a multiple of 8: a segment is all valid or all past the end
+                    *reinterpret_cast<uint4*>(VqT + (int64_t)(j * 32 + col) * rows + row0 + rs) =
+                        *reinterpret_cast<const uint4*>(&tt[col][rs]);
+            }
+            __syncthreads();
         }
-        __syncthreads();
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xFFFFFFFFu, sq, o);

@@ -68,14 +68,32 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// kind::f16, D = f32, A = B = bf16, both K-major, M = 256 (pair), N = 256
-__host__ __device__ constexpr uint32_t idesc_m256n256_bf16() {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+// kind::f16, D = f32, A = B = bf16, M = 256 (pair), N = 256; bit 15 / 16: A / B stored MN-major
+__host__ __device__ constexpr uint32_t idesc_m256n256_bf16(bool a_mn = false, bool b_mn = false) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((256u >> 3) << 17) | ((256u >> 4) << 24);
+}
+// MN-major operand tile, 128-byte swizzle: a TMA box of 64 MN-elements (128 bytes, the contiguous
+// direction in memory) x 64 K-rows lands as 64 rows of 128 bytes; 8-row groups are 1024 bytes apart
+// (stride byte offset) and the next 64 MN-elements are the next box, 8 KB further (leading byte
+// offset).  One K = 16 instruction covers 16 rows = 2048 bytes.
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)(8192 >> 4) << 16;       // leading byte offset: next 64 elements along M / N
+    d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset: next 8 rows along K
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+    return d;
 }
 
-// p.tiles_m counts 256-row tiles here.  gridDim.x = 2 x (number of pairs); cluster size 2.
+// C[M][N] = sum_k A(m, k) B(n, k).  A_MN = false: A is stored [M][K] (K contiguous), tmap_a boxes are
+// 64 K-elements x 128 rows; A_MN = true: A is stored [K][M] (M contiguous), tmap_a boxes are 64
+// M-elements x 64 K-rows and two of them make this CTA's 128 rows.  Likewise B_MN for B ([N][K] or
+// [K][N]).  p.tiles_m counts 256-row tiles.  gridDim.x = 2 x (number of pairs); cluster size 2.
+template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_nt_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+gemm_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const GemmProblem p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -135,8 +153,19 @@ gemm_nt_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint32_t dst = base + s * kGemm2StageBytes;
                     const uint32_t leader_full = mapa_shared(bar_full(s), 0);
                     if (rank == 0) mbar_expect_tx(bar_full(s), 2 * kGemm2StageBytes);   // both CTAs' bytes
-                    tma_load_2d_pair(dst, &tmap_a, kb * kGemmBK, tm * kGemm2BM + (int)rank * 128, leader_full);
-                    tma_load_2d_pair(dst + kGemm2ABytes, &tmap_b, kb * kGemmBK, tn * kGemmBN + (int)rank * 128, leader_full);
+                    const int m0 = tm * kGemm2BM + (int)rank * 128, n0 = tn * kGemmBN + (int)rank * 128;
+                    if (A_MN) {
+                        tma_load_2d_pair(dst, &tmap_a, m0, kb * kGemmBK, leader_full);
+                        tma_load_2d_pair(dst + 8192, &tmap_a, m0 + 64, kb * kGemmBK, leader_full);
+                    } else {
+                        tma_load_2d_pair(dst, &tmap_a, kb * kGemmBK, m0, leader_full);
+                    }
+                    if (B_MN) {
+                        tma_load_2d_pair(dst + kGemm2ABytes, &tmap_b, n0, kb * kGemmBK, leader_full);
+                        tma_load_2d_pair(dst + kGemm2ABytes + 8192, &tmap_b, n0 + 64, kb * kGemmBK, leader_full);
+                    } else {
+                        tma_load_2d_pair(dst + kGemm2ABytes, &tmap_b, kb * kGemmBK, n0, leader_full);
+                    }
                     issued = it + 1;
                 }
             }
@@ -144,8 +173,9 @@ gemm_nt_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader CTA only) ----------------
         if (lane == 0 && rank == 0) {
-            const uint64_t a_desc0 = smem_desc_sw128(base);
-            const uint64_t b_desc0 = smem_desc_sw128(base + kGemm2ABytes);
+            const uint64_t a_desc0 = A_MN ? smem_desc_sw128_mn(base) : smem_desc_sw128(base);
+            const uint64_t b_desc0 = B_MN ? smem_desc_sw128_mn(base + kGemm2ABytes) : smem_desc_sw128(base + kGemm2ABytes);
+            constexpr uint64_t a_step = A_MN ? (2048 >> 4) : 2, b_step = B_MN ? (2048 >> 4) : 2;   // per K = 16
             int it = 0;
             bool ok = true;
             for (int i = 0; ok && i < my_tiles; ++i) {
@@ -167,8 +197,8 @@ gemm_nt_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     const uint64_t off = (uint64_t)((s * kGemm2StageBytes) >> 4);
 #pragma unroll
                     for (int k = 0; k < kGemmBK / 16; ++k)
-                        tc_mma_bf16_pair(d_addr, a_desc0 + off + (uint64_t)(2 * k), b_desc0 + off + (uint64_t)(2 * k),
-                                         idesc_m256n256_bf16(), (uint32_t)((kb | k) != 0));
+                        tc_mma_bf16_pair(d_addr, a_desc0 + off + a_step * k, b_desc0 + off + b_step * k,
+                                         idesc_m256n256_bf16(A_MN, B_MN), (uint32_t)((kb | k) != 0));
                     tc_commit_pair(bar_empty(s));
                 }
                 if (ok) tc_commit_pair(bar_tfull(acc));

@@ -31,6 +31,8 @@ struct kroquant_calib {
     // "_b" = 256-row boxes (B operand of the one-CTA kernel)
     CUtensorMap tm_A_a, tm_W_b, tm_Yq_a, tm_Zq_b, tm_dO_a, tm_ZqT_b, tm_dOT_a, tm_YqT_b;
     CUtensorMap tm_W_a, tm_Zq_a, tm_ZqT_a, tm_YqT_a;
+    // paired kernel, operands read in their stored orientation: boxes of 64 contiguous elements x 64 rows
+    CUtensorMap tm_Zq_mn, tm_dO_mn, tm_Yq_mn;
 };
 
 kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
@@ -57,22 +59,42 @@ bool make_operand_map(CUtensorMap* tm, const void* ptr, int64_t rows, int64_t K,
 std::atomic<int> g_gemm_pair{1};       // 1: two-CTA 256 x 256 tiles (default); 0: one-CTA 128 x 256 tiles
 
 // tb = B operand map with 256-row boxes (one-CTA kernel), tb2 = the same tensor with 128-row boxes
+// [K][MN] bf16 row-major (MN contiguous) as an MN-major operand of the paired kernel
+bool make_operand_map_mn(CUtensorMap* tm, const void* ptr, int64_t k_rows, int64_t mn) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)mn, (cuuint64_t)k_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)mn * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kq::kGemmBK};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// mode 0: A [M][K], B [N][K] (both K contiguous; ta / tb / tb2 as described below);
+// paired kernel only: mode 1: B given as [K][N] (tb2 = its MN-major map); mode 2: A as [K][M] and B as [K][N]
+// (ta, tb2 = MN-major maps)
 kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& tb2, int M, int N, int K,
                         const float* aux, int64_t ld_aux, const float* coef_ptr, float coef_mul, float out_scale,
                         float* out_f32, __nv_bfloat16* out_bf16, int64_t ld_out, double* sumsq, cudaStream_t st,
-                        __nv_bfloat16* out_bf16_t = nullptr, int64_t ld_out_t = 0) {
+                        __nv_bfloat16* out_bf16_t = nullptr, int64_t ld_out_t = 0, int mode = 0) {
     static std::atomic<int> attr_done{0};
     if (!attr_done.load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kq::gemm_nt_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kGemmDynBytes) !=
                 cudaSuccess ||
-            cudaFuncSetAttribute(kq::gemm_nt_umma_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kGemm2DynBytes) !=
-                cudaSuccess) {
+            cudaFuncSetAttribute(kq::gemm_umma_pair<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kq::kGemm2DynBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(kq::gemm_umma_pair<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kq::kGemm2DynBytes) != cudaSuccess ||
+            cudaFuncSetAttribute(kq::gemm_umma_pair<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kq::kGemm2DynBytes) != cudaSuccess) {
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
         }
         attr_done.store(1, std::memory_order_release);
     }
-    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0;
+    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0 || mode != 0;
     const int bm = pair ? kq::kGemm2BM : kq::kGemmBM;
     kq::GemmProblem p;
     p.M = M; p.N = N; p.K = K;
@@ -99,7 +121,10 @@ kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, kq::gemm_nt_umma_pair, ta, tb2, p) != cudaSuccess) {
+        const cudaError_t lrc = mode == 0   ? cudaLaunchKernelEx(&cfg, kq::gemm_umma_pair<false, false>, ta, tb2, p)
+                                : mode == 1 ? cudaLaunchKernelEx(&cfg, kq::gemm_umma_pair<false, true>, ta, tb2, p)
+                                            : cudaLaunchKernelEx(&cfg, kq::gemm_umma_pair<true, true>, ta, tb2, p);
+        if (lrc != cudaSuccess) {
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
         }
@@ -161,15 +186,19 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
         if (gx < 1) gx = 1;
         return dim3((unsigned)gx, (unsigned)nb);
     };
-    kq::calib_fakequant<<<fq_grid(M), 128, 0, st>>>(c->A, c->Kd, c->n_sets, M, d, c->Yq, c->YqT, c->ResY, c->sums + 1);
+    // the paired GEMM reads Yq, Zq and dO in either orientation; only the one-CTA GEMM needs transposed copies
+    const bool pair_mode = g_gemm_pair.load(std::memory_order_relaxed) != 0;
+    kq::calib_fakequant<<<fq_grid(M), 128, 0, st>>>(c->A, c->Kd, c->n_sets, M, d, c->Yq, pair_mode ? nullptr : c->YqT,
+                                                   c->ResY, c->sums + 1);
     if (!launched()) return KQ_ERR_CUDA;
-    kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, c->ZqT, c->ResZ, c->sums + 2);
+    kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, pair_mode ? nullptr : c->ZqT,
+                                                   c->ResZ, c->sums + 2);
     if (!launched()) return KQ_ERR_CUDA;
     // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o)) and its transpose.  Yq and Zq are MXFP4 values,
     // so with the paired kernels the product runs on the FP4 tensor-core path: re-encoding Yq, Zq with the
     // bare MXFP4 encoder returns their codes and scales exactly (the encoder is idempotent on its own output)
     kq_status_t rc;
-    if (g_gemm_pair.load(std::memory_order_relaxed) != 0) {
+    if (pair_mode) {
         rc = run_stream<kq::MODE_PLAIN, false>(c->Yq, false, M, d, nullptr, nullptr, c->qY, c->sY, true, nullptr, st);
         if (rc != KQ_OK) return rc;
         rc = run_stream<kq::MODE_PLAIN, false>(c->Zq, false, o, d, nullptr, nullptr, c->qZ, c->sZ, true, nullptr, st);
@@ -179,7 +208,7 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
         e.aux = c->R; e.ld_aux = o; e.coef_ptr = nullptr; e.coef_mul = -1.0f;
         e.out_scale = (float)(2.0 / ((double)M * o));
         e.out_f32 = nullptr; e.out_bf16 = backward ? c->dO : nullptr; e.ld_out = o;
-        e.out_bf16_t = backward ? c->dOT : nullptr; e.ld_out_t = M;
+        e.out_bf16_t = nullptr; e.ld_out_t = 0;
         e.sumsq = c->sums;
         rc = launch_gemm_fp4(c->qY, c->sY, c->qZ, c->sZ, M, o, d, nullptr, nullptr, KQ_OUT_BF16, &e, st);
     } else {
@@ -193,12 +222,21 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
         return KQ_ERR_CUDA;
     if (!backward) return KQ_OK;
     // dY = dO Zq + lambda_A 2 (Y - Yq) / (M d);  dZ = dO^T Yq + lambda_W 2 (Z - Zq) / (o d)
-    rc = launch_gemm(c->tm_dO_a, c->tm_ZqT_b, c->tm_ZqT_a, (int)M, d, o, c->ResY, d, c->lam, (float)(2.0 / ((double)M * d)), 1.0f,
-                     c->dY, nullptr, d, nullptr, st);
-    if (rc != KQ_OK) return rc;
-    rc = launch_gemm(c->tm_dOT_a, c->tm_YqT_b, c->tm_YqT_a, o, d, (int)M, c->ResZ, d, c->lam + 1, (float)(2.0 / ((double)o * d)), 1.0f,
-                     c->dZ, nullptr, d, nullptr, st);
-    if (rc != KQ_OK) return rc;
+    if (pair_mode) {
+        rc = launch_gemm(c->tm_dO_a, c->tm_Zq_mn, c->tm_Zq_mn, (int)M, d, o, c->ResY, d, c->lam,
+                         (float)(2.0 / ((double)M * d)), 1.0f, c->dY, nullptr, d, nullptr, st, nullptr, 0, 1);
+        if (rc != KQ_OK) return rc;
+        rc = launch_gemm(c->tm_dO_mn, c->tm_Yq_mn, c->tm_Yq_mn, o, d, (int)M, c->ResZ, d, c->lam + 1,
+                         (float)(2.0 / ((double)o * d)), 1.0f, c->dZ, nullptr, d, nullptr, st, nullptr, 0, 2);
+        if (rc != KQ_OK) return rc;
+    } else {
+        rc = launch_gemm(c->tm_dO_a, c->tm_ZqT_b, c->tm_ZqT_a, (int)M, d, o, c->ResY, d, c->lam,
+                         (float)(2.0 / ((double)M * d)), 1.0f, c->dY, nullptr, d, nullptr, st);
+        if (rc != KQ_OK) return rc;
+        rc = launch_gemm(c->tm_dOT_a, c->tm_YqT_b, c->tm_YqT_a, o, d, (int)M, c->ResZ, d, c->lam + 1,
+                         (float)(2.0 / ((double)o * d)), 1.0f, c->dZ, nullptr, d, nullptr, st);
+        if (rc != KQ_OK) return rc;
+    }
     rc = run_block_grad(c->A, c->dY, M, d, c->n_sets, c->chunksK, c->rpcK, c->partK, c->dK, st);
     if (rc != KQ_OK) return rc;
     rc = run_block_grad(c->W, c->dZ, o, d, c->n_sets, c->chunksP, c->rpcP, c->partP, c->dP, st);
@@ -446,7 +484,9 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
               make_operand_map(&c->tm_dO_a, c->dO, M, o, kq::kGemmBM) && make_operand_map(&c->tm_ZqT_b, c->ZqT, d, o, kq::kGemmBN) &&
               make_operand_map(&c->tm_dOT_a, c->dOT, o, M, kq::kGemmBM) && make_operand_map(&c->tm_YqT_b, c->YqT, d, M, kq::kGemmBN) &&
               make_operand_map(&c->tm_W_a, c->W, o, d, 128) && make_operand_map(&c->tm_Zq_a, c->Zq, o, d, 128) &&
-              make_operand_map(&c->tm_ZqT_a, c->ZqT, d, o, 128) && make_operand_map(&c->tm_YqT_a, c->YqT, d, M, 128);
+              make_operand_map(&c->tm_ZqT_a, c->ZqT, d, o, 128) && make_operand_map(&c->tm_YqT_a, c->YqT, d, M, 128) &&
+              make_operand_map_mn(&c->tm_Zq_mn, c->Zq, o, d) && make_operand_map_mn(&c->tm_dO_mn, c->dO, M, o) &&
+              make_operand_map_mn(&c->tm_Yq_mn, c->Yq, M, d);
     kq_status_t rc = ok ? KQ_OK : KQ_ERR_CUDA;
     std::vector<float> th;
     hadamard_theta(th, n_sets);
