@@ -562,6 +562,8 @@ def run_calib(args):
     dev = torch.device("cuda:0")
     A_t = torch.from_numpy(A_bits.view(np.int16)).to(dev).view(torch.bfloat16)
     W_t = torch.from_numpy(W_bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    side = torch.cuda.Stream()          # a capturable stream: the library replays one captured step per Adam step
+    torch.cuda.set_stream(side)
     stream = torch.cuda.current_stream()
     launches0 = B.kroquant_launch_count()
     cal = B.Calibrator(A_t, W_t, n_sets)

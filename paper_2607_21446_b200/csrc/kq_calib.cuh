@@ -331,6 +331,9 @@ struct CalibStepArgs {
     const float* dP;           // [n_sets][32][32]
     float* theta; float* adam_m; float* adam_v; float* grad_out;
     float lr; int t; int do_update;
+    // when ctl != null the step count and the learning rate come from device memory (ctl[0] = Adam steps
+    // taken so far, *lr_ptr), so that the same launch can be replayed from a CUDA graph
+    const int* ctl; const float* lr_ptr;
 };
 
 __global__ void __launch_bounds__(1024)
@@ -398,11 +401,24 @@ calib_param_step(const CalibStepArgs a) {
             const double v = b2 * (double)a.adam_v[idx] + (1.0 - b2) * g * g;
             a.adam_m[idx] = (float)m;
             a.adam_v[idx] = (float)v;
-            const double mhat = m / (1.0 - pow(b1, (double)a.t));
-            const double vhat = v / (1.0 - pow(b2, (double)a.t));
-            const double th = (which == 0 ? aa : which == 1 ? bb : cc) - (double)a.lr * mhat / (sqrt(vhat) + eps);
+            const double t = a.ctl ? (double)(a.ctl[0] + 1) : (double)a.t;
+            const double lr = a.lr_ptr ? (double)*a.lr_ptr : (double)a.lr;
+            const double mhat = m / (1.0 - pow(b1, t));
+            const double vhat = v / (1.0 - pow(b2, t));
+            const double th = (which == 0 ? aa : which == 1 ? bb : cc) - lr * mhat / (sqrt(vhat) + eps);
             a.theta[idx] = (float)th;
         }
+    }
+}
+
+// End of a step that is replayed from a graph: file the step's three sums of squares in the next
+// history row and count the step (ctl[0] = Adam steps taken, ctl[1] = next history row).
+__global__ void calib_advance(const double* __restrict__ sums, double* __restrict__ hist, int* __restrict__ ctl, int hist_cap) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        const int row = ctl[1];
+        if (row < hist_cap) { hist[3 * row] = sums[0]; hist[3 * row + 1] = sums[1]; hist[3 * row + 2] = sums[2]; }
+        ctl[1] = row + 1;
+        ctl[0] = ctl[0] + 1;
     }
 }
 

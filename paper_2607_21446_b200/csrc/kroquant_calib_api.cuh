@@ -26,7 +26,11 @@ struct kroquant_calib {
     int64_t rpcK = 0, rpcP = 0;
     double* sums = nullptr;            // [3] sums of squares of the evaluation in flight
     double* hist = nullptr;            // [kHistCap][3]
-    int t = 0;                         // Adam steps taken
+    int t = 0;                         // Adam steps taken (host mirror of ctl[0])
+    int* ctl = nullptr;                // device: {Adam steps taken, next history row}
+    float* lr_dev = nullptr;           // device: learning rate of the run in flight
+    cudaGraphExec_t step_graph[2] = {nullptr, nullptr};   // one captured Adam step per GEMM variant
+    int launches_per_step = 0;         // kernels in one captured step (for the launch counter)
     // GEMM operands: "_a" = 128-row boxes (A operand, and both operands of the paired kernel),
     // "_b" = 256-row boxes (B operand of the one-CTA kernel)
     CUtensorMap tm_A_a, tm_W_b, tm_Yq_a, tm_Zq_b, tm_dO_a, tm_ZqT_b, tm_dOT_a, tm_YqT_b;
@@ -171,7 +175,10 @@ kq_status_t run_block_grad(const uint16_t* X, const float* G, int64_t rows, int 
 
 // One evaluation at the current parameters.  backward: also the gradient; update: Adam step.
 // hist_row >= 0: copy the three sums of squares to that history row.
-kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr, int hist_row, cudaStream_t st) {
+// device_ctl (with update): step count, learning rate and history row come from device memory and the
+// step ends with calib_advance - the launch sequence is then identical for every step (graph replay).
+kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr, int hist_row, cudaStream_t st,
+                       bool device_ctl = false) {
     const int64_t M = c->M;
     const int o = c->o, d = c->d, nb = c->nb;
     const int sms = sm_count();
@@ -245,9 +252,15 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
     a.dK = c->dK; a.dP = c->dP;
     a.theta = c->theta; a.adam_m = c->adam_m; a.adam_v = c->adam_v; a.grad_out = c->grad;
     a.lr = lr; a.t = c->t + 1; a.do_update = update ? 1 : 0;
+    a.ctl = device_ctl ? c->ctl : nullptr;
+    a.lr_ptr = device_ctl ? c->lr_dev : nullptr;
     kq::calib_param_step<<<c->n_sets, 1024, 0, st>>>(a);
     if (!launched()) return KQ_ERR_CUDA;
-    if (update) c->t += 1;
+    if (device_ctl) {
+        kq::calib_advance<<<1, 32, 0, st>>>(c->sums, c->hist, c->ctl, kHistCap);
+        if (!launched()) return KQ_ERR_CUDA;
+    }
+    if (update && !device_ctl) c->t += 1;      // with device_ctl the caller keeps the host mirror
     return KQ_OK;
 }
 
@@ -454,6 +467,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     auto take = [&](size_t bytes) { const size_t at = off; off += (bytes + 255) & ~(size_t)255; return at; };
     const size_t Md = (size_t)M * d, od = (size_t)o * d, Mo = (size_t)M * o, np = (size_t)n_sets * 15;
     const size_t o_theta = take(np * 4), o_m = take(np * 4), o_v = take(np * 4), o_grad = take(np * 4), o_lam = take(8);
+    const size_t o_ctl = take(8), o_lr = take(4);
     const size_t o_K = take((size_t)n_sets * 4096), o_P = take((size_t)n_sets * 4096);
     const size_t o_Yq = take(Md * 2), o_YqT = take(Md * 2), o_Zq = take(od * 2), o_ZqT = take(od * 2);
     const size_t o_dO = take(Mo * 2), o_dOT = take(Mo * 2);
@@ -468,6 +482,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     uint8_t* b = c->pool;
     c->theta = (float*)(b + o_theta); c->adam_m = (float*)(b + o_m); c->adam_v = (float*)(b + o_v);
     c->grad = (float*)(b + o_grad); c->lam = (float*)(b + o_lam);
+    c->ctl = (int*)(b + o_ctl); c->lr_dev = (float*)(b + o_lr);
     c->Kd = (float*)(b + o_K); c->Pd = (float*)(b + o_P);
     c->Yq = (__nv_bfloat16*)(b + o_Yq); c->YqT = (__nv_bfloat16*)(b + o_YqT);
     c->Zq = (__nv_bfloat16*)(b + o_Zq); c->ZqT = (__nv_bfloat16*)(b + o_ZqT);
@@ -513,6 +528,8 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
 
 void kroquant_calib_destroy(kroquant_calib_t* c) {
     if (!c) return;
+    for (int i = 0; i < 2; ++i)
+        if (c->step_graph[i]) (void)cudaGraphExecDestroy(c->step_graph[i]);
     if (c->pool) (void)cudaFree(c->pool);
     delete c;
 }
@@ -527,7 +544,8 @@ kq_status_t kroquant_calib_set_theta(kroquant_calib_t* c, const float* theta_hos
             !std::isfinite(theta_host[i + 2]))
             return KQ_ERR_FACTORS;                       // a = 0 has no LU form
     if (cudaMemcpy(c->theta, theta_host, np * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemset(c->adam_m, 0, np * 4) != cudaSuccess || cudaMemset(c->adam_v, 0, np * 4) != cudaSuccess)
+        cudaMemset(c->adam_m, 0, np * 4) != cudaSuccess || cudaMemset(c->adam_v, 0, np * 4) != cudaSuccess ||
+        cudaMemset(c->ctl, 0, 8) != cudaSuccess)
         return KQ_ERR_CUDA;
     c->t = 0;
     return KQ_OK;
@@ -611,10 +629,42 @@ kq_status_t kroquant_calib_run(kroquant_calib_t* c, int steps, float lr, double*
     if (rc != KQ_OK) return rc;
     if (steps < 1 || steps > kHistCap - 1 || !(lr > 0.f)) return KQ_ERR_SHAPE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    for (int i = 0; i < steps; ++i) {
-        rc = calib_eval(c, true, true, lr, i, st);
-        if (rc != KQ_OK) return rc;
+    // learning rate and history row for this run live on the device; the step count is already there
+    if (cudaMemcpyAsync(c->lr_dev, &lr, 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||      // pageable source: staged
+        cudaMemsetAsync(c->ctl + 1, 0, 4, st) != cudaSuccess)
+        return KQ_ERR_CUDA;
+    // One Adam step is the same sequence of launches every time, so it is captured once per GEMM variant
+    // and replayed.  A stream that cannot be captured (the legacy default stream, or one that is being
+    // captured by the caller) gets the launches directly.
+    const int variant = g_gemm_pair.load(std::memory_order_relaxed) != 0 ? 1 : 0;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    const bool can_capture = st != nullptr && st != cudaStreamLegacy && cudaStreamIsCapturing(st, &cap) == cudaSuccess &&
+                             cap == cudaStreamCaptureStatusNone;
+    if (can_capture && !c->step_graph[variant]) {
+        cudaGraph_t g = nullptr;
+        if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+            const int64_t before = g_launches.load(std::memory_order_relaxed);
+            const kq_status_t crc = calib_eval(c, true, true, lr, -1, st, true);
+            c->launches_per_step = (int)(g_launches.load(std::memory_order_relaxed) - before);
+            g_launches.store(before, std::memory_order_relaxed);              // captured, not launched
+            const cudaError_t erc = cudaStreamEndCapture(st, &g);
+            if (crc == KQ_OK && erc == cudaSuccess && g &&
+                cudaGraphInstantiate(&c->step_graph[variant], g, 0) != cudaSuccess)
+                c->step_graph[variant] = nullptr;
+            if (g) (void)cudaGraphDestroy(g);
+            (void)cudaGetLastError();
+        }
     }
+    for (int i = 0; i < steps; ++i) {
+        if (can_capture && c->step_graph[variant]) {
+            if (cudaGraphLaunch(c->step_graph[variant], st) != cudaSuccess) { (void)cudaGetLastError(); return KQ_ERR_CUDA; }
+            g_launches.fetch_add(c->launches_per_step, std::memory_order_relaxed);
+        } else {
+            rc = calib_eval(c, true, true, lr, -1, st, true);
+            if (rc != KQ_OK) return rc;
+        }
+    }
+    c->t += steps;
     if (!history_host_out) return KQ_OK;
     rc = calib_eval(c, false, false, 0.f, steps, st);
     if (rc != KQ_OK) return rc;

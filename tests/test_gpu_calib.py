@@ -147,6 +147,31 @@ def test_calibration_run_lowers_the_objective_like_the_oracle(shared):
     cal.destroy()
 
 
+@pytest.mark.parametrize("shared", [True, False])
+def test_run_on_a_side_stream_replays_a_captured_step(shared):
+    """On a capturable stream one Adam step is captured once and replayed; the result must be the same as
+    on the default stream, where every step is launched directly."""
+    M, o, d, seed = 512, 96, 256, 52
+    A, W, A_t, W_t = _case(M, o, d, seed)
+    n_sets = 1 if shared else d // 32
+    ref = kb.Calibrator(A_t, W_t, n_sets)
+    h_ref = ref.run(7, lr=1e-2)
+    h_ref2 = ref.run(3, lr=5e-3)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        cal = kb.Calibrator(A_t, W_t, n_sets, stream=side)
+        h = cal.run(7, lr=1e-2, stream=side)
+        h2 = cal.run(3, lr=5e-3, stream=side)          # second run: replay of the same graph, new learning rate
+        side.synchronize()
+    # same kernels in the same order; only atomics on the loss sums may reorder
+    assert np.allclose(h, h_ref, rtol=1e-9) and np.allclose(h2, h_ref2, rtol=1e-9)
+    assert np.allclose(cal.theta, ref.theta, rtol=0, atol=1e-6)
+    _no_device_error()
+    cal.destroy()
+    ref.destroy()
+
+
 def test_calibrated_factors_feed_the_quantizer():
     """get_factors -> factors_create -> quantize equals the oracle quantizer with the same G."""
     from oracle import c_oracle
