@@ -222,7 +222,7 @@ kq_status_t kroquant_linear_w4a4(const void *X, kq_xdtype_t x_dtype, int64_t tok
  * must stay valid and unchanged for the life of the object.  M is the number of calibration
  * rows (all samples stacked), a multiple of 8; o and d are multiples of 32; n_sets is 1 (one
  * factor set for the layer) or d/32 (one per block).  create allocates all work space
- * (about 12 M d + 8 M o bytes), forms A W^T, evaluates the three terms at the initialisation and
+ * (about 13 M d + 8 M o bytes), forms A W^T, evaluates the three terms at the initialisation and
  * sets lambda_A = L_out/L_A, lambda_W = L_out/L_W there; it synchronizes `stream`.  The object is
  * tied to the device that was current at creation.  All three contractions of a step run on the
  * tensor cores in bf16 with fp32 accumulation (exact products for the forward one); the output
@@ -263,7 +263,11 @@ kq_status_t kroquant_calib_loss_grad(kroquant_calib_t *c, double *losses_host_ou
 /* `steps` Adam steps (1 <= steps <= 4096) with learning rate lr.  history_host_out, if not NULL,
  * receives [steps + 1][3] doubles: the three terms before each step and, in the last row, at the
  * final parameters (one more forward pass).  Asynchronous on `stream` if history_host_out is NULL,
- * otherwise synchronizes it. */
+ * otherwise synchronizes it.  Step count, learning rate and history row are kept in device memory, so
+ * every step is the same sequence of launches: on a stream that can be captured (not the legacy
+ * default stream, not one the caller is capturing) the first call records that sequence once as a
+ * CUDA graph, owned by the object, and each step replays it; elsewhere the launches are issued
+ * directly. */
 kq_status_t kroquant_calib_run(kroquant_calib_t *c, int steps, float lr, double *history_host_out,
                                void *stream);
 
