@@ -18,8 +18,23 @@ namespace kq {
 // One CTA of 1024 threads per factor set; thread (r, c).  G_k = [[a, b], [a c, b c - 1/a]]
 // (Section 3.2, L_k U_k multiplied out); H_k = G_k^-T = [[1/a - b c, a c], [b, -a]] (det G_k = -1).
 // K[r][c] = prod_k G_k[bit(r)][bit(c)] with G_1 on the most significant index bit.
+// imgK / imgP (optional): the same blocks as operand images of the tensor-core quantizer (kq_umma.cuh):
+// K^T split into three bf16 terms, [term][n = column of K][k = row of K] with 64-byte rows in the
+// 64-byte-swizzle layout, 6 KB per set.
+__device__ __forceinline__ void store_image_entry(uint8_t* img, int r, int c, float v) {
+    const __nv_bfloat16 h0 = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(h0);
+    const __nv_bfloat16 h1 = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 h2 = __float2bfloat16_rn(r1 - __bfloat162float(h1));
+    uint32_t off = (uint32_t)(c * 64 + 2 * r);
+    off ^= ((off >> 7) & 3u) << 4;
+    *reinterpret_cast<__nv_bfloat16*>(img + off) = h0;
+    *reinterpret_cast<__nv_bfloat16*>(img + 2048 + off) = h1;
+    *reinterpret_cast<__nv_bfloat16*>(img + 4096 + off) = h2;
+}
 __global__ void __launch_bounds__(1024)
-calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, float* __restrict__ Pout) {
+calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, float* __restrict__ Pout,
+                   uint8_t* __restrict__ imgK, uint8_t* __restrict__ imgP) {
     const int s = blockIdx.x;
     const int r = threadIdx.x >> 5, c = threadIdx.x & 31;
     double k = 1.0, p = 1.0;
@@ -34,6 +49,8 @@ calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, fl
     }
     Kout[s * 1024 + threadIdx.x] = (float)k;
     Pout[s * 1024 + threadIdx.x] = (float)p;
+    if (imgK) store_image_entry(imgK + (size_t)s * 6144, r, c, (float)k);
+    if (imgP) store_image_entry(imgP + (size_t)s * 6144, r, c, (float)p);
 }
 
 // ---- transform + fake quantisation ---------------------------------------------------------
@@ -44,12 +61,6 @@ calib_build_blocks(const float* __restrict__ theta, float* __restrict__ Kout, fl
 // quantizer kernels followed by its decoder; Vq is exact in bf16.  Outputs: Vq [rows][d],
 // optionally its transpose VqT [d][rows] (staged through shared memory, 16-byte segments; only the
 // one-CTA GEMM needs it, the paired GEMM reads Vq in either orientation), R = V - Vq, and the sum of R^2.
-// two E2M1 codes (one byte, even element in the low nibble) -> two floats, by the hardware convert
-__device__ __forceinline__ float2 e2m1x2_to_float2(uint32_t byte) {
-    uint32_t h2;
-    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(byte));
-    return __half22float2(*reinterpret_cast<const __half2*>(&h2));
-}
 __device__ __forceinline__ void split3_bf16(float x, uint32_t (&t)[3]) {
     const __nv_bfloat16 h0 = __float2bfloat16_rn(x);
     const float r1 = x - __bfloat162float(h0);

@@ -72,6 +72,12 @@ __device__ __forceinline__ uint32_t e2m1x8(float v0, float v1, float v2, float v
     return out;
 }
 
+// two E2M1 codes (one byte, even element in the low nibble) -> two floats, by the hardware convert
+__device__ __forceinline__ float2 e2m1x2_to_float2(uint32_t byte) {
+    uint32_t h2;
+    asm("{\n\t.reg .b8 b;\n\tcvt.u8.u32 b, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, b;\n\t}" : "=r"(h2) : "r"(byte));
+    return __half22float2(*reinterpret_cast<const __half2*>(&h2));
+}
 __device__ __forceinline__ float absmax8(const float (&y)[8]) {
     float m = fmaxf(fabsf(y[0]), fabsf(y[1]));
     m = fmaxf(m, fmaxf(fabsf(y[2]), fabsf(y[3])));

@@ -262,6 +262,48 @@ __device__ __forceinline__ void encode_block_regs(uint32_t (&acc)[32], int e, ui
     codes = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// Calibration outputs of one block (y = acc, bf16 image: no normalisation exponent): q = decode(codes) 2^(S-127)
+// as 32 bf16 (64 bytes), r = y - q as 32 floats (128 bytes), and the block's sum of r^2.  Full-sector stores
+// when the buffers are 32-byte aligned.
+__device__ __forceinline__ float store_block_calib(const uint32_t (&acc)[32], const uint4& codes, uint32_t S,
+                                                   uint4* vq_dst, float* res_dst) {
+    const float sc = scale_from_e8m0(S);
+    const uint32_t cw[4] = {codes.x, codes.y, codes.z, codes.w};
+    uint32_t wq[16];
+    uint32_t wr[32];
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float2 dq = e2m1x2_to_float2((cw[i >> 2] >> (8 * (i & 3))) & 0xFFu);
+        const float q0 = dq.x * sc, q1 = dq.y * sc;
+        const float r0 = __uint_as_float(acc[2 * i]) - q0, r1 = __uint_as_float(acc[2 * i + 1]) - q1;
+        sq = fmaf(r0, r0, fmaf(r1, r1, sq));
+        const __nv_bfloat162 h = __floats2bfloat162_rn(q0, q1);
+        wq[i] = *reinterpret_cast<const uint32_t*>(&h);
+        wr[2 * i] = __float_as_uint(r0);
+        wr[2 * i + 1] = __float_as_uint(r1);
+    }
+    if (((reinterpret_cast<uintptr_t>(vq_dst) | reinterpret_cast<uintptr_t>(res_dst)) & 31u) == 0) {
+#pragma unroll
+        for (int v = 0; v < 2; ++v)
+            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                         ::"l"(vq_dst + 2 * v), "r"(wq[8 * v]), "r"(wq[8 * v + 1]), "r"(wq[8 * v + 2]), "r"(wq[8 * v + 3]),
+                           "r"(wq[8 * v + 4]), "r"(wq[8 * v + 5]), "r"(wq[8 * v + 6]), "r"(wq[8 * v + 7]) : "memory");
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                         ::"l"(res_dst + 8 * v), "r"(wr[8 * v]), "r"(wr[8 * v + 1]), "r"(wr[8 * v + 2]), "r"(wr[8 * v + 3]),
+                           "r"(wr[8 * v + 4]), "r"(wr[8 * v + 5]), "r"(wr[8 * v + 6]), "r"(wr[8 * v + 7]) : "memory");
+    } else {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) vq_dst[v] = make_uint4(wq[4 * v], wq[4 * v + 1], wq[4 * v + 2], wq[4 * v + 3]);
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+            reinterpret_cast<uint4*>(res_dst)[v] = make_uint4(wr[4 * v], wr[4 * v + 1], wr[4 * v + 2], wr[4 * v + 3]);
+    }
+    return sq;
+}
+
 // Work decomposition.  CTA b takes work units b, b + gridDim.x, ...
 //   PB = false (one shared factor set): X is the flat matrix [n_rows = tokens*d/32][32];
 //     unit = tile w = flat rows 128w .. 128w+127; outputs of flat row r: 16 B of codes at
@@ -296,14 +338,23 @@ struct UmmaProblem {
 // Grid: any size <= number of tiles; CTA b takes tiles b, b + gridDim.x, ...
 // XF16: X and the factor image are fp16 (else bf16); e_norm: per-set normalisation exponents of
 // the image (all zero for bf16 images).
-// DUAL: also write the 16-bit transformed activations (at_out); a separate instantiation, because the
-// extra conversion code costs registers that would take a resident CTA away from the default kernel.
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, bool DUAL = false>
+// EXTRA = 1 (second output): also write the 16-bit transformed activations (at_out).
+// EXTRA = 2 (calibration, Section 3.3): besides codes and scales write the fake-quantised block Q(y) in
+//   bf16 (at_out, 64 bytes per block), the residual y - Q(y) in fp32 (Y, 128 bytes per block) and add the
+//   sum of squared residuals to *sumsq - the calibration loop's forward pass is this production kernel
+//   followed by its own decode, so it sees exactly the rounding that inference will see.
+// Separate instantiations, because the extra code costs registers that would take a resident CTA away
+// from the default kernel.
+constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone>
 __global__ void __launch_bounds__(128 + 128 * NG, 1)
 quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
               const uint8_t* __restrict__ b_image, const int* __restrict__ e_norm, const UmmaProblem prob,
               uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y,
-              uint4* __restrict__ at_out) {
+              uint4* __restrict__ at_out, double* __restrict__ sumsq) {
+    constexpr bool DUAL = EXTRA == kExtraDual;
+    constexpr bool CALIB = EXTRA == kExtraCalib;
+    static_assert(!CALIB || (!XF16 && !WRITE_Y), "calibration outputs: bf16 images, quantizing path");
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
     // A slot must always be served by the same issuer warp and the same epilogue group:
     // only then does program order inside that warp guarantee that a parity wait never
@@ -447,6 +498,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
         const int e_shared = PB ? 0 : __ldg(e_norm);
+        double sq_sum = 0.0;                       // CALIB: this thread's sum of squared residuals
         for (int n = g; n < my_tiles; n += NG) {
             const int s = n % NS;
             if (!mbar_wait(bar_done(s), (n / NS) & 1, abort_flag)) {
@@ -474,6 +526,10 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     (int64_t)tt * kTileRows + r < prob.n_rows)
                     store_block_16bit<XF16>(acc, e_j, at_out + (((int64_t)tt * kTileRows + r) * prob.blocks_per_row + j) * 4);
                 encode_block_regs(acc, e_j, codes, S);
+                if (CALIB && j < prob.blocks_per_row && (int64_t)tt * kTileRows + r < prob.n_rows) {
+                    const int64_t blk_c = ((int64_t)tt * kTileRows + r) * prob.blocks_per_row + j;
+                    sq_sum += (double)store_block_calib(acc, codes, S, at_out + blk_c * 4, Y + blk_c * 32);
+                }
                 if (c == 0) {
                     // the previous group's TMA store must have finished reading the staging tile
                     if (elected) bulk_wait_group_read<0>();
@@ -563,6 +619,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                         uint32_t S;
                         if (DUAL) store_block_16bit<XF16>(acc, e, at_out + blk * 4);
                         encode_block_regs(acc, e, codes, S);
+                        if (CALIB) sq_sum += (double)store_block_calib(acc, codes, S, at_out + blk * 4, Y + blk * 32);
                         st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
                         int64_t si = blk;
                         if (prob.tiled_scales) {      // flat block index -> (token, block column)
@@ -577,6 +634,11 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         }
         // the staging tile must not be released while a TMA store still reads it
         if (PB && !WRITE_Y && threadIdx.x == 128) bulk_wait_group_read<0>();
+        if (CALIB) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sq_sum += __shfl_xor_sync(0xFFFFFFFFu, sq_sum, o);
+            if (lane == 0 && sq_sum != 0.0) atomicAdd(sumsq, sq_sum);
+        }
     }
 
     // ---------------- teardown ----------------

@@ -181,13 +181,13 @@ kq_status_t finish_factors(kroquant_factors_t* f, const std::vector<double>& K,
     return KQ_OK;
 }
 
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, bool DUAL = false>
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kq::kExtraNone>
 kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
                         const int* enorm, const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, void* at_out, int ctas_per_sm, bool pdl,
-                        cudaStream_t st) {
+                        cudaStream_t st, double* sumsq = nullptr) {
     using L = kq::UmmaSmem<NS, PB>;
-    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, DUAL>;
+    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA>;
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, [&] {
@@ -211,7 +211,8 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, enorm, prob, q, scales, Y, reinterpret_cast<uint4*>(at_out)) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, enorm, prob, q, scales, Y, reinterpret_cast<uint4*>(at_out),
+                           sumsq) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -221,9 +222,10 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
 
 // Tensor-core path.  Shared factor set: flat [tokens*d/32][32] view of X.  Per-block
 // factor sets: 2-D view [tokens][d] with one 32-channel column per tile.
+// calib_sumsq != null: calibration outputs (bf16 X only): at_out receives Q(y) in bf16, Y the residual y - Q(y)
 template <bool WRITE_Y>
 kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f, uint8_t* q,
-                     uint8_t* scales, bool tiled, float* Y, void* at_out, cudaStream_t st) {
+                     uint8_t* scales, bool tiled, float* Y, void* at_out, cudaStream_t st, double* calib_sumsq = nullptr) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
     const bool pb = f->n_sets != 1;
@@ -269,7 +271,16 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
 #define KQ_LAUNCH(NS, NM, NG, PB, XF) \
     launch_umma<NS, NM, NG, PB, XF, WRITE_Y>(tmap, tmap_q, b, en, prob, q, scales, Y, nullptr, cps, pdl, st)
 #define KQ_LAUNCH_DUAL(NS, NM, NG, PB, XF) \
-    launch_umma<NS, NM, NG, PB, XF, false, true>(tmap, tmap_q, b, en, prob, q, scales, nullptr, at_out, cps, pdl, st)
+    launch_umma<NS, NM, NG, PB, XF, false, kq::kExtraDual>(tmap, tmap_q, b, en, prob, q, scales, nullptr, at_out, cps, pdl, st)
+    if (!WRITE_Y && calib_sumsq != nullptr) {
+        if (xf16 || !at_out || !Y) return KQ_ERR_UNSUPPORTED;
+        // the calibration epilogue needs about twice the registers: two CTAs per SM.  No programmatic
+        // dependent launch: the operand image is written by the kernel just before this one
+        return pb ? launch_umma<4, 1, 1, true, false, false, kq::kExtraCalib>(tmap, tmap_q, b, en, prob, q, scales, Y, at_out,
+                                                                          2, false, st, calib_sumsq)
+                  : launch_umma<4, 2, 1, false, false, false, kq::kExtraCalib>(tmap, tmap_q, b, en, prob, q, scales, Y, at_out,
+                                                                           2, false, st, calib_sumsq);
+    }
     if (!WRITE_Y && at_out != nullptr) {
         if (xf16) return pb ? KQ_LAUNCH_DUAL(4, 1, 1, true, true) : KQ_LAUNCH_DUAL(4, 2, 1, false, true);
         return pb ? KQ_LAUNCH_DUAL(4, 1, 1, true, false) : KQ_LAUNCH_DUAL(4, 2, 1, false, false);

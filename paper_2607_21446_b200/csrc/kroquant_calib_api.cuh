@@ -22,6 +22,11 @@ struct kroquant_calib {
     float *dK = nullptr, *dP = nullptr;           // reduced block gradients [n_sets][32][32]
     // Q(AT) and Q(WT^-T) once more as packed codes + tiled scale bytes: operands of the FP4 forward GEMM
     uint8_t *qY = nullptr, *sY = nullptr, *qZ = nullptr, *sZ = nullptr;
+    // K and P = K^-T once more as operand images of the tensor-core quantizer, rebuilt every step, and two
+    // factor handles that point at them (not created through the API: they own nothing)
+    uint8_t *imgK = nullptr, *imgP = nullptr;
+    int* enorm0 = nullptr;
+    kroquant_factors fK, fP;
     int chunksK = 0, chunksP = 0;
     int64_t rpcK = 0, rpcP = 0;
     double* sums = nullptr;            // [3] sums of squares of the evaluation in flight
@@ -183,7 +188,7 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
     const int o = c->o, d = c->d, nb = c->nb;
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
-    kq::calib_build_blocks<<<c->n_sets, 1024, 0, st>>>(c->theta, c->Kd, c->Pd);
+    kq::calib_build_blocks<<<c->n_sets, 1024, 0, st>>>(c->theta, c->Kd, c->Pd, c->imgK, c->imgP);
     if (!launched()) return KQ_ERR_CUDA;
     if (cudaMemsetAsync(c->sums, 0, 3 * sizeof(double), st) != cudaSuccess) return KQ_ERR_CUDA;
     auto fq_grid = [&](int64_t rows) {
@@ -193,23 +198,28 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
         if (gx < 1) gx = 1;
         return dim3((unsigned)gx, (unsigned)nb);
     };
-    // the paired GEMM reads Yq, Zq and dO in either orientation; only the one-CTA GEMM needs transposed copies
+    // Fake quantisation.  Paired mode: the production tensor-core quantizer itself, with the blocks K (resp.
+    // P = K^-T) as its operand images and an epilogue that, besides codes and tiled scale bytes, writes the
+    // decoded block in bf16, the residual in fp32 and the sum of squared residuals - calibration sees exactly
+    // the rounding inference will see, and the codes feed the FP4 forward contraction directly.
+    // One-CTA mode: the mma.sync kernel, which also writes the transposed copies that GEMM needs.
     const bool pair_mode = g_gemm_pair.load(std::memory_order_relaxed) != 0;
-    kq::calib_fakequant<<<fq_grid(M), 128, 0, st>>>(c->A, c->Kd, c->n_sets, M, d, c->Yq, pair_mode ? nullptr : c->YqT,
-                                                   c->ResY, c->sums + 1);
-    if (!launched()) return KQ_ERR_CUDA;
-    kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, pair_mode ? nullptr : c->ZqT,
-                                                   c->ResZ, c->sums + 2);
-    if (!launched()) return KQ_ERR_CUDA;
-    // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o)) and its transpose.  Yq and Zq are MXFP4 values,
-    // so with the paired kernels the product runs on the FP4 tensor-core path: re-encoding Yq, Zq with the
-    // bare MXFP4 encoder returns their codes and scales exactly (the encoder is idempotent on its own output)
     kq_status_t rc;
     if (pair_mode) {
-        rc = run_stream<kq::MODE_PLAIN, false>(c->Yq, false, M, d, nullptr, nullptr, c->qY, c->sY, true, nullptr, st);
+        rc = run_umma<false>(c->A, false, M, d, &c->fK, c->qY, c->sY, true, c->ResY, c->Yq, st, c->sums + 1);
         if (rc != KQ_OK) return rc;
-        rc = run_stream<kq::MODE_PLAIN, false>(c->Zq, false, o, d, nullptr, nullptr, c->qZ, c->sZ, true, nullptr, st);
+        rc = run_umma<false>(c->W, false, o, d, &c->fP, c->qZ, c->sZ, true, c->ResZ, c->Zq, st, c->sums + 2);
         if (rc != KQ_OK) return rc;
+    } else {
+        kq::calib_fakequant<<<fq_grid(M), 128, 0, st>>>(c->A, c->Kd, c->n_sets, M, d, c->Yq, c->YqT, c->ResY, c->sums + 1);
+        if (!launched()) return KQ_ERR_CUDA;
+        kq::calib_fakequant<<<fq_grid(o), 128, 0, st>>>(c->W, c->Pd, c->n_sets, o, d, c->Zq, c->ZqT, c->ResZ, c->sums + 2);
+        if (!launched()) return KQ_ERR_CUDA;
+    }
+    // E = Yq Zq^T - A W^T; sum E^2; dO = bf16(2 E / (M o)) (one-CTA mode: and its transpose).  Yq and Zq are
+    // MXFP4 values, so with the paired kernels the product runs on the FP4 tensor-core path, straight from
+    // the codes and scale bytes the quantizer just wrote
+    if (pair_mode) {
         kq::GemmProblem e{};
         e.M = (int)M; e.N = o; e.K = d;
         e.aux = c->R; e.ld_aux = o; e.coef_ptr = nullptr; e.coef_mul = -1.0f;
@@ -476,6 +486,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     const size_t o_dK = take((size_t)n_sets * 4096), o_dP = take((size_t)n_sets * 4096);
     const size_t kt = (size_t)((d + 127) / 128) * 512;                       // scale bytes per 128-row tile
     const size_t sY_bytes = (size_t)((M + 127) / 128) * kt, sZ_bytes = (size_t)((o + 127) / 128) * kt;
+    const size_t o_imgK = take((size_t)n_sets * 6144), o_imgP = take((size_t)n_sets * 6144), o_en = take((size_t)n_sets * 4);
     const size_t o_qY = take(Md / 2), o_sY = take(sY_bytes), o_qZ = take(od / 2), o_sZ = take(sZ_bytes);
     const size_t o_sums = take(3 * 8), o_hist = take((size_t)kHistCap * 3 * 8);
     if (cudaMalloc(&c->pool, off) != cudaSuccess) { (void)cudaGetLastError(); delete c; return KQ_ERR_CUDA; }
@@ -492,6 +503,13 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     c->partK = (float*)(b + o_pK); c->partP = (float*)(b + o_pP);
     c->dK = (float*)(b + o_dK); c->dP = (float*)(b + o_dP);
     c->qY = b + o_qY; c->sY = b + o_sY; c->qZ = b + o_qZ; c->sZ = b + o_sZ;
+    c->imgK = b + o_imgK; c->imgP = b + o_imgP; c->enorm0 = (int*)(b + o_en);
+    for (kroquant_factors* f : {&c->fK, &c->fP}) {
+        f->n_sets = n_sets; f->device = c->device; f->identity = false; f->dense = true;
+        f->d_enorm = c->enorm0;
+    }
+    c->fK.d_bimage = c->imgK;
+    c->fP.d_bimage = c->imgP;
     c->sums = (double*)(b + o_sums); c->hist = (double*)(b + o_hist);
 
     bool ok = make_operand_map(&c->tm_A_a, c->A, M, d, kq::kGemmBM) && make_operand_map(&c->tm_W_b, c->W, o, d, kq::kGemmBN) &&
@@ -505,6 +523,7 @@ kq_status_t kroquant_calib_create(const void* A, const void* W, int64_t M, int o
     kq_status_t rc = ok ? KQ_OK : KQ_ERR_CUDA;
     std::vector<float> th;
     hadamard_theta(th, n_sets);
+    if (rc == KQ_OK && cudaMemsetAsync(c->enorm0, 0, (size_t)n_sets * 4, st) != cudaSuccess) rc = KQ_ERR_CUDA;
     if (rc == KQ_OK && (cudaMemsetAsync(c->sY, 0, sY_bytes, st) != cudaSuccess ||    // padding bytes stay zero
                         cudaMemsetAsync(c->sZ, 0, sZ_bytes, st) != cudaSuccess))
         rc = KQ_ERR_CUDA;
