@@ -86,6 +86,27 @@ def test_loss_and_gradient_at_random_parameters(M, o, d, seed, shared):
     cal.destroy()
 
 
+@pytest.mark.parametrize("M,o,d,seed", [(8, 32, 32, 1), (16, 32, 64, 2), (136, 160, 96, 3), (264, 32, 4608, 4)])
+@pytest.mark.parametrize("shared", [True, False])
+def test_smallest_and_ragged_shapes(M, o, d, seed, shared):
+    """One row tile or less, one block, d far larger than M: every tile is ragged.  With so few rows the bf16
+    rounding of the output error averages over few terms, hence the wider gradient tolerance (measured
+    up to 6.4e-4 at M = 16)."""
+    A, W, A_t, W_t = _case(M, o, d, seed)
+    n_sets = 1 if shared else d // 32
+    theta = wl.gen_lu_params(seed, n_sets)
+    cal = kb.Calibrator(A_t, W_t, n_sets)
+    cal.theta = theta
+    cal.lambdas = (2.5, 40.0)
+    lam = cal.lambdas.astype(np.float64)
+    losses, g = cal.loss_grad()
+    _, terms, g_ref = co.loss_and_grad(A, W, theta.astype(np.float64), lam[0], lam[1])
+    assert np.allclose(losses, terms, rtol=LOSS_RTOL, atol=0), (losses, terms)
+    assert np.abs(g - g_ref).max() <= 2e-3 * np.abs(g_ref).max()
+    _no_device_error()
+    cal.destroy()
+
+
 def test_gradient_of_the_regularisers_alone():
     """W = 0 makes the output term and its gradient vanish: what is left is lambda_A dL_A/dtheta,
     which involves no bf16 rounding of the output error."""
