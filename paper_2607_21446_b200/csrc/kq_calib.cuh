@@ -226,10 +226,11 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[a][b][c] = 0.f;
     // staging roles: X tile = 64 rows x 4 segments of 8 channels (2 per thread);
-    // G tile = 64 rows x 8 segments of 4 channels (4 per thread)
-    uint4 px[2];
-    float4 pg[4];
-    auto fetch = [&](int64_t t0) {
+    // G tile = 64 rows x 8 segments of 4 channels (4 per thread).  Two tiles ahead of the one being
+    // multiplied are in flight in registers (two alternating register sets).
+    uint4 px0[2], px1[2];
+    float4 pg0[4], pg1[4];
+    auto fetch = [&](uint4 (&px)[2], float4 (&pg)[4], int64_t t0) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int seg = threadIdx.x + 128 * i;
@@ -244,14 +245,15 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
                                 : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     };
-    if (r_begin < r_end) fetch(r_begin);
     const uint32_t xs_base = (uint32_t)__cvta_generic_to_shared(&xs[0][0]);
     const uint32_t gs_base = (uint32_t)__cvta_generic_to_shared(&gs[0][0][0]);
     // ldmatrix lane addresses inside this warp's 16 rows (see the header comment)
     const int mid = lane >> 3, l7 = lane & 7;
     const uint32_t a_off = (uint32_t)(((16 * warp + (mid >> 1) * 8 + l7) * kGradPitch + (mid & 1) * 8) * 2);
     const uint32_t b_off = (uint32_t)(((16 * warp + (mid & 1) * 8 + l7) * kGradPitch + (mid >> 1) * 8) * 2);
-    for (int64_t t0 = r_begin; t0 < r_end; t0 += kGradTileRows) {
+    // one tile: registers -> shared memory (G split into its three bf16 terms), refill the register set
+    // with the tile two steps ahead, multiply
+    auto step = [&](uint4 (&px)[2], float4 (&pg)[4], int64_t t0) {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int seg = threadIdx.x + 128 * i;
@@ -270,7 +272,7 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
                     make_uint2(t[0][m] | (t[1][m] << 16), t[2][m] | (t[3][m] << 16));
         }
         __syncthreads();
-        if (t0 + kGradTileRows < r_end) fetch(t0 + kGradTileRows);       // lands while this tile is multiplied
+        if (t0 + 2 * kGradTileRows < r_end) fetch(px, pg, t0 + 2 * kGradTileRows);
         uint32_t af[2][4];
         ldmatrix_x4_trans(af[0], xs_base + a_off);                       // channels 0..15 of X
         ldmatrix_x4_trans(af[1], xs_base + a_off + 32);                  // channels 16..31
@@ -287,6 +289,12 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
                     mma_bf16_16816(acc[mt][nt], af[mt], bfr[nt >> 1][(nt & 1) * 2], bfr[nt >> 1][(nt & 1) * 2 + 1]);
         }
         __syncthreads();
+    };
+    if (r_begin < r_end) fetch(px0, pg0, r_begin);
+    if (r_begin + kGradTileRows < r_end) fetch(px1, pg1, r_begin + kGradTileRows);
+    for (int64_t t0 = r_begin; t0 < r_end; t0 += 2 * kGradTileRows) {
+        step(px0, pg0, t0);
+        if (t0 + kGradTileRows < r_end) step(px1, pg1, t0 + kGradTileRows);
     }
     // accumulator fragment: c0, c1 = (m = g, n = 2q, 2q + 1); c2, c3 = (m = g + 8, same n)
     {
