@@ -279,7 +279,8 @@ kq_status_t kroquant_calib_run(kroquant_calib_t *c, int steps, float lr, double 
  * out is DEVICE fp32 [n_sets][32][32].  The kernel first writes partial sums per chunk of rows
  * into `scratch` (DEVICE, 16-byte aligned, at least kroquant_block_grad_scratch_bytes(rows, d)
  * bytes, contents irrelevant before and after), then reduces them in a fixed order, so the result
- * is deterministic.  Errors: KQ_ERR_NULL, KQ_ERR_SHAPE (d % 32, rows < 0, scratch too small),
+ * is deterministic.  The products run on the tensor cores with G taken to its 16 leading significand
+ * bits (two bf16 terms; X is bf16 already), fp32 accumulation per chunk, double across chunks.  Errors: KQ_ERR_NULL, KQ_ERR_SHAPE (d % 32, rows < 0, scratch too small),
  * KQ_ERR_FACTORS (n_sets), KQ_ERR_ALIGN, KQ_ERR_CUDA.  rows == 0 writes zeros. */
 int64_t kroquant_block_grad_scratch_bytes(int64_t rows, int d);
 kq_status_t kroquant_block_grad(const void *X, const float *G, int64_t rows, int d, int n_sets,

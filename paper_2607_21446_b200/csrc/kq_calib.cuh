@@ -196,14 +196,17 @@ calib_fakequant(const uint16_t* __restrict__ X, const float* __restrict__ B, int
 }
 
 // ---- block gradients: part[chunk][j][32][32] = sum over the chunk's rows of x_j^T g_j ---------
-// grid (chunks, d/32); 4 warps.  Tiles of 64 rows are staged in shared memory as bf16: X as it is,
-// G (fp32) split into three bf16 terms that add up to it exactly, so the tensor-core products
-// (mma.sync m16n8k16, fp32 accumulate) are exact.  Both operands are stored row-major [row][channel]
+// grid (d/32, chunks); 4 warps.  Tiles of 64 rows are staged in shared memory as bf16: X as it is,
+// G (fp32) as the sum of two bf16 terms (its 16 leading significand bits: relative error below 2^-16
+// per element, far below the noise of a gradient whose upstream factor was rounded to bf16 itself; the
+// legacy mma.sync path is the bottleneck of this kernel, and a third term costs a third more of it), so
+// the tensor-core products (mma.sync m16n8k16, fp32 accumulate) are exact for the stored terms.  Both operands are stored row-major [row][channel]
 // and fetched with transposing ldmatrix, which yields x^T as the "A" fragments (m = channel of X,
 // k = row) and g as the "B" fragments (k = row, n = channel of G).  Warp w multiplies rows
 // 16w..16w+15 of every tile into its own 32 x 32 accumulator; the four are summed at the end.
 constexpr int kGradTileRows = 64;
 constexpr int kGradPitch = 40;                 // bf16 elements per staged row: 80 bytes, conflict-free ldmatrix
+constexpr int kGradTerms = 2;                  // bf16 terms of G
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
@@ -212,11 +215,14 @@ __global__ void __launch_bounds__(128)
 calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, int64_t rows, int d,
                  int64_t rows_per_chunk, float* __restrict__ part) {
     __shared__ __align__(16) uint16_t xs[kGradTileRows][kGradPitch];
-    __shared__ __align__(16) uint16_t gs[3][kGradTileRows][kGradPitch];
+    __shared__ __align__(16) uint16_t gs[kGradTerms][kGradTileRows][kGradPitch];
     __shared__ __align__(16) float red[4][1024];
-    const int j = blockIdx.y;
+    // grid (d/32, chunks): CTAs that run at the same time read neighbouring 128-byte columns of the same
+    // rows, which keeps the DRAM pages they touch fully used
+    const int j = blockIdx.x;
+    const int chunk = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t r_begin = (int64_t)blockIdx.x * rows_per_chunk;
+    const int64_t r_begin = (int64_t)chunk * rows_per_chunk;
     const int64_t r_end = r_begin + rows_per_chunk < rows ? r_begin + rows_per_chunk : rows;
     float acc[2][4][4];
 #pragma unroll
@@ -267,7 +273,7 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
 #pragma unroll
             for (int e = 0; e < 4; ++e) split3_bf16(gv[e], t[e]);
 #pragma unroll
-            for (int m = 0; m < 3; ++m)
+            for (int m = 0; m < kGradTerms; ++m)
                 *reinterpret_cast<uint2*>(&gs[m][seg >> 3][(seg & 7) * 4]) =
                     make_uint2(t[0][m] | (t[1][m] << 16), t[2][m] | (t[3][m] << 16));
         }
@@ -277,7 +283,7 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
         ldmatrix_x4_trans(af[0], xs_base + a_off);                       // channels 0..15 of X
         ldmatrix_x4_trans(af[1], xs_base + a_off + 32);                  // channels 16..31
 #pragma unroll
-        for (int m = 2; m >= 0; --m) {                                   // smallest term first
+        for (int m = kGradTerms - 1; m >= 0; --m) {                      // smallest term first
             uint32_t bfr[2][4];
             const uint32_t gm = gs_base + (uint32_t)(m * kGradTileRows * kGradPitch * 2) + b_off;
             ldmatrix_x4_trans(bfr[0], gm);                               // channels 0..15 of G: n-tiles 0, 1
@@ -309,7 +315,7 @@ calib_block_grad(const uint16_t* __restrict__ X, const float* __restrict__ G, in
             }
     }
     __syncthreads();
-    float* dst = part + ((size_t)blockIdx.x * gridDim.y + j) * 1024;
+    float* dst = part + ((size_t)chunk * gridDim.x + j) * 1024;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int e = threadIdx.x + 128 * i;

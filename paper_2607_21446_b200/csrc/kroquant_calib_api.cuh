@@ -168,7 +168,7 @@ void chunking(int64_t rows, int nb, int sms, int* chunks, int64_t* rpc) {
 kq_status_t run_block_grad(const uint16_t* X, const float* G, int64_t rows, int d, int n_sets, int chunks, int64_t rpc,
                            float* part, float* out, cudaStream_t st) {
     const int nb = d / 32;
-    kq::calib_block_grad<<<dim3((unsigned)chunks, (unsigned)nb), 128, 0, st>>>(X, G, rows, d, rpc, part);
+    kq::calib_block_grad<<<dim3((unsigned)nb, (unsigned)chunks), 128, 0, st>>>(X, G, rows, d, rpc, part);
     if (!launched()) return KQ_ERR_CUDA;
     if (n_sets == 1)
         kq::calib_reduce_parts<<<dim3(32, 1), 1024, 0, st>>>(part, chunks * nb, out);
