@@ -192,6 +192,15 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t *a_codes, const uint8_t *a_scales,
                                 const uint8_t *b_scales, int64_t M, int N, int K, const void *add_bf16,
                                 void *out, kq_dtype_t out_dtype, void *stream);
 
+/* Plain bf16 GEMM on the same tensor-core kernels the calibration loop uses, offered for the 16-bit
+ * low-rank branch A T L R of Section 3.4 (two skinny products whose result goes into the `add`
+ * argument of kroquant_gemm_mxfp4):  out[m][n] = sum_k A[m][k] B[n][k]  (+ add[m][n]).
+ * A [M][K], B [N][K]: DEVICE bf16, row-major, 16-byte aligned; K % 8 == 0, N % 32 == 0;
+ * add: optional DEVICE fp32 [M][N]; out: DEVICE [M][N] bf16 or fp32.  fp32 accumulation.
+ * Asynchronous on `stream`, allocates nothing. */
+kq_status_t kroquant_gemm_bf16(const void *A, const void *B, int64_t M, int N, int K, const float *add_f32,
+                               void *out, kq_dtype_t out_dtype, void *stream);
+
 /* The quantized linear layer of Section 3.4 in one call:
  *     out = Q(X T) Q(W~)^T (+ add),   Q(X T) by kroquant_quantize_ex (tensor path, tiled scales),
  *                                     the product by kroquant_gemm_mxfp4,

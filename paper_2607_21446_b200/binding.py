@@ -34,7 +34,7 @@ EXPORTS = [
     "kroquant_calib_loss_grad", "kroquant_calib_run",
     "kroquant_block_grad_scratch_bytes", "kroquant_block_grad", "kroquant_block_grad_static",
     "kroquant_debug_set_gemm_pair", "kroquant_calib_get_weight_factors", "kroquant_gemm_mxfp4",
-    "kroquant_linear_w4a4",
+    "kroquant_linear_w4a4", "kroquant_gemm_bf16",
 ]
 
 
@@ -98,6 +98,7 @@ def load_library() -> C.CDLL:
     L.kroquant_block_grad_static.argtypes = [vp, vp, i64, i32, i32, vp, vp]
     L.kroquant_debug_set_gemm_pair.argtypes = [i32]
     L.kroquant_gemm_mxfp4.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, vp]
+    L.kroquant_gemm_bf16.argtypes = [vp, vp, i64, i32, i32, vp, vp, i32, vp]
     L.kroquant_linear_w4a4.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, i32, vp]
     _lib = L
     return L
@@ -438,6 +439,28 @@ def kroquant_gemm_mxfp4(a_codes: torch.Tensor, a_scales: torch.Tensor, b_codes: 
     _check(load_library().kroquant_gemm_mxfp4(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), M, N, K,
                                               _ptr(add), _ptr(out), 1 if out.dtype == torch.bfloat16 else 0,
                                               _stream(stream)), "kroquant_gemm_mxfp4")
+    return out
+
+
+def kroquant_gemm_bf16(A: torch.Tensor, Bm: torch.Tensor, add: Optional[torch.Tensor] = None,
+                       out: Optional[torch.Tensor] = None, out_dtype=torch.bfloat16, stream=None) -> torch.Tensor:
+    """out[M, N] = A[M, K] @ Bm[N, K]^T (+ add, float32): bf16 operands, fp32 accumulation, on this library's
+    tensor-core GEMM (for the 16-bit low-rank branch of the quantized layer)."""
+    for t in (A, Bm):
+        if t.dim() != 2 or t.dtype != torch.bfloat16 or not t.is_cuda or not t.is_contiguous():
+            raise ValueError("A and Bm must be contiguous 2-D CUDA bfloat16 tensors")
+    M, K = A.shape
+    N = Bm.shape[0]
+    if Bm.shape[1] != K:
+        raise ValueError("A [M, K] and Bm [N, K] must share K")
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    if out.dtype not in (torch.bfloat16, torch.float32) or tuple(out.shape) != (M, N) or not out.is_contiguous():
+        raise ValueError("out must be a contiguous bfloat16 or float32 tensor [M, N]")
+    if add is not None and (add.dtype != torch.float32 or tuple(add.shape) != (M, N) or not add.is_contiguous()):
+        raise ValueError("add must be a contiguous float32 tensor [M, N]")
+    _check(load_library().kroquant_gemm_bf16(_ptr(A), _ptr(Bm), M, N, K, _ptr(add), _ptr(out),
+                                             1 if out.dtype == torch.bfloat16 else 0, _stream(stream)), "kroquant_gemm_bf16")
     return out
 
 

@@ -436,6 +436,23 @@ kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, con
 
 extern "C" {
 
+kq_status_t kroquant_gemm_bf16(const void* A, const void* B, int64_t M, int N, int K, const float* add_f32, void* out,
+                               kq_dtype_t out_dtype, void* stream) {
+    if (!A || !B || !out) return KQ_ERR_NULL;
+    if (M < 0 || N <= 0 || K <= 0 || K % 8 || N % 32 || M > (1 << 30)) return KQ_ERR_SHAPE;
+    if (out_dtype != KQ_OUT_F32 && out_dtype != KQ_OUT_BF16) return KQ_ERR_UNSUPPORTED;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(out) || (add_f32 && !aligned16(add_f32))) return KQ_ERR_ALIGN;
+    if (M == 0) return KQ_OK;
+    CUtensorMap ta, tb, tb2;
+    if (!make_operand_map(&ta, A, M, K, kq::kGemmBM) || !make_operand_map(&tb, B, N, K, kq::kGemmBN) ||
+        !make_operand_map(&tb2, B, N, K, 128))
+        return KQ_ERR_CUDA;
+    return launch_gemm(ta, tb, tb2, (int)M, N, K, add_f32, N, nullptr, 1.0f, 1.0f,
+                       out_dtype == KQ_OUT_F32 ? static_cast<float*>(out) : nullptr,
+                       out_dtype == KQ_OUT_BF16 ? static_cast<__nv_bfloat16*>(out) : nullptr, N, nullptr,
+                       reinterpret_cast<cudaStream_t>(stream));
+}
+
 kq_status_t kroquant_linear_w4a4(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const kroquant_factors_t* f,
                                  const uint8_t* w_codes, const uint8_t* w_scales, int o, uint8_t* q_work, uint8_t* s_work,
                                  const void* add_bf16, void* out, kq_dtype_t out_dtype, void* stream) {

@@ -171,6 +171,62 @@ def test_linear_layer_call_equals_the_two_separate_calls(dtype):
     assert kb.kroquant_last_device_error() == 0
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 128, 1152), (257, 96, 136), (1000, 512, 128), (64, 32, 8)])
+def test_bf16_gemm_for_the_low_rank_branch(M, N, K):
+    g = torch.Generator(device="cuda")
+    g.manual_seed(M + N + K)
+    A = torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
+    Bm = torch.randn(N, K, device="cuda", generator=g).to(torch.bfloat16)
+    add = torch.randn(M, N, device="cuda", generator=g)
+    ref = A.double().cpu().numpy() @ Bm.double().cpu().numpy().T
+    bound = np.abs(A.double().cpu().numpy()) @ np.abs(Bm.double().cpu().numpy()).T
+    out = kb.kroquant_gemm_bf16(A, Bm, out_dtype=torch.float32).double().cpu().numpy()
+    assert np.all(np.abs(out - ref) <= 1e-6 * bound + 1e-30)          # exact products, fp32 accumulation
+    out2 = kb.kroquant_gemm_bf16(A, Bm, add=add, out_dtype=torch.float32).double().cpu().numpy()
+    assert np.all(np.abs(out2 - (ref + add.double().cpu().numpy())) <= 1e-6 * (bound + np.abs(add.double().cpu().numpy())))
+    out16 = kb.kroquant_gemm_bf16(A, Bm)
+    assert torch.equal(out16, kb.kroquant_gemm_bf16(A, Bm, out_dtype=torch.float32).to(torch.bfloat16))
+    assert kb.kroquant_last_device_error() == 0
+
+
+def test_whole_layer_with_low_rank_branch():
+    """Section 3.4's inference form with this library's kernels only:
+    O = Q(A T) Q(W~ - L R)^T + (A T) R^T L^T, the second term in 16 bit with rank 128."""
+    M, o, d, r, seed = 384, 256, 1152, 128, 17
+    rng = np.random.default_rng(seed)
+    A_bits = wl.gen_activations(wl.calib_spec(M, d, seed))
+    A_t = torch.from_numpy(A_bits.view(np.int16)).cuda().view(torch.bfloat16)
+    W = wl.bf16_bits_to_f32(wl.gen_weights(seed, o, d)).astype(np.float64)
+    theta = wl.gen_lu_params(seed, 1).astype(np.float64)
+    G = cal.lu_factors(theta).astype(np.float32)
+    K_, P_ = cal.blocks_of(theta)
+    Wt = cal.apply_blocks(W, P_)                                   # W~ = W T^-T
+    U_, s_, Vt_ = np.linalg.svd(Wt, full_matrices=False)            # a rank-r split of W~ stands in for LoRaQ's L, R
+    Lm = (U_[:, :r] * s_[:r]).astype(np.float32)                    # [o, r]
+    Rm = Vt_[:r].astype(np.float32)                                 # [r, d]
+    L_t = torch.from_numpy(Lm).cuda().to(torch.bfloat16).contiguous()
+    R_t = torch.from_numpy(Rm).cuda().to(torch.bfloat16).contiguous()
+    resid = torch.from_numpy((Wt - L_t.double().cpu().numpy() @ R_t.double().cpu().numpy()).astype(np.float32)).cuda().to(torch.bfloat16)
+    qw, sw = kb.kroquant_mxfp4_quantize(resid.contiguous(), scale_layout="tiled")       # Q(W~ - L R), offline
+    fa = kb.Factors.create(G)
+    qa, sa, AT = kb.kroquant_quantize_dual(A_t, fa, scale_layout="tiled")               # codes, scales, A T in bf16
+    low = kb.kroquant_gemm_bf16(kb.kroquant_gemm_bf16(AT, R_t), L_t)                    # (A T R^T) L^T, bf16 [M, o]
+    out = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, add=low, out_dtype=torch.float32).double().cpu().numpy()
+    # oracle: decode both quantized operands, float64 products; the 16-bit branch from the same bf16 inputs
+    qa_r, sa_r = kb.kroquant_quantize(A_t, fa)
+    qw_r, sw_r = kb.kroquant_mxfp4_quantize(resid.contiguous())
+    main = co.dequantize(qa_r.cpu().numpy(), sa_r.cpu().numpy()).astype(np.float64) @ \
+        co.dequantize(qw_r.cpu().numpy(), sw_r.cpu().numpy()).astype(np.float64).T
+    branch = (AT.double().cpu().numpy() @ R_t.double().cpu().numpy().T) @ L_t.double().cpu().numpy().T
+    ref = main + branch
+    # two bf16 roundings on the branch (2^-9 relative each); the W4A4 part is exact up to accumulation order
+    assert np.abs(out - ref).max() <= 1e-2 * np.abs(branch).max() + 1e-6 * np.abs(main).max()
+    # and the layer does what it is for: close to the unquantized product A W^T
+    exact = wl.bf16_bits_to_f32(A_bits).astype(np.float64) @ W.T
+    assert np.linalg.norm(out - exact) < 0.25 * np.linalg.norm(exact)
+    fa.destroy()
+
+
 def test_argument_checks():
     A, W = _operand(128, 128, 1), _operand(128, 128, 2)
     qa, sa, _ = _decoded(A)
