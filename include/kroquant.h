@@ -174,7 +174,14 @@ kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes,
 /* Tuning hook for the tensor-core kernel.  config 0..7 selects (pipeline slots, MMA
  * issuer warps, epilogue warpgroups) = (2,2,1) (8,2,1) (8,2,2) (2,1,1) (4,1,1) (4,2,1)
  * (16,2,2) (16,2,4); the default is config 5 with 3 CTAs per SM; ctas_per_sm in 1..8 caps the persistent grid; use_pdl != 0
- * launches with programmatic stream serialization.  Process-wide. */
+ * (default) launches the quantizer kernels with programmatic stream serialization and lets them signal
+ * launch completion at their start, so that consecutive calls overlap their set-up with the tail of the
+ * call before; every kernel of this library waits for its prerequisite grids before it touches memory.
+ * Ordinary launches behind them (plain <<<>>> kernels, the framework's and the vendor libraries' kernels)
+ * were checked to start only after the outputs are complete.  One exception was measured on driver 580: a
+ * kernel launched by the caller with cudaLaunchKernelEx and a cluster dimension directly behind such a
+ * chain began early; a kernel like that has to call cudaGridDependencySynchronize() first, or the caller
+ * turns the early signal off with use_pdl = 0.  Process-wide. */
 kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl);
 
 /* The W4A4 product of the quantized layer (Section 3.4: O = Q(A T) Q(W~)^T + A T L R):

@@ -216,6 +216,7 @@ gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
+            pdl_wait_prior_grid();      // nothing is read before every earlier grid in the stream is complete
             int it = 0;
             for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
                 int tm, tn;
@@ -271,6 +272,7 @@ gemm_nt_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__
         // ---------------- epilogue: warps 2..9, TMEM lane quarter = warp % 4 ----------------
         const int quarter = warp & 3;
         const int chalf = (warp - 2) >> 2;                  // which half of the tile's columns
+        pdl_wait_prior_grid();
         const float coef = p.coef_mul * (p.coef_ptr ? __ldg(p.coef_ptr) : 1.0f);
         double sq = 0.0;
         for (int i = 0; i < my_tiles; ++i) {

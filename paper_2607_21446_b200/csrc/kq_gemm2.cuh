@@ -140,6 +140,11 @@ gemm_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (warp == 0) {
         // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
+            // Measured on this driver: a cluster kernel launched right behind a chain of programmatically
+            // dependent launches (the quantizer kernels trigger their dependents early) can begin before
+            // that chain has finished, although it was launched without the attribute.  Every thread that
+            // touches global memory therefore waits for the prerequisite grids first (a no-op otherwise).
+            pdl_wait_prior_grid();
             int it = 0;
             for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
                 int tm, tn;
@@ -208,6 +213,7 @@ gemm_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // ---------------- epilogue: warps 2..9 of both CTAs, each CTA its own 128 rows ----------------
         const int quarter = warp & 3;
         const int chalf = (warp - 2) >> 2;
+        pdl_wait_prior_grid();          // see the producer
         const float coef = p.coef_mul * (p.coef_ptr ? __ldg(p.coef_ptr) : 1.0f);
         double sq = 0.0;
         for (int i = 0; i < my_tiles; ++i) {

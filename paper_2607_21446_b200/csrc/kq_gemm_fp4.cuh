@@ -129,6 +129,7 @@ gemm_mxfp4_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     if (warp == 0) {
         // ---------------- producer ----------------
         if (lane == 0) {
+            pdl_wait_prior_grid();      // nothing is read before every earlier grid in the stream is complete
             int it = 0;
             for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
                 int tm, tn;
@@ -194,6 +195,7 @@ gemm_mxfp4_umma(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         // ---------------- epilogue: warps 2..9 ----------------
         const int quarter = warp & 3;
         const int chalf = (warp - 2) >> 2;
+        pdl_wait_prior_grid();
         for (int i = 0; i < my_tiles; ++i) {
             const int acc = i & 1;
             int tm, tn;

@@ -139,6 +139,9 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     if (warp == 0) {
         // ---------------- producer (both CTAs) ----------------
         if (lane == 0) {
+            // launched with programmatic stream serialization: everything up to here overlapped the tail of
+            // the kernel before (typically the quantizer that writes A's codes and scales)
+            pdl_wait_prior_grid();
             int it = 0;
             for (int i = 0; i < my_tiles && !*abort_flag; ++i) {
                 int tm, tn;
@@ -228,6 +231,7 @@ gemm_mxfp4_umma_pair(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         const int chalf = (warp - 2) >> 2;
         // full-sector (32-byte) stores when the output base allows it; row pitches and column offsets always do
         const bool wide = ((reinterpret_cast<uintptr_t>(p.out_bf16) | reinterpret_cast<uintptr_t>(p.out_f32)) & 31u) == 0;
+        pdl_wait_prior_grid();          // outputs and epilogue inputs may still be in use by the kernel before
         const float epi_coef = p.use_epi ? p.epi.coef_mul * (p.epi.coef_ptr ? __ldg(p.epi.coef_ptr) : 1.0f) : 0.f;
         double sq = 0.0;
         for (int i = 0; i < my_tiles; ++i) {

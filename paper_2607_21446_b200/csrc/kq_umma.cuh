@@ -322,6 +322,7 @@ struct UmmaProblem {
     int n_ttiles;        // PB=true: token tiles (ceil(tokens/128))
     int blocks_per_row;  // d/32
     int tiled_scales;    // 0: scales[t][d/32] row-major; 1: 128 x 4 tiled layout for GEMM consumers
+    int early_trigger;   // 1: signal programmatic launch completion at the start of the kernel (see below)
 };
 
 // NS pipeline slots: slot s = one shared-memory stage + one 32-column TMEM accumulator
@@ -404,7 +405,11 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         }
     };
 
-    pdl_launch_dependents();
+    // Early trigger: a following kernel that was launched with programmatic stream serialization may then
+    // run its set-up while this one still works (it must wait for the prerequisite grids before it touches
+    // memory, as this kernel does).  Off when the library's programmatic-launch switch is off, and for
+    // launches whose operand image was written by the kernel just before.
+    if (prob.early_trigger) pdl_launch_dependents();
     int issued = 0;   // tiles whose TMA load the producer thread has issued
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_done(s), 1); mbar_init(bar_tempty(s), 4); }

@@ -233,6 +233,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     kq::UmmaProblem prob;
     prob.blocks_per_row = nb;
     prob.tiled_scales = tiled ? 1 : 0;
+    prob.early_trigger = (g_umma_pdl.load() != 0 && calib_sumsq == nullptr) ? 1 : 0;
     CUtensorMap tmap;
     cuuint64_t dims[2], strides[1];
     if (pb) {

@@ -123,13 +123,17 @@ kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
         cfg.blockDim = dim3(kq::kGemmThreads);
         cfg.dynamicSmemBytes = kq::kGemm2DynBytes;
         cfg.stream = st;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        // the kernel's set-up may overlap the tail of the kernel before it (it waits for that kernel's
+        // memory before its first global access)
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
         const cudaError_t lrc = mode == 0   ? cudaLaunchKernelEx(&cfg, kq::gemm_umma_pair<false, false>, ta, tb2, p)
                                 : mode == 1 ? cudaLaunchKernelEx(&cfg, kq::gemm_umma_pair<false, true>, ta, tb2, p)
                                             : cudaLaunchKernelEx(&cfg, kq::gemm_umma_pair<true, true>, ta, tb2, p);
@@ -415,13 +419,17 @@ kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, con
         cfg.blockDim = dim3(kq::kF4PThreads);
         cfg.dynamicSmemBytes = kq::kF4PDynBytes;
         cfg.stream = st;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        // the kernel's set-up may overlap the tail of the kernel before it (it waits for that kernel's
+        // memory before its first global access)
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 2;
         if (cudaLaunchKernelEx(&cfg, kq::gemm_mxfp4_umma_pair, ta, tb, tsa, tsb, p) != cudaSuccess) {
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
