@@ -65,6 +65,28 @@ def test_against_the_decoded_float64_product(M, N, K):
     assert torch.equal(out16, out.to(torch.bfloat16))
 
 
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    return [(int(rng.integers(1, 700)), 32 * int(rng.integers(1, 34)), 32 * int(rng.integers(1, 66))) for _ in range(n)]
+
+
+@pytest.mark.parametrize("M,N,K", _random_shapes(14, 2024))
+def test_seeded_random_shapes(M, N, K):
+    A, W = _operand(M, K, M + K), _operand(N, K, N + K)
+    qa, sa, Ad = _decoded(A)
+    qw, sw, Wd = _decoded(W)
+    out = kb.kroquant_gemm_mxfp4(qa, sa, qw, sw, out_dtype=torch.float32).double().cpu().numpy()
+    assert np.all(np.abs(out - Ad @ Wd.T) <= TOL * (np.abs(Ad) @ np.abs(Wd).T) + 1e-300)
+    low = kb.kroquant_gemm_bf16(A, W, out_dtype=torch.float32).double().cpu().numpy()
+    Af, Wf = A.double().cpu().numpy(), W.double().cpu().numpy()
+    # 16-bit operands with outlier channels: the products span many binades, and the tensor core drops the bits
+    # below its accumulator's last place once per 16-deep instruction, so the bound grows with K/16 roundings of
+    # at most 2^-23 of the running sum of magnitudes (seen: 1.7e-6 of that sum at K = 2048)
+    low_tol = (K // 16 + 2) * 2.0 ** -23
+    assert np.all(np.abs(low - Af @ Wf.T) <= low_tol * (np.abs(Af) @ np.abs(Wf).T) + 1e-300)
+    assert kb.kroquant_last_device_error() == 0
+
+
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 def test_output_base_that_is_only_16_byte_aligned(dtype):
     """The epilogue uses 32-byte stores when the output base allows it and 16-byte stores otherwise."""
