@@ -184,6 +184,24 @@ kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes,
  * turns the early signal off with use_pdl = 0.  Process-wide. */
 kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl);
 
+/* Tuning knobs for what happens at the boundary between two consecutive quantizer kernels (both only act
+ * while use_pdl is on).  trigger: 0 = a kernel never signals launch completion before it ends; 1 = every
+ * CTA signals at its start; 2 = a CTA signals once it has no tile load left to issue, so that the next
+ * kernel's CTAs become resident shortly before this one ends.  prefetch_tiles (0..64):
+ * before a CTA waits for its prerequisite grids it asks the L2 cache for its first prefetch_tiles tiles of
+ * X (a prefetch moves no data into the SM and the L2 is where the previous kernel's writes land, so the
+ * request is safe even if that kernel still produces X).  KQ_ERR_UNSUPPORTED outside the ranges.
+ * Process-wide. */
+kq_status_t kroquant_debug_set_boundary(int trigger, int prefetch_tiles);
+
+/* How the tensor-core quantizer hands its tiles (128 blocks of 32 channels) to CTAs.  A unit is unit_tiles
+ * (1..16) consecutive tiles (always 4 column tiles with per-block factor sets).  dynamic = 0: a persistent
+ * grid of at most ctas_per_sm CTAs per SM, CTA b takes units b, b + grid, ...  dynamic = 1: one CTA per unit
+ * in the grid; the CTAs that the hardware starts first take over, besides their own unit, the units of CTAs
+ * that have not started (cluster launch control), so that a CTA on a slower path to memory simply takes fewer.
+ * Results do not depend on either setting.  KQ_ERR_UNSUPPORTED outside the ranges.  Process-wide. */
+kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles);
+
 /* The W4A4 product of the quantized layer (Section 3.4: O = Q(A T) Q(W~)^T + A T L R):
  *     out[m][n] = sum_k a[m][k] 2^(sa[m][k/32] - 127) * b[n][k] 2^(sb[n][k/32] - 127)  (+ add[m][n])
  * on the block-scaled FP4 tensor-core path (fp32 accumulation).  a_codes [M][K/2] and b_codes

@@ -172,6 +172,7 @@ __device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcon
 // ---- shared memory plan ----------------------------------------------------------
 // PB = false: one factor image for the whole launch at offset 0, stages of 8 KB (A only).
 // PB = true : every stage carries its own factor image: 8 KB of A + 6 KB of B.
+constexpr int kRingEntries = 32;
 template <int NS, bool PB>
 struct UmmaSmem {
     static constexpr int kStageBytes = kTileBytes + (PB ? kBImageBytes : 0);   // multiple of 1024
@@ -182,9 +183,11 @@ struct UmmaSmem {
     static constexpr int kStoreOff = kAOff + NS * kStageBytes;
     static constexpr int kStoreBytes = PB ? (kTileRows * 64 + kTileRows * 4) : 0;
     static constexpr int kBarOff = kStoreOff + kStoreBytes;
-    // barriers: full[NS], done[NS], tempty[NS], bfull
-    static constexpr int kNumBars = 3 * NS + 1;
-    static constexpr int kTmemSlotOff = kBarOff + 8 * kNumBars;
+    // barriers: full[NS], done[NS], tempty[NS], bfull, clc
+    static constexpr int kNumBars = 3 * NS + 2;
+    static constexpr int kClcOff = kBarOff + ((8 * kNumBars + 15) & ~15);     // 16-byte response of a cancel request
+    static constexpr int kRingOff = kClcOff + 16;                             // kRingEntries ints: work item of local tile n
+    static constexpr int kTmemSlotOff = kRingOff + 4 * kRingEntries;
     static constexpr int kAbortOff = kTmemSlotOff + 4;
     static constexpr int kBytes = kAbortOff + 4;
     static constexpr int kDynBytes = kBytes + 1024;                  // slack for manual alignment
@@ -322,7 +325,13 @@ struct UmmaProblem {
     int n_ttiles;        // PB=true: token tiles (ceil(tokens/128))
     int blocks_per_row;  // d/32
     int tiled_scales;    // 0: scales[t][d/32] row-major; 1: 128 x 4 tiled layout for GEMM consumers
-    int early_trigger;   // 1: signal programmatic launch completion at the start of the kernel (see below)
+    int early_trigger;   // 0: never; 1: signal programmatic launch completion at the start of the kernel;
+                         // 2: each CTA signals once its producer has no tile left to issue
+    int prefetch_tiles;  // tiles of X each CTA asks the L2 for before it waits for the prerequisite grids
+    int64_t n_tiles;     // PB=false: 128-row tiles
+    int unit_tiles;      // PB=false: consecutive tiles per work unit (PB: kPbCols)
+    int dynamic;         // 1: the grid has one CTA per unit and running CTAs take over the units of CTAs that
+                         // have not started yet (cluster launch control); 0: CTA b takes units b, b + gridDim.x, ...
 };
 
 // NS pipeline slots: slot s = one shared-memory stage + one 32-column TMEM accumulator
@@ -336,7 +345,14 @@ struct UmmaProblem {
 // Per slot: full (TMA landed) -> done (one tcgen05.commit: the MMAs have read the stage
 // and written the accumulator; frees the stage for the producer and hands the
 // accumulator to the epilogue) -> tempty (4 epilogue warps have read the accumulator).
-// Grid: any size <= number of tiles; CTA b takes tiles b, b + gridDim.x, ...
+// Work distribution: a unit is unit_tiles consecutive tiles (PB: the kPbCols tiles of one column group).
+// Static: any grid size <= number of units; CTA b takes units b, b + gridDim.x, ...  Dynamic: the grid has
+// one CTA per unit; the hardware starts as many as fit, and each of them, besides its own unit, takes over
+// the units of CTAs that have not started yet (clusterlaunchcontrol.try_cancel: one request in flight per
+// CTA, none after the first refusal), so that all CTAs finish within about one tile time of each other
+// whatever their individual memory throughput.  The producer writes the work item of local tile n into
+// ring[n % kRingEntries] before it arms the tile's barrier; the end of the stream is a run of sentinel
+// tiles (-1) that the MMA warps pass on to the epilogue groups.
 // XF16: X and the factor image are fp16 (else bf16); e_norm: per-set normalisation exponents of
 // the image (all zero for bf16 images).
 // EXTRA = 1 (second output): also write the 16-bit transformed activations (at_out).
@@ -376,32 +392,114 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int my_units = (int)((prob.n_units - blockIdx.x + gridDim.x - 1) / gridDim.x);
-    const int my_tiles = PB ? my_units * kPbCols : my_units;
     static_assert(!PB || NG == 1, "a column group is staged by one epilogue warpgroup");
+    static_assert(kRingEntries >= 2 * NS, "a ring entry must outlive the tile it describes");
+    // sentinel tiles at the end of the stream: every MMA warp gets the same number, every epilogue group at least one
+    constexpr int kSentinels = ((NM > NG ? NM : NG) + NM - 1) / NM * NM;
+    volatile int* ring = reinterpret_cast<volatile int*>(base_ptr + L::kRingOff);
+    const uint32_t bar_clc = bar0 + 8u * (3 * NS + 1);
+    const uint32_t clc_resp = base + L::kClcOff;
+    const int tpu = PB ? kPbCols : prob.unit_tiles;                   // tiles per unit
 
-    // issue the TMA copies of local tile n into slot n % NS (producer thread only)
-    // PB: local tile n -> column j (may be >= blocks_per_row in the last, ragged group: such a
+    // PB: unit u, column c of its group -> column j (may be >= blocks_per_row in the last, ragged group: such a
     // tile loads zeros and stores nothing), column group jg, token tile tt
-    auto pb_coords = [&](int n, int& j, int& jg, int& tt) {
-        const int64_t u = blockIdx.x + (int64_t)(n / kPbCols) * gridDim.x;
-        jg = (int)(u / prob.n_ttiles);
-        tt = (int)(u % prob.n_ttiles);
-        j = jg * kPbCols + (n % kPbCols);
+    auto pb_coords = [&](int u, int c, int& j, int& jg, int& tt) {
+        jg = u / prob.n_ttiles;
+        tt = u % prob.n_ttiles;
+        j = jg * kPbCols + c;
     };
-    auto issue_tile = [&](int n) {
+    // issue the TMA copies of local tile n into slot n % NS (producer thread only); item = global tile index
+    // (PB: unit index, the column is n % kPbCols)
+    auto issue_tile = [&](int n, int item) {
         const int s = n % NS;
         const uint32_t dst = base + L::kAOff + s * L::kStageBytes;
+        ring[n % kRingEntries] = item;
         mbar_expect_tx(bar_full(s), L::kStageBytes);
         if (PB) {
             int j, jg, tt;
-            pb_coords(n, j, jg, tt);
+            pb_coords(item, n % kPbCols, j, jg, tt);
             const int jb = j < prob.blocks_per_row ? j : prob.blocks_per_row - 1;
             tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));      // zero-filled if j is out of range
             bulk_load(dst + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(s));
         } else {
-            const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
-            tma_load_2d(dst, &tmap_x, 0, (int)(w * kTileRows), bar_full(s));
+            tma_load_2d(dst, &tmap_x, 0, item * kTileRows, bar_full(s));
+        }
+    };
+    auto prefetch_tile = [&](int item, int c) {
+        int x = 0, y = item * kTileRows;
+        if (PB) {
+            int j, jg, tt;
+            pb_coords(item, c, j, jg, tt);
+            if (j >= prob.blocks_per_row) return;
+            x = j * 32;
+            y = tt * kTileRows;
+        }
+        asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+                     ::"l"(&tmap_x), "r"(x), "r"(y) : "memory");
+    };
+    auto unit_count = [&](int64_t u) -> int {                       // tiles of unit u
+        if (PB) return kPbCols;
+        const int64_t rem = prob.n_tiles - u * tpu;
+        return rem < tpu ? (int)rem : tpu;
+    };
+    auto clc_request = [&]() {
+        mbar_expect_tx(bar_clc, 16);
+        asm volatile("clusterlaunchcontrol.try_cancel.async.shared::cta.mbarrier::complete_tx::bytes.b128 [%0], [%1];"
+                     ::"r"(clc_resp), "r"(bar_clc) : "memory");
+    };
+
+    // Producer state (thread 0 only).  The work stream of this CTA: its own unit, then static strides or the
+    // units of the CTAs it cancels.
+    int64_t unit = blockIdx.x;
+    int unit_left = unit_count(unit);      // tiles of `unit` not yet issued; 0: the next unit has to be fetched
+    int t_in = 0;                          // tiles of `unit` already issued
+    int issued = 0;                        // tiles whose TMA load the producer thread has issued
+    uint32_t clc_parity = 0;
+    bool producer_failed = false;
+    auto next_unit = [&]() -> int64_t {
+        if (!prob.dynamic) {
+            const int64_t u = unit + gridDim.x;
+            return u < prob.n_units ? u : -1;
+        }
+        if (!mbar_wait(bar_clc, clc_parity, abort_flag)) {
+            if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
+            producer_failed = true;
+            return -1;
+        }
+        clc_parity ^= 1u;
+        uint32_t valid = 0, x = 0;
+        asm volatile("{\n\t.reg .pred p1;\n\t.reg .b128 resp;\n\t"
+                     "ld.shared.b128 resp, [%2];\n\t"
+                     "clusterlaunchcontrol.query_cancel.is_canceled.pred.b128 p1, resp;\n\t"
+                     "selp.u32 %1, 1, 0, p1;\n\t"
+                     "@p1 clusterlaunchcontrol.query_cancel.get_first_ctaid.v4.b32.b128 {%0, _, _, _}, resp;\n\t}"
+                     : "+r"(x), "=r"(valid) : "r"(clc_resp) : "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the next response overwrites the buffer
+        if (!valid) return -1;                                            // refused: nothing is pending any more
+        clc_request();
+        return (int64_t)x;
+    };
+    // Issue tiles until the stream ends.  before_sync: only tiles that need neither a free slot nor a blocking
+    // request (the first NS at most).  Returns false when the stream has ended (or a wait gave up).
+    auto produce = [&](bool before_sync) -> bool {
+        for (;;) {
+            if (before_sync && issued >= NS) return true;
+            if (unit_left == 0) {
+                if (before_sync && prob.dynamic) return true;
+                unit = next_unit();
+                if (unit < 0) return false;
+                unit_left = unit_count(unit);
+                t_in = 0;
+            }
+            if (issued >= NS && !mbar_wait(bar_done(issued % NS), ((issued / NS) - 1) & 1, abort_flag)) {
+                if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
+                producer_failed = true;
+                return false;
+            }
+            issue_tile(issued, PB ? (int)unit : (int)(unit * tpu) + t_in);
+            ++issued;
+            ++t_in;
+            --unit_left;
         }
     };
 
@@ -409,11 +507,12 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     // run its set-up while this one still works (it must wait for the prerequisite grids before it touches
     // memory, as this kernel does).  Off when the library's programmatic-launch switch is off, and for
     // launches whose operand image was written by the kernel just before.
-    if (prob.early_trigger) pdl_launch_dependents();
-    int issued = 0;   // tiles whose TMA load the producer thread has issued
+    if (prob.early_trigger == 1) pdl_launch_dependents();
+    bool more = true;
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_done(s), 1); mbar_init(bar_tempty(s), 4); }
         mbar_init(bar_b, 1);
+        mbar_init(bar_clc, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -423,14 +522,22 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // (and, in the epilogue, the outputs) may not.
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
         if (PB && !WRITE_Y) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
+        if (prob.dynamic) clc_request();       // concerns this grid's own CTAs only
         if (!PB) {
             mbar_expect_tx(bar_b, kBImageBytes);
             bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
         }
+        // An L2 prefetch moves nothing into this SM: if the previous kernel still writes X, the lines it
+        // writes afterwards are updated in the same L2, so asking early is safe and keeps the memory
+        // system busy across the kernel boundary.
+        for (int k = 0; k < prob.prefetch_tiles; ++k) {
+            if (prob.dynamic && k >= tpu) break;
+            const int64_t u = blockIdx.x + (int64_t)(k / tpu) * gridDim.x;
+            if (u >= prob.n_units || k % tpu >= unit_count(u)) break;
+            prefetch_tile(PB ? (int)u : (int)(u * tpu) + k % tpu, k % tpu);
+        }
         pdl_wait_prior_grid();
-        const int first = my_tiles < NS ? my_tiles : NS;
-        for (int n = 0; n < first; ++n) issue_tile(n);
-        issued = first;
+        more = produce(true);
     }
     if (warp == 1) {
         __syncwarp();
@@ -446,13 +553,16 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            for (int n = NS; n < my_tiles; ++n) {
-                if (!mbar_wait(bar_done(n % NS), ((n / NS) - 1) & 1, abort_flag)) {
-                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
+            if (more) (void)produce(false);
+            if (prob.early_trigger == 2) pdl_launch_dependents();
+            // end of the stream: sentinel tiles (no copy, a plain arrival on the tile's barrier)
+            for (int k = 0, n = issued; k < kSentinels && !producer_failed; ++k, ++n) {
+                if (n >= NS && !mbar_wait(bar_done(n % NS), ((n / NS) - 1) & 1, abort_flag)) {
+                    if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
                     break;
                 }
-                issue_tile(n);
-                issued = n + 1;
+                ring[n % kRingEntries] = -1;
+                mbar_arrive(bar_full(n % NS));
             }
         }
     } else if (warp <= NM) {
@@ -461,7 +571,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             bool ok = true;
             if (!PB) {
                 ok = mbar_wait(bar_b, 0, abort_flag);
-                if (!ok && !*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
+                if (!ok && !*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
             }
             // descriptors of slot 0; slot s adds s*kStageBytes to the start-address field
             uint64_t b_desc[3][2];
@@ -472,15 +582,24 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     b_desc[t][kk] = smem_desc_sw64(base + (PB ? L::kAOff + kTileBytes : L::kBOff) +
                                                    t * kBTermBytes + kk * 32);
             const uint64_t a_desc0 = smem_desc_sw64(base + L::kAOff);
-            for (int n = warp - 1; ok && n < my_tiles; n += NM) {
+            int sentinels_seen = 0;
+            for (int n = warp - 1; ok; n += NM) {
                 const int s = n % NS;
                 if (!mbar_wait(bar_full(s), (n / NS) & 1, abort_flag)) {
-                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_MMA_FULL); *abort_flag = 1; }
+                    if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_MMA_FULL); *abort_flag = 1; }
                     break;
                 }
+                const bool sentinel = ring[n % kRingEntries] < 0;
+                // also before a sentinel: the slot's "done" barrier must not complete another phase before
+                // the epilogue has taken the previous one, or the epilogue's parity wait would miss it
                 if (n >= NS && !mbar_wait(bar_tempty(s), ((n / NS) - 1) & 1, abort_flag)) {
-                    if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_MMA_TMEM); *abort_flag = 1; }
+                    if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_MMA_TMEM); *abort_flag = 1; }
                     break;
+                }
+                if (sentinel) {                            // pass the end of the stream on to the epilogue
+                    mbar_arrive(bar_done(s));
+                    if (++sentinels_seen == kSentinels / NM) break;
+                    continue;
                 }
                 tc_fence_after();
                 const uint64_t slot_off = (uint64_t)((s * L::kStageBytes) >> 4);
@@ -504,12 +623,14 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
         const int e_shared = PB ? 0 : __ldg(e_norm);
         double sq_sum = 0.0;                       // CALIB: this thread's sum of squared residuals
-        for (int n = g; n < my_tiles; n += NG) {
+        for (int n = g;; n += NG) {
             const int s = n % NS;
             if (!mbar_wait(bar_done(s), (n / NS) & 1, abort_flag)) {
-                if (!*abort_flag) { atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_EPILOGUE); *abort_flag = 1; }
+                if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_EPILOGUE); *abort_flag = 1; }
                 break;
             }
+            const int item = ring[n % kRingEntries];
+            if (item < 0) break;
             tc_fence_after();
             uint32_t acc[32];
             tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * 32), acc);
@@ -518,8 +639,8 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             if (lane == 0) mbar_arrive(bar_tempty(s));
             if (PB && !WRITE_Y) {
                 int j, jg, tt;
-                pb_coords(n, j, jg, tt);
                 const int c = n % kPbCols;
+                pb_coords(item, c, j, jg, tt);
                 const int r = quarter * 32 + lane;                 // token row inside the tile
                 const uint32_t st_codes = base + L::kStoreOff;
                 const uint32_t st_scale = st_codes + kTileRows * 64;
@@ -587,13 +708,12 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 bool valid;
                 if (PB) {
                     int j, jg, tt;
-                    pb_coords(n, j, jg, tt);
+                    pb_coords(item, n % kPbCols, j, jg, tt);
                     row = (int64_t)tt * kTileRows + quarter * 32 + lane;
                     blk = row * prob.blocks_per_row + j;
                     valid = row < prob.n_rows && j < prob.blocks_per_row;
                 } else {
-                    const int64_t w = blockIdx.x + (int64_t)n * gridDim.x;
-                    row = w * kTileRows + quarter * 32 + lane;
+                    row = (int64_t)item * kTileRows + quarter * 32 + lane;
                     blk = row;
                     valid = row < prob.n_rows;
                 }
@@ -656,7 +776,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (!PB) (void)mbar_wait(bar_b, 0, &never);
         for (int m = (issued > NS ? issued - NS : 0); m < issued; ++m)
             if (!mbar_wait(bar_full(m % NS), (m / NS) & 1, &never))
-                atomicExch(&g_kq_device_error, KQ_DEV_TIMEOUT_DRAIN);
+                atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_DRAIN);
     }
     __syncthreads();
     if (warp == 1) {

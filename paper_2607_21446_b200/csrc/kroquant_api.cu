@@ -38,6 +38,10 @@ std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_umma_cfg{5};
 std::atomic<int> g_umma_ctas_per_sm{3};
 std::atomic<int> g_umma_pdl{1};
+std::atomic<int> g_umma_trigger{2};     // UmmaProblem::early_trigger of ordinary launches
+std::atomic<int> g_umma_prefetch{2};    // UmmaProblem::prefetch_tiles
+std::atomic<int> g_umma_dynamic{1};     // UmmaProblem::dynamic
+std::atomic<int> g_umma_unit_tiles{1};  // UmmaProblem::unit_tiles
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -190,8 +194,13 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA>;
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
+    // Dynamic distribution: the grid has one CTA per unit and the hardware decides how many run at once, so the
+    // number of resident CTAs per SM is set through the shared memory each CTA asks for: just too much for
+    // ctas_per_sm + 1 of them (228 KB per SM, 1 KB reserved per CTA).
+    constexpr int kSmemPerSm = 233472, kSmemReserved = 1024, kMaxDyn = kSmemPerSm / 2 - kSmemReserved + 128;
     std::call_once(once, [&] {
-        attr_rc = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynBytes);
+        attr_rc = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       L::kDynBytes > kMaxDyn ? L::kDynBytes : kMaxDyn);
     });
     if (attr_rc != cudaSuccess) return KQ_ERR_CUDA;
     const int sms = sm_count();
@@ -200,11 +209,16 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     // gets the same number of units was measured and is no faster: fewer resident CTAs hide
     // less latency than the shorter last round saves)
     const int64_t cap = (int64_t)sms * ctas_per_sm;
-    const int64_t grid = prob.n_units < cap ? prob.n_units : cap;
+    const int64_t grid = (prob.dynamic || prob.n_units < cap) ? prob.n_units : cap;
+    int smem = L::kDynBytes;
+    if (prob.dynamic) {
+        const int limit = ((kSmemPerSm / (ctas_per_sm + 1) - kSmemReserved) & ~127) + 128;
+        if (limit > smem) smem = limit;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(128 + 128 * NG);
-    cfg.dynamicSmemBytes = L::kDynBytes;
+    cfg.dynamicSmemBytes = (size_t)smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -233,18 +247,23 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     kq::UmmaProblem prob;
     prob.blocks_per_row = nb;
     prob.tiled_scales = tiled ? 1 : 0;
-    prob.early_trigger = (g_umma_pdl.load() != 0 && calib_sumsq == nullptr) ? 1 : 0;
+    prob.early_trigger = (g_umma_pdl.load() != 0 && calib_sumsq == nullptr) ? g_umma_trigger.load() : 0;
+    prob.prefetch_tiles = g_umma_pdl.load() != 0 ? g_umma_prefetch.load() : 0;
+    prob.dynamic = g_umma_dynamic.load();
+    prob.unit_tiles = pb ? kq::kPbCols : g_umma_unit_tiles.load();
     CUtensorMap tmap;
     cuuint64_t dims[2], strides[1];
     if (pb) {
         prob.n_rows = tokens;
         prob.n_ttiles = (int)((tokens + kq::kTileRows - 1) / kq::kTileRows);
         prob.n_units = (int64_t)prob.n_ttiles * ((nb + kq::kPbCols - 1) / kq::kPbCols);
+        prob.n_tiles = prob.n_units * kq::kPbCols;
         dims[0] = (cuuint64_t)d; dims[1] = (cuuint64_t)tokens; strides[0] = (cuuint64_t)d * 2;
     } else {
         prob.n_rows = tokens * (int64_t)nb;
         prob.n_ttiles = 1;
-        prob.n_units = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
+        prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
+        prob.n_units = (prob.n_tiles + prob.unit_tiles - 1) / prob.unit_tiles;
         dims[0] = 32; dims[1] = (cuuint64_t)prob.n_rows; strides[0] = 64;
     }
     const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
@@ -700,6 +719,20 @@ kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_
     g_umma_cfg.store(config);
     g_umma_ctas_per_sm.store(ctas_per_sm);
     g_umma_pdl.store(use_pdl != 0);
+    return KQ_OK;
+}
+
+kq_status_t kroquant_debug_set_boundary(int trigger, int prefetch_tiles) {
+    if (trigger < 0 || trigger > 2 || prefetch_tiles < 0 || prefetch_tiles > 64) return KQ_ERR_UNSUPPORTED;
+    g_umma_trigger.store(trigger);
+    g_umma_prefetch.store(prefetch_tiles);
+    return KQ_OK;
+}
+
+kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles) {
+    if (dynamic < 0 || dynamic > 1 || unit_tiles < 1 || unit_tiles > 16) return KQ_ERR_UNSUPPORTED;
+    g_umma_dynamic.store(dynamic);
+    g_umma_unit_tiles.store(unit_tiles);
     return KQ_OK;
 }
 
