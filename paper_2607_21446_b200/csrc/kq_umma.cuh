@@ -530,11 +530,18 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // An L2 prefetch moves nothing into this SM: if the previous kernel still writes X, the lines it
         // writes afterwards are updated in the same L2, so asking early is safe and keeps the memory
         // system busy across the kernel boundary.
-        for (int k = 0; k < prob.prefetch_tiles; ++k) {
-            if (prob.dynamic && k >= tpu) break;
-            const int64_t u = blockIdx.x + (int64_t)(k / tpu) * gridDim.x;
-            if (u >= prob.n_units || k % tpu >= unit_count(u)) break;
-            prefetch_tile(PB ? (int)u : (int)(u * tpu) + k % tpu, k % tpu);
+        {
+            int64_t u = unit;
+            int t = 0, cnt = unit_left;
+            for (int k = 0; k < prob.prefetch_tiles; ++k) {
+                prefetch_tile(PB ? (int)u : (int)(u * tpu) + t, t);
+                if (++t == cnt) {                  // the units after the first are known only with static strides
+                    u += gridDim.x;
+                    if (prob.dynamic || u >= prob.n_units) break;
+                    t = 0;
+                    cnt = unit_count(u);
+                }
+            }
         }
         pdl_wait_prior_grid();
         more = produce(true);

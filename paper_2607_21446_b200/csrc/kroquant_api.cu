@@ -286,6 +286,13 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     }
     const int cps = g_umma_ctas_per_sm.load();
     const bool pdl = g_umma_pdl.load() != 0;
+    // A launch whose units all fit the GPU at once has nothing to hand out: static distribution (no cancel
+    // request, no shared-memory padding), and the completion signal goes back to the kernel's start, where it
+    // lets the launches of a chain of very short kernels run ahead of one another.
+    if (prob.dynamic && prob.n_units <= (int64_t)sm_count() * cps) {
+        prob.dynamic = 0;
+        if (prob.early_trigger == 2) prob.early_trigger = 1;
+    }
     const uint8_t* b = f->d_bimage + (xf16 ? (size_t)f->n_sets * kq::kBImageBytes : 0);
     const int* en = f->d_enorm + (xf16 ? f->n_sets : 0);
 #define KQ_LAUNCH(NS, NM, NG, PB, XF) \
