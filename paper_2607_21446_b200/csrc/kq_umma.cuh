@@ -230,16 +230,32 @@ __device__ __forceinline__ void store_block_16bit(const uint32_t (&acc)[32], int
 // Common case: the true scale byte S = biased_exp(amax_acc) - 2 - e needs no clamping;
 // then v = acc * 2^(129 - biased_exp(amax_acc)) does not depend on e at all.  Otherwise
 // (block amax below 2^-125, or above fp32's range) the values are first brought back to y.
+// max(|a|, |b|, |c|) in one instruction (sm_100: three-input max with the .abs modifier)
+__device__ __forceinline__ float max3_abs(float a, float b, float c) {
+    float d;
+    asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// {a0 * b, a1 * b}: one packed multiply (sm_100 mul.f32x2; each half is an ordinary round-to-nearest product)
+__device__ __forceinline__ void mul2(uint32_t a0, uint32_t a1, uint64_t bb, float& r0, float& r1) {
+    uint64_t aa, d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(aa) : "r"(a0), "r"(a1));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(aa), "l"(bb));
+    uint32_t lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(d));
+    r0 = __uint_as_float(lo);
+    r1 = __uint_as_float(hi);
+}
 __device__ __forceinline__ void encode_block_regs(uint32_t (&acc)[32], int e, uint4& codes, uint32_t& S) {
-    float m[4] = {0.f, 0.f, 0.f, 0.f};      // four independent max chains
+    // amax of 32 values in 16 three-input instructions: ten over fresh triples, then a tree over their results
+    // and the two values left over
+    float m[10];
 #pragma unroll
-    for (int c = 0; c < 32; c += 4) {
-        m[0] = fmaxf(m[0], fabsf(__uint_as_float(acc[c + 0])));
-        m[1] = fmaxf(m[1], fabsf(__uint_as_float(acc[c + 1])));
-        m[2] = fmaxf(m[2], fabsf(__uint_as_float(acc[c + 2])));
-        m[3] = fmaxf(m[3], fabsf(__uint_as_float(acc[c + 3])));
-    }
-    float amax = fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+    for (int c = 0; c < 10; ++c)
+        m[c] = max3_abs(__uint_as_float(acc[3 * c]), __uint_as_float(acc[3 * c + 1]), __uint_as_float(acc[3 * c + 2]));
+    const float n0 = max3_abs(m[0], m[1], m[2]), n1 = max3_abs(m[3], m[4], m[5]), n2 = max3_abs(m[6], m[7], m[8]);
+    const float n3 = max3_abs(m[9], __uint_as_float(acc[30]), __uint_as_float(acc[31]));
+    float amax = max3_abs(max3_abs(n0, n1, n2), n3, n3);
     const int ea = (int)((__float_as_uint(amax) >> 23) & 0xFFu);
     const int s_raw = ea - 2 - e;
     float inv;
@@ -254,13 +270,15 @@ __device__ __forceinline__ void encode_block_regs(uint32_t (&acc)[32], int e, ui
         S = e8m0_from_amax(amax);
         inv = inv_scale_from_e8m0(S);
     }
+    uint64_t inv2;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(inv2) : "r"(__float_as_uint(inv)));
     uint32_t w[4];
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
-        w[g] = e2m1x8(__uint_as_float(acc[8 * g + 0]) * inv, __uint_as_float(acc[8 * g + 1]) * inv,
-                      __uint_as_float(acc[8 * g + 2]) * inv, __uint_as_float(acc[8 * g + 3]) * inv,
-                      __uint_as_float(acc[8 * g + 4]) * inv, __uint_as_float(acc[8 * g + 5]) * inv,
-                      __uint_as_float(acc[8 * g + 6]) * inv, __uint_as_float(acc[8 * g + 7]) * inv);
+        float v[8];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) mul2(acc[8 * g + 2 * h], acc[8 * g + 2 * h + 1], inv2, v[2 * h], v[2 * h + 1]);
+        w[g] = e2m1x8(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7]);
     }
     codes = make_uint4(w[0], w[1], w[2], w[3]);
 }
@@ -328,6 +346,7 @@ struct UmmaProblem {
     int early_trigger;   // 0: never; 1: signal programmatic launch completion at the start of the kernel;
                          // 2: each CTA signals once its producer has no tile left to issue
     int prefetch_tiles;  // tiles of X each CTA asks the L2 for before it waits for the prerequisite grids
+    int prefetch_stride; // dynamic distribution: number of CTAs that run at once (see the prefetch loop)
     int64_t n_tiles;     // PB=false: 128-row tiles
     int unit_tiles;      // PB=false: consecutive tiles per work unit (PB: kPbCols)
     int dynamic;         // 1: the grid has one CTA per unit and running CTAs take over the units of CTAs that
@@ -530,18 +549,23 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // An L2 prefetch moves nothing into this SM: if the previous kernel still writes X, the lines it
         // writes afterwards are updated in the same L2, so asking early is safe and keeps the memory
         // system busy across the kernel boundary.
-        {
+        // (With dynamic distribution nobody knows who will take the units after the first wave; the CTAs of the
+        // first wave ask for them by position, prefetch_stride = number of CTAs that run at once: the L2 is shared.)
+        if (!prob.dynamic || (int64_t)blockIdx.x < prob.prefetch_stride) {
+            const int64_t stride = prob.dynamic ? prob.prefetch_stride : (int64_t)gridDim.x;
             int64_t u = unit;
             int t = 0, cnt = unit_left;
             for (int k = 0; k < prob.prefetch_tiles; ++k) {
                 prefetch_tile(PB ? (int)u : (int)(u * tpu) + t, t);
-                if (++t == cnt) {                  // the units after the first are known only with static strides
-                    u += gridDim.x;
-                    if (prob.dynamic || u >= prob.n_units) break;
+                if (++t == cnt) {
+                    u += stride;
+                    if (u >= prob.n_units) break;
                     t = 0;
                     cnt = unit_count(u);
                 }
             }
+        } else if (prob.prefetch_tiles > 0) {
+            prefetch_tile(PB ? (int)unit : (int)(unit * tpu), 0);
         }
         pdl_wait_prior_grid();
         more = produce(true);

@@ -289,6 +289,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     // A launch whose units all fit the GPU at once has nothing to hand out: static distribution (no cancel
     // request, no shared-memory padding), and the completion signal goes back to the kernel's start, where it
     // lets the launches of a chain of very short kernels run ahead of one another.
+    prob.prefetch_stride = sm_count() * cps;
     if (prob.dynamic && prob.n_units <= (int64_t)sm_count() * cps) {
         prob.dynamic = 0;
         if (prob.early_trigger == 2) prob.early_trigger = 1;
