@@ -88,6 +88,28 @@ def test_multi_tile_ctas_against_the_oracle(B, mode):
     assert B.kroquant_last_device_error() == 0
 
 
+def test_dynamic_launches_that_overlap_on_two_streams(B):
+    """A running CTA may only take over CTAs of its own grid: two dynamic launches that share the GPU must
+    each produce their own complete result."""
+    set_mode(B, MODES[3])
+    shapes = [(4608, 3072), (3000, 2240)]
+    X = [dev(W.gen_activations(spec(t, d, 40 + i))) for i, (t, d) in enumerate(shapes)]
+    f = [B.Factors.create(W.gen_factors(50 + i)) for i in range(2)]
+    ref = [B.kroquant_quantize(X[i], f[i], path="tensor") for i in range(2)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    outs = [[], []]
+    for rep in range(12):
+        for i in range(2):
+            with torch.cuda.stream(streams[i]):
+                outs[i].append(B.kroquant_quantize(X[i], f[i], path="tensor", stream=streams[i]))
+    torch.cuda.synchronize()
+    for i in range(2):
+        for q, s in outs[i]:
+            assert torch.equal(q, ref[i][0]) and torch.equal(s, ref[i][1])
+    assert B.kroquant_last_device_error() == 0
+
+
 def test_knob_ranges(B):
     for args in [(-1, 0), (3, 0), (0, -1), (0, 65)]:
         with pytest.raises(RuntimeError):
