@@ -187,7 +187,8 @@ struct UmmaSmem {
     static constexpr int kNumBars = 3 * NS + 2;
     static constexpr int kClcOff = kBarOff + ((8 * kNumBars + 15) & ~15);     // 16-byte response of a cancel request
     static constexpr int kRingOff = kClcOff + 16;                             // kRingEntries ints: work item of local tile n
-    static constexpr int kTmemSlotOff = kRingOff + 4 * kRingEntries;
+    static constexpr int kRing2Off = kRingOff + 4 * kRingEntries;             // PB: column group of local tile n
+    static constexpr int kTmemSlotOff = kRing2Off + 4 * kRingEntries;
     static constexpr int kAbortOff = kTmemSlotOff + 4;
     static constexpr int kBytes = kAbortOff + 4;
     static constexpr int kDynBytes = kBytes + 1024;                  // slack for manual alignment
@@ -416,6 +417,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     // sentinel tiles at the end of the stream: every MMA warp gets the same number, every epilogue group at least one
     constexpr int kSentinels = ((NM > NG ? NM : NG) + NM - 1) / NM * NM;
     volatile int* ring = reinterpret_cast<volatile int*>(base_ptr + L::kRingOff);
+    volatile int* ring_jg = reinterpret_cast<volatile int*>(base_ptr + L::kRing2Off);
     const uint32_t bar_clc = bar0 + 8u * (3 * NS + 1);
     const uint32_t clc_resp = base + L::kClcOff;
     const int tpu = PB ? kPbCols : prob.unit_tiles;                   // tiles per unit
@@ -428,15 +430,19 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         j = jg * kPbCols + c;
     };
     // issue the TMA copies of local tile n into slot n % NS (producer thread only); item = global tile index
-    // (PB: unit index, the column is n % kPbCols)
+    // (PB: unit index, the column is n % kPbCols).  The ring tells the consumers what the tile is: the global
+    // tile index, or (PB) token tile and column group, so that only this thread divides.
     auto issue_tile = [&](int n, int item) {
         const int s = n % NS;
         const uint32_t dst = base + L::kAOff + s * L::kStageBytes;
-        ring[n % kRingEntries] = item;
+        int j = 0, jg = 0, tt = 0;
+        if (PB) {
+            pb_coords(item, n % kPbCols, j, jg, tt);
+            ring_jg[n % kRingEntries] = jg;
+        }
+        ring[n % kRingEntries] = PB ? tt : item;
         mbar_expect_tx(bar_full(s), L::kStageBytes);
         if (PB) {
-            int j, jg, tt;
-            pb_coords(item, n % kPbCols, j, jg, tt);
             const int jb = j < prob.blocks_per_row ? j : prob.blocks_per_row - 1;
             tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));      // zero-filled if j is out of range
             bulk_load(dst + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(s));
@@ -652,7 +658,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
-        const int e_shared = PB ? 0 : __ldg(e_norm);
+        const int e_shared = (PB || !XF16) ? 0 : __ldg(e_norm);
         double sq_sum = 0.0;                       // CALIB: this thread's sum of squared residuals
         for (int n = g;; n += NG) {
             const int s = n % NS;
@@ -669,16 +675,16 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_tempty(s));
             if (PB && !WRITE_Y) {
-                int j, jg, tt;
                 const int c = n % kPbCols;
-                pb_coords(item, c, j, jg, tt);
+                const int tt = item, jg = ring_jg[n % kRingEntries], j = jg * kPbCols + c;
                 const int r = quarter * 32 + lane;                 // token row inside the tile
                 const uint32_t st_codes = base + L::kStoreOff;
                 const uint32_t st_scale = st_codes + kTileRows * 64;
                 const bool elected = threadIdx.x == 128;
                 uint4 codes;
                 uint32_t S;
-                const int e_j = __ldg(e_norm + (j < prob.blocks_per_row ? j : 0));
+                // (bf16 images carry no normalisation exponent)
+                const int e_j = XF16 ? __ldg(e_norm + (j < prob.blocks_per_row ? j : 0)) : 0;
                 if (DUAL && j < prob.blocks_per_row &&
                     (int64_t)tt * kTileRows + r < prob.n_rows)
                     store_block_16bit<XF16>(acc, e_j, at_out + (((int64_t)tt * kTileRows + r) * prob.blocks_per_row + j) * 4);
@@ -738,8 +744,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 int64_t row, blk;       // row inside the tiled dimension; flat index of the 32-channel block
                 bool valid;
                 if (PB) {
-                    int j, jg, tt;
-                    pb_coords(item, n % kPbCols, j, jg, tt);
+                    const int tt = item, j = ring_jg[n % kRingEntries] * kPbCols + n % kPbCols;
                     row = (int64_t)tt * kTileRows + quarter * 32 + lane;
                     blk = row * prob.blocks_per_row + j;
                     valid = row < prob.n_rows && j < prob.blocks_per_row;
@@ -749,7 +754,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     valid = row < prob.n_rows;
                 }
                 if (valid) {
-                    const int e = PB ? __ldg(e_norm + (int)(blk % prob.blocks_per_row)) : e_shared;
+                    const int e = (PB && XF16) ? __ldg(e_norm + (int)(blk % prob.blocks_per_row)) : e_shared;
                     if (WRITE_Y) {
                         const float back = __uint_as_float((uint32_t)(127 - e) << 23);    // 2^-e
                         float* yp = Y + blk * 32;
