@@ -178,10 +178,12 @@ struct UmmaSmem {
     static constexpr int kStageBytes = kTileBytes + (PB ? kBImageBytes : 0);   // multiple of 1024
     static constexpr int kBOff = 0;                                  // shared image (PB = false)
     static constexpr int kAOff = PB ? 0 : 8192;                      // NS stages
-    // PB only: staging of one column group's outputs: 128 rows x 64 B of codes (64-byte
-    // swizzle, leaves by TMA store) and 128 x 4 scale bytes
+    // PB only: staging of a column group's outputs: 128 rows x 64 B of codes (64-byte
+    // swizzle, leaves by TMA store) and 128 x 4 scale bytes; two tiles, so that a group can be staged while
+    // the TMA store of the group before still reads its tile
     static constexpr int kStoreOff = kAOff + NS * kStageBytes;
-    static constexpr int kStoreBytes = PB ? (kTileRows * 64 + kTileRows * 4) : 0;
+    static constexpr int kStoreTile = kTileRows * 64 + kTileRows * 4;          // one staging tile
+    static constexpr int kStoreBytes = PB ? 2 * kStoreTile : 0;                // two of them, used alternately
     static constexpr int kBarOff = kStoreOff + kStoreBytes;
     // barriers: full[NS], done[NS], tempty[NS], bfull, clc
     static constexpr int kNumBars = 3 * NS + 2;
@@ -678,7 +680,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 const int c = n % kPbCols;
                 const int tt = item, jg = ring_jg[n % kRingEntries], j = jg * kPbCols + c;
                 const int r = quarter * 32 + lane;                 // token row inside the tile
-                const uint32_t st_codes = base + L::kStoreOff;
+                const uint32_t st_codes = base + L::kStoreOff + (uint32_t)((n / kPbCols) & 1) * L::kStoreTile;
                 const uint32_t st_scale = st_codes + kTileRows * 64;
                 const bool elected = threadIdx.x == 128;
                 uint4 codes;
@@ -693,11 +695,6 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     const int64_t blk_c = ((int64_t)tt * kTileRows + r) * prob.blocks_per_row + j;
                     sq_sum += (double)store_block_calib(acc, codes, S, at_out + blk_c * 4, Y + blk_c * 32);
                 }
-                if (c == 0) {
-                    // the previous group's TMA store must have finished reading the staging tile
-                    if (elected) bulk_wait_group_read<0>();
-                    named_barrier_sync(1, 128);
-                }
                 // 64-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3)
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
                              ::"r"(st_codes + 64u * r + 16u * (uint32_t)(c ^ ((r >> 1) & 3))),
@@ -710,6 +707,10 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                                                          : (uint32_t)(4 * r + c);
                 asm volatile("st.shared.u8 [%0], %1;" ::"r"(st_scale + s_off), "r"(S_st) : "memory");
                 if (c == kPbCols - 1) {
+                    // One barrier per group.  Before it the elected thread makes sure that the store of the
+                    // group before (issued a whole group ago) has finished reading the other staging tile, so
+                    // past the barrier every thread may write there.
+                    if (elected) bulk_wait_group_read<0>();
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     named_barrier_sync(1, 128);
                     if (elected) {
