@@ -352,6 +352,11 @@ def run_ours(args):
                                stream)
     B.kroquant_debug_set_distribution(True, 1)
     ms_ovl, _ = time_graph(torch, None, g_ovl, stream, args.steps, 3)
+    # the headline step again right after an idle second (not the headline: it shows what the 1 kW power cap
+    # costs; the timed region above starts only after seconds of load, with the SM clock already lowered)
+    torch.cuda.synchronize()
+    time.sleep(1.5)
+    ms_burst, _ = time_graph(torch, None, g_kq, stream, min(args.steps, 50), 3)
     # end to end: pinned host inputs -> device -> quantize -> pinned host outputs
     e2e_steps = max(1, min(args.steps, 3))
     hx = [torch.empty(c["X"].shape, dtype=torch.bfloat16).pin_memory() for c in calls[:2]]
@@ -421,6 +426,11 @@ def run_ours(args):
         "frac_of_hbm_peak": value / world / peak,
         "speedup_vs_scale_kernel": ms_scale / ms_step,
         "speedup_vs_plain_mxfp4": ms_plain / ms_step,
+        "after_idle": {
+            "ms_per_step": round(ms_burst, 5), "GB/s": round(byts / (ms_burst * 1e-3) / 1e9, 1),
+            "frac_of_hbm_peak": round(byts / (ms_burst * 1e-3) / 1e9 / peak, 4),
+            "note": "the same graph, 3 warm-up + at most 50 timed steps after 1.5 s of idle: before the power cap "
+                    "lowers the SM clock; not the headline"},
         "independent_calls_overlapped": {
             "ms_per_step": round(ms_ovl, 5), "GB/s": round(byts / (ms_ovl * 1e-3) / 1e9, 1),
             "frac_of_hbm_peak": round(byts / (ms_ovl * 1e-3) / 1e9 / peak, 4),
