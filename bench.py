@@ -40,7 +40,7 @@ SHAPES = [(4608, 3072), (4608, 12288)]
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch of the tensor-core kernel from the Nsight Compute captures
 # summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
-NCU_TRAFFIC_BYTES = {(4608, 3072): 28.35e6, (4608, 12288): 125.5e6}
+NCU_TRAFFIC_BYTES = {(4608, 3072): 28.36e6, (4608, 12288): 125.3e6}
 
 
 def measured_peak():
