@@ -762,23 +762,31 @@ def run_layer(args):
     q = torch.empty((t, d // 2), dtype=torch.uint8, device="cuda")
     sc = torch.zeros(B.tiled_scale_bytes(t, d), dtype=torch.uint8, device="cuda")
 
+    stream = torch.cuda.Stream()
+    per_graph = 2 * nbuf
+
     def timed(fn):
-        for i in range(max(args.warmup, 3)):
-            fn(i % nbuf)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for i in range(args.steps):
-            fn(i % nbuf)
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / args.steps * 1e3
+        """One CUDA graph of 2 * nbuf calls over the rotating buffers, replayed: the host's launch cost
+        (about 10 us per call from Python) stays out of the number."""
+        g = capture(torch, [lambda i=i: fn(i % nbuf) for i in range(per_graph)], stream)
+        reps = max(1, args.steps // per_graph)
+        with torch.cuda.stream(stream):
+            for _ in range(max(args.warmup, 3)):
+                g.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(reps):
+                g.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / (reps * per_graph) * 1e3
 
     l0 = B.kroquant_launch_count()
-    us_layer = timed(lambda i: layer(Xs[i], out=outs[i]))
-    launches = B.kroquant_launch_count() - l0
-    us_quant = timed(lambda i: B.kroquant_quantize(Xs[i], layer.factors, q, sc, scale_layout="tiled"))
-    us_gemm = timed(lambda i: B.kroquant_gemm_mxfp4(q, sc, layer.w_codes, layer.w_scales, out=outs[i]))
+    us_layer = timed(lambda i: layer(Xs[i], out=outs[i], stream=stream))
+    launches = (B.kroquant_launch_count() - l0) / 2 / per_graph      # eager pass + captured pass
+    us_quant = timed(lambda i: B.kroquant_quantize(Xs[i], layer.factors, q, sc, scale_layout="tiled", stream=stream))
+    us_gemm = timed(lambda i: B.kroquant_gemm_mxfp4(q, sc, layer.w_codes, layer.w_scales, out=outs[i], stream=stream))
     us_bf16 = timed(lambda i: torch.matmul(Xs[i], Wt.t(), out=outs[i]))
     flop = 2.0 * t * o * d
     print(json.dumps({
@@ -787,7 +795,7 @@ def run_layer(args):
         "dtype": "bf16 activations -> MXFP4 x MXFP4, fp32 accumulate, bf16 output",
         "config": {"workload": f"linear layer tokens={t} d={d} o={o}, n_sets={G.shape[0]}",
                    "l2": f"{nbuf} rotating input/output buffer pairs ({nbuf * t * (d + o) * 2 / 1e6:.0f} MB)"},
-        "gpu_launches": int(launches), "launches_per_step": launches / (args.steps + max(args.warmup, 3)),
+        "gpu_launches": int(round(launches * per_graph * max(1, args.steps // per_graph))), "launches_per_step": launches,
         "quantizer_us": round(us_quant, 2), "w4a4_gemm_us": round(us_gemm, 2), "cublas_bf16_gemm_us": round(us_bf16, 2),
         "speedup_vs_bf16_gemm": round(us_bf16 / us_layer, 3), "effective_tflops": round(flop / us_layer / 1e6, 1),
         "device_error": B.kroquant_last_device_error()}), flush=True)
