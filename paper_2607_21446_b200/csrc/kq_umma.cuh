@@ -386,7 +386,7 @@ struct UmmaProblem {
 // from the default kernel.
 constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
 template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone>
-__global__ void __launch_bounds__(128 + 128 * NG, 1)
+__global__ void __launch_bounds__(128 + 128 * NG, (NS == 8 && NG == 2) ? 2 : 1)      // (8,2,2) runs two per SM
 quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
               const uint8_t* __restrict__ b_image, const int* __restrict__ e_norm, const UmmaProblem prob,
               uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y,
@@ -395,6 +395,9 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     constexpr bool CALIB = EXTRA == kExtraCalib;
     static_assert(!CALIB || (!XF16 && !WRITE_Y), "calibration outputs: bf16 images, quantizing path");
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
+    // TMEM is handed out in powers of two
+    constexpr int kTmemCols = NS * 32 <= 32 ? 32 : NS * 32 <= 64 ? 64 : NS * 32 <= 128 ? 128 : NS * 32 <= 256 ? 256 : 512;
+    static_assert(NS * 32 <= 512, "at most 16 accumulators of 32 columns");
     // A slot must always be served by the same issuer warp and the same epilogue group:
     // only then does program order inside that warp guarantee that a parity wait never
     // runs a whole phase ahead of the barrier it polls.
@@ -581,7 +584,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     if (warp == 1) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(base + (uint32_t)L::kTmemSlotOff), "r"((uint32_t)(NS * 32)) : "memory");
+                     ::"r"(base + (uint32_t)L::kTmemSlotOff), "r"((uint32_t)kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -820,7 +823,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                     ::"r"(tmem_base), "r"((uint32_t)(NS * 32)) : "memory");
+                     ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
     }
 }
 

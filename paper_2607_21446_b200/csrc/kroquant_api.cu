@@ -35,13 +35,17 @@ namespace {
 std::atomic<int64_t> g_launches{0};
 
 // ---- tensor-core kernel configuration ----------------------------------------
-std::atomic<int> g_umma_cfg{5};
-std::atomic<int> g_umma_ctas_per_sm{3};
+// Defaults (measured on the 28-call FLUX step): the shared-factor bf16 kernel runs as (8 slots, 2 MMA warps,
+// 2 epilogue warpgroups) with 2 CTAs per SM, every other variant as compiled for it with 3 CTAs per SM.
+// ctas_per_sm 0 = that automatic choice; kroquant_debug_set_umma_config makes both explicit for all variants.
+std::atomic<int> g_umma_cfg{2};
+std::atomic<int> g_umma_ctas_per_sm{0};
 std::atomic<int> g_umma_pdl{1};
 std::atomic<int> g_umma_trigger{2};     // UmmaProblem::early_trigger of ordinary launches
-std::atomic<int> g_umma_prefetch{2};    // UmmaProblem::prefetch_tiles
+std::atomic<int> g_umma_prefetch{4};    // UmmaProblem::prefetch_tiles
 std::atomic<int> g_umma_dynamic{1};     // UmmaProblem::dynamic
-std::atomic<int> g_umma_unit_tiles{1};  // UmmaProblem::unit_tiles
+std::atomic<int> g_umma_unit_tiles{3};  // UmmaProblem::unit_tiles
+std::atomic<int> g_umma_unit_auto{1};   // 1: small launches use single-tile units (until the caller sets the unit)
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -263,6 +267,8 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
         prob.n_rows = tokens * (int64_t)nb;
         prob.n_ttiles = 1;
         prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
+        // units of several tiles save cancel requests, but a launch of a few tiles per CTA wants them spread out
+        if (g_umma_unit_auto.load() && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
         prob.n_units = (prob.n_tiles + prob.unit_tiles - 1) / prob.unit_tiles;
         dims[0] = 32; dims[1] = (cuuint64_t)prob.n_rows; strides[0] = 64;
     }
@@ -284,7 +290,13 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return KQ_ERR_CUDA;
     }
-    const int cps = g_umma_ctas_per_sm.load();
+    const bool main_variant = !pb && calib_sumsq == nullptr;      // shared factor set: bf16 or fp16, one or two outputs
+    const int cps_set = g_umma_ctas_per_sm.load();
+    // (a launch that fits the GPU in one wave of the smaller CTAs keeps those: more of them run at once)
+    // (the fp16 two-output kernel would spill registers at two large CTAs per SM)
+    const bool big_ctas = main_variant && !(xf16 && at_out != nullptr && !WRITE_Y) && cps_set == 0 &&
+                          prob.n_tiles > (int64_t)3 * sm_count();
+    const int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
     const bool pdl = g_umma_pdl.load() != 0;
     // A launch whose units all fit the GPU at once has nothing to hand out: static distribution (no cancel
     // request, no shared-memory padding), and the completion signal goes back to the kernel's start, where it
@@ -311,9 +323,11 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     }
     if (!WRITE_Y && at_out != nullptr) {
         if (xf16) return pb ? KQ_LAUNCH_DUAL(4, 1, 1, true, true) : KQ_LAUNCH_DUAL(4, 2, 1, false, true);
-        return pb ? KQ_LAUNCH_DUAL(4, 1, 1, true, false) : KQ_LAUNCH_DUAL(4, 2, 1, false, false);
+        return pb ? KQ_LAUNCH_DUAL(4, 1, 1, true, false)
+                  : big_ctas ? KQ_LAUNCH_DUAL(8, 2, 2, false, false) : KQ_LAUNCH_DUAL(4, 2, 1, false, false);
     }
-    if (xf16) return pb ? KQ_LAUNCH(4, 1, 1, true, true) : KQ_LAUNCH(4, 2, 1, false, true);
+    if (xf16) return pb ? KQ_LAUNCH(4, 1, 1, true, true)
+                        : big_ctas ? KQ_LAUNCH(8, 2, 2, false, true) : KQ_LAUNCH(4, 2, 1, false, true);
     if (pb) {
         switch (g_umma_cfg.load()) {
             default:
@@ -322,7 +336,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
             case 1: return KQ_LAUNCH(8, 2, 1, true, false);
         }
     }
-    switch (g_umma_cfg.load()) {
+    switch (cps_set == 0 && !big_ctas ? 5 : g_umma_cfg.load()) {
         default:
         case 0: return KQ_LAUNCH(2, 2, 1, false, false);
         case 1: return KQ_LAUNCH(8, 2, 1, false, false);
@@ -741,6 +755,7 @@ kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles) {
     if (dynamic < 0 || dynamic > 1 || unit_tiles < 1 || unit_tiles > 16) return KQ_ERR_UNSUPPORTED;
     g_umma_dynamic.store(dynamic);
     g_umma_unit_tiles.store(unit_tiles);
+    g_umma_unit_auto.store(0);
     return KQ_OK;
 }
 
