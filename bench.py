@@ -445,7 +445,7 @@ def run_ours(args):
         "gpu_launches": n_launch,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                     "kernel": "quantize_umma<4,2,1,false,false>", "launches": n_launch,
+                     "kernel": "quantize_umma<8,2,2,false,false>", "launches": n_launch,
                      "avg_launch_us": us_per_launch, "algorithmic_bytes_per_launch": alg_per_launch},
         "cpu_baseline": {"value": cpu_gbs, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{SAMPLE}, {cpu_dt:.2f} s per pass, 5 passes, "
