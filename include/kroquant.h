@@ -173,7 +173,10 @@ kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes,
 
 /* Tuning hook for the tensor-core kernel.  config 0..7 selects (pipeline slots, MMA
  * issuer warps, epilogue warpgroups) = (2,2,1) (8,2,1) (8,2,2) (2,1,1) (4,1,1) (4,2,1)
- * (16,2,2) (16,2,4); the default is config 5 with 3 CTAs per SM; ctas_per_sm in 1..8 is the number of CTAs
+ * (16,2,2) (16,2,4).  Until this function is called the library chooses by itself: (8,2,2) with 2 CTAs per SM
+ * for shared-factor launches of more than one wave, (4,2,1) with 3 per SM otherwise (per-block sets: (4,1,1));
+ * a call with ctas_per_sm > 0 makes config and ctas_per_sm explicit for every variant, ctas_per_sm = 0 returns
+ * to the automatic choice (config is then ignored unless it is the default 2).  ctas_per_sm in 1..8 is the number of CTAs
  * that run on an SM at once (a cap on the persistent grid with the static distribution, a shared-memory
  * request that lets no more of them fit with the dynamic one); use_pdl != 0 (default) launches the quantizer
  * kernels with programmatic stream serialization and lets them signal launch completion before they end
@@ -192,18 +195,19 @@ kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_
  * kernel's CTAs become resident shortly before this one ends.  prefetch_tiles (0..64):
  * before a CTA waits for its prerequisite grids it asks the L2 cache for its first prefetch_tiles tiles of
  * X (a prefetch moves no data into the SM and the L2 is where the previous kernel's writes land, so the
- * request is safe even if that kernel still produces X).  Defaults: trigger 2, prefetch_tiles 2; a launch
+ * request is safe even if that kernel still produces X).  Defaults: trigger 2, prefetch_tiles 4; a launch
  * whose tiles all run at once signals at its start whatever the setting (unless trigger is 0).
  * KQ_ERR_UNSUPPORTED outside the ranges.  Process-wide. */
 kq_status_t kroquant_debug_set_boundary(int trigger, int prefetch_tiles);
 
 /* How the tensor-core quantizer hands its tiles (128 blocks of 32 channels) to CTAs.  A unit is unit_tiles
- * (1..16) consecutive tiles (always 4 column tiles with per-block factor sets).  dynamic = 0: a persistent
+ * (1..16, or 0 = automatic) consecutive tiles (always 4 column tiles with per-block factor sets).  dynamic = 0: a persistent
  * grid of at most ctas_per_sm CTAs per SM, CTA b takes units b, b + grid, ...  dynamic = 1: one CTA per unit
  * in the grid; the CTAs that the hardware starts first take over, besides their own unit, the units of CTAs
  * that have not started (cluster launch control), so that a CTA on a slower path to memory simply takes fewer.
- * Results do not depend on either setting.  Default: dynamic, 1 tile per unit; a launch whose units all fit the
- * GPU at once uses the static form.  The dynamic form is the faster one for calls that follow one another in a
+ * Results do not depend on either setting.  Default: dynamic, 3 tiles per unit (1 for launches of fewer than 8
+ * tiles per SM; unit_tiles = 0 selects that automatic rule again); a launch whose units all fit the GPU at once
+ * uses the static form.  The dynamic form is the faster one for calls that follow one another in a
  * stream; calls that are meant to overlap on several streams want the static one, because a dynamic launch
  * claims every CTA slot of the GPU.  KQ_ERR_UNSUPPORTED outside the ranges.  Process-wide. */
 kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles);

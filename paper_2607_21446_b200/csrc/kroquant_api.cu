@@ -737,7 +737,7 @@ kq_status_t kroquant_debug_e2m1_codes(const float* v, int64_t n, uint8_t* codes,
 }
 
 kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl) {
-    if (config < 0 || config > 7 || ctas_per_sm < 1 || ctas_per_sm > 8) return KQ_ERR_UNSUPPORTED;
+    if (config < 0 || config > 7 || ctas_per_sm < 0 || ctas_per_sm > 8) return KQ_ERR_UNSUPPORTED;
     g_umma_cfg.store(config);
     g_umma_ctas_per_sm.store(ctas_per_sm);
     g_umma_pdl.store(use_pdl != 0);
@@ -752,10 +752,10 @@ kq_status_t kroquant_debug_set_boundary(int trigger, int prefetch_tiles) {
 }
 
 kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles) {
-    if (dynamic < 0 || dynamic > 1 || unit_tiles < 1 || unit_tiles > 16) return KQ_ERR_UNSUPPORTED;
+    if (dynamic < 0 || dynamic > 1 || unit_tiles < 0 || unit_tiles > 16) return KQ_ERR_UNSUPPORTED;
     g_umma_dynamic.store(dynamic);
-    g_umma_unit_tiles.store(unit_tiles);
-    g_umma_unit_auto.store(0);
+    g_umma_unit_tiles.store(unit_tiles > 0 ? unit_tiles : 3);
+    g_umma_unit_auto.store(unit_tiles > 0 ? 0 : 1);
     return KQ_OK;
 }
 

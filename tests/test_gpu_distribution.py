@@ -20,9 +20,9 @@ def B():
     from paper_2607_21446_b200 import binding
     binding.load_library()
     yield binding
-    binding.kroquant_debug_set_distribution(True, 1)
-    binding.kroquant_debug_set_boundary(2, 2)
-    binding.kroquant_debug_set_umma_config(5, 3, True)
+    binding.kroquant_debug_set_distribution(True, 0)         # back to the library's own choices
+    binding.kroquant_debug_set_boundary(2, 4)
+    binding.kroquant_debug_set_umma_config(2, 0, True)
 
 
 def dev(bits):
@@ -34,14 +34,15 @@ def spec(tokens, d, seed):
                             outlier_gain=50.0, spike_rows=min(2, tokens), spike_gain=8.0)
 
 
-# (dynamic, unit_tiles, trigger, prefetch_tiles, ctas_per_sm)
-MODES = [(False, 1, 1, 0, 3), (False, 3, 2, 4, 3), (False, 2, 0, 1, 2), (True, 1, 2, 2, 3), (True, 2, 1, 0, 3),
-         (True, 4, 0, 3, 2), (True, 1, 2, 1, 4), (True, 16, 2, 64, 1)]
+# (dynamic, unit_tiles, trigger, prefetch_tiles, ctas_per_sm, config); unit_tiles 0 and ctas_per_sm 0: automatic
+MODES = [(False, 1, 1, 0, 3, 5), (False, 3, 2, 4, 3, 5), (False, 2, 0, 1, 2, 5), (True, 1, 2, 2, 3, 5), (True, 2, 1, 0, 3, 5),
+         (True, 4, 0, 3, 2, 5), (True, 1, 2, 1, 4, 5), (True, 16, 2, 64, 1, 5), (True, 0, 2, 4, 0, 2), (True, 3, 2, 4, 2, 2),
+         (False, 1, 1, 0, 2, 2), (True, 5, 1, 2, 2, 1)]
 
 
 def set_mode(B, mode):
-    dyn, unit, trigger, prefetch, cps = mode
-    B.kroquant_debug_set_umma_config(5, cps, True)
+    dyn, unit, trigger, prefetch, cps, cfg = mode
+    B.kroquant_debug_set_umma_config(cfg, cps, True)
     B.kroquant_debug_set_boundary(trigger, prefetch)
     B.kroquant_debug_set_distribution(dyn, unit)
 
@@ -73,7 +74,7 @@ def test_every_mode_gives_the_same_bits(B, tokens, d, per_block):
         assert B.kroquant_last_device_error() == 0, mode
 
 
-@pytest.mark.parametrize("mode", [MODES[0], MODES[3], MODES[5]])
+@pytest.mark.parametrize("mode", [MODES[0], MODES[3], MODES[5], MODES[8], MODES[9]])
 def test_multi_tile_ctas_against_the_oracle(B, mode):
     tokens, d = 1500, 3072           # 1125 tiles: 2 to 3 per CTA of a 444-CTA grid, ragged last tile
     Xb = W.gen_activations(spec(tokens, d, 11))
@@ -114,6 +115,6 @@ def test_knob_ranges(B):
     for args in [(-1, 0), (3, 0), (0, -1), (0, 65)]:
         with pytest.raises(RuntimeError):
             B.kroquant_debug_set_boundary(*args)
-    for args in [(True, 0), (True, 17)]:
+    for args in [(True, -1), (True, 17)]:
         with pytest.raises(RuntimeError):
             B.kroquant_debug_set_distribution(*args)
