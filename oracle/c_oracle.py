@@ -25,17 +25,12 @@ def lib() -> C.CDLL:
         L.kq_oracle_dense_k.restype = None
         L.kq_oracle_dense_kinv.argtypes = [vp, vp]
         L.kq_oracle_dense_kinv.restype = None
-        L.kq_oracle_transform.argtypes = [vp, i64, i32, vp, i32, vp]
         L.kq_oracle_transform_x.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp]
         L.kq_oracle_scale_transform_x.argtypes = [vp, i32, i64, i32, vp, vp]
         L.kq_oracle_widen_x.argtypes = [vp, i32, i64, i32, vp]
-        L.kq_oracle_scale_transform.argtypes = [vp, i64, i32, vp, vp]
-        L.kq_oracle_widen.argtypes = [vp, i64, i32, vp]
         L.kq_oracle_encode_block.argtypes = [vp, vp, vp]
         L.kq_oracle_encode_block.restype = None
         L.kq_oracle_mx_encode.argtypes = [vp, i64, i32, vp, vp]
-        L.kq_oracle_quantize.argtypes = [vp, i64, i32, vp, i32, vp, vp, vp]
-        L.kq_oracle_scale_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
         L.kq_oracle_dequantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, i32]
         L.kq_oracle_hadamard_transform_x.argtypes = [vp, i32, i64, i32, vp]
         L.kq_oracle_round_y_to_16bit.argtypes = [vp, i64, i32, vp]

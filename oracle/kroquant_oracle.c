@@ -26,9 +26,23 @@
  * double in ascending index order; the transformed value is rounded once to
  * float ("pre-rounding value"), and everything after that is exact in float.
  *
- * Parity pins: every function here is pinned by tests/test_oracle_*.py
- * (closed forms, hand-worked encodings, brute force, invariants); nothing is
- * "parity unpinned".
+ * Parity pins (tests/test_oracle_*.py), function by function:
+ *   kq_oracle_lu_to_factors         L U product written out, det = -1, |det K| = 1
+ *   kq_oracle_dense_k               np.kron chain; two shear hand vectors (factor <-> bit order, row-vector
+ *                                   convention); Hadamard closed form (-1)^popcount(r & c) / sqrt(32)
+ *   kq_oracle_dense_kinv            K K^-1 = I; numpy.linalg.inv
+ *   kq_oracle_transform_x           exact rational (Fraction) sums; pair form P^T X Q and five-stage butterfly
+ *   kq_oracle_scale_transform_x,
+ *   kq_oracle_widen_x               NumPy casts (one correctly rounded product / exact widening)
+ *   kq_oracle_encode_block,
+ *   kq_oracle_mx_encode             hand-worked blocks (tests/golden/mxfp4_handworked.txt); brute force over every
+ *                                   bf16 value in (-8, 8) with exact rationals; tie table; invariants
+ *   kq_oracle_dequantize            the E2M1 grid written out; numpy.linalg.inv round trip; torch's bf16 cast
+ *   kq_oracle_hadamard_transform_x  scipy's Sylvester matrix
+ *   kq_oracle_round_y_to_16bit      NumPy / torch casts, all ties
+ *   kq_oracle_tiled_scale_*,
+ *   kq_oracle_scales_to_tiled       hand indices; reshape/permute restatement
+ * Nothing is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -163,12 +177,6 @@ int kq_oracle_transform_x(const uint16_t *X, int x_dtype, int64_t tokens, int d,
     return 0;
 }
 
-int kq_oracle_transform(const uint16_t *X, int64_t tokens, int d,
-                        const float *G, int n_sets, float *Y)
-{
-    return kq_oracle_transform_x(X, 0, tokens, d, G, NULL, n_sets, Y);
-}
-
 /* per-channel scaling (SmoothQuant-style diagonal T, Appendix D "Smoothing"):
  * Y[t, i] = float( x * s_i ); the double product is exact, so this is one
  * correctly rounded float product. */
@@ -183,22 +191,12 @@ int kq_oracle_scale_transform_x(const uint16_t *X, int x_dtype, int64_t tokens, 
     return 0;
 }
 
-int kq_oracle_scale_transform(const uint16_t *X, int64_t tokens, int d, const float *s, float *Y)
-{
-    return kq_oracle_scale_transform_x(X, 0, tokens, d, s, Y);
-}
-
 /* no transform (bare MXFP4 quantizer, the paper's "Q4" column): Y = X widened. */
 int kq_oracle_widen_x(const uint16_t *X, int x_dtype, int64_t tokens, int d, float *Y)
 {
     if (d <= 0 || d % KQ_BLOCK || tokens < 0) return -1;
     for (int64_t i = 0; i < tokens * d; ++i) Y[i] = load_x(X, i, x_dtype);
     return 0;
-}
-
-int kq_oracle_widen(const uint16_t *X, int64_t tokens, int d, float *Y)
-{
-    return kq_oracle_widen_x(X, 0, tokens, d, Y);
 }
 
 /* ---- MXFP4 encode -------------------------------------------------------- */
@@ -260,24 +258,6 @@ int kq_oracle_mx_encode(const float *Y, int64_t tokens, int d, uint8_t *q, uint8
                                    q + t * (d / 2) + (int64_t)j * 16,
                                    scales + t * nb + j);
     return 0;
-}
-
-/* whole path: transform (factors), then encode.  Y_scratch: float [tokens][d]
- * supplied by the caller and left holding the pre-rounding values. */
-int kq_oracle_quantize(const uint16_t *X, int64_t tokens, int d, const float *G, int n_sets,
-                       float *Y_scratch, uint8_t *q, uint8_t *scales)
-{
-    int rc = kq_oracle_transform(X, tokens, d, G, n_sets, Y_scratch);
-    if (rc) return rc;
-    return kq_oracle_mx_encode(Y_scratch, tokens, d, q, scales);
-}
-
-int kq_oracle_scale_quantize(const uint16_t *X, int64_t tokens, int d, const float *s,
-                             float *Y_scratch, uint8_t *q, uint8_t *scales)
-{
-    int rc = kq_oracle_scale_transform(X, tokens, d, s, Y_scratch);
-    if (rc) return rc;
-    return kq_oracle_mx_encode(Y_scratch, tokens, d, q, scales);
 }
 
 /* ---- decode ---------------------------------------------------------------- */

@@ -8,6 +8,19 @@ The two must agree bit for bit; the tests check that.
 Paper passages: blockwise quantizer Q_b (Section 3.1); K = G1 (x) ... (x) G5
 (Section 3.2); y = x K on each 32-channel slice (Section 3.5); MXFP4 = E2M1 +
 E8M0 per 32 block following OCP Microscaling (Section 4.1, Appendix D).
+
+Parity pins (tests that fix each function to something other than itself):
+  dense_k            np.kron chain vs the bit formula of the C twin; shear hand vectors; Hadamard closed form
+  lu_to_factors      L U product written out, det = -1
+  transform          exact Fraction sums on small blocks; the C twin bit for bit
+  scale_transform    NumPy casts; the C twin
+  mx_encode          hand-worked blocks (tests/golden/mxfp4_handworked.txt); brute force over every bf16
+                     value in (-8, 8) with exact rationals; tie table
+  decode             the E2M1 grid written out; np.linalg.inv round trip
+  encode_with_scale  hand-worked blocks under imposed scale bytes (tests/golden/mxfp4_imposed_scale.txt);
+                     brute force over every bf16 value in (-8, 8) at three scale bytes; equality with the
+                     C encoder when the imposed byte is the block's own
+Nothing here is "parity unpinned".
 """
 from __future__ import annotations
 

@@ -254,3 +254,55 @@ def test_dequantize_bf16_rounding_matches_torch(small):
     # without factors every decoded value is exactly representable in bf16
     b0 = co.dequantize(q, s, None, out_bf16=True)
     assert np.array_equal(W.bf16_bits_to_f32(b0), co.dequantize(q, s))
+
+
+# ---- codes under an imposed scale byte (the helper of parity rule P3) ----------------------
+IMPOSED = os.path.join(os.path.dirname(__file__), "golden", "mxfp4_imposed_scale.txt")
+
+
+def _imposed_rows():
+    rows = []
+    with open(IMPOSED) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            name, vals, S, codes = [p.strip() for p in line.split("|")]
+            rows.append((name, [float(v) for v in vals.split()], int(S), [int(c, 16) for c in codes.split()]))
+    return rows
+
+
+@pytest.mark.parametrize("row", _imposed_rows(), ids=lambda r: r[0])
+def test_encode_with_scale_handworked(row):
+    name, vals, S, codes = row
+    got = no.encode_with_scale(block32(vals)[None, :], np.array([[S]], np.uint8))
+    assert list(got[0, :len(codes)]) == codes
+    assert not got[0, len(vals):].any()
+
+
+def test_encode_with_scale_at_own_scale_is_the_encoder(small):
+    # with S = the block's own scale byte it must reproduce the C oracle's encoder on whole tensors
+    Xb, G = small
+    q, s, Y = co.quantize(Xb, G)
+    codes = np.empty(Y.shape, np.uint8)
+    codes[:, 0::2] = q & 15
+    codes[:, 1::2] = q >> 4
+    assert np.array_equal(no.encode_with_scale(Y, s), codes)
+    spec = W.tiny_spec()
+    Xt = W.gen_activations(spec)
+    qt, st, Yt = co.quantize(Xt, W.gen_factors(0))
+    ct = np.empty(Yt.shape, np.uint8)
+    ct[:, 0::2] = qt & 15
+    ct[:, 1::2] = qt >> 4
+    assert np.array_equal(no.encode_with_scale(Yt, st), ct)
+
+
+def test_encode_with_scale_brute_force_neighbouring_scales():
+    # every bf16 value in (-8, 8) at S = 126, 127, 128 against the exact-rational nearest-code search
+    vals = all_bf16_in_open_8()
+    Y = np.zeros((len(vals), 32), np.float32)
+    Y[:, 0] = vals
+    for S in (126, 127, 128):
+        got = no.encode_with_scale(Y, np.full((len(vals), 1), S, np.uint8))[:, 0]
+        expect = np.array([brute_code(float(v) * 2.0 ** (127 - S)) for v in vals], dtype=np.uint8)
+        assert np.array_equal(got, expect)
