@@ -57,8 +57,9 @@ typedef enum { KQ_X_BF16 = 0, KQ_X_FP16 = 1 } kq_xdtype_t;
  * tensor-core GEMMs read (the consumer of the paper's W4A4 product, Section 3.4): tiles of 128 rows x
  * 4 blocks = 512 bytes, row-tile-major; byte of (t, j) at
  *   ((t/128) * ceil(d/128) + j/4) * 512 + (t%32)*16 + ((t%128)/32)*4 + j%4.
- * The buffer then holds ceil(tokens/128)*128 * ceil(d/128)*4 bytes (16-byte aligned for per-block
- * factor sets); padding bytes are left untouched or written as 0.
+ * The buffer then holds ceil(tokens/128)*128 * ceil(d/128)*4 bytes and must be 16-byte aligned
+ * (KQ_ERR_ALIGN otherwise: whole tiles leave by vector stores); padding bytes are left untouched
+ * or written as 0.
  * kroquant_dequantize reads ROWMAJOR only. */
 typedef enum { KQ_SCALES_ROWMAJOR = 0, KQ_SCALES_TILED_128X4 = 1 } kq_scale_layout_t;
 
@@ -211,6 +212,13 @@ kq_status_t kroquant_debug_set_boundary(int trigger, int prefetch_tiles);
  * stream; calls that are meant to overlap on several streams want the static one, because a dynamic launch
  * claims every CTA slot of the GPU.  KQ_ERR_UNSUPPORTED outside the ranges.  Process-wide. */
 kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles);
+
+/* Which device code runs the two comparison quantizers of Section 4.4 (bare MXFP4 "Q4", per-channel "Scale"):
+ * staged = 1 (default): the KroQuant kernel's own pipeline (TMA-staged tiles, same tile distribution and
+ * kernel-boundary handling) with the tensor-core stage left out, so that the comparison measures the
+ * transform and not the pipeline; staged = 0: plain grid-stride CUDA-core kernels.  Same bits either way.
+ * Process-wide; other values give KQ_ERR_UNSUPPORTED. */
+kq_status_t kroquant_debug_set_compare_kernels(int staged);
 
 /* The W4A4 product of the quantized layer (Section 3.4: O = Q(A T) Q(W~)^T + A T L R):
  *     out[m][n] = sum_k a[m][k] 2^(sa[m][k/32] - 127) * b[n][k] 2^(sb[n][k/32] - 127)  (+ add[m][n])

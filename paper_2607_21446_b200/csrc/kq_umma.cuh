@@ -2,8 +2,8 @@
 // (accumulators in TMEM) -> tcgen05.ld -> fused MXFP4 encoder in registers.
 //
 // Shared factor set (one K per layer; the per-block variant is described at the
-// kernel).  Because every 32-channel block of every token is multiplied by the same K (paper Section 3.5: "many column blocks share
-// the same Kronecker factors"), X[tokens][d] is viewed as a flat matrix of
+// kernel).  Because every 32-channel block of every token is multiplied by the same K (paper Section 3.5:
+// one factor set shared by the column blocks of a layer), X[tokens][d] is viewed as a flat matrix of
 // n_blocks = tokens*d/32 rows of 32 bf16 (64 contiguous bytes each), and the whole
 // layer is one tall GEMM  Y[n_blocks][32] = Xflat[n_blocks][32] * K[32][32]
 // (Section 3.5: y = x K per block).  In this view the inputs, the 16-byte code
@@ -146,10 +146,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr) {
     return d;
 }
 // kind::f16 instruction descriptor: D=f32, A and B both bf16 (format code 1) or both fp16 (0),
-// both K-major, N=32, M=128.
-__host__ __device__ constexpr uint32_t idesc_m128n32(bool fp16) {
-    return (1u << 4) | ((fp16 ? 0u : 1u) << 7) | ((fp16 ? 0u : 1u) << 10) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+// both K-major, M=128, N = n (a multiple of 16).
+__host__ __device__ constexpr uint32_t idesc_m128(bool fp16, uint32_t n) {
+    return (1u << 4) | ((fp16 ? 0u : 1u) << 7) | ((fp16 ? 0u : 1u) << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
+__host__ __device__ constexpr uint32_t idesc_m128n32(bool fp16) { return idesc_m128(fp16, 32u); }
 
 // TMA store of a 2-D box from shared memory (bulk async group of the issuing thread).
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, uint32_t src, int x, int y) {
@@ -385,14 +386,26 @@ struct UmmaProblem {
 // Separate instantiations, because the extra code costs registers that would take a resident CTA away
 // from the default kernel.
 constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone>
-__global__ void __launch_bounds__(128 + 128 * NG, (NS == 8 && NG == 2) ? 2 : 1)      // (8,2,2) runs two per SM
+// OP: what happens between the staged tile and the encoder.
+//   kOpKron   the block transform on the tensor core (everything described above).
+//   kOpPlain  nothing: the bare MXFP4 quantizer ("Q4", Section 4.4).
+// The bare quantizer is this kernel minus the tensor-core stage: the same producer (TMA tiles into the same
+// swizzled stages, the same work distribution and kernel-boundary handling), no TMEM, no MMA warps; an
+// epilogue thread reads the 64 bytes of its block from the stage (conflict-free thanks to the swizzle), widens
+// them and runs the same encoder.  Shared-set flat view only.
+constexpr int kOpKron = 0, kOpPlain = 1;
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone, int OP = kOpKron>
+// resident CTAs per SM the register budget must allow: (8,2,2) two; the one-warpgroup shapes three (two with the
+// calibration epilogue)
+__global__ void __launch_bounds__(128 + 128 * NG, (NS == 8 && NG == 2) ? 2 : NG == 1 ? (EXTRA == kExtraCalib ? 2 : 3) : 1)
 quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
               const uint8_t* __restrict__ b_image, const int* __restrict__ e_norm, const UmmaProblem prob,
               uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y,
               uint4* __restrict__ at_out, double* __restrict__ sumsq) {
     constexpr bool DUAL = EXTRA == kExtraDual;
     constexpr bool CALIB = EXTRA == kExtraCalib;
+    constexpr bool TC = OP == kOpKron;            // tensor-core stage present
+    static_assert(TC || (!PB && !WRITE_Y && EXTRA == kExtraNone), "comparison kernels: flat view, quantizing path only");
     static_assert(!CALIB || (!XF16 && !WRITE_Y), "calibration outputs: bf16 images, quantizing path");
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
     // TMEM is handed out in powers of two
@@ -420,7 +433,8 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     static_assert(!PB || NG == 1, "a column group is staged by one epilogue warpgroup");
     static_assert(kRingEntries >= 2 * NS, "a ring entry must outlive the tile it describes");
     // sentinel tiles at the end of the stream: every MMA warp gets the same number, every epilogue group at least one
-    constexpr int kSentinels = ((NM > NG ? NM : NG) + NM - 1) / NM * NM;
+    // (without the tensor-core stage the epilogue groups read the producer's sentinels themselves: one each)
+    constexpr int kSentinels = TC ? ((NM > NG ? NM : NG) + NM - 1) / NM * NM : NG;
     volatile int* ring = reinterpret_cast<volatile int*>(base_ptr + L::kRingOff);
     volatile int* ring_jg = reinterpret_cast<volatile int*>(base_ptr + L::kRing2Off);
     const uint32_t bar_clc = bar0 + 8u * (3 * NS + 1);
@@ -540,7 +554,9 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     if (prob.early_trigger == 1) pdl_launch_dependents();
     bool more = true;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_done(s), 1); mbar_init(bar_tempty(s), 4); }
+        // "done" = the stage may be refilled: one tcgen05.commit, or (no tensor-core stage) the four epilogue
+        // warps that have read it
+        for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_done(s), TC ? 1 : 4); mbar_init(bar_tempty(s), 4); }
         mbar_init(bar_b, 1);
         mbar_init(bar_clc, 1);
         *abort_flag = 0;
@@ -553,7 +569,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
         if (PB && !WRITE_Y) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
         if (prob.dynamic) clc_request();       // concerns this grid's own CTAs only
-        if (!PB) {
+        if (TC && !PB) {
             mbar_expect_tx(bar_b, kBImageBytes);
             bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
         }
@@ -581,7 +597,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         pdl_wait_prior_grid();
         more = produce(true);
     }
-    if (warp == 1) {
+    if (TC && warp == 1) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(base + (uint32_t)L::kTmemSlotOff), "r"((uint32_t)kTmemCols) : "memory");
@@ -590,7 +606,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = TC ? *tmem_slot : 0u;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -607,7 +623,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 mbar_arrive(bar_full(n % NS));
             }
         }
-    } else if (warp <= NM) {
+    } else if (TC && warp <= NM) {
         // ---------------- MMA issuers ----------------
         if (lane == 0) {
             bool ok = true;
@@ -663,22 +679,45 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
-        const int e_shared = (PB || !XF16) ? 0 : __ldg(e_norm);
+        const int e_shared = (PB || !XF16 || !TC) ? 0 : __ldg(e_norm);
         double sq_sum = 0.0;                       // CALIB: this thread's sum of squared residuals
         for (int n = g;; n += NG) {
             const int s = n % NS;
-            if (!mbar_wait(bar_done(s), (n / NS) & 1, abort_flag)) {
+            if (!mbar_wait(TC ? bar_done(s) : bar_full(s), (n / NS) & 1, abort_flag)) {
                 if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_EPILOGUE); *abort_flag = 1; }
                 break;
             }
             const int item = ring[n % kRingEntries];
             if (item < 0) break;
-            tc_fence_after();
             uint32_t acc[32];
-            tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * 32), acc);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty(s));
+            if (TC) {
+                tc_fence_after();
+                tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * 32), acc);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty(s));
+            } else {
+                // the block's 64 bytes straight from the stage: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3)
+                const int r = quarter * 32 + lane;
+                const uint32_t row_addr = base + L::kAOff + s * L::kStageBytes + 64u * r;
+                uint32_t w[16];
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(w[4 * c]), "=r"(w[4 * c + 1]), "=r"(w[4 * c + 2]), "=r"(w[4 * c + 3])
+                                 : "r"(row_addr + 16u * (uint32_t)(c ^ ((r >> 1) & 3))) : "memory");
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    if (XF16) {
+                        const float2 f2 = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+                        acc[2 * i] = __float_as_uint(f2.x);
+                        acc[2 * i + 1] = __float_as_uint(f2.y);
+                    } else {
+                        acc[2 * i] = w[i] << 16;
+                        acc[2 * i + 1] = w[i] & 0xFFFF0000u;
+                    }
+                }
+            }
             if (PB && !WRITE_Y) {
                 const int c = n % kPbCols;
                 const int tt = item, jg = ring_jg[n % kRingEntries], j = jg * kPbCols + c;
@@ -796,6 +835,13 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     }
                 }
             }
+            if (!TC) {
+                // The stage may be refilled.  Released only here, behind the stores of the results: they depend
+                // on every value read from the stage, so the reads have certainly been performed (an arrival
+                // right after the shared-memory loads were issued let the next TMA copy overtake them).
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_done(s));
+            }
         }
         // the staging tile must not be released while a TMA store still reads it
         if (PB && !WRITE_Y && threadIdx.x == 128) bulk_wait_group_read<0>();
@@ -813,13 +859,13 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // abort path only: let the copies this thread issued land before the CTA's shared
         // memory goes away (load m went to slot m % NS and completes phase (m / NS) & 1)
         int never = 0;
-        if (!PB) (void)mbar_wait(bar_b, 0, &never);
+        if (TC && !PB) (void)mbar_wait(bar_b, 0, &never);
         for (int m = (issued > NS ? issued - NS : 0); m < issued; ++m)
             if (!mbar_wait(bar_full(m % NS), (m / NS) & 1, &never))
                 atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_DRAIN);
     }
     __syncthreads();
-    if (warp == 1) {
+    if (TC && warp == 1) {
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"

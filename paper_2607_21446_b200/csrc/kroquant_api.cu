@@ -46,6 +46,8 @@ std::atomic<int> g_umma_prefetch{4};    // UmmaProblem::prefetch_tiles
 std::atomic<int> g_umma_dynamic{1};     // UmmaProblem::dynamic
 std::atomic<int> g_umma_unit_tiles{3};  // UmmaProblem::unit_tiles
 std::atomic<int> g_umma_unit_auto{1};   // 1: small launches use single-tile units (until the caller sets the unit)
+std::atomic<int> g_compare_staged{1};   // comparison quantizers: 1 = the tensor-core kernel's pipeline without its MMA stage,
+                                        // 0 = the plain grid-stride kernels
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -76,6 +78,20 @@ int sm_count() {
     }
     return cached[dev];
 }
+
+// Per-device "do once" for set-up that belongs to a device (function attributes).  needed() is true until
+// done() has been called with the same device current; a race between two first calls only repeats the set-up.
+struct DeviceOnce {
+    std::atomic<int> flag[64];
+    DeviceOnce() { for (auto& f : flag) f.store(0); }
+    static int dev() {
+        int d = -1;
+        if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= 64) return -1;
+        return d;
+    }
+    bool needed() const { const int d = dev(); return d < 0 || !flag[d].load(std::memory_order_acquire); }
+    void done() { const int d = dev(); if (d >= 0) flag[d].store(1, std::memory_order_release); }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -189,24 +205,27 @@ kq_status_t finish_factors(kroquant_factors_t* f, const std::vector<double>& K,
     return KQ_OK;
 }
 
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kq::kExtraNone>
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kq::kExtraNone, int OP = kq::kOpKron>
 kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
                         const int* enorm, const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, void* at_out, int ctas_per_sm, bool pdl,
                         cudaStream_t st, double* sumsq = nullptr) {
     using L = kq::UmmaSmem<NS, PB>;
-    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA>;
-    static std::once_flag once;
-    static cudaError_t attr_rc = cudaSuccess;
+    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA, OP>;
     // Dynamic distribution: the grid has one CTA per unit and the hardware decides how many run at once, so the
     // number of resident CTAs per SM is set through the shared memory each CTA asks for: just too much for
     // ctas_per_sm + 1 of them (228 KB per SM, 1 KB reserved per CTA).
     constexpr int kSmemPerSm = 233472, kSmemReserved = 1024, kMaxDyn = kSmemPerSm / 2 - kSmemReserved + 128;
-    std::call_once(once, [&] {
-        attr_rc = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       L::kDynBytes > kMaxDyn ? L::kDynBytes : kMaxDyn);
-    });
-    if (attr_rc != cudaSuccess) return KQ_ERR_CUDA;
+    // function attributes belong to a device: set once per device and instantiation
+    static DeviceOnce attr_done;
+    if (attr_done.needed()) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 L::kDynBytes > kMaxDyn ? L::kDynBytes : kMaxDyn) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KQ_ERR_CUDA;
+        }
+        attr_done.done();
+    }
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
     // persistent grid: at most ctas_per_sm CTAs per SM (shrinking it further so that every CTA
@@ -349,6 +368,52 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     }
 #undef KQ_LAUNCH
 #undef KQ_LAUNCH_DUAL
+}
+
+// The bare MXFP4 quantizer on the tensor-core kernel's own pipeline minus the tensor-core stage: same flat view,
+// tile distribution, CTA shapes and kernel-boundary handling as run_umma.
+kq_status_t run_plain_staged(const void* X, bool xf16, int64_t tokens, int d, uint8_t* q, uint8_t* scales, bool tiled,
+                             cudaStream_t st) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return KQ_ERR_CUDA;
+    const int nb = d / 32;
+    kq::UmmaProblem prob;
+    prob.blocks_per_row = nb;
+    prob.tiled_scales = tiled ? 1 : 0;
+    prob.early_trigger = g_umma_pdl.load() != 0 ? g_umma_trigger.load() : 0;
+    prob.prefetch_tiles = g_umma_pdl.load() != 0 ? g_umma_prefetch.load() : 0;
+    prob.dynamic = g_umma_dynamic.load();
+    prob.unit_tiles = g_umma_unit_tiles.load();
+    prob.n_rows = tokens * (int64_t)nb;
+    prob.n_ttiles = 1;
+    prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
+    if (g_umma_unit_auto.load() && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
+    prob.n_units = (prob.n_tiles + prob.unit_tiles - 1) / prob.unit_tiles;
+    CUtensorMap tmap;
+    const cuuint64_t dims[2] = {32, (cuuint64_t)prob.n_rows}, strides[1] = {64};
+    const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, xf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void*>(X), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return KQ_ERR_CUDA;
+    const int cps_set = g_umma_ctas_per_sm.load();
+    const bool big_ctas = cps_set == 0 && prob.n_tiles > (int64_t)3 * sm_count();
+    const int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
+    const bool pdl = g_umma_pdl.load() != 0;
+    prob.prefetch_stride = sm_count() * cps;
+    if (prob.dynamic && prob.n_units <= (int64_t)sm_count() * cps) {
+        prob.dynamic = 0;
+        if (prob.early_trigger == 2) prob.early_trigger = 1;
+    }
+#define KQ_LAUNCH_CMP(NS, NM, NG, XF) \
+    launch_umma<NS, NM, NG, false, XF, false, kq::kExtraNone, kq::kOpPlain>(tmap, tmap, nullptr, nullptr, prob, q, scales, \
+                                                                            nullptr, nullptr, cps, pdl, st)
+    const bool big = cps_set == 0 ? big_ctas : g_umma_cfg.load() == 2;
+    if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true) : KQ_LAUNCH_CMP(4, 2, 1, true);
+    return big ? KQ_LAUNCH_CMP(8, 2, 2, false) : KQ_LAUNCH_CMP(4, 2, 1, false);
+#undef KQ_LAUNCH_CMP
 }
 
 template <int MODE, bool WRITE_Y, bool XF16, bool TILED>
@@ -515,12 +580,16 @@ kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tok
     if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
     if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
     if (path == KQ_PATH_ALU && f->dense) return KQ_ERR_UNSUPPORTED;
+    // whole 512-byte scale tiles leave by 16-byte vector stores
+    if (scale_layout == KQ_SCALES_TILED_128X4 && !aligned16(scales)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
     const bool tiled = scale_layout == KQ_SCALES_TILED_128X4;
-    if (path == KQ_PATH_AUTO && f->identity)
+    if (path == KQ_PATH_AUTO && f->identity) {
+        if (g_compare_staged.load()) return run_plain_staged(X, xf16, tokens, d, q_packed, scales, tiled, st);
         return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, tiled, nullptr, st);
+    }
     if (path != KQ_PATH_ALU)
         return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, tiled, nullptr, nullptr, st);
     return run_stream<kq::MODE_KRON, false>(X, xf16, tokens, d, f, nullptr, q_packed, scales, tiled, nullptr, st);
@@ -536,6 +605,7 @@ kq_status_t kroquant_quantize_dual(const void* X, kq_xdtype_t x_dtype, int64_t t
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed) || !aligned16(AT_out)) return KQ_ERR_ALIGN;
     if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
+    if (scale_layout == KQ_SCALES_TILED_128X4 && !aligned16(scales)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
     return run_umma<false>(X, x_dtype == KQ_X_FP16, tokens, d, f, q_packed, scales,
                            scale_layout == KQ_SCALES_TILED_128X4, nullptr, AT_out, static_cast<cudaStream_t>(stream));
@@ -585,6 +655,7 @@ kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed) || !aligned16(s)) return KQ_ERR_ALIGN;
     if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
+    if (scale_layout == KQ_SCALES_TILED_128X4 && !aligned16(scales)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
@@ -633,7 +704,11 @@ kq_status_t kroquant_mxfp4_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
     if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
+    if (scale_layout == KQ_SCALES_TILED_128X4 && !aligned16(scales)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
+    if (g_compare_staged.load())
+        return run_plain_staged(X, x_dtype == KQ_X_FP16, tokens, d, q_packed, scales,
+                                scale_layout == KQ_SCALES_TILED_128X4, static_cast<cudaStream_t>(stream));
     return run_stream<kq::MODE_PLAIN, false>(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, nullptr, q_packed, scales,
                                              scale_layout == KQ_SCALES_TILED_128X4, nullptr,
                                              static_cast<cudaStream_t>(stream));
@@ -756,6 +831,12 @@ kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles) {
     g_umma_dynamic.store(dynamic);
     g_umma_unit_tiles.store(unit_tiles > 0 ? unit_tiles : 3);
     g_umma_unit_auto.store(unit_tiles > 0 ? 0 : 1);
+    return KQ_OK;
+}
+
+kq_status_t kroquant_debug_set_compare_kernels(int staged) {
+    if (staged < 0 || staged > 1) return KQ_ERR_UNSUPPORTED;
+    g_compare_staged.store(staged);
     return KQ_OK;
 }
 

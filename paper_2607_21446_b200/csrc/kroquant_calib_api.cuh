@@ -88,8 +88,8 @@ kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
                         const float* aux, int64_t ld_aux, const float* coef_ptr, float coef_mul, float out_scale,
                         float* out_f32, __nv_bfloat16* out_bf16, int64_t ld_out, double* sumsq, cudaStream_t st,
                         __nv_bfloat16* out_bf16_t = nullptr, int64_t ld_out_t = 0, int mode = 0) {
-    static std::atomic<int> attr_done{0};
-    if (!attr_done.load(std::memory_order_acquire)) {
+    static DeviceOnce attr_done;
+    if (attr_done.needed()) {
         if (cudaFuncSetAttribute(kq::gemm_nt_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kGemmDynBytes) !=
                 cudaSuccess ||
             cudaFuncSetAttribute(kq::gemm_umma_pair<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -101,7 +101,7 @@ kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
         }
-        attr_done.store(1, std::memory_order_release);
+        attr_done.done();
     }
     const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0 || mode != 0;
     const int bm = pair ? kq::kGemm2BM : kq::kGemmBM;
@@ -347,8 +347,8 @@ kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, con
     if (M == 0) return KQ_OK;
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
-    static std::atomic<int> attr_done{0};
-    if (!attr_done.load(std::memory_order_acquire)) {
+    static DeviceOnce attr_done;
+    if (attr_done.needed()) {
         if (cudaFuncSetAttribute(kq::gemm_mxfp4_umma, cudaFuncAttributeMaxDynamicSharedMemorySize, kq::kF4DynBytes) !=
                 cudaSuccess ||
             cudaFuncSetAttribute(kq::gemm_mxfp4_umma_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -356,7 +356,7 @@ kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, con
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
         }
-        attr_done.store(1, std::memory_order_release);
+        attr_done.done();
     }
     CUtensorMap ta, tb;
     const cuuint32_t estr[2] = {1, 1};

@@ -215,7 +215,20 @@ def test_error_codes(B):
     assert L.kroquant_quantize(px, 4, 64, f3._h, pq, ps, st) == 4
     assert L.kroquant_quantize_path(px, 4, 64, f._h, pq, ps, 7, st) == 5
     assert L.kroquant_quantize(px, 0, 64, f._h, pq, ps, st) == 0            # empty input: ok, no launch
+    # tiled scale bytes leave by 16-byte vector stores: a misaligned buffer is refused, never launched
+    big = torch.zeros(4096 + 16, dtype=torch.uint8, device="cuda")
+    ps_odd = C.c_void_p(big.data_ptr() + 4)
+    pat = C.c_void_p(torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda").data_ptr())
+    f2 = B.Factors.create(W.gen_factors(0, n_sets=2))
+    for h in (f._h, f2._h):
+        assert L.kroquant_quantize_ex(px, 0, 4, 64, h, pq, ps_odd, 1, 0, st) == 3
+        assert L.kroquant_quantize_dual(px, 0, 4, 64, h, pq, ps_odd, 1, pat, st) == 3
+    assert L.kroquant_mxfp4_quantize_ex(px, 0, 4, 64, pq, ps_odd, 1, st) == 3
     assert B.kroquant_launch_count() == n0
+    assert L.kroquant_quantize_ex(px, 0, 4, 64, f._h, pq, ps_odd, 0, 0, st) == 0     # row-major scales: any address
+    torch.cuda.synchronize()
+    assert B.kroquant_launch_count() == n0 + 1
+    n0 += 1
     bad = W.gen_factors(0)
     bad[0, 2] = np.array([[1, 2], [2, 4]], np.float32)                       # singular
     with pytest.raises(B.KroQuantError) as e:
