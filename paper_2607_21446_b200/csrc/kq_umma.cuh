@@ -393,15 +393,21 @@ constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
 // swizzled stages, the same work distribution and kernel-boundary handling), no TMEM, no MMA warps; an
 // epilogue thread reads the 64 bytes of its block from the stage (conflict-free thanks to the swizzle), widens
 // them and runs the same encoder.  Shared-set flat view only.
-constexpr int kOpKron = 0, kOpPlain = 1;
+//   kOpScale  the per-channel "Scale" comparison (Section 4.4; Appendix D, Smoothing): y = x * s, one correctly
+//     rounded float product per element.  In the flat view every block of a tile belongs to a different block
+//     column, so each thread needs its own 32 multipliers (128 bytes, twice the bytes of its activations): the
+//     whole vector s[d] is copied once per CTA into shared memory (behind the stages; 16-byte chunk v of column j
+//     at chunk v ^ (j & 7), so that the eight lanes of a quarter warp, which hold consecutive columns, read eight
+//     different bank groups), and a thread reads its column's 128 bytes from there.
+constexpr int kOpKron = 0, kOpPlain = 1, kOpScale = 2;
 template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone, int OP = kOpKron>
 // resident CTAs per SM the register budget must allow: (8,2,2) two; the one-warpgroup shapes three (two with the
 // calibration epilogue)
-__global__ void __launch_bounds__(128 + 128 * NG, (NS == 8 && NG == 2) ? 2 : NG == 1 ? (EXTRA == kExtraCalib ? 2 : 3) : 1)
+__global__ void __launch_bounds__(128 + 128 * NG, (NS <= 8 && NG == 2) ? 2 : NG == 1 ? (EXTRA == kExtraCalib ? 2 : 3) : 1)
 quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_q,
               const uint8_t* __restrict__ b_image, const int* __restrict__ e_norm, const UmmaProblem prob,
               uint8_t* __restrict__ q_packed, uint8_t* __restrict__ scales, float* __restrict__ Y,
-              uint4* __restrict__ at_out, double* __restrict__ sumsq) {
+              uint4* __restrict__ at_out, double* __restrict__ sumsq, const float* __restrict__ chan_scale) {
     constexpr bool DUAL = EXTRA == kExtraDual;
     constexpr bool CALIB = EXTRA == kExtraCalib;
     constexpr bool TC = OP == kOpKron;            // tensor-core stage present
@@ -679,6 +685,18 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
+        const uint32_t vec_base = base + (uint32_t)((L::kBytes + 127) & ~127);
+        if (OP == kOpScale) {
+            // the multiplier vector -> shared memory (it is an ordinary input: read after the dependency wait)
+            const int n_chunks = prob.blocks_per_row * 8;
+            for (int i = (int)threadIdx.x - 128; i < n_chunks; i += 128 * NG) {
+                const float4 m = __ldg(reinterpret_cast<const float4*>(chan_scale) + i);
+                const uint32_t j = (uint32_t)i >> 3, v = (uint32_t)i & 7u;
+                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};"
+                             ::"r"(vec_base + 128u * j + 16u * (v ^ (j & 7u))), "f"(m.x), "f"(m.y), "f"(m.z), "f"(m.w) : "memory");
+            }
+            named_barrier_sync(2, 128 * NG);
+        }
         const int e_shared = (PB || !XF16 || !TC) ? 0 : __ldg(e_norm);
         double sq_sum = 0.0;                       // CALIB: this thread's sum of squared residuals
         for (int n = g;; n += NG) {
@@ -715,6 +733,23 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     } else {
                         acc[2 * i] = w[i] << 16;
                         acc[2 * i + 1] = w[i] & 0xFFFF0000u;
+                    }
+                }
+                if (OP == kOpScale) {
+                    const uint32_t blk = (uint32_t)item * kTileRows + (uint32_t)r;       // flat block index (< 2^31 is enforced)
+                    const uint32_t j = blk % (uint32_t)prob.blocks_per_row;             // its block column
+                    const uint32_t col_addr = vec_base + 128u * j, sw = j & 7u;
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        uint64_t m01, m23;
+                        asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(m01), "=l"(m23) : "r"(col_addr + 16u * ((uint32_t)v ^ sw)) : "memory");
+                        float p0, p1, p2, p3;
+                        mul2(acc[4 * v], acc[4 * v + 1], m01, p0, p1);               // each half an ordinary rounded product
+                        mul2(acc[4 * v + 2], acc[4 * v + 3], m23, p2, p3);
+                        acc[4 * v] = __float_as_uint(p0);
+                        acc[4 * v + 1] = __float_as_uint(p1);
+                        acc[4 * v + 2] = __float_as_uint(p2);
+                        acc[4 * v + 3] = __float_as_uint(p3);
                     }
                 }
             }

@@ -209,7 +209,7 @@ template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = 
 kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
                         const int* enorm, const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, void* at_out, int ctas_per_sm, bool pdl,
-                        cudaStream_t st, double* sumsq = nullptr) {
+                        cudaStream_t st, double* sumsq = nullptr, const float* chan_scale = nullptr, int extra_smem = 0) {
     using L = kq::UmmaSmem<NS, PB>;
     auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA, OP>;
     // Dynamic distribution: the grid has one CTA per unit and the hardware decides how many run at once, so the
@@ -220,7 +220,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     static DeviceOnce attr_done;
     if (attr_done.needed()) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 L::kDynBytes > kMaxDyn ? L::kDynBytes : kMaxDyn) != cudaSuccess) {
+                                 OP == kq::kOpScale ? 232448 : (L::kDynBytes > kMaxDyn ? L::kDynBytes : kMaxDyn)) != cudaSuccess) {
             (void)cudaGetLastError();
             return KQ_ERR_CUDA;
         }
@@ -233,7 +233,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     // less latency than the shorter last round saves)
     const int64_t cap = (int64_t)sms * ctas_per_sm;
     const int64_t grid = (prob.dynamic || prob.n_units < cap) ? prob.n_units : cap;
-    int smem = L::kDynBytes;
+    int smem = L::kDynBytes + extra_smem;
     if (prob.dynamic) {
         const int limit = ((kSmemPerSm / (ctas_per_sm + 1) - kSmemReserved) & ~127) + 128;
         if (limit > smem) smem = limit;
@@ -249,7 +249,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
     if (cudaLaunchKernelEx(&cfg, kern, tmap, tmap_q, bimg, enorm, prob, q, scales, Y, reinterpret_cast<uint4*>(at_out),
-                           sumsq) != cudaSuccess) {
+                           sumsq, chan_scale) != cudaSuccess) {
         (void)cudaGetLastError();
         return KQ_ERR_CUDA;
     }
@@ -370,10 +370,11 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
 #undef KQ_LAUNCH_DUAL
 }
 
-// The bare MXFP4 quantizer on the tensor-core kernel's own pipeline minus the tensor-core stage: same flat view,
-// tile distribution, CTA shapes and kernel-boundary handling as run_umma.
-kq_status_t run_plain_staged(const void* X, bool xf16, int64_t tokens, int d, uint8_t* q, uint8_t* scales, bool tiled,
-                             cudaStream_t st) {
+// The comparison quantizers (bare MXFP4; per-channel scale when chan_scale != null) on the tensor-core kernel's own
+// pipeline minus the tensor-core stage: same flat view, tile distribution, CTA shapes and kernel-boundary handling
+// as run_umma.  KQ_ERR_UNSUPPORTED: the multiplier vector does not fit beside the stages (the caller falls back).
+kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, const float* chan_scale, uint8_t* q,
+                            uint8_t* scales, bool tiled, cudaStream_t st) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
     const int nb = d / 32;
@@ -400,19 +401,34 @@ kq_status_t run_plain_staged(const void* X, bool xf16, int64_t tokens, int d, ui
         return KQ_ERR_CUDA;
     const int cps_set = g_umma_ctas_per_sm.load();
     const bool big_ctas = cps_set == 0 && prob.n_tiles > (int64_t)3 * sm_count();
-    const int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
+    int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
     const bool pdl = g_umma_pdl.load() != 0;
+    bool big = cps_set == 0 ? big_ctas : g_umma_cfg.load() == 2;
+    const int vec = chan_scale ? d * 4 + 128 : 0;              // the multiplier vector behind the stages
+    if (chan_scale) {
+        constexpr int kSmemPerSm = 233472, kSmemReserved = 1024;
+        const int big_bytes = kq::UmmaSmem<8, false>::kDynBytes + vec, small_bytes = kq::UmmaSmem<4, false>::kDynBytes + vec;
+        if (big && 2 * (big_bytes + kSmemReserved) > kSmemPerSm) big = false;      // eight stages would leave one CTA per SM
+        if (!big) {
+            if (small_bytes + kSmemReserved > kSmemPerSm / 2) return KQ_ERR_UNSUPPORTED;
+            while (cps > 2 && cps * (small_bytes + kSmemReserved) > kSmemPerSm) --cps;
+            if (big_ctas) cps = 2;
+        }
+    }
     prob.prefetch_stride = sm_count() * cps;
     if (prob.dynamic && prob.n_units <= (int64_t)sm_count() * cps) {
         prob.dynamic = 0;
         if (prob.early_trigger == 2) prob.early_trigger = 1;
     }
-#define KQ_LAUNCH_CMP(NS, NM, NG, XF) \
-    launch_umma<NS, NM, NG, false, XF, false, kq::kExtraNone, kq::kOpPlain>(tmap, tmap, nullptr, nullptr, prob, q, scales, \
-                                                                            nullptr, nullptr, cps, pdl, st)
-    const bool big = cps_set == 0 ? big_ctas : g_umma_cfg.load() == 2;
-    if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true) : KQ_LAUNCH_CMP(4, 2, 1, true);
-    return big ? KQ_LAUNCH_CMP(8, 2, 2, false) : KQ_LAUNCH_CMP(4, 2, 1, false);
+#define KQ_LAUNCH_CMP(NS, NM, NG, XF, OPC) \
+    launch_umma<NS, NM, NG, false, XF, false, kq::kExtraNone, OPC>(tmap, tmap, nullptr, nullptr, prob, q, scales, nullptr, \
+                                                                   nullptr, cps, pdl, st, nullptr, chan_scale, vec)
+    if (chan_scale) {
+        if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true, kq::kOpScale) : KQ_LAUNCH_CMP(4, 2, 2, true, kq::kOpScale);
+        return big ? KQ_LAUNCH_CMP(8, 2, 2, false, kq::kOpScale) : KQ_LAUNCH_CMP(4, 2, 2, false, kq::kOpScale);
+    }
+    if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true, kq::kOpPlain) : KQ_LAUNCH_CMP(4, 2, 1, true, kq::kOpPlain);
+    return big ? KQ_LAUNCH_CMP(8, 2, 2, false, kq::kOpPlain) : KQ_LAUNCH_CMP(4, 2, 1, false, kq::kOpPlain);
 #undef KQ_LAUNCH_CMP
 }
 
@@ -587,7 +603,7 @@ kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tok
     const bool xf16 = x_dtype == KQ_X_FP16;
     const bool tiled = scale_layout == KQ_SCALES_TILED_128X4;
     if (path == KQ_PATH_AUTO && f->identity) {
-        if (g_compare_staged.load()) return run_plain_staged(X, xf16, tokens, d, q_packed, scales, tiled, st);
+        if (g_compare_staged.load()) return run_flat_staged(X, xf16, tokens, d, nullptr, q_packed, scales, tiled, st);
         return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, tiled, nullptr, st);
     }
     if (path != KQ_PATH_ALU)
@@ -660,6 +676,10 @@ kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
     const int tiled = scale_layout == KQ_SCALES_TILED_128X4 ? 1 : 0;
+    if (g_compare_staged.load()) {
+        const kq_status_t rc_staged = run_flat_staged(X, xf16, tokens, d, s, q_packed, scales, tiled != 0, st);
+        if (rc_staged != KQ_ERR_UNSUPPORTED) return rc_staged;       // (a vector too long for shared memory: grid-stride kernel)
+    }
     const int64_t n_quads = tokens * (int64_t)(d / 8);
     const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
@@ -707,8 +727,8 @@ kq_status_t kroquant_mxfp4_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     if (scale_layout == KQ_SCALES_TILED_128X4 && !aligned16(scales)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
     if (g_compare_staged.load())
-        return run_plain_staged(X, x_dtype == KQ_X_FP16, tokens, d, q_packed, scales,
-                                scale_layout == KQ_SCALES_TILED_128X4, static_cast<cudaStream_t>(stream));
+        return run_flat_staged(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, q_packed, scales,
+                               scale_layout == KQ_SCALES_TILED_128X4, static_cast<cudaStream_t>(stream));
     return run_stream<kq::MODE_PLAIN, false>(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, nullptr, q_packed, scales,
                                              scale_layout == KQ_SCALES_TILED_128X4, nullptr,
                                              static_cast<cudaStream_t>(stream));
