@@ -102,6 +102,17 @@ int kroquant_factors_n_sets(const kroquant_factors_t *f);
 kq_status_t kroquant_quantize(const void *X, int64_t tokens, int d, const kroquant_factors_t *f,
                               uint8_t *q_packed, uint8_t *scales, void *stream);
 
+/* Sections 3.1 + 3.5 for a caller whose tensors live in HOST memory: X_host (bf16 [tokens][d]) is copied into
+ * the caller's DEVICE work buffer X_work, quantized there into q_work / scales_work (DEVICE, same sizes and
+ * alignment rules as kroquant_quantize), and the results are copied to q_host [tokens][d/2] and scales_host
+ * [tokens][d/32] -- three copies and one launch, all asynchronous and in order on `stream`; nothing is
+ * allocated.  The host buffers must stay valid until the stream has passed the call (page-locked memory makes
+ * the copies truly asynchronous); calls on different streams with different work buffers overlap their copies
+ * and kernels.  The copies dominate: this path runs at the host link's rate, not the kernel's. */
+kq_status_t kroquant_quantize_host(const void *X_host, int64_t tokens, int d, const kroquant_factors_t *f,
+                                   uint8_t *q_host, uint8_t *scales_host, void *X_work, uint8_t *q_work,
+                                   uint8_t *scales_work, void *stream);
+
 /* Same, with the transform code path chosen by the caller (tests and ablations). */
 kq_status_t kroquant_quantize_path(const void *X, int64_t tokens, int d,
                                    const kroquant_factors_t *f, uint8_t *q_packed,

@@ -24,7 +24,7 @@ EXPORTS = [
     "kroquant_factors_destroy", "kroquant_quantize_ex", "kroquant_transform_f32_ex",
     "kroquant_scale_quantize_ex", "kroquant_mxfp4_quantize_ex", "kroquant_quantize_dual",
     "kroquant_fwht_quantize", "kroquant_fwht_transform_f32",
-    "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize",
+    "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize", "kroquant_quantize_host",
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
     "kroquant_debug_set_umma_config", "kroquant_debug_set_boundary", "kroquant_debug_set_distribution", "kroquant_debug_set_compare_kernels", "kroquant_launch_count", "kroquant_last_device_error",
@@ -74,6 +74,7 @@ def load_library() -> C.CDLL:
     L.kroquant_factors_n_sets.argtypes = [vp]
     L.kroquant_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
     L.kroquant_quantize_path.argtypes = [vp, i64, i32, vp, vp, vp, i32, vp]
+    L.kroquant_quantize_host.argtypes = [vp, i64, i32, vp, vp, vp, vp, vp, vp, vp]
     L.kroquant_dequantize.argtypes = [vp, vp, i64, i32, vp, vp, i32, vp]
     L.kroquant_scale_quantize.argtypes = [vp, i64, i32, vp, vp, vp, vp]
     L.kroquant_mxfp4_quantize.argtypes = [vp, i64, i32, vp, vp, vp]
@@ -356,46 +357,18 @@ def quantize_from_host(X_host: torch.Tensor, factors: Factors, X_dev: torch.Tens
     return q_host, s_host
 
 
-class HostPipeline:
-    """Host-to-host quantization with the three phases on their own streams, so that the upload of
-    call i+1, the kernel of call i and the download of call i-1 overlap (PCIe is full duplex).
-    Buffers may be reused from call to call: a buffer's next writer waits for its last reader."""
-
-    def __init__(self, device=None):
-        self.h2d = torch.cuda.Stream(device)
-        self.compute = torch.cuda.Stream(device)
-        self.d2h = torch.cuda.Stream(device)
-        self._last_kernel = {}      # X_dev.data_ptr() -> event after the kernel that read it
-        self._last_download = {}    # q_dev.data_ptr() -> event after the copy that read it
-
-    def submit(self, X_host, factors: Factors, X_dev, q_dev, s_dev, q_host, s_host):
-        ev = self._last_kernel.get(X_dev.data_ptr())
-        if ev is not None:
-            self.h2d.wait_event(ev)
-        with torch.cuda.stream(self.h2d):
-            X_dev.copy_(X_host, non_blocking=True)
-        up = torch.cuda.Event()
-        up.record(self.h2d)
-        self.compute.wait_event(up)
-        ev = self._last_download.get(q_dev.data_ptr())
-        if ev is not None:
-            self.compute.wait_event(ev)
-        kroquant_quantize(X_dev, factors, q_dev, s_dev, stream=self.compute)
-        done = torch.cuda.Event()
-        done.record(self.compute)
-        self._last_kernel[X_dev.data_ptr()] = done
-        self.d2h.wait_event(done)
-        with torch.cuda.stream(self.d2h):
-            q_host.copy_(q_dev, non_blocking=True)
-            s_host.copy_(s_dev, non_blocking=True)
-        down = torch.cuda.Event()
-        down.record(self.d2h)
-        self._last_download[q_dev.data_ptr()] = down
-
-    def synchronize(self):
-        self.h2d.synchronize()
-        self.compute.synchronize()
-        self.d2h.synchronize()
+def kroquant_quantize_host(X_host: torch.Tensor, factors: Factors, q_host: torch.Tensor, s_host: torch.Tensor,
+                           X_work: torch.Tensor, q_work: torch.Tensor, s_work: torch.Tensor, stream=None) -> None:
+    """Host tensors in, host tensors out, through the caller's device work buffers: one C call that issues the
+    upload, the kernel and the two downloads in order on `stream` (asynchronous when the host tensors are pinned)."""
+    tokens, d = X_host.shape
+    assert X_host.dtype == torch.bfloat16 and X_host.is_contiguous() and not X_host.is_cuda
+    assert q_host.shape == (tokens, d // 2) and s_host.shape == (tokens, d // 32) and not q_host.is_cuda
+    assert X_work.is_cuda and X_work.shape == X_host.shape and q_work.shape == q_host.shape and s_work.shape == s_host.shape
+    _check(load_library().kroquant_quantize_host(
+        C.c_void_p(X_host.data_ptr()), tokens, d, factors._h, C.c_void_p(q_host.data_ptr()), C.c_void_p(s_host.data_ptr()),
+        C.c_void_p(X_work.data_ptr()), C.c_void_p(q_work.data_ptr()), C.c_void_p(s_work.data_ptr()), C.c_void_p(_stream(stream))),
+        "kroquant_quantize_host")
 
 
 def kroquant_block_grad(X: torch.Tensor, G: torch.Tensor, n_sets: int = 1, out: Optional[torch.Tensor] = None,

@@ -637,6 +637,29 @@ kq_status_t kroquant_quantize(const void* X, int64_t tokens, int d, const kroqua
     return kroquant_quantize_ex(X, KQ_X_BF16, tokens, d, f, q_packed, scales, KQ_SCALES_ROWMAJOR, KQ_PATH_AUTO, stream);
 }
 
+kq_status_t kroquant_quantize_host(const void* X_host, int64_t tokens, int d, const kroquant_factors_t* f,
+                                   uint8_t* q_host, uint8_t* scales_host, void* X_work, uint8_t* q_work,
+                                   uint8_t* scales_work, void* stream) {
+    if (!X_host || !q_host || !scales_host || !X_work || !q_work || !scales_work) return KQ_ERR_NULL;
+    kq_status_t rc = check_shape(tokens, d);
+    if (rc != KQ_OK) return rc;
+    rc = check_factors_for(f, d);
+    if (rc != KQ_OK) return rc;
+    if (!aligned16(X_work) || !aligned16(q_work)) return KQ_ERR_ALIGN;
+    if (tokens == 0) return KQ_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t n = (size_t)tokens * (size_t)d;
+    if (cudaMemcpyAsync(X_work, X_host, n * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) { (void)cudaGetLastError(); return KQ_ERR_CUDA; }
+    rc = kroquant_quantize(X_work, tokens, d, f, q_work, scales_work, stream);
+    if (rc != KQ_OK) return rc;
+    if (cudaMemcpyAsync(q_host, q_work, n / 2, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(scales_host, scales_work, n / 32, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KQ_ERR_CUDA;
+    }
+    return KQ_OK;
+}
+
 kq_status_t kroquant_transform_f32_ex(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d,
                                       const kroquant_factors_t* f, float* Y, kq_path_t path, void* stream) {
     if (!X || !Y) return KQ_ERR_NULL;

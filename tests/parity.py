@@ -103,3 +103,32 @@ def check_codes(q_gpu, s_gpu, q_or, s_or, Y_or, exact: bool, x_dtype: str = "bf1
         assert n_diff <= max(1, MAX_FRACTION * t * d), f"P2: {n_diff} code mismatches"
     return {"code_mismatches": n_diff, "scale_mismatches": n_sdiff,
             "zero_sign_only": int(zero_sign.sum())}
+
+
+def check_codes_chunked(q_gpu, s_gpu, x_bits_rows, oracle_quantize, tokens: int, exact: bool, x_dtype: str = "bf16",
+                        chunk: int = 2048) -> dict:
+    """Whole-tensor P0/P2/P3 check with bounded host memory: the oracle runs on `chunk` token rows at a time.
+
+    q_gpu, s_gpu: the device results (anything sliceable by row range that yields NumPy arrays through
+    ``np.asarray`` / ``.cpu().numpy()``); x_bits_rows(r0, r1) -> uint16 input rows; oracle_quantize(bits) ->
+    (q, s, Y).  Every row is compared.  A chunk whose bytes are identical to the oracle's is accepted at once;
+    the others go through check_codes, and the 1e-4 limits are applied to the chunk and to the whole tensor."""
+    total = {"code_mismatches": 0, "scale_mismatches": 0, "zero_sign_only": 0, "rows": 0}
+    d = None
+    for r0 in range(0, tokens, chunk):
+        r1 = min(tokens, r0 + chunk)
+        q_or, s_or, Y = oracle_quantize(x_bits_rows(r0, r1))
+        qg, sg = q_gpu[r0:r1], s_gpu[r0:r1]
+        if hasattr(qg, "cpu"):
+            qg, sg = qg.cpu().numpy(), sg.cpu().numpy()
+        d = Y.shape[1]
+        total["rows"] += r1 - r0
+        if np.array_equal(qg, q_or) and np.array_equal(sg, s_or):
+            continue
+        r = check_codes(qg, sg, q_or, s_or, Y, exact=exact, x_dtype=x_dtype)
+        for k in ("code_mismatches", "scale_mismatches", "zero_sign_only"):
+            total[k] += r[k]
+    assert total["rows"] == tokens
+    assert total["code_mismatches"] <= max(1, MAX_FRACTION * tokens * d), f"P2: {total['code_mismatches']} code mismatches"
+    assert total["scale_mismatches"] <= max(1, MAX_FRACTION * tokens * d / 32), f"P3: {total['scale_mismatches']} scale mismatches"
+    return total

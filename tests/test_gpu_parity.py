@@ -244,3 +244,22 @@ def test_error_codes(B):
     assert L.kroquant_quantize(px, 4, 64, f._h, pq, ps, st) == 0
     assert B.kroquant_launch_count() == n0 + 1
     torch.cuda.synchronize()
+
+
+def test_host_buffer_entry_point_equals_device_path(B):
+    """kroquant_quantize_host: pinned host tensors in and out through caller-owned device work buffers, one C call."""
+    Xb = W.gen_activations(spec(300, 1152, seed=12))
+    f = B.Factors.create(W.gen_factors(12))
+    X = dev_bf16(Xb)
+    q_ref, s_ref = B.kroquant_quantize(X, f)
+    hx = torch.from_numpy(Xb.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    hq = torch.empty((300, 576), dtype=torch.uint8).pin_memory()
+    hs = torch.empty((300, 36), dtype=torch.uint8).pin_memory()
+    xw, qw, sw = torch.empty_like(X), torch.empty_like(q_ref), torch.empty_like(s_ref)
+    st = torch.cuda.Stream()
+    n0 = B.kroquant_launch_count()
+    for _ in range(2):
+        B.kroquant_quantize_host(hx, f, hq, hs, xw, qw, sw, stream=st)
+    st.synchronize()
+    assert B.kroquant_launch_count() == n0 + 2
+    assert np.array_equal(hq.numpy(), host(q_ref)) and np.array_equal(hs.numpy(), host(s_ref))
