@@ -958,12 +958,77 @@ def run_layer(args):
         "device_error": B.kroquant_last_device_error()}), flush=True)
 
 
+def run_timeline(args):
+    """Where a call's time goes at the kernel boundary: eight back-to-back calls of one shape in a CUDA graph, run on
+    the timeline build of the library (per-CTA global-timer marks, see kroquant_debug_set_timeline).  For the KroQuant
+    kernel and the two comparison kernels: time of each mark relative to the end of the LAST CTA of the call before,
+    minimum / median / maximum over the CTAs, averaged over calls 2..7; and the call period.  The marks cost a few
+    per cent; this is a diagnosis, never a bench value."""
+    import torch
+    from paper_2607_21446_b200 import binding as B, build as kbuild
+    if not os.path.exists(kbuild.LIB_TIMELINE):
+        kbuild.build_timeline()
+    B.use_library(kbuild.LIB_TIMELINE)
+    B.load_library()
+    t, d = (int(v) for v in args.timeline.lower().split("x"))
+    ncall = 8
+    stream = torch.cuda.Stream()
+    sp = W.ActivationSpec("tl", min(t, 8192), d, seed=3, outlier_channels=max(1, d // 200), outlier_gain=100.0)
+    x0 = torch.from_numpy(W.gen_activations(sp).view(np.int16)).cuda().view(torch.bfloat16)
+    x0 = x0.repeat((t + x0.shape[0] - 1) // x0.shape[0], 1)[:t].contiguous()
+    Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, ncall)]
+    q = torch.empty((t, d // 2), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((t, d // 32), dtype=torch.uint8, device="cuda")
+    f = B.Factors.create(W.gen_factors(3))
+    sv = torch.from_numpy(W.gen_channel_scales(3, d)).cuda()
+    marks = torch.zeros(64 * 4096 * 8, dtype=torch.int64, device="cuda")
+    names = ["cta_start", "wait_returned", "first_tile_ready", "producer_done", "epilogue_done", "cta_end"]
+    out = {"timeline": args.timeline, "calls": ncall, "unit": "us after the last CTA of the previous call ended (min/median/max over CTAs)"}
+    for kname, fn in (("kroquant", lambda x: B.kroquant_quantize(x, f, q, sc, stream=stream)),
+                      ("plain_mxfp4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)),
+                      ("scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream))):
+        B.kroquant_debug_set_timeline(None)
+        with torch.cuda.stream(stream):
+            for x in Xs:
+                fn(x)
+            torch.cuda.synchronize()
+            B.kroquant_debug_set_timeline(marks)           # launch slots restart at 0: the captured calls get 0..7
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for x in Xs:
+                    fn(x)
+            for _ in range(5):
+                g.replay()
+            torch.cuda.synchronize()
+            marks.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+        a = marks.cpu().numpy().reshape(64, 4096, 8)
+        ends = [a[k, a[k, :, 0] > 0, 5].max() for k in range(ncall)]
+        rows = {n: np.zeros(3) for n in names}
+        periods = []
+        for k in range(2, ncall):
+            live = a[k, :, 0] > 0
+            for i, n in enumerate(names):
+                v = (a[k, live, i] - ends[k - 1]) / 1e3
+                rows[n] += np.array([v.min(), np.median(v), v.max()]) / (ncall - 2)
+            periods.append((ends[k] - ends[k - 1]) / 1e3)
+        out[kname] = {"period_us": round(float(np.mean(periods)), 2), "ctas": int((a[2, :, 0] > 0).sum()),
+                      "tiles_per_cta_max": int(a[2, :, 6].max()),
+                      **{n: [round(float(x), 2) for x in rows[n]] for n in names}}
+    B.kroquant_debug_set_timeline(None)
+    out["device_error"] = B.kroquant_last_device_error()
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", action="store_true",
                     help="the paper's two latency tables (Q4 / Scale / K1 / K2, FP16) on this GPU")
     ap.add_argument("--sweep", action="store_true",
                     help="tokens x d sweep of KroQuant / Scale / bare MXFP4 (one JSON line per point)")
+    ap.add_argument("--timeline", default=None, metavar="TOKENSxD",
+                    help="per-CTA timeline of back-to-back calls at the kernel boundary (timeline build of the library)")
     ap.add_argument("--points", default=None, metavar="TOKENSxD,...", help="with --sweep: only these points")
     ap.add_argument("--single", default=None, metavar="TOKENSxD",
                     help="profiling aid: a few eager launches of one shape, e.g. 4608x12288")
@@ -986,12 +1051,14 @@ def main():
                     help="run the multi-rank launch / barrier / reduction logic on CPU ranks (gloo) with a stub step")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.table or args.sweep or args.single or args.calib
-                                                                  or args.gemm_fp4 or args.layer):
+                                                                  or args.gemm_fp4 or args.layer or args.timeline):
         sys.exit(relaunch_under_torchrun(sys.argv[1:], args.gpus))
     if args.dist_selftest:
         return run_dist_selftest(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.table:
+    if args.timeline:
+        run_timeline(args)
+    elif args.table:
         run_table(args)
     elif args.sweep:
         run_sweep(args)

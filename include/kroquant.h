@@ -231,6 +231,13 @@ kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles);
  * Process-wide; other values give KQ_ERR_UNSUPPORTED. */
 kq_status_t kroquant_debug_set_compare_kernels(int staged);
 
+/* Timeline builds only (the library compiled with -DKQ_TIMELINE, `python -m paper_2607_21446_b200.build
+ * --timeline`; the ordinary build returns KQ_ERR_UNSUPPORTED): every CTA of the quantizer kernels writes the
+ * global timer at six points of its life (start, dependency wait returned, first tile ready, producer done,
+ * epilogue done, end) into marks, DEVICE int64 [64 launch slots][4096 CTAs][8]; launch k after this call writes
+ * slot k % 64.  NULL switches the marks off.  Synchronize before reading.  A measuring aid, not a product path. */
+kq_status_t kroquant_debug_set_timeline(void *marks);
+
 /* The W4A4 product of the quantized layer (Section 3.4: O = Q(A T) Q(W~)^T + A T L R):
  *     out[m][n] = sum_k a[m][k] 2^(sa[m][k/32] - 127) * b[n][k] 2^(sb[n][k/32] - 127)  (+ add[m][n])
  * on the block-scaled FP4 tensor-core path (fp32 accumulation).  a_codes [M][K/2] and b_codes

@@ -27,7 +27,7 @@ EXPORTS = [
     "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize", "kroquant_quantize_host",
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
-    "kroquant_debug_set_umma_config", "kroquant_debug_set_boundary", "kroquant_debug_set_distribution", "kroquant_debug_set_compare_kernels", "kroquant_launch_count", "kroquant_last_device_error",
+    "kroquant_debug_set_umma_config", "kroquant_debug_set_boundary", "kroquant_debug_set_distribution", "kroquant_debug_set_compare_kernels", "kroquant_debug_set_timeline", "kroquant_launch_count", "kroquant_last_device_error",
     "kroquant_status_string",
     "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
@@ -84,6 +84,7 @@ def load_library() -> C.CDLL:
     L.kroquant_debug_set_boundary.argtypes = [i32, i32]
     L.kroquant_debug_set_distribution.argtypes = [i32, i32]
     L.kroquant_debug_set_compare_kernels.argtypes = [i32]
+    L.kroquant_debug_set_timeline.argtypes = [vp]
     L.kroquant_launch_count.argtypes = []
     L.kroquant_launch_count.restype = i64
     L.kroquant_last_device_error.argtypes = [vp, C.POINTER(i32)]
@@ -329,6 +330,16 @@ def kroquant_debug_set_boundary(trigger: int, prefetch_tiles: int) -> None:
 
 def kroquant_debug_set_distribution(dynamic: bool, unit_tiles: int = 1) -> None:
     _check(load_library().kroquant_debug_set_distribution(int(dynamic), unit_tiles), "kroquant_debug_set_distribution")
+
+
+def use_library(path: str) -> None:
+    """Load another build of the library (the timeline build) instead of libkroquant.so; call before anything else."""
+    global LIB_PATH, _lib
+    LIB_PATH, _lib = path, None
+
+
+def kroquant_debug_set_timeline(marks: Optional[torch.Tensor]) -> None:
+    _check(load_library().kroquant_debug_set_timeline(_ptr(marks)), "kroquant_debug_set_timeline")
 
 
 def kroquant_debug_set_compare_kernels(staged: bool) -> None:

@@ -32,6 +32,20 @@ def _stale() -> bool:
     return any(os.path.getmtime(p) > t for p in SOURCES + HEADERS + [os.path.abspath(__file__)])
 
 
+LIB_TIMELINE = os.path.join(PKG, "libkroquant_timeline.so")
+
+
+def build_timeline() -> str:
+    """The same library with per-CTA timeline marks compiled in (-DKQ_TIMELINE): a measuring aid for
+    `bench.py --timeline`, never loaded by the product path."""
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    res = subprocess.run([nvcc] + NVCC_FLAGS + ["-DKQ_TIMELINE", "-o", LIB_TIMELINE] + SOURCES, capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed building libkroquant_timeline.so")
+    return LIB_TIMELINE
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
@@ -46,4 +60,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    if "--timeline" in sys.argv[1:]:
+        print(build_timeline())
+    else:
+        print(build(force=True, verbose=True))

@@ -38,6 +38,31 @@ namespace kq {
 
 __device__ int g_kq_device_error = 0;
 
+// Timeline marks (build with -DKQ_TIMELINE; compiled out otherwise): every CTA of a launch writes %globaltimer
+// at six points of its life into a caller-supplied buffer, 8 words per CTA, 4096 CTAs per launch slot:
+//   0 CTA start   1 dependency wait returned (producer)   2 first tile ready for the epilogue
+//   3 producer has issued its last tile   4 epilogue group 0 finished   5 CTA end   6 tiles issued
+#ifdef KQ_TIMELINE
+__device__ long long* g_kq_timeline = nullptr;
+__device__ __forceinline__ void tl_mark(int slot, int i) {
+    long long* p = g_kq_timeline;
+    if (p && blockIdx.x < 4096) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p[((size_t)slot * 4096 + blockIdx.x) * 8 + i] = (long long)t;
+    }
+}
+__device__ __forceinline__ void tl_value(int slot, int i, long long v) {
+    long long* p = g_kq_timeline;
+    if (p && blockIdx.x < 4096) p[((size_t)slot * 4096 + blockIdx.x) * 8 + i] = v;
+}
+#define KQ_TL_MARK(slot, i) tl_mark(slot, i)
+#define KQ_TL_VALUE(slot, i, v) tl_value(slot, i, v)
+#else
+#define KQ_TL_MARK(slot, i) ((void)0)
+#define KQ_TL_VALUE(slot, i, v) ((void)0)
+#endif
+
 constexpr int kTileRows = 128;                    // blocks (flat rows) per MMA tile = TMEM lanes
 constexpr int kTileBytes = kTileRows * 64;        // 8 KB of bf16 per tile
 constexpr int kBTermBytes = 32 * 64;              // one bf16 term of K^T: 32 rows (n) x 64 B (k)
@@ -353,6 +378,7 @@ struct UmmaProblem {
     int prefetch_stride; // dynamic distribution: number of CTAs that run at once (see the prefetch loop)
     int64_t n_tiles;     // PB=false: 128-row tiles
     int unit_tiles;      // PB=false: consecutive tiles per work unit (PB: kPbCols)
+    int tl_slot;         // timeline builds: which launch slot of the mark buffer this launch writes
     int dynamic;         // 1: the grid has one CTA per unit and running CTAs take over the units of CTAs that
                          // have not started yet (cluster launch control); 0: CTA b takes units b, b + gridDim.x, ...
 };
@@ -396,9 +422,11 @@ constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
 //   kOpScale  the per-channel "Scale" comparison (Section 4.4; Appendix D, Smoothing): y = x * s, one correctly
 //     rounded float product per element.  In the flat view every block of a tile belongs to a different block
 //     column, so each thread needs its own 32 multipliers (128 bytes, twice the bytes of its activations): the
-//     whole vector s[d] is copied once per CTA into shared memory (behind the stages; 16-byte chunk v of column j
-//     at chunk v ^ (j & 7), so that the eight lanes of a quarter warp, which hold consecutive columns, read eight
-//     different bank groups), and a thread reads its column's 128 bytes from there.
+//     whole vector s[d] is copied once per CTA into shared memory (behind the stages) by TMA, as a matrix of
+//     d/32 rows of 128 bytes in the 128-byte-swizzle layout (16-byte chunk v of column j at chunk v ^ (j & 7), so
+//     that the eight lanes of a quarter warp, which hold consecutive columns, read eight different bank groups;
+//     tmap_q is that matrix's map), issued right behind the dependency wait so that it lands with the first tiles;
+//     a thread reads its column's 128 bytes from there.
 constexpr int kOpKron = 0, kOpPlain = 1, kOpScale = 2;
 template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone, int OP = kOpKron>
 // resident CTAs per SM the register budget must allow: (8,2,2) two; the one-warpgroup shapes three (two with the
@@ -557,6 +585,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     // run its set-up while this one still works (it must wait for the prerequisite grids before it touches
     // memory, as this kernel does).  Off when the library's programmatic-launch switch is off, and for
     // launches whose operand image was written by the kernel just before.
+    if (threadIdx.x == 0) KQ_TL_MARK(prob.tl_slot, 0);
     if (prob.early_trigger == 1) pdl_launch_dependents();
     bool more = true;
     if (threadIdx.x == 0) {
@@ -601,6 +630,18 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             prefetch_tile(PB ? (int)unit : (int)(unit * tpu), 0);
         }
         pdl_wait_prior_grid();
+        KQ_TL_MARK(prob.tl_slot, 1);
+        if (OP == kOpScale) {
+            // the multiplier vector is an ordinary input (it may come from the kernel before): fetched behind the wait
+            const uint32_t vec = (base + (uint32_t)L::kBytes + 1023u) & ~1023u;
+            // (boxes of all d/32 rows when there are at most 256, else of 128 rows; a box is always written whole,
+            //  rows beyond the vector as zeros, and the host sizes the buffer for whole boxes)
+            const int box_rows = prob.blocks_per_row <= 256 ? prob.blocks_per_row : 128;
+            const int n_boxes = (prob.blocks_per_row + box_rows - 1) / box_rows;
+            mbar_expect_tx(bar_b, (uint32_t)(n_boxes * box_rows) * 128u);
+            for (int bx = 0; bx < n_boxes; ++bx)
+                tma_load_2d(vec + 128u * (uint32_t)(bx * box_rows), &tmap_q, 0, bx * box_rows, bar_b);
+        }
         more = produce(true);
     }
     if (TC && warp == 1) {
@@ -618,6 +659,8 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             if (more) (void)produce(false);
+            KQ_TL_MARK(prob.tl_slot, 3);
+            KQ_TL_VALUE(prob.tl_slot, 6, issued);
             if (prob.early_trigger == 2) pdl_launch_dependents();
             // end of the stream: sentinel tiles (no copy, a plain arrival on the tile's barrier)
             for (int k = 0, n = issued; k < kSentinels && !producer_failed; ++k, ++n) {
@@ -685,17 +728,9 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
-        const uint32_t vec_base = base + (uint32_t)((L::kBytes + 127) & ~127);
+        const uint32_t vec_base = (base + (uint32_t)L::kBytes + 1023u) & ~1023u;
         if (OP == kOpScale) {
-            // the multiplier vector -> shared memory (it is an ordinary input: read after the dependency wait)
-            const int n_chunks = prob.blocks_per_row * 8;
-            for (int i = (int)threadIdx.x - 128; i < n_chunks; i += 128 * NG) {
-                const float4 m = __ldg(reinterpret_cast<const float4*>(chan_scale) + i);
-                const uint32_t j = (uint32_t)i >> 3, v = (uint32_t)i & 7u;
-                asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};"
-                             ::"r"(vec_base + 128u * j + 16u * (v ^ (j & 7u))), "f"(m.x), "f"(m.y), "f"(m.z), "f"(m.w) : "memory");
-            }
-            named_barrier_sync(2, 128 * NG);
+            if (!mbar_wait(bar_b, 0, abort_flag) && !*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
         }
         const int e_shared = (PB || !XF16 || !TC) ? 0 : __ldg(e_norm);
         double sq_sum = 0.0;                       // CALIB: this thread's sum of squared residuals
@@ -706,6 +741,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 break;
             }
             const int item = ring[n % kRingEntries];
+            if (n == 0 && threadIdx.x == 128) KQ_TL_MARK(prob.tl_slot, 2);
             if (item < 0) break;
             uint32_t acc[32];
             if (TC) {
@@ -878,6 +914,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 if (lane == 0) mbar_arrive(bar_done(s));
             }
         }
+        if (threadIdx.x == 128) KQ_TL_MARK(prob.tl_slot, 4);
         // the staging tile must not be released while a TMA store still reads it
         if (PB && !WRITE_Y && threadIdx.x == 128) bulk_wait_group_read<0>();
         if (CALIB) {
@@ -890,11 +927,12 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     // ---------------- teardown ----------------
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) KQ_TL_MARK(prob.tl_slot, 5);
     if (*abort_flag && threadIdx.x == 0) {
         // abort path only: let the copies this thread issued land before the CTA's shared
         // memory goes away (load m went to slot m % NS and completes phase (m / NS) & 1)
         int never = 0;
-        if (TC && !PB) (void)mbar_wait(bar_b, 0, &never);
+        if ((TC && !PB) || OP == kOpScale) (void)mbar_wait(bar_b, 0, &never);
         for (int m = (issued > NS ? issued - NS : 0); m < issued; ++m)
             if (!mbar_wait(bar_full(m % NS), (m / NS) & 1, &never))
                 atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_DRAIN);

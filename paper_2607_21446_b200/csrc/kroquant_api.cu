@@ -46,7 +46,8 @@ std::atomic<int> g_umma_prefetch{4};    // UmmaProblem::prefetch_tiles
 std::atomic<int> g_umma_dynamic{1};     // UmmaProblem::dynamic
 std::atomic<int> g_umma_unit_tiles{3};  // UmmaProblem::unit_tiles
 std::atomic<int> g_umma_unit_auto{1};   // 1: small launches use single-tile units (until the caller sets the unit)
-std::atomic<int> g_compare_staged{1};   // comparison quantizers: 1 = the tensor-core kernel's pipeline without its MMA stage,
+std::atomic<int> g_compare_staged{1};
+std::atomic<int> g_tl_next{0};          // timeline builds: next launch slot   // comparison quantizers: 1 = the tensor-core kernel's pipeline without its MMA stage,
                                         // 0 = the plain grid-stride kernels
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -273,6 +274,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     prob.early_trigger = (g_umma_pdl.load() != 0 && calib_sumsq == nullptr) ? g_umma_trigger.load() : 0;
     prob.prefetch_tiles = g_umma_pdl.load() != 0 ? g_umma_prefetch.load() : 0;
     prob.dynamic = g_umma_dynamic.load();
+    prob.tl_slot = g_tl_next.fetch_add(1) % 64;
     prob.unit_tiles = pb ? kq::kPbCols : g_umma_unit_tiles.load();
     CUtensorMap tmap;
     cuuint64_t dims[2], strides[1];
@@ -384,6 +386,7 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     prob.early_trigger = g_umma_pdl.load() != 0 ? g_umma_trigger.load() : 0;
     prob.prefetch_tiles = g_umma_pdl.load() != 0 ? g_umma_prefetch.load() : 0;
     prob.dynamic = g_umma_dynamic.load();
+    prob.tl_slot = g_tl_next.fetch_add(1) % 64;
     prob.unit_tiles = g_umma_unit_tiles.load();
     prob.n_rows = tokens * (int64_t)nb;
     prob.n_ttiles = 1;
@@ -404,7 +407,18 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
     const bool pdl = g_umma_pdl.load() != 0;
     bool big = cps_set == 0 ? big_ctas : g_umma_cfg.load() == 2;
-    const int vec = chan_scale ? d * 4 + 128 : 0;              // the multiplier vector behind the stages
+    const int box_rows = nb <= 256 ? nb : 128;                 // rows of one TMA box of the multiplier matrix
+    const int vec = chan_scale ? (nb + box_rows - 1) / box_rows * box_rows * 128 + 1024 : 0;   // whole boxes, 1 KB-aligned
+    CUtensorMap tmap_s = tmap;
+    if (chan_scale) {
+        // s[d] as [d/32 rows][32 floats]: one 128-byte-swizzled row per block column
+        const cuuint64_t sdims[2] = {32, (cuuint64_t)nb}, sstrides[1] = {128};
+        const cuuint32_t sbox[2] = {32, (cuuint32_t)box_rows};
+        if (enc(&tmap_s, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(chan_scale), sdims, sstrides, sbox, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return KQ_ERR_CUDA;
+    }
     if (chan_scale) {
         constexpr int kSmemPerSm = 233472, kSmemReserved = 1024;
         const int big_bytes = kq::UmmaSmem<8, false>::kDynBytes + vec, small_bytes = kq::UmmaSmem<4, false>::kDynBytes + vec;
@@ -421,7 +435,7 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
         if (prob.early_trigger == 2) prob.early_trigger = 1;
     }
 #define KQ_LAUNCH_CMP(NS, NM, NG, XF, OPC) \
-    launch_umma<NS, NM, NG, false, XF, false, kq::kExtraNone, OPC>(tmap, tmap, nullptr, nullptr, prob, q, scales, nullptr, \
+    launch_umma<NS, NM, NG, false, XF, false, kq::kExtraNone, OPC>(tmap, tmap_s, nullptr, nullptr, prob, q, scales, nullptr, \
                                                                    nullptr, cps, pdl, st, nullptr, chan_scale, vec)
     if (chan_scale) {
         if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true, kq::kOpScale) : KQ_LAUNCH_CMP(4, 2, 2, true, kq::kOpScale);
@@ -881,6 +895,17 @@ kq_status_t kroquant_debug_set_compare_kernels(int staged) {
     if (staged < 0 || staged > 1) return KQ_ERR_UNSUPPORTED;
     g_compare_staged.store(staged);
     return KQ_OK;
+}
+
+kq_status_t kroquant_debug_set_timeline(void* marks) {
+#ifdef KQ_TIMELINE
+    g_tl_next.store(0);
+    long long* p = static_cast<long long*>(marks);
+    return cudaMemcpyToSymbol(kq::g_kq_timeline, &p, sizeof(p)) == cudaSuccess ? KQ_OK : KQ_ERR_CUDA;
+#else
+    (void)marks;
+    return KQ_ERR_UNSUPPORTED;
+#endif
 }
 
 int64_t kroquant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -95,7 +95,7 @@ def run_kroquant(B, Xb, G, path):
     return {**v, **c}
 
 
-@pytest.mark.parametrize("path", ["tensor", "alu"])
+@pytest.mark.parametrize("path", ["auto", "tensor", "alu"])
 def test_tiny_config(B, path):
     Xb = W.gen_activations(W.tiny_spec())
     r = run_kroquant(B, Xb, W.gen_factors(0), path)
@@ -109,7 +109,7 @@ def test_ragged_shapes(B, path, tokens, d):
     run_kroquant(B, Xb, W.gen_factors(tokens), path)
 
 
-@pytest.mark.parametrize("path", ["tensor", "alu"])
+@pytest.mark.parametrize("path", ["auto", "tensor", "alu"])
 def test_hadamard_and_lu_factors(B, path):
     Xb = W.gen_activations(spec(512, 1152, seed=9))
     X = dev_bf16(Xb)
