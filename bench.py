@@ -458,7 +458,7 @@ def run_ours(args):
     ms_burst, _ = time_graph(torch, None, g_kq, stream, min(args.steps, 50), 3)
     # the same graph for at least a second (its own clock samples): what the step costs once the power cap has
     # settled the SM clock; the headline above is the K steps the caller asked for
-    n_sus = max(args.steps, int(1.2 / (ms_step * 1e-3)))
+    n_sus = max(args.steps, int(args.sustained_seconds / (ms_step * 1e-3)))
     ms_sus, clocks_sus = time_graph(torch, dist, g_kq, stream, n_sus, 3, ClockSampler(smi_index))
     ms_sus = ranks.max(ms_sus)
     # end to end: pinned host inputs -> device -> quantize -> pinned host outputs
@@ -541,7 +541,7 @@ def run_ours(args):
                      "which the quantizer exceeds on its largest launches); frac_of_nominal_8tbs by the data-sheet figure",
         "sustained": {"steps": n_sus, "ms_per_step": round(ms_sus, 5), "GB/s": round(world * byts / (ms_sus * 1e-3) / 1e9, 1),
                       "frac_of_hbm_peak": round(byts / (ms_sus * 1e-3) / 1e9 / peak, 4), "clocks": clocks_sus,
-                      "note": "the same graph timed for at least 1.2 s, after the headline region"},
+                      "note": f"the same graph timed for at least {args.sustained_seconds} s, after the headline region"},
         "speedup_vs_scale_kernel": ms_scale / ms_step,
         "speedup_vs_plain_mxfp4": ms_plain / ms_step,
         "after_idle": {
@@ -608,12 +608,81 @@ def run_single(args):
                       "device_error": B.kroquant_last_device_error()}), flush=True)
 
 
+def run_point(torch, B, co, P, args, label, bits, tokens, G, seed, peak, peak_kind, stream, idx):
+    """One measured and parity-checked point: KroQuant (factor sets G: one shared set or one per block), Scale and bare
+    MXFP4 on the same input, each as a CUDA graph of back-to-back calls over rotating buffers (> 3 x L2).  `bits` holds
+    the first n0 <= tokens host rows; device row r is host row r % n0.  The C oracle then goes over EVERY row in
+    chunks of 2048 (that pass is its measured time, all host cores) and all three outputs are compared with it
+    (rules P0-P3 of tests/parity.py).  Prints one JSON line."""
+    n0, d = bits.shape
+    nbuf = min(28, max(3, int(400e6 // (tokens * d * 2)) + 1))
+    x0 = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    x0 = x0.repeat((tokens + n0 - 1) // n0, 1)[:tokens].contiguous()
+    Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, nbuf)]
+    q = torch.empty((tokens, d // 2), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((tokens, d // 32), dtype=torch.uint8, device="cuda")
+    f = B.Factors.create(G)
+    svh = W.gen_channel_scales(seed, d)
+    sv = torch.from_numpy(svh).cuda()
+    kernels = (("kroquant", lambda x: B.kroquant_quantize(x, f, q, sc, stream=stream)),
+               ("scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
+               ("plain_mxfp4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)))
+    res, clk = {}, {}
+    for name, fn in kernels:
+        g = capture(torch, [lambda x=x, fn=fn: fn(x) for x in Xs], stream)
+        # (every kernel is timed with the clock sampler running: the sampler's start-up keeps the GPU under
+        #  load for some hundred milliseconds before the timed region, and all three must see the same regime)
+        ms, c = time_graph(torch, None, g, stream, max(5, args.steps // 10), 3, ClockSampler(idx))
+        res[name] = ms * 1e3 / nbuf
+        clk[name] = {"sm_mhz": c.get("sm_mhz"), "reasons": c.get("reasons")}
+
+    def rows(r0, r1):
+        return bits[np.arange(r0, r1) % n0]
+    oracle_s = [0.0]
+
+    def timed(fn_or):
+        def run(b):
+            t0 = time.perf_counter()
+            out = fn_or(b)
+            oracle_s[0] += time.perf_counter() - t0
+            return out
+        return run
+    parity = {}
+    try:
+        with torch.cuda.stream(stream):
+            for name, fn in kernels:
+                fn(x0)
+                stream.synchronize()
+                if name == "kroquant":
+                    parity[name] = P.check_codes_chunked(q, sc, rows, timed(lambda b: co.quantize(b, G)), tokens, exact=False)
+                elif name == "scale":
+                    parity[name] = P.check_codes_chunked(q, sc, rows, lambda b: co.scale_quantize(b, svh), tokens, exact=True)
+                else:
+                    parity[name] = P.check_codes_chunked(q, sc, rows, co.plain_quantize, tokens, exact=True)
+        parity["status"] = "ok"
+    except AssertionError as e:          # report, never hide
+        parity["status"] = "FAILED"
+        parity["error"] = str(e)[:200]
+    byt = W.algorithmic_bytes(tokens, d)
+    print(json.dumps({
+        "point": label, "shape": f"{tokens}x{d}", "factor_sets": int(G.shape[0]),
+        "us": {k: round(v, 2) for k, v in res.items()},
+        "GB/s": {k: round(byt / v / 1e3, 1) for k, v in res.items()},
+        "frac_of_hbm_peak": {k: round(byt / v / 1e3 / peak, 4) for k, v in res.items()},
+        "frac_of_nominal_8tbs": {k: round(byt / v / 1e3 / 8000.0, 4) for k, v in res.items()},
+        "tokens_per_s": round(tokens / (res["kroquant"] * 1e-6)),
+        "scale_over_kroquant": round(res["scale"] / res["kroquant"], 3),
+        "plain_over_kroquant": round(res["plain_mxfp4"] / res["kroquant"], 3),
+        "parity": parity,
+        "cpu_oracle_s": round(oracle_s[0], 3), "cpu_oracle_rows": tokens, "cpu_cores": os.cpu_count(),
+        "clocks": clk, "peak": f"{peak} GB/s of {peak_kind}", "buffers": nbuf,
+        "device_error": B.kroquant_last_device_error()}), flush=True)
+
+
 def run_sweep(args):
-    """The sweep config: tokens x d grid; KroQuant (one shared set), Scale and bare MXFP4 on the same input, each
-    as a CUDA graph of back-to-back calls over rotating buffers (> 3 x L2).  Every timed point is parity-checked
-    in the same run: the C oracle goes over EVERY row of the tensor in chunks of 2048 rows (that pass is also the
-    oracle's measured time, all host cores), and all three kernels' outputs are compared with it (rules P0-P3 of
-    tests/parity.py).  One JSON line per point; --points TOKENSxD,... restricts the grid."""
+    """The sweep config (tokens x d grid, one shared factor set), or with --configs the PixArt-, SANA- and
+    FLUX-shaped tensors of the other workload configs (SANA also with one factor set per block): see run_point.
+    --points TOKENSxD,... restricts the sweep grid."""
     import torch
     from oracle import c_oracle as co
     from paper_2607_21446_b200 import binding as B
@@ -622,75 +691,23 @@ def run_sweep(args):
     peak, peak_kind = measured_peak()
     stream = torch.cuda.Stream()
     idx = torch.cuda.current_device()
+    if args.configs:
+        todo = [("tiny", W.tiny_spec(), 0, 0, False)]
+        todo += [(sp.name, sp, 1, i, False) for i, sp in enumerate(W.pixart_specs())]
+        for i, sp in enumerate(W.sana_specs()):
+            todo += [(sp.name, sp, 2, i, False), (sp.name + "_per_block", sp, 2, i, True)]
+        todo += [(sp.name, sp, 3, i, False) for i, sp in enumerate(W.flux_specs())]
+        for label, sp, seed, layer, per_block in todo:
+            bits = W.gen_activations(sp)
+            G = W.gen_factors(seed, n_sets=sp.d // 32 if per_block else 1, layer=layer)
+            run_point(torch, B, co, P, args, label, bits, sp.tokens, G, seed, peak, peak_kind, stream, idx)
+        return
     points = [(t, d) for t in W.SWEEP_TOKENS for d in W.SWEEP_D]
     if args.points:
         points = [tuple(int(v) for v in p.lower().split("x")) for p in args.points.split(",")]
     for tokens, d in points:
-        nbuf = min(28, max(3, int(400e6 // (tokens * d * 2)) + 1))
-        n0 = min(tokens, 4096)
-        bits = W.gen_activations(W.sweep_spec(n0, d))          # host generator on <= 4096 rows, tiled on the device
-        x0 = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
-        x0 = x0.repeat((tokens + n0 - 1) // n0, 1)[:tokens].contiguous()
-        Xs = [x0] + [torch.roll(x0, shifts=i, dims=0).contiguous() for i in range(1, nbuf)]
-        q = torch.empty((tokens, d // 2), dtype=torch.uint8, device="cuda")
-        sc = torch.empty((tokens, d // 32), dtype=torch.uint8, device="cuda")
-        G = W.gen_factors(4)
-        f = B.Factors.create(G)
-        svh = W.gen_channel_scales(4, d)
-        sv = torch.from_numpy(svh).cuda()
-        kernels = (("kroquant", lambda x: B.kroquant_quantize(x, f, q, sc, stream=stream)),
-                   ("scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
-                   ("plain_mxfp4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)))
-        res, clk = {}, None
-        for name, fn in kernels:
-            g = capture(torch, [lambda x=x, fn=fn: fn(x) for x in Xs], stream)
-            # (every kernel is timed with the clock sampler running: the sampler's start-up keeps the GPU under
-            #  load for some hundred milliseconds before the timed region, and all three must see the same regime)
-            ms, c = time_graph(torch, None, g, stream, max(5, args.steps // 10), 3, ClockSampler(idx))
-            res[name] = ms * 1e3 / nbuf
-            clk = clk or {}
-            clk[name] = {"sm_mhz": c.get("sm_mhz"), "reasons": c.get("reasons")}
-        # parity of the timed configuration, whole tensor; row r of the device tensor is host row r % n0
-        def rows(r0, r1):
-            return bits[np.arange(r0, r1) % n0]
-        oracle_s = [0.0]
-
-        def timed(fn_or):
-            def run(b):
-                t0 = time.perf_counter()
-                out = fn_or(b)
-                oracle_s[0] += time.perf_counter() - t0
-                return out
-            return run
-        parity = {}
-        try:
-            with torch.cuda.stream(stream):
-                for name, fn in kernels:
-                    fn(x0)
-                    stream.synchronize()
-                    if name == "kroquant":
-                        parity[name] = P.check_codes_chunked(q, sc, rows, timed(lambda b: co.quantize(b, G)), tokens, exact=False)
-                    elif name == "scale":
-                        parity[name] = P.check_codes_chunked(q, sc, rows, lambda b: co.scale_quantize(b, svh), tokens, exact=True)
-                    else:
-                        parity[name] = P.check_codes_chunked(q, sc, rows, co.plain_quantize, tokens, exact=True)
-            parity["status"] = "ok"
-        except AssertionError as e:          # report, never hide
-            parity["status"] = "FAILED"
-            parity["error"] = str(e)[:200]
-        byt = W.algorithmic_bytes(tokens, d)
-        print(json.dumps({
-            "sweep": f"{tokens}x{d}", "us": {k: round(v, 2) for k, v in res.items()},
-            "GB/s": {k: round(byt / v / 1e3, 1) for k, v in res.items()},
-            "frac_of_hbm_peak": {k: round(byt / v / 1e3 / peak, 4) for k, v in res.items()},
-            "tokens_per_s": round(tokens / (res["kroquant"] * 1e-6)),
-            "scale_over_kroquant": round(res["scale"] / res["kroquant"], 3),
-            "plain_over_kroquant": round(res["plain_mxfp4"] / res["kroquant"], 3),
-            "parity": parity,
-            "cpu_oracle_s": round(oracle_s[0], 3), "cpu_oracle_rows": tokens, "cpu_cores": os.cpu_count(),
-            "clocks": clk, "peak": f"{peak} GB/s of {peak_kind}", "buffers": nbuf,
-            "device_error": B.kroquant_last_device_error()}), flush=True)
-        del Xs, x0, q, sc
+        bits = W.gen_activations(W.sweep_spec(min(tokens, 4096), d))     # host generator on <= 4096 rows, tiled on the device
+        run_point(torch, B, co, P, args, f"sweep_{tokens}x{d}", bits, tokens, W.gen_factors(4), 4, peak, peak_kind, stream, idx)
 
 
 # The paper's two latency tables (Section 4.4 and Appendix A): (m, d) and its MI350 / FP16 numbers in
@@ -966,9 +983,7 @@ def run_timeline(args):
     per cent; this is a diagnosis, never a bench value."""
     import torch
     from paper_2607_21446_b200 import binding as B, build as kbuild
-    if not os.path.exists(kbuild.LIB_TIMELINE):
-        kbuild.build_timeline()
-    B.use_library(kbuild.LIB_TIMELINE)
+    B.use_library(kbuild.build_timeline())           # (re)built when missing or older than the sources
     B.load_library()
     t, d = (int(v) for v in args.timeline.lower().split("x"))
     ncall = 8
@@ -1029,6 +1044,8 @@ def main():
                     help="tokens x d sweep of KroQuant / Scale / bare MXFP4 (one JSON line per point)")
     ap.add_argument("--timeline", default=None, metavar="TOKENSxD",
                     help="per-CTA timeline of back-to-back calls at the kernel boundary (timeline build of the library)")
+    ap.add_argument("--configs", action="store_true",
+                    help="the tiny, PixArt-, SANA- (shared and per-block sets) and FLUX-shaped tensors, measured and parity-checked like --sweep")
     ap.add_argument("--points", default=None, metavar="TOKENSxD,...", help="with --sweep: only these points")
     ap.add_argument("--single", default=None, metavar="TOKENSxD",
                     help="profiling aid: a few eager launches of one shape, e.g. 4608x12288")
@@ -1047,10 +1064,12 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sustained-seconds", type=float, default=1.2,
+                    help="length of the extra sustained measurement of the headline graph (0: only --steps replays; for profilers)")
     ap.add_argument("--dist-selftest", action="store_true",
                     help="run the multi-rank launch / barrier / reduction logic on CPU ranks (gloo) with a stub step")
     args = ap.parse_args()
-    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.table or args.sweep or args.single or args.calib
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.table or args.sweep or args.configs or args.single or args.calib
                                                                   or args.gemm_fp4 or args.layer or args.timeline):
         sys.exit(relaunch_under_torchrun(sys.argv[1:], args.gpus))
     if args.dist_selftest:
@@ -1060,7 +1079,7 @@ def main():
         run_timeline(args)
     elif args.table:
         run_table(args)
-    elif args.sweep:
+    elif args.sweep or args.configs:
         run_sweep(args)
     elif args.single:
         run_single(args)

@@ -35,9 +35,13 @@ def _stale() -> bool:
 LIB_TIMELINE = os.path.join(PKG, "libkroquant_timeline.so")
 
 
-def build_timeline() -> str:
+def build_timeline(force: bool = False) -> str:
     """The same library with per-CTA timeline marks compiled in (-DKQ_TIMELINE): a measuring aid for
-    `bench.py --timeline`, never loaded by the product path."""
+    `bench.py --timeline`, never loaded by the product path.  Rebuilt when any source is newer."""
+    if not force and os.path.exists(LIB_TIMELINE):
+        t = os.path.getmtime(LIB_TIMELINE)
+        if not any(os.path.getmtime(p) > t for p in SOURCES + HEADERS + [os.path.abspath(__file__)]):
+            return LIB_TIMELINE
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     res = subprocess.run([nvcc] + NVCC_FLAGS + ["-DKQ_TIMELINE", "-o", LIB_TIMELINE] + SOURCES, capture_output=True, text=True)
     if res.returncode != 0:
@@ -61,6 +65,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 if __name__ == "__main__":
     if "--timeline" in sys.argv[1:]:
-        print(build_timeline())
+        print(build_timeline(force=True))
     else:
         print(build(force=True, verbose=True))
