@@ -48,6 +48,23 @@ def test_own_arm_line():
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     assert d["parity"]["status"] == "ok" and d["device_error"] == 0
     assert 0.05 < d["frac_of_hbm_peak"] < 1.3
+    assert abs(d["frac_of_nominal_8tbs"] - d["value"] / 8000.0) < 1e-9
+    su = d["sustained"]
+    assert su["steps"] >= d["steps"] and su["steps"] * su["ms_per_step"] >= 1000.0 and 0.05 < su["frac_of_hbm_peak"] < 1.3
+    one = c["one_thread"]
+    assert one is None or (one["cores"] == 1 and 0 < one["value"] < c["value"])
+    assert "kroquant_quantize_host" in e["api"]
+
+
+def test_sweep_point_line_carries_parity():
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--sweep", "--points", "1024x1152", "--steps", "50"],
+                         cwd=ROOT, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stderr[-2000:]
+    d = json.loads([l for l in res.stdout.strip().splitlines() if l.startswith("{")][0])
+    assert d["shape"] == "1024x1152" and d["parity"]["status"] == "ok" and d["device_error"] == 0
+    assert d["parity"]["scale"]["code_mismatches"] == 0 and d["parity"]["plain_mxfp4"]["code_mismatches"] == 0
+    assert d["parity"]["kroquant"]["rows"] == 1024 and d["cpu_oracle_rows"] == 1024 and d["cpu_oracle_s"] > 0
+    assert set(d["us"]) == {"kroquant", "scale", "plain_mxfp4"}
 
 
 def test_reference_arm_line():
