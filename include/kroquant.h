@@ -183,53 +183,76 @@ kq_status_t kroquant_transform_f32(const void *X, int64_t tokens, int d,
  * the 4-bit code the encoder's convert instruction gives (DEVICE uint8 [n]). */
 kq_status_t kroquant_debug_e2m1_codes(const float *v, int64_t n, uint8_t *codes, void *stream);
 
-/* Tuning hook for the tensor-core kernel.  config 0..7 selects (pipeline slots, MMA
- * issuer warps, epilogue warpgroups) = (2,2,1) (8,2,1) (8,2,2) (2,1,1) (4,1,1) (4,2,1)
- * (16,2,2) (16,2,4).  Until this function is called the library chooses by itself: (8,2,2) with 2 CTAs per SM
- * for shared-factor launches of more than one wave, (4,2,1) with 3 per SM otherwise (per-block sets: (4,1,1));
- * a call with ctas_per_sm > 0 makes config and ctas_per_sm explicit for every variant, ctas_per_sm = 0 returns
- * to the automatic choice (config is then ignored unless it is the default 2).  ctas_per_sm in 1..8 is the number of CTAs
- * that run on an SM at once (a cap on the persistent grid with the static distribution, a shared-memory
- * request that lets no more of them fit with the dynamic one); use_pdl != 0 (default) launches the quantizer
- * kernels with programmatic stream serialization and lets them signal launch completion before they end
- * (when: kroquant_debug_set_boundary), so that consecutive calls overlap their set-up with the tail of the
- * call before; every kernel of this library waits for its prerequisite grids before it touches memory.
- * Ordinary launches behind them (plain <<<>>> kernels, the framework's and the vendor libraries' kernels)
- * were checked to start only after the outputs are complete.  One exception was measured on driver 580: a
- * kernel launched by the caller with cudaLaunchKernelEx and a cluster dimension directly behind such a
- * chain began early; a kernel like that has to call cudaGridDependencySynchronize() first, or the caller
- * turns the early signal off with use_pdl = 0.  Process-wide. */
-kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl);
+/* Per-call tuning of the quantizer kernels (measurements, ablations, tests).  Results never depend on it.  A caller
+ * fills the struct with kroquant_tuning_default and changes what it wants; the *_tuned entry points below take it
+ * (NULL = defaults) and apply it to that one call on the calling thread: there is no process-wide tuning state.
+ * A field outside its range gives KQ_ERR_UNSUPPORTED and nothing is launched.
+ *
+ * config, ctas_per_sm: CTA shape of the tensor-core kernel.  config 0..7 selects (pipeline slots, MMA issuer warps,
+ *   epilogue warpgroups) = (2,2,1) (8,2,1) (8,2,2) (2,1,1) (4,1,1) (4,2,1) (16,2,2) (16,2,4).  ctas_per_sm = 0
+ *   (default): the library chooses: (8,2,2) with 2 CTAs per SM for shared-set launches of more than one wave,
+ *   (4,2,1) with 3 per SM otherwise (per-block sets: (4,1,1)); config is then ignored.  ctas_per_sm in 1..8 makes
+ *   both explicit: the number of CTAs that run on an SM at once (a cap on the persistent grid with the static
+ *   distribution, a shared-memory request that lets no more of them fit with the dynamic one).
+ * use_pdl (default 1): launch with programmatic stream serialization and let a kernel signal launch completion
+ *   before it ends, so that consecutive calls overlap their set-up with the tail of the call before; every kernel
+ *   of this library waits for its prerequisite grids before it touches memory.  Ordinary launches behind them
+ *   (plain <<<>>> kernels, the framework's and the vendor libraries' kernels) were checked to start only after the
+ *   outputs are complete.  One exception was measured on driver 580: a kernel launched by the caller with
+ *   cudaLaunchKernelEx and a cluster dimension directly behind such a chain began early; a kernel like that has to
+ *   call cudaGridDependencySynchronize() first, or the caller passes use_pdl = 0.
+ * trigger (default 2; acts while use_pdl is on): 0 = never signal before the end; 1 = every CTA signals at its
+ *   start; 2 = a CTA signals once it has no tile load left to issue, so that the next kernel's CTAs become
+ *   resident shortly before this one ends.  A launch whose tiles all run at once signals at its start unless 0.
+ * prefetch_tiles (0..64, default 4): before a CTA waits for its prerequisite grids it asks the L2 cache for its
+ *   first tiles of X (a prefetch moves no data into the SM and the L2 is where the previous kernel's writes land,
+ *   so the request is safe even if that kernel still produces X).
+ * dynamic, unit_tiles: how tiles (128 blocks of 32 channels) are handed to CTAs.  A unit is unit_tiles (1..16;
+ *   0 = automatic: 3, or 1 for launches of fewer than 8 tiles per SM) consecutive tiles (always 4 column tiles
+ *   with per-block sets).  dynamic = 0: a persistent grid, CTA b takes units b, b + grid, ...  dynamic = 1
+ *   (default): one CTA per unit in the grid; the CTAs that the hardware starts first take over the units of CTAs
+ *   that have not started (cluster launch control), so that a CTA on a slower path to memory simply takes fewer.
+ *   A launch whose units all fit the GPU at once uses the static form.  Calls that are meant to overlap on
+ *   several streams want the static one: a dynamic launch claims every CTA slot of the GPU.
+ * compare_staged (default 1): the two comparison quantizers of Section 4.4 (bare MXFP4 "Q4", per-channel "Scale")
+ *   run on the KroQuant kernel's own pipeline (TMA-staged tiles, same tile distribution and kernel-boundary
+ *   handling) with the tensor-core stage left out, so that the comparison measures the transform and not the
+ *   pipeline; 0: plain grid-stride CUDA-core kernels (also the fall-back for d > about 18 000, where the Scale
+ *   multipliers do not fit shared memory).  Same bits either way. */
+typedef struct kq_tuning {
+    int config;
+    int ctas_per_sm;
+    int use_pdl;
+    int trigger;
+    int prefetch_tiles;
+    int dynamic;
+    int unit_tiles;
+    int compare_staged;
+} kq_tuning_t;
 
-/* Tuning knobs for what happens at the boundary between two consecutive quantizer kernels (both only act
- * while use_pdl is on).  trigger: 0 = a kernel never signals launch completion before it ends; 1 = every
- * CTA signals at its start; 2 = a CTA signals once it has no tile load left to issue, so that the next
- * kernel's CTAs become resident shortly before this one ends.  prefetch_tiles (0..64):
- * before a CTA waits for its prerequisite grids it asks the L2 cache for its first prefetch_tiles tiles of
- * X (a prefetch moves no data into the SM and the L2 is where the previous kernel's writes land, so the
- * request is safe even if that kernel still produces X).  Defaults: trigger 2, prefetch_tiles 4; a launch
- * whose tiles all run at once signals at its start whatever the setting (unless trigger is 0).
- * KQ_ERR_UNSUPPORTED outside the ranges.  Process-wide. */
-kq_status_t kroquant_debug_set_boundary(int trigger, int prefetch_tiles);
+/* Writes the defaults {2, 0, 1, 2, 4, 1, 0, 1}.  NULL is ignored. */
+void kroquant_tuning_default(kq_tuning_t *t);
 
-/* How the tensor-core quantizer hands its tiles (128 blocks of 32 channels) to CTAs.  A unit is unit_tiles
- * (1..16, or 0 = automatic) consecutive tiles (always 4 column tiles with per-block factor sets).  dynamic = 0: a persistent
- * grid of at most ctas_per_sm CTAs per SM, CTA b takes units b, b + grid, ...  dynamic = 1: one CTA per unit
- * in the grid; the CTAs that the hardware starts first take over, besides their own unit, the units of CTAs
- * that have not started (cluster launch control), so that a CTA on a slower path to memory simply takes fewer.
- * Results do not depend on either setting.  Default: dynamic, 3 tiles per unit (1 for launches of fewer than 8
- * tiles per SM; unit_tiles = 0 selects that automatic rule again); a launch whose units all fit the GPU at once
- * uses the static form.  The dynamic form is the faster one for calls that follow one another in a
- * stream; calls that are meant to overlap on several streams want the static one, because a dynamic launch
- * claims every CTA slot of the GPU.  KQ_ERR_UNSUPPORTED outside the ranges.  Process-wide. */
-kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles);
-
-/* Which device code runs the two comparison quantizers of Section 4.4 (bare MXFP4 "Q4", per-channel "Scale"):
- * staged = 1 (default): the KroQuant kernel's own pipeline (TMA-staged tiles, same tile distribution and
- * kernel-boundary handling) with the tensor-core stage left out, so that the comparison measures the
- * transform and not the pipeline; staged = 0: plain grid-stride CUDA-core kernels.  Same bits either way.
- * Process-wide; other values give KQ_ERR_UNSUPPORTED. */
-kq_status_t kroquant_debug_set_compare_kernels(int staged);
+/* kroquant_quantize_ex, kroquant_quantize_dual, kroquant_transform_f32_ex, kroquant_scale_quantize_ex and
+ * kroquant_mxfp4_quantize_ex with the tuning of this one call (NULL = defaults).  Same arguments, layouts and
+ * error codes otherwise. */
+kq_status_t kroquant_quantize_tuned(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                    const kroquant_factors_t *f, uint8_t *q_packed, uint8_t *scales,
+                                    kq_scale_layout_t scale_layout, kq_path_t path, const kq_tuning_t *tuning,
+                                    void *stream);
+kq_status_t kroquant_quantize_dual_tuned(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                         const kroquant_factors_t *f, uint8_t *q_packed, uint8_t *scales,
+                                         kq_scale_layout_t scale_layout, void *AT_out, const kq_tuning_t *tuning,
+                                         void *stream);
+kq_status_t kroquant_transform_f32_tuned(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                         const kroquant_factors_t *f, float *Y, kq_path_t path,
+                                         const kq_tuning_t *tuning, void *stream);
+kq_status_t kroquant_scale_quantize_tuned(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d, const float *s,
+                                          uint8_t *q_packed, uint8_t *scales, kq_scale_layout_t scale_layout,
+                                          const kq_tuning_t *tuning, void *stream);
+kq_status_t kroquant_mxfp4_quantize_tuned(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
+                                          uint8_t *q_packed, uint8_t *scales, kq_scale_layout_t scale_layout,
+                                          const kq_tuning_t *tuning, void *stream);
 
 /* Timeline builds only (the library compiled with -DKQ_TIMELINE, `python -m paper_2607_21446_b200.build
  * --timeline`; the ordinary build returns KQ_ERR_UNSUPPORTED): every CTA of the quantizer kernels writes the

@@ -27,7 +27,8 @@ EXPORTS = [
     "kroquant_factors_get", "kroquant_factors_n_sets", "kroquant_quantize", "kroquant_quantize_host",
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
-    "kroquant_debug_set_umma_config", "kroquant_debug_set_boundary", "kroquant_debug_set_distribution", "kroquant_debug_set_compare_kernels", "kroquant_debug_set_timeline", "kroquant_launch_count", "kroquant_last_device_error",
+    "kroquant_tuning_default", "kroquant_quantize_tuned", "kroquant_quantize_dual_tuned", "kroquant_transform_f32_tuned",
+    "kroquant_scale_quantize_tuned", "kroquant_mxfp4_quantize_tuned", "kroquant_debug_set_timeline", "kroquant_launch_count", "kroquant_last_device_error",
     "kroquant_status_string",
     "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
@@ -80,10 +81,13 @@ def load_library() -> C.CDLL:
     L.kroquant_mxfp4_quantize.argtypes = [vp, i64, i32, vp, vp, vp]
     L.kroquant_transform_f32.argtypes = [vp, i64, i32, vp, vp, i32, vp]
     L.kroquant_debug_e2m1_codes.argtypes = [vp, i64, vp, vp]
-    L.kroquant_debug_set_umma_config.argtypes = [i32, i32, i32]
-    L.kroquant_debug_set_boundary.argtypes = [i32, i32]
-    L.kroquant_debug_set_distribution.argtypes = [i32, i32]
-    L.kroquant_debug_set_compare_kernels.argtypes = [i32]
+    L.kroquant_tuning_default.argtypes = [vp]
+    L.kroquant_tuning_default.restype = None
+    L.kroquant_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, i32, vp, vp]
+    L.kroquant_quantize_dual_tuned.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp, vp]
+    L.kroquant_transform_f32_tuned.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, vp]
+    L.kroquant_scale_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp]
+    L.kroquant_mxfp4_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, vp]
     L.kroquant_debug_set_timeline.argtypes = [vp]
     L.kroquant_launch_count.argtypes = []
     L.kroquant_launch_count.restype = i64
@@ -205,9 +209,28 @@ class Factors:
             pass
 
 
+class Tuning(C.Structure):
+    """kq_tuning_t: per-call tuning of the quantizer kernels (see include/kroquant.h).  ``Tuning()`` holds the
+    library's defaults; keyword arguments override single fields."""
+    _fields_ = [(n, C.c_int) for n in ("config", "ctas_per_sm", "use_pdl", "trigger", "prefetch_tiles", "dynamic",
+                                       "unit_tiles", "compare_staged")]
+
+    def __init__(self, **kw):
+        super().__init__()
+        load_library().kroquant_tuning_default(C.byref(self))
+        for k, v in kw.items():
+            if k not in dict(self._fields_):
+                raise TypeError(f"unknown tuning field {k}")
+            setattr(self, k, int(v))
+
+
+def _tuning(t: Optional["Tuning"]):
+    return None if t is None else C.cast(C.pointer(t), C.c_void_p)
+
+
 def kroquant_quantize(X: torch.Tensor, factors: Factors, q_packed: Optional[torch.Tensor] = None,
                       scales: Optional[torch.Tensor] = None, path: str = "auto", stream=None,
-                      scale_layout: str = "rowmajor"):
+                      scale_layout: str = "rowmajor", tuning: Optional[Tuning] = None):
     """(X bf16/fp16 [tokens, d], factors) -> (q_packed uint8 [tokens, d/2], scales uint8 [tokens, d/32]
     or, with scale_layout="tiled", a flat uint8 buffer in the 128 x 4 tiled layout)."""
     tokens, d = _x_shape(X)
@@ -215,15 +238,15 @@ def kroquant_quantize(X: torch.Tensor, factors: Factors, q_packed: Optional[torc
         q_packed = torch.empty((tokens, max(d // 2, 0)), dtype=torch.uint8, device=X.device)
     if scales is None:
         scales = _scale_buffer(tokens, d, scale_layout, X.device)
-    _check(load_library().kroquant_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(q_packed),
-                                               _ptr(scales), SCALE_LAYOUTS[scale_layout], PATHS[path],
-                                               C.c_void_p(_stream(stream))),
+    _check(load_library().kroquant_quantize_tuned(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(q_packed),
+                                                  _ptr(scales), SCALE_LAYOUTS[scale_layout], PATHS[path], _tuning(tuning),
+                                                  C.c_void_p(_stream(stream))),
            "kroquant_quantize")
     return q_packed, scales
 
 
 def kroquant_quantize_dual(X: torch.Tensor, factors: Factors, q_packed=None, scales=None, AT=None, stream=None,
-                           scale_layout: str = "rowmajor"):
+                           scale_layout: str = "rowmajor", tuning: Optional[Tuning] = None):
     """One pass: MXFP4(X T) and X T itself in X's dtype -> (q_packed, scales, AT)."""
     tokens, d = _x_shape(X)
     if q_packed is None:
@@ -232,9 +255,9 @@ def kroquant_quantize_dual(X: torch.Tensor, factors: Factors, q_packed=None, sca
         scales = _scale_buffer(tokens, d, scale_layout, X.device)
     if AT is None:
         AT = torch.empty_like(X)
-    _check(load_library().kroquant_quantize_dual(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(q_packed),
-                                                 _ptr(scales), SCALE_LAYOUTS[scale_layout], _ptr(AT),
-                                                 C.c_void_p(_stream(stream))), "kroquant_quantize_dual")
+    _check(load_library().kroquant_quantize_dual_tuned(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(q_packed),
+                                                       _ptr(scales), SCALE_LAYOUTS[scale_layout], _ptr(AT), _tuning(tuning),
+                                                       C.c_void_p(_stream(stream))), "kroquant_quantize_dual")
     return q_packed, scales, AT
 
 
@@ -260,7 +283,7 @@ def kroquant_fwht_transform_f32(X: torch.Tensor, Y=None, stream=None):
 
 
 def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, scales=None, stream=None,
-                            scale_layout: str = "rowmajor"):
+                            scale_layout: str = "rowmajor", tuning: Optional[Tuning] = None):
     tokens, d = _x_shape(X)
     if s.dtype != torch.float32 or not s.is_cuda or s.numel() != d or not s.is_contiguous():
         raise ValueError("s must be a contiguous CUDA float32 tensor [d]")
@@ -268,33 +291,34 @@ def kroquant_scale_quantize(X: torch.Tensor, s: torch.Tensor, q_packed=None, sca
         q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
     if scales is None:
         scales = _scale_buffer(tokens, d, scale_layout, X.device)
-    _check(load_library().kroquant_scale_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(s), _ptr(q_packed),
-                                                     _ptr(scales), SCALE_LAYOUTS[scale_layout],
-                                                     C.c_void_p(_stream(stream))),
+    _check(load_library().kroquant_scale_quantize_tuned(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(s), _ptr(q_packed),
+                                                        _ptr(scales), SCALE_LAYOUTS[scale_layout], _tuning(tuning),
+                                                        C.c_void_p(_stream(stream))),
            "kroquant_scale_quantize")
     return q_packed, scales
 
 
 def kroquant_mxfp4_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=None,
-                            scale_layout: str = "rowmajor"):
+                            scale_layout: str = "rowmajor", tuning: Optional[Tuning] = None):
     tokens, d = _x_shape(X)
     if q_packed is None:
         q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
     if scales is None:
         scales = _scale_buffer(tokens, d, scale_layout, X.device)
-    _check(load_library().kroquant_mxfp4_quantize_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(q_packed),
-                                                     _ptr(scales), SCALE_LAYOUTS[scale_layout],
-                                                     C.c_void_p(_stream(stream))),
+    _check(load_library().kroquant_mxfp4_quantize_tuned(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(q_packed),
+                                                        _ptr(scales), SCALE_LAYOUTS[scale_layout], _tuning(tuning),
+                                                        C.c_void_p(_stream(stream))),
            "kroquant_mxfp4_quantize")
     return q_packed, scales
 
 
-def kroquant_transform_f32(X: torch.Tensor, factors: Factors, Y=None, path: str = "auto", stream=None):
+def kroquant_transform_f32(X: torch.Tensor, factors: Factors, Y=None, path: str = "auto", stream=None,
+                           tuning: Optional[Tuning] = None):
     tokens, d = _x_shape(X)
     if Y is None:
         Y = torch.empty((tokens, d), dtype=torch.float32, device=X.device)
-    _check(load_library().kroquant_transform_f32_ex(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(Y),
-                                                    PATHS[path], C.c_void_p(_stream(stream))),
+    _check(load_library().kroquant_transform_f32_tuned(_ptr(X), X_DTYPES[X.dtype], tokens, d, factors._h, _ptr(Y),
+                                                       PATHS[path], _tuning(tuning), C.c_void_p(_stream(stream))),
            "kroquant_transform_f32")
     return Y
 
@@ -319,19 +343,6 @@ def kroquant_debug_e2m1_codes(v: torch.Tensor, stream=None) -> torch.Tensor:
     return codes
 
 
-def kroquant_debug_set_umma_config(config: int, ctas_per_sm: int, use_pdl: bool = True) -> None:
-    _check(load_library().kroquant_debug_set_umma_config(config, ctas_per_sm, int(use_pdl)),
-           "kroquant_debug_set_umma_config")
-
-
-def kroquant_debug_set_boundary(trigger: int, prefetch_tiles: int) -> None:
-    _check(load_library().kroquant_debug_set_boundary(trigger, prefetch_tiles), "kroquant_debug_set_boundary")
-
-
-def kroquant_debug_set_distribution(dynamic: bool, unit_tiles: int = 1) -> None:
-    _check(load_library().kroquant_debug_set_distribution(int(dynamic), unit_tiles), "kroquant_debug_set_distribution")
-
-
 def use_library(path: str) -> None:
     """Load another build of the library (the timeline build) instead of libkroquant.so; call before anything else."""
     global LIB_PATH, _lib
@@ -340,10 +351,6 @@ def use_library(path: str) -> None:
 
 def kroquant_debug_set_timeline(marks: Optional[torch.Tensor]) -> None:
     _check(load_library().kroquant_debug_set_timeline(_ptr(marks)), "kroquant_debug_set_timeline")
-
-
-def kroquant_debug_set_compare_kernels(staged: bool) -> None:
-    _check(load_library().kroquant_debug_set_compare_kernels(int(staged)), "kroquant_debug_set_compare_kernels")
 
 
 def kroquant_launch_count() -> int:

@@ -37,16 +37,21 @@ std::atomic<int64_t> g_launches{0};
 // ---- tensor-core kernel configuration ----------------------------------------
 // Defaults (measured on the 28-call FLUX step): the shared-factor bf16 kernel runs as (8 slots, 2 MMA warps,
 // 2 epilogue warpgroups) with 2 CTAs per SM, every other variant as compiled for it with 3 CTAs per SM.
-// ctas_per_sm 0 = that automatic choice; kroquant_debug_set_umma_config makes both explicit for all variants.
-std::atomic<int> g_umma_cfg{2};
-std::atomic<int> g_umma_ctas_per_sm{0};
-std::atomic<int> g_umma_pdl{1};
-std::atomic<int> g_umma_trigger{2};     // UmmaProblem::early_trigger of ordinary launches
-std::atomic<int> g_umma_prefetch{4};    // UmmaProblem::prefetch_tiles
-std::atomic<int> g_umma_dynamic{1};     // UmmaProblem::dynamic
-std::atomic<int> g_umma_unit_tiles{3};  // UmmaProblem::unit_tiles
-std::atomic<int> g_umma_unit_auto{1};   // 1: small launches use single-tile units (until the caller sets the unit)
-std::atomic<int> g_compare_staged{1};
+// ctas_per_sm 0 = that automatic choice; a tuning struct with ctas_per_sm > 0 makes both explicit for all variants.
+// The tuning of the current call.  The *_tuned entry points install the caller's struct for the duration of the call
+// on the calling thread; every other entry point sees the defaults.  Nothing here is process-wide.
+constexpr kq_tuning_t kDefaultTuning = {2, 0, 1, 2, 4, 1, 0, 1};
+thread_local kq_tuning_t t_tuning = kDefaultTuning;
+struct TuningScope {
+    kq_tuning_t saved;
+    explicit TuningScope(const kq_tuning_t* t) : saved(t_tuning) { t_tuning = t ? *t : kDefaultTuning; }
+    ~TuningScope() { t_tuning = saved; }
+};
+bool valid_tuning(const kq_tuning_t* t) {
+    return !t || (t->config >= 0 && t->config <= 7 && t->ctas_per_sm >= 0 && t->ctas_per_sm <= 8 && (t->use_pdl | 1) == 1 &&
+                  t->trigger >= 0 && t->trigger <= 2 && t->prefetch_tiles >= 0 && t->prefetch_tiles <= 64 &&
+                  (t->dynamic | 1) == 1 && t->unit_tiles >= 0 && t->unit_tiles <= 16 && (t->compare_staged | 1) == 1);
+}
 std::atomic<int> g_tl_next{0};          // timeline builds: next launch slot   // comparison quantizers: 1 = the tensor-core kernel's pipeline without its MMA stage,
                                         // 0 = the plain grid-stride kernels
 
@@ -271,11 +276,11 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     kq::UmmaProblem prob;
     prob.blocks_per_row = nb;
     prob.tiled_scales = tiled ? 1 : 0;
-    prob.early_trigger = (g_umma_pdl.load() != 0 && calib_sumsq == nullptr) ? g_umma_trigger.load() : 0;
-    prob.prefetch_tiles = g_umma_pdl.load() != 0 ? g_umma_prefetch.load() : 0;
-    prob.dynamic = g_umma_dynamic.load();
+    prob.early_trigger = (t_tuning.use_pdl != 0 && calib_sumsq == nullptr) ? t_tuning.trigger : 0;
+    prob.prefetch_tiles = t_tuning.use_pdl != 0 ? t_tuning.prefetch_tiles : 0;
+    prob.dynamic = t_tuning.dynamic;
     prob.tl_slot = g_tl_next.fetch_add(1) % 64;
-    prob.unit_tiles = pb ? kq::kPbCols : g_umma_unit_tiles.load();
+    prob.unit_tiles = pb ? kq::kPbCols : (t_tuning.unit_tiles > 0 ? t_tuning.unit_tiles : 3);
     CUtensorMap tmap;
     cuuint64_t dims[2], strides[1];
     if (pb) {
@@ -289,7 +294,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
         prob.n_ttiles = 1;
         prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
         // units of several tiles save cancel requests, but a launch of a few tiles per CTA wants them spread out
-        if (g_umma_unit_auto.load() && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
+        if ((t_tuning.unit_tiles == 0) && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
         prob.n_units = (prob.n_tiles + prob.unit_tiles - 1) / prob.unit_tiles;
         dims[0] = 32; dims[1] = (cuuint64_t)prob.n_rows; strides[0] = 64;
     }
@@ -312,13 +317,13 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
             return KQ_ERR_CUDA;
     }
     const bool main_variant = !pb && calib_sumsq == nullptr;      // shared factor set: bf16 or fp16, one or two outputs
-    const int cps_set = g_umma_ctas_per_sm.load();
+    const int cps_set = t_tuning.ctas_per_sm;
     // (a launch that fits the GPU in one wave of the smaller CTAs keeps those: more of them run at once)
     // (the fp16 two-output kernel would spill registers at two large CTAs per SM)
     const bool big_ctas = main_variant && !(xf16 && at_out != nullptr && !WRITE_Y) && cps_set == 0 &&
                           prob.n_tiles > (int64_t)3 * sm_count();
     const int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
-    const bool pdl = g_umma_pdl.load() != 0;
+    const bool pdl = t_tuning.use_pdl != 0;
     // A launch whose units all fit the GPU at once has nothing to hand out: static distribution (no cancel
     // request, no shared-memory padding), and the completion signal goes back to the kernel's start, where it
     // lets the launches of a chain of very short kernels run ahead of one another.
@@ -350,14 +355,14 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     if (xf16) return pb ? KQ_LAUNCH(4, 1, 1, true, true)
                         : big_ctas ? KQ_LAUNCH(8, 2, 2, false, true) : KQ_LAUNCH(4, 2, 1, false, true);
     if (pb) {
-        switch (g_umma_cfg.load()) {
+        switch (t_tuning.config) {
             default:
             case 4: return KQ_LAUNCH(4, 1, 1, true, false);
             case 0: return KQ_LAUNCH(4, 2, 1, true, false);
             case 1: return KQ_LAUNCH(8, 2, 1, true, false);
         }
     }
-    switch (cps_set == 0 && !big_ctas ? 5 : g_umma_cfg.load()) {
+    switch (cps_set == 0 && !big_ctas ? 5 : t_tuning.config) {
         default:
         case 0: return KQ_LAUNCH(2, 2, 1, false, false);
         case 1: return KQ_LAUNCH(8, 2, 1, false, false);
@@ -383,15 +388,15 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     kq::UmmaProblem prob;
     prob.blocks_per_row = nb;
     prob.tiled_scales = tiled ? 1 : 0;
-    prob.early_trigger = g_umma_pdl.load() != 0 ? g_umma_trigger.load() : 0;
-    prob.prefetch_tiles = g_umma_pdl.load() != 0 ? g_umma_prefetch.load() : 0;
-    prob.dynamic = g_umma_dynamic.load();
+    prob.early_trigger = t_tuning.use_pdl != 0 ? t_tuning.trigger : 0;
+    prob.prefetch_tiles = t_tuning.use_pdl != 0 ? t_tuning.prefetch_tiles : 0;
+    prob.dynamic = t_tuning.dynamic;
     prob.tl_slot = g_tl_next.fetch_add(1) % 64;
-    prob.unit_tiles = g_umma_unit_tiles.load();
+    prob.unit_tiles = (t_tuning.unit_tiles > 0 ? t_tuning.unit_tiles : 3);
     prob.n_rows = tokens * (int64_t)nb;
     prob.n_ttiles = 1;
     prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
-    if (g_umma_unit_auto.load() && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
+    if ((t_tuning.unit_tiles == 0) && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
     prob.n_units = (prob.n_tiles + prob.unit_tiles - 1) / prob.unit_tiles;
     CUtensorMap tmap;
     const cuuint64_t dims[2] = {32, (cuuint64_t)prob.n_rows}, strides[1] = {64};
@@ -402,11 +407,11 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
-    const int cps_set = g_umma_ctas_per_sm.load();
+    const int cps_set = t_tuning.ctas_per_sm;
     const bool big_ctas = cps_set == 0 && prob.n_tiles > (int64_t)3 * sm_count();
     int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
-    const bool pdl = g_umma_pdl.load() != 0;
-    bool big = cps_set == 0 ? big_ctas : g_umma_cfg.load() == 2;
+    const bool pdl = t_tuning.use_pdl != 0;
+    bool big = cps_set == 0 ? big_ctas : t_tuning.config == 2;
     const int box_rows = nb <= 256 ? nb : 128;                 // rows of one TMA box of the multiplier matrix
     const int vec = chan_scale ? (nb + box_rows - 1) / box_rows * box_rows * 128 + 1024 : 0;   // whole boxes, 1 KB-aligned
     CUtensorMap tmap_s = tmap;
@@ -460,7 +465,7 @@ kq_status_t run_stream_t(const void* X, int64_t tokens, int d, const kroquant_fa
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
+    cfg.numAttrs = t_tuning.use_pdl ? 1 : 0;
     if (cudaLaunchKernelEx(&cfg, kq::quantize_stream<MODE, WRITE_Y, XF16, TILED>, reinterpret_cast<const uint4*>(X),
                            n_quads, d / 32, f ? (const kq::FactorSet*)f->d_G : (const kq::FactorSet*)nullptr,
                            f ? f->n_sets : 0, s, reinterpret_cast<uint32_t*>(q), scales, Y) != cudaSuccess) {
@@ -617,7 +622,7 @@ kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tok
     const bool xf16 = x_dtype == KQ_X_FP16;
     const bool tiled = scale_layout == KQ_SCALES_TILED_128X4;
     if (path == KQ_PATH_AUTO && f->identity) {
-        if (g_compare_staged.load()) return run_flat_staged(X, xf16, tokens, d, nullptr, q_packed, scales, tiled, st);
+        if (t_tuning.compare_staged) return run_flat_staged(X, xf16, tokens, d, nullptr, q_packed, scales, tiled, st);
         return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, tiled, nullptr, st);
     }
     if (path != KQ_PATH_ALU)
@@ -713,7 +718,7 @@ kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
     const int tiled = scale_layout == KQ_SCALES_TILED_128X4 ? 1 : 0;
-    if (g_compare_staged.load()) {
+    if (t_tuning.compare_staged) {
         const kq_status_t rc_staged = run_flat_staged(X, xf16, tokens, d, s, q_packed, scales, tiled != 0, st);
         if (rc_staged != KQ_ERR_UNSUPPORTED) return rc_staged;       // (a vector too long for shared memory: grid-stride kernel)
     }
@@ -730,7 +735,7 @@ kq_status_t kroquant_scale_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
+    cfg.numAttrs = t_tuning.use_pdl ? 1 : 0;
     const uint4* x4 = reinterpret_cast<const uint4*>(X);
     uint32_t* q32 = reinterpret_cast<uint32_t*>(q_packed);
     cudaError_t err;
@@ -763,7 +768,7 @@ kq_status_t kroquant_mxfp4_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64
     if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
     if (scale_layout == KQ_SCALES_TILED_128X4 && !aligned16(scales)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
-    if (g_compare_staged.load())
+    if (t_tuning.compare_staged)
         return run_flat_staged(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, q_packed, scales,
                                scale_layout == KQ_SCALES_TILED_128X4, static_cast<cudaStream_t>(stream));
     return run_stream<kq::MODE_PLAIN, false>(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, nullptr, q_packed, scales,
@@ -798,7 +803,7 @@ static kq_status_t run_fwht(const void* X, kq_xdtype_t x_dtype, int64_t tokens, 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = g_umma_pdl.load() ? 1 : 0;
+    cfg.numAttrs = t_tuning.use_pdl ? 1 : 0;
     const float norm = (float)(1.0 / std::sqrt((double)d));
     const uint4* x4 = reinterpret_cast<const uint4*>(X);
     uint32_t* q32 = reinterpret_cast<uint32_t*>(q_packed);
@@ -868,33 +873,47 @@ kq_status_t kroquant_debug_e2m1_codes(const float* v, int64_t n, uint8_t* codes,
     return KQ_OK;
 }
 
-kq_status_t kroquant_debug_set_umma_config(int config, int ctas_per_sm, int use_pdl) {
-    if (config < 0 || config > 7 || ctas_per_sm < 0 || ctas_per_sm > 8) return KQ_ERR_UNSUPPORTED;
-    g_umma_cfg.store(config);
-    g_umma_ctas_per_sm.store(ctas_per_sm);
-    g_umma_pdl.store(use_pdl != 0);
-    return KQ_OK;
+void kroquant_tuning_default(kq_tuning_t* t) {
+    if (t) *t = kDefaultTuning;
 }
 
-kq_status_t kroquant_debug_set_boundary(int trigger, int prefetch_tiles) {
-    if (trigger < 0 || trigger > 2 || prefetch_tiles < 0 || prefetch_tiles > 64) return KQ_ERR_UNSUPPORTED;
-    g_umma_trigger.store(trigger);
-    g_umma_prefetch.store(prefetch_tiles);
-    return KQ_OK;
+kq_status_t kroquant_quantize_tuned(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const kroquant_factors_t* f,
+                                    uint8_t* q_packed, uint8_t* scales, kq_scale_layout_t scale_layout, kq_path_t path,
+                                    const kq_tuning_t* tuning, void* stream) {
+    if (!valid_tuning(tuning)) return KQ_ERR_UNSUPPORTED;
+    TuningScope scope(tuning);
+    return kroquant_quantize_ex(X, x_dtype, tokens, d, f, q_packed, scales, scale_layout, path, stream);
 }
 
-kq_status_t kroquant_debug_set_distribution(int dynamic, int unit_tiles) {
-    if (dynamic < 0 || dynamic > 1 || unit_tiles < 0 || unit_tiles > 16) return KQ_ERR_UNSUPPORTED;
-    g_umma_dynamic.store(dynamic);
-    g_umma_unit_tiles.store(unit_tiles > 0 ? unit_tiles : 3);
-    g_umma_unit_auto.store(unit_tiles > 0 ? 0 : 1);
-    return KQ_OK;
+kq_status_t kroquant_quantize_dual_tuned(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const kroquant_factors_t* f,
+                                         uint8_t* q_packed, uint8_t* scales, kq_scale_layout_t scale_layout, void* AT_out,
+                                         const kq_tuning_t* tuning, void* stream) {
+    if (!valid_tuning(tuning)) return KQ_ERR_UNSUPPORTED;
+    TuningScope scope(tuning);
+    return kroquant_quantize_dual(X, x_dtype, tokens, d, f, q_packed, scales, scale_layout, AT_out, stream);
 }
 
-kq_status_t kroquant_debug_set_compare_kernels(int staged) {
-    if (staged < 0 || staged > 1) return KQ_ERR_UNSUPPORTED;
-    g_compare_staged.store(staged);
-    return KQ_OK;
+kq_status_t kroquant_transform_f32_tuned(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const kroquant_factors_t* f,
+                                         float* Y, kq_path_t path, const kq_tuning_t* tuning, void* stream) {
+    if (!valid_tuning(tuning)) return KQ_ERR_UNSUPPORTED;
+    TuningScope scope(tuning);
+    return kroquant_transform_f32_ex(X, x_dtype, tokens, d, f, Y, path, stream);
+}
+
+kq_status_t kroquant_scale_quantize_tuned(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, const float* s,
+                                          uint8_t* q_packed, uint8_t* scales, kq_scale_layout_t scale_layout,
+                                          const kq_tuning_t* tuning, void* stream) {
+    if (!valid_tuning(tuning)) return KQ_ERR_UNSUPPORTED;
+    TuningScope scope(tuning);
+    return kroquant_scale_quantize_ex(X, x_dtype, tokens, d, s, q_packed, scales, scale_layout, stream);
+}
+
+kq_status_t kroquant_mxfp4_quantize_tuned(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, uint8_t* q_packed,
+                                          uint8_t* scales, kq_scale_layout_t scale_layout, const kq_tuning_t* tuning,
+                                          void* stream) {
+    if (!valid_tuning(tuning)) return KQ_ERR_UNSUPPORTED;
+    TuningScope scope(tuning);
+    return kroquant_mxfp4_quantize_ex(X, x_dtype, tokens, d, q_packed, scales, scale_layout, stream);
 }
 
 kq_status_t kroquant_debug_set_timeline(void* marks) {

@@ -19,10 +19,7 @@ pytestmark = pytest.mark.gpu
 def B():
     from paper_2607_21446_b200 import binding
     binding.load_library()
-    yield binding
-    binding.kroquant_debug_set_distribution(True, 0)         # back to the library's own choices
-    binding.kroquant_debug_set_boundary(2, 4)
-    binding.kroquant_debug_set_umma_config(2, 0, True)
+    return binding
 
 
 def dev(bits):
@@ -40,11 +37,10 @@ MODES = [(False, 1, 1, 0, 3, 5), (False, 3, 2, 4, 3, 5), (False, 2, 0, 1, 2, 5),
          (False, 1, 1, 0, 2, 2), (True, 5, 1, 2, 2, 1)]
 
 
-def set_mode(B, mode):
+def tuning_of(B, mode):
+    """The per-call tuning struct of a mode: nothing in the library is changed for anybody else."""
     dyn, unit, trigger, prefetch, cps, cfg = mode
-    B.kroquant_debug_set_umma_config(cfg, cps, True)
-    B.kroquant_debug_set_boundary(trigger, prefetch)
-    B.kroquant_debug_set_distribution(dyn, unit)
+    return B.Tuning(config=cfg, ctas_per_sm=cps, use_pdl=1, trigger=trigger, prefetch_tiles=prefetch, dynamic=dyn, unit_tiles=unit)
 
 
 # 4608 x 3072: 3456 tiles (7 to 8 per CTA of a 444-CTA grid); 2500 x 2240: ragged last tile; 700 x 5600 per block
@@ -56,10 +52,10 @@ def test_every_mode_gives_the_same_bits(B, tokens, d, per_block):
     f = B.Factors.create(W.gen_factors(7, n_sets=d // 32 if per_block else 1))
     ref = None
     for mode in MODES:
-        set_mode(B, mode)
+        tn = tuning_of(B, mode)
         for layout in ("rowmajor", "tiled"):
-            outs = [B.kroquant_quantize(X, f, path="tensor", scale_layout=layout) for _ in range(3)]   # back to back
-            dual = B.kroquant_quantize_dual(X, f, scale_layout=layout)
+            outs = [B.kroquant_quantize(X, f, path="tensor", scale_layout=layout, tuning=tn) for _ in range(3)]   # back to back
+            dual = B.kroquant_quantize_dual(X, f, scale_layout=layout, tuning=tn)
             got = [t.clone() for t in outs[-1]] + [dual[2].clone()]
             for q, s in outs[:-1]:
                 assert torch.equal(q, got[0]) and torch.equal(s, got[1])
@@ -79,10 +75,10 @@ def test_multi_tile_ctas_against_the_oracle(B, mode):
     tokens, d = 1500, 3072           # 1125 tiles: 2 to 3 per CTA of a 444-CTA grid, ragged last tile
     Xb = W.gen_activations(spec(tokens, d, 11))
     G = W.gen_factors(11)
-    set_mode(B, mode)
+    tn = tuning_of(B, mode)
     X, f = dev(Xb), B.Factors.create(G)
-    q, s = B.kroquant_quantize(X, f, path="tensor")
-    Yg = B.kroquant_transform_f32(X, f, path="tensor")
+    q, s = B.kroquant_quantize(X, f, path="tensor", tuning=tn)
+    Yg = B.kroquant_transform_f32(X, f, path="tensor", tuning=tn)
     qo, so, Y = co.quantize(Xb, G)
     P.check_values(Yg.cpu().numpy(), Y)
     P.check_codes(q.cpu().numpy(), s.cpu().numpy(), qo, so, Y, exact=False)
@@ -92,7 +88,7 @@ def test_multi_tile_ctas_against_the_oracle(B, mode):
 def test_dynamic_launches_that_overlap_on_two_streams(B):
     """A running CTA may only take over CTAs of its own grid: two dynamic launches that share the GPU must
     each produce their own complete result."""
-    set_mode(B, MODES[3])
+    tn = tuning_of(B, MODES[3])
     shapes = [(4608, 3072), (3000, 2240)]
     X = [dev(W.gen_activations(spec(t, d, 40 + i))) for i, (t, d) in enumerate(shapes)]
     f = [B.Factors.create(W.gen_factors(50 + i)) for i in range(2)]
@@ -103,7 +99,7 @@ def test_dynamic_launches_that_overlap_on_two_streams(B):
     for rep in range(12):
         for i in range(2):
             with torch.cuda.stream(streams[i]):
-                outs[i].append(B.kroquant_quantize(X[i], f[i], path="tensor", stream=streams[i]))
+                outs[i].append(B.kroquant_quantize(X[i], f[i], path="tensor", stream=streams[i], tuning=tn))
     torch.cuda.synchronize()
     for i in range(2):
         for q, s in outs[i]:
@@ -111,10 +107,16 @@ def test_dynamic_launches_that_overlap_on_two_streams(B):
     assert B.kroquant_last_device_error() == 0
 
 
-def test_knob_ranges(B):
-    for args in [(-1, 0), (3, 0), (0, -1), (0, 65)]:
+def test_tuning_ranges_and_scope(B):
+    X = dev(W.gen_activations(spec(64, 64, 3)))
+    f = B.Factors.create(W.gen_factors(3))
+    n0 = B.kroquant_launch_count()
+    for bad in [dict(trigger=-1), dict(trigger=3), dict(prefetch_tiles=-1), dict(prefetch_tiles=65), dict(unit_tiles=-1),
+                dict(unit_tiles=17), dict(dynamic=2), dict(config=8), dict(ctas_per_sm=9), dict(use_pdl=2), dict(compare_staged=-1)]:
         with pytest.raises(RuntimeError):
-            B.kroquant_debug_set_boundary(*args)
-    for args in [(True, -1), (True, 17)]:
-        with pytest.raises(RuntimeError):
-            B.kroquant_debug_set_distribution(*args)
+            B.kroquant_quantize(X, f, tuning=B.Tuning(**bad))
+    assert B.kroquant_launch_count() == n0                     # refused: nothing launched
+    # a tuned call leaves no trace: the next plain call runs with the defaults and gives the same bits
+    a = B.kroquant_quantize(X, f, tuning=B.Tuning(dynamic=0, unit_tiles=1, ctas_per_sm=1, config=3, use_pdl=0))
+    b = B.kroquant_quantize(X, f)
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])

@@ -267,19 +267,16 @@ def test_host_buffer_entry_point_equals_device_path(B):
 
 @pytest.mark.parametrize("tokens,d", [(3, 1152), (257, 96), (640, 1152), (2048, 2240)])
 def test_grid_stride_comparison_kernels_bit_exact(B, tokens, d):
-    """The plain grid-stride kernels behind kroquant_debug_set_compare_kernels(0) (the fall-back for a multiplier
-    vector that does not fit shared memory) give the same bits as the staged ones and as the oracle."""
+    """The plain grid-stride kernels (tuning field compare_staged = 0; also the fall-back for a multiplier vector
+    that does not fit shared memory) give the same bits as the staged ones and as the oracle."""
     Xb = W.gen_activations(spec(tokens, d, seed=31))
     sv = W.gen_channel_scales(31, d)
     X, svd = dev_bf16(Xb), torch.from_numpy(sv).cuda()
     qs, ss = B.kroquant_scale_quantize(X, svd)
     qp, sp = B.kroquant_mxfp4_quantize(X)
-    B.kroquant_debug_set_compare_kernels(False)
-    try:
-        qs0, ss0 = B.kroquant_scale_quantize(X, svd)
-        qp0, sp0 = B.kroquant_mxfp4_quantize(X)
-    finally:
-        B.kroquant_debug_set_compare_kernels(True)
+    plain = B.Tuning(compare_staged=0)
+    qs0, ss0 = B.kroquant_scale_quantize(X, svd, tuning=plain)
+    qp0, sp0 = B.kroquant_mxfp4_quantize(X, tuning=plain)
     assert torch.equal(qs, qs0) and torch.equal(ss, ss0) and torch.equal(qp, qp0) and torch.equal(sp, sp0)
     q_or, s_or, Y = co.scale_quantize(Xb, sv)
     P.check_codes(host(qs0), host(ss0), q_or, s_or, Y, exact=True)
