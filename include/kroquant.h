@@ -261,6 +261,13 @@ kq_status_t kroquant_mxfp4_quantize_tuned(const void *X, kq_xdtype_t x_dtype, in
  * slot k % 64.  NULL switches the marks off.  Synchronize before reading.  A measuring aid, not a product path. */
 kq_status_t kroquant_debug_set_timeline(void *marks);
 
+/* Diagnostic builds only (same build as above; KQ_ERR_UNSUPPORTED otherwise): while on != 0, CTA 0 of every
+ * quantizer launch withholds its first tile, so that the waits on it run out (after 20 ms in that build) and the
+ * kernel leaves through its give-up path: the code is then read with kroquant_last_device_error
+ * (2 = the MMA warp's wait for a tile), the context stays usable and the other CTAs' outputs are complete.
+ * This is how the bounded waits are tested without a fault or a hang. */
+kq_status_t kroquant_debug_withhold_arrival(int on);
+
 /* The W4A4 product of the quantized layer (Section 3.4: O = Q(A T) Q(W~)^T + A T L R):
  *     out[m][n] = sum_k a[m][k] 2^(sa[m][k/32] - 127) * b[n][k] 2^(sb[n][k/32] - 127)  (+ add[m][n])
  * on the block-scaled FP4 tensor-core path (fp32 accumulation).  a_codes [M][K/2] and b_codes

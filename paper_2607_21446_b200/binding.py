@@ -28,7 +28,7 @@ EXPORTS = [
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
     "kroquant_tuning_default", "kroquant_quantize_tuned", "kroquant_quantize_dual_tuned", "kroquant_transform_f32_tuned",
-    "kroquant_scale_quantize_tuned", "kroquant_mxfp4_quantize_tuned", "kroquant_debug_set_timeline", "kroquant_launch_count", "kroquant_last_device_error",
+    "kroquant_scale_quantize_tuned", "kroquant_mxfp4_quantize_tuned", "kroquant_debug_set_timeline", "kroquant_debug_withhold_arrival", "kroquant_launch_count", "kroquant_last_device_error",
     "kroquant_status_string",
     "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
@@ -81,6 +81,7 @@ def load_library() -> C.CDLL:
     L.kroquant_mxfp4_quantize.argtypes = [vp, i64, i32, vp, vp, vp]
     L.kroquant_transform_f32.argtypes = [vp, i64, i32, vp, vp, i32, vp]
     L.kroquant_debug_e2m1_codes.argtypes = [vp, i64, vp, vp]
+    L.kroquant_debug_withhold_arrival.argtypes = [i32]
     L.kroquant_tuning_default.argtypes = [vp]
     L.kroquant_tuning_default.restype = None
     L.kroquant_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, i32, vp, vp]
@@ -351,6 +352,10 @@ def use_library(path: str) -> None:
 
 def kroquant_debug_set_timeline(marks: Optional[torch.Tensor]) -> None:
     _check(load_library().kroquant_debug_set_timeline(_ptr(marks)), "kroquant_debug_set_timeline")
+
+
+def kroquant_debug_withhold_arrival(on: bool) -> None:
+    _check(load_library().kroquant_debug_withhold_arrival(int(on)), "kroquant_debug_withhold_arrival")
 
 
 def kroquant_launch_count() -> int:

@@ -43,6 +43,9 @@ __device__ int g_kq_device_error = 0;
 //   0 CTA start   1 dependency wait returned (producer)   2 first tile ready for the epilogue
 //   3 producer has issued its last tile   4 epilogue group 0 finished   5 CTA end   6 tiles issued
 #ifdef KQ_TIMELINE
+// Diagnostic builds: non-zero makes CTA 0 of every launch withhold its first tile (no copy, no arrival), so that the
+// waits on that tile run out and the give-up path (error word, abort flag, drain, TMEM release) executes.
+__device__ int g_kq_withhold = 0;
 __device__ long long* g_kq_timeline = nullptr;
 __device__ __forceinline__ void tl_mark(int slot, int i) {
     long long* p = g_kq_timeline;
@@ -67,7 +70,11 @@ constexpr int kTileRows = 128;                    // blocks (flat rows) per MMA 
 constexpr int kTileBytes = kTileRows * 64;        // 8 KB of bf16 per tile
 constexpr int kBTermBytes = 32 * 64;              // one bf16 term of K^T: 32 rows (n) x 64 B (k)
 constexpr int kBImageBytes = 3 * kBTermBytes;     // 6 KB per factor set
+#ifdef KQ_TIMELINE
+constexpr uint64_t kWaitLimitNs = 20ull * 1000ull * 1000ull;    // diagnostic build: every mbarrier wait gives up after 20 ms
+#else
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // every mbarrier wait gives up after 1 s
+#endif
 
 enum {
     KQ_DEV_OK = 0,
@@ -494,6 +501,9 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             ring_jg[n % kRingEntries] = jg;
         }
         ring[n % kRingEntries] = PB ? tt : item;
+#ifdef KQ_TIMELINE
+        if (n == 0 && blockIdx.x == 0 && g_kq_withhold) return;
+#endif
         mbar_expect_tx(bar_full(s), L::kStageBytes);
         if (PB) {
             const int jb = j < prob.blocks_per_row ? j : prob.blocks_per_row - 1;

@@ -927,6 +927,16 @@ kq_status_t kroquant_debug_set_timeline(void* marks) {
 #endif
 }
 
+kq_status_t kroquant_debug_withhold_arrival(int on) {
+#ifdef KQ_TIMELINE
+    const int v = on ? 1 : 0;
+    return cudaMemcpyToSymbol(kq::g_kq_withhold, &v, sizeof(v)) == cudaSuccess ? KQ_OK : KQ_ERR_CUDA;
+#else
+    (void)on;
+    return KQ_ERR_UNSUPPORTED;
+#endif
+}
+
 int64_t kroquant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 kq_status_t kroquant_last_device_error(void* stream, int* code_out) {
