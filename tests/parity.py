@@ -3,7 +3,7 @@
 P0  exact kernels (bare MXFP4, per-channel scale, identity factors): every code
     and scale byte identical (a zero's sign may differ only where the oracle's
     value is exactly +-0).
-P1  pre-rounding values: |y_gpu - y| <= 1e-5 * max(|y|, amax_block / 32)   (amax_block / 8 for
+P1  pre-rounding values: |y_gpu - y| <= 1e-5 * max(|y|, amax_block / 32)   (amax_block / 16 for
     fp16 activations, see FLOOR_DIV).
     A code 0x0 vs 0x8 (signed zero) is not a mismatch where the oracle's value is
     exactly +-0 or, for the inexact kernels, within the P1 tolerance of zero.
@@ -23,12 +23,16 @@ from oracle import np_oracle as no
 BOUNDS = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0])
 REL = 1e-5
 MAX_FRACTION = 1e-4
-# Floor of the value tolerance, as a fraction of the block amax.  bf16 activations (the case the
-# 1e-5 rule is stated for): amax/32.  fp16 activations: amax/8 -- their products with the 11-bit
-# factor terms carry 22 significant bits, so the tensor core's fp32 accumulation of 96 of them
-# rounds at every step (with bf16 activations most partial sums are still exact); measured worst
-# error 1.1x the bf16 floor.
-FLOOR_DIV = {"bf16": 32.0, "fp16": 8.0}
+# Floor of the value tolerance, as a fraction of the block amax.  bf16 activations (the case the 1e-5 rule is stated
+# for): amax/32.  fp16 activations: amax/16, from the accumulation model: an fp16 activation times an 11-bit factor
+# term is a 22-bit product, so (unlike the 16-bit products of bf16 activations, whose sums mostly stay exact in 24
+# bits) every one of the 32 additions of leading-term products rounds in the tensor core's fp32 accumulator.  With
+# partial sums growing like sqrt(k) sigma_p (sigma_p = rms product) and a rounding of +-2^-24 relative each, the
+# error's standard deviation is sqrt(sum_{k<=32} k / 3) 2^-24 sigma_p = 7.9e-7 sigma_p, while a block's amax is
+# about 13.6 sigma_p (the largest of 32 sums of 32 products; outlier channels only raise it): amax/32 puts the
+# tolerance at 5.4 standard deviations, which 10^8 elements do exceed now and then (measured worst: 1.1 times
+# that floor), amax/16 at 10.8.
+FLOOR_DIV = {"bf16": 32.0, "fp16": 16.0}
 
 
 def unpack(q: np.ndarray) -> np.ndarray:
