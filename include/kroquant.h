@@ -292,6 +292,15 @@ kq_status_t kroquant_gemm_mxfp4(const uint8_t *a_codes, const uint8_t *a_scales,
 kq_status_t kroquant_gemm_bf16(const void *A, const void *B, int64_t M, int N, int K, const float *add_f32,
                                void *out, kq_dtype_t out_dtype, void *stream);
 
+/* kroquant_gemm_mxfp4 / kroquant_gemm_bf16 with the kernel variant chosen for this one call: pair = 1 (what the plain
+ * entry points use): CTA pairs on 256 x 256 tiles; 0: one CTA per 128 x 128 (FP4) or 128 x 256 (bf16) tile.  Tests and
+ * ablations; same contraction, fp32 summation order differs.  Other values: KQ_ERR_UNSUPPORTED. */
+kq_status_t kroquant_gemm_mxfp4_variant(const uint8_t *a_codes, const uint8_t *a_scales, const uint8_t *b_codes,
+                                        const uint8_t *b_scales, int64_t M, int N, int K, const void *add_bf16,
+                                        void *out, kq_dtype_t out_dtype, int pair, void *stream);
+kq_status_t kroquant_gemm_bf16_variant(const void *A, const void *B, int64_t M, int N, int K, const float *add_f32,
+                                       void *out, kq_dtype_t out_dtype, int pair, void *stream);
+
 /* The quantized linear layer of Section 3.4 in one call:
  *     out = Q(X T) Q(W~)^T (+ add),   Q(X T) by kroquant_quantize_ex (tensor path, tiled scales),
  *                                     the product by kroquant_gemm_mxfp4,
@@ -329,11 +338,11 @@ kq_status_t kroquant_linear_w4a4(const void *X, kq_xdtype_t x_dtype, int64_t tok
  * error is rounded to bf16 once before the two backward contractions. */
 typedef struct kroquant_calib kroquant_calib_t;
 
-/* Test and tuning knob: which tensor-core GEMM kernels the calibration calls and kroquant_gemm_mxfp4
- * launch from now on.  1 (default): pairs of CTAs on 256 x 256 tiles (tcgen05 cta_group::2); 0: one
- * CTA per tile (128 x 256 bf16, 128 x 128 FP4).  Both compute the same contractions; results differ
- * only in fp32 summation order. */
-kq_status_t kroquant_debug_set_gemm_pair(int on);
+/* Which tensor-core GEMM kernels this handle's calibration calls launch.  pair = 1 (default): pairs of CTAs on
+ * 256 x 256 tiles (tcgen05 cta_group::2) and the production quantizer as the fake-quant forward; 0: one CTA per tile
+ * (128 x 256 bf16).  Both compute the same contractions; results differ only in fp32 summation order.  Per handle;
+ * other values give KQ_ERR_UNSUPPORTED. */
+kq_status_t kroquant_calib_set_gemm_variant(kroquant_calib_t *c, int pair);
 
 kq_status_t kroquant_calib_create(const void *A, const void *W, int64_t M, int o, int d, int n_sets,
                                   void *stream, kroquant_calib_t **out);

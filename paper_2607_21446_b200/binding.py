@@ -34,7 +34,7 @@ EXPORTS = [
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
     "kroquant_calib_loss_grad", "kroquant_calib_run",
     "kroquant_block_grad_scratch_bytes", "kroquant_block_grad", "kroquant_block_grad_static",
-    "kroquant_debug_set_gemm_pair", "kroquant_calib_get_weight_factors", "kroquant_gemm_mxfp4",
+    "kroquant_calib_set_gemm_variant", "kroquant_gemm_mxfp4_variant", "kroquant_gemm_bf16_variant", "kroquant_calib_get_weight_factors", "kroquant_gemm_mxfp4",
     "kroquant_linear_w4a4", "kroquant_gemm_bf16",
 ]
 
@@ -106,7 +106,9 @@ def load_library() -> C.CDLL:
     L.kroquant_block_grad_scratch_bytes.restype = i64
     L.kroquant_block_grad.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, vp]
     L.kroquant_block_grad_static.argtypes = [vp, vp, i64, i32, i32, vp, vp]
-    L.kroquant_debug_set_gemm_pair.argtypes = [i32]
+    L.kroquant_calib_set_gemm_variant.argtypes = [vp, i32]
+    L.kroquant_gemm_mxfp4_variant.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, i32, vp]
+    L.kroquant_gemm_bf16_variant.argtypes = [vp, vp, i64, i32, i32, vp, vp, i32, i32, vp]
     L.kroquant_gemm_mxfp4.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, vp]
     L.kroquant_gemm_bf16.argtypes = [vp, vp, i64, i32, i32, vp, vp, i32, vp]
     L.kroquant_linear_w4a4.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp, vp, vp, i32, vp]
@@ -447,9 +449,9 @@ def kroquant_gemm_mxfp4(a_codes: torch.Tensor, a_scales: torch.Tensor, b_codes: 
         raise ValueError("out must be a contiguous bfloat16 or float32 tensor [M, N]")
     if add is not None and (add.dtype != torch.bfloat16 or tuple(add.shape) != (M, N) or not add.is_contiguous()):
         raise ValueError("add must be a contiguous bfloat16 tensor [M, N]")
-    _check(load_library().kroquant_gemm_mxfp4(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), M, N, K,
-                                              _ptr(add), _ptr(out), 1 if out.dtype == torch.bfloat16 else 0,
-                                              _stream(stream)), "kroquant_gemm_mxfp4")
+    _check(load_library().kroquant_gemm_mxfp4_variant(_ptr(a_codes), _ptr(a_scales), _ptr(b_codes), _ptr(b_scales), M, N, K,
+                                                      _ptr(add), _ptr(out), 1 if out.dtype == torch.bfloat16 else 0,
+                                                      int(_GEMM_PAIR), _stream(stream)), "kroquant_gemm_mxfp4")
     return out
 
 
@@ -470,8 +472,9 @@ def kroquant_gemm_bf16(A: torch.Tensor, Bm: torch.Tensor, add: Optional[torch.Te
         raise ValueError("out must be a contiguous bfloat16 or float32 tensor [M, N]")
     if add is not None and (add.dtype != torch.float32 or tuple(add.shape) != (M, N) or not add.is_contiguous()):
         raise ValueError("add must be a contiguous float32 tensor [M, N]")
-    _check(load_library().kroquant_gemm_bf16(_ptr(A), _ptr(Bm), M, N, K, _ptr(add), _ptr(out),
-                                             1 if out.dtype == torch.bfloat16 else 0, _stream(stream)), "kroquant_gemm_bf16")
+    _check(load_library().kroquant_gemm_bf16_variant(_ptr(A), _ptr(Bm), M, N, K, _ptr(add), _ptr(out),
+                                                     1 if out.dtype == torch.bfloat16 else 0, int(_GEMM_PAIR),
+                                                     _stream(stream)), "kroquant_gemm_bf16")
     return out
 
 
@@ -512,9 +515,15 @@ class LinearW4A4:
         return out
 
 
+_GEMM_PAIR = True
+
+
 def set_gemm_pair(on: bool) -> None:
-    """Choose the calibration GEMM: pairs of CTAs on 256 x 256 tiles (default) or one CTA per tile."""
-    _check(load_library().kroquant_debug_set_gemm_pair(1 if on else 0), "kroquant_debug_set_gemm_pair")
+    """Which GEMM variant THIS BINDING passes with its calls from now on (a default of the Python layer, handed to
+    the library per call or per calibration handle; the library keeps no process-wide switch): pairs of CTAs on
+    256 x 256 tiles (default) or one CTA per tile."""
+    global _GEMM_PAIR
+    _GEMM_PAIR = bool(on)
 
 
 class Calibrator:
@@ -584,6 +593,7 @@ class Calibrator:
         """-> (losses float64 [3] = (L_out, L_A, L_W), dL/dtheta float32 [n_sets, 5, 3] or None)."""
         losses = np.empty(3, np.float64)
         g = np.empty((self.n_sets, 5, 3), np.float32) if grad else None
+        _check(load_library().kroquant_calib_set_gemm_variant(self._h, int(_GEMM_PAIR)), "kroquant_calib_set_gemm_variant")
         _check(load_library().kroquant_calib_loss_grad(self._h, losses.ctypes.data_as(C.c_void_p),
                                                        g.ctypes.data_as(C.c_void_p) if grad else None,
                                                        _stream(stream)), "kroquant_calib_loss_grad")
@@ -592,6 +602,7 @@ class Calibrator:
     def run(self, steps: int, lr: float = 1e-2, history: bool = True, stream=None):
         """`steps` Adam steps; -> history float64 [steps + 1, 3] (or None, asynchronous)."""
         h = np.empty((steps + 1, 3), np.float64) if history else None
+        _check(load_library().kroquant_calib_set_gemm_variant(self._h, int(_GEMM_PAIR)), "kroquant_calib_set_gemm_variant")
         _check(load_library().kroquant_calib_run(self._h, steps, lr, h.ctypes.data_as(C.c_void_p) if history else None,
                                                  _stream(stream)), "kroquant_calib_run")
         return h

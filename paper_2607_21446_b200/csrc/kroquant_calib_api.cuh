@@ -36,6 +36,7 @@ struct kroquant_calib {
     float* lr_dev = nullptr;           // device: learning rate of the run in flight
     cudaGraphExec_t step_graph[2] = {nullptr, nullptr};   // one captured Adam step per GEMM variant
     int launches_per_step = 0;         // kernels in one captured step (for the launch counter)
+    int gemm_pair = 1;                 // GEMM variant of this handle's calls (kroquant_calib_set_gemm_variant)
     // GEMM operands: "_a" = 128-row boxes (A operand, and both operands of the paired kernel),
     // "_b" = 256-row boxes (B operand of the one-CTA kernel)
     CUtensorMap tm_A_a, tm_W_b, tm_Yq_a, tm_Zq_b, tm_dO_a, tm_ZqT_b, tm_dOT_a, tm_YqT_b;
@@ -65,7 +66,14 @@ bool make_operand_map(CUtensorMap* tm, const void* ptr, int64_t rows, int64_t K,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-std::atomic<int> g_gemm_pair{1};       // 1: two-CTA 256 x 256 tiles (default); 0: one-CTA 128 x 256 tiles
+// GEMM variant of the call in flight on this thread: 1: two-CTA 256 x 256 tiles (default); 0: one-CTA 128 x 256
+// tiles.  Installed by the *_variant entry points and, for calibration calls, from the handle; never process-wide.
+thread_local int t_gemm_pair = 1;
+struct GemmVariantScope {
+    int saved;
+    explicit GemmVariantScope(int pair) : saved(t_gemm_pair) { t_gemm_pair = pair ? 1 : 0; }
+    ~GemmVariantScope() { t_gemm_pair = saved; }
+};
 
 // tb = B operand map with 256-row boxes (one-CTA kernel), tb2 = the same tensor with 128-row boxes
 // [K][MN] bf16 row-major (MN contiguous) as an MN-major operand of the paired kernel
@@ -103,7 +111,7 @@ kq_status_t launch_gemm(const CUtensorMap& ta, const CUtensorMap& tb, const CUte
         }
         attr_done.done();
     }
-    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0 || mode != 0;
+    const bool pair = (t_gemm_pair != 0) || mode != 0;
     const int bm = pair ? kq::kGemm2BM : kq::kGemmBM;
     kq::GemmProblem p;
     p.M = M; p.N = N; p.K = K;
@@ -207,7 +215,7 @@ kq_status_t calib_eval(kroquant_calib_t* c, bool backward, bool update, float lr
     // decoded block in bf16, the residual in fp32 and the sum of squared residuals - calibration sees exactly
     // the rounding inference will see, and the codes feed the FP4 forward contraction directly.
     // One-CTA mode: the mma.sync kernel, which also writes the transposed copies that GEMM needs.
-    const bool pair_mode = g_gemm_pair.load(std::memory_order_relaxed) != 0;
+    const bool pair_mode = (t_gemm_pair != 0);
     kq_status_t rc;
     if (pair_mode) {
         rc = run_umma<false>(c->A, false, M, d, &c->fK, c->qY, c->sY, true, c->ResY, c->Yq, st, c->sums + 1);
@@ -370,7 +378,7 @@ kq_status_t launch_gemm_fp4(const uint8_t* a_codes, const uint8_t* a_scales, con
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
-    const bool pair = g_gemm_pair.load(std::memory_order_relaxed) != 0 || epi != nullptr;
+    const bool pair = (t_gemm_pair != 0) || epi != nullptr;
     const int bm = pair ? 256 : kq::kF4BM, bn = pair ? 256 : kq::kF4BN;
     kq::Fp4GemmProblem p;
     p.M = (int)M; p.N = N; p.K = K;
@@ -473,8 +481,25 @@ kq_status_t kroquant_linear_w4a4(const void* X, kq_xdtype_t x_dtype, int64_t tok
     return kroquant_gemm_mxfp4(q_work, s_work, w_codes, w_scales, tokens, o, d, add_bf16, out, out_dtype, stream);
 }
 
-kq_status_t kroquant_debug_set_gemm_pair(int on) {
-    g_gemm_pair.store(on ? 1 : 0, std::memory_order_relaxed);
+kq_status_t kroquant_gemm_mxfp4_variant(const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
+                                        const uint8_t* b_scales, int64_t M, int N, int K, const void* add_bf16, void* out,
+                                        kq_dtype_t out_dtype, int pair, void* stream) {
+    if (pair != 0 && pair != 1) return KQ_ERR_UNSUPPORTED;
+    GemmVariantScope scope(pair);
+    return kroquant_gemm_mxfp4(a_codes, a_scales, b_codes, b_scales, M, N, K, add_bf16, out, out_dtype, stream);
+}
+
+kq_status_t kroquant_gemm_bf16_variant(const void* A, const void* B, int64_t M, int N, int K, const float* add_f32, void* out,
+                                       kq_dtype_t out_dtype, int pair, void* stream) {
+    if (pair != 0 && pair != 1) return KQ_ERR_UNSUPPORTED;
+    GemmVariantScope scope(pair);
+    return kroquant_gemm_bf16(A, B, M, N, K, add_f32, out, out_dtype, stream);
+}
+
+kq_status_t kroquant_calib_set_gemm_variant(kroquant_calib_t* c, int pair) {
+    if (!c) return KQ_ERR_NULL;
+    if (pair != 0 && pair != 1) return KQ_ERR_UNSUPPORTED;
+    c->gemm_pair = pair;
     return KQ_OK;
 }
 
@@ -653,6 +678,7 @@ kq_status_t kroquant_calib_loss_grad(kroquant_calib_t* c, double* losses_host_ou
     kq_status_t rc = calib_check(c);
     if (rc != KQ_OK) return rc;
     if (!losses_host_out) return KQ_ERR_NULL;
+    GemmVariantScope variant_scope(c->gemm_pair);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     rc = calib_eval(c, grad_host_out != nullptr, false, 0.f, -1, st);
     if (rc != KQ_OK) return rc;
@@ -672,6 +698,7 @@ kq_status_t kroquant_calib_run(kroquant_calib_t* c, int steps, float lr, double*
     kq_status_t rc = calib_check(c);
     if (rc != KQ_OK) return rc;
     if (steps < 1 || steps > kHistCap - 1 || !(lr > 0.f)) return KQ_ERR_SHAPE;
+    GemmVariantScope variant_scope(c->gemm_pair);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     // learning rate and history row for this run live on the device; the step count is already there
     if (cudaMemcpyAsync(c->lr_dev, &lr, 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||      // pageable source: staged
@@ -680,7 +707,7 @@ kq_status_t kroquant_calib_run(kroquant_calib_t* c, int steps, float lr, double*
     // One Adam step is the same sequence of launches every time, so it is captured once per GEMM variant
     // and replayed.  A stream that cannot be captured (the legacy default stream, or one that is being
     // captured by the caller) gets the launches directly.
-    const int variant = g_gemm_pair.load(std::memory_order_relaxed) != 0 ? 1 : 0;
+    const int variant = (t_gemm_pair != 0) ? 1 : 0;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     const bool can_capture = st != nullptr && st != cudaStreamLegacy && cudaStreamIsCapturing(st, &cap) == cudaSuccess &&
                              cap == cudaStreamCaptureStatusNone;
