@@ -606,8 +606,8 @@ def run_single(args):
 
 
 def run_point(torch, B, co, P, args, label, bits, tokens, G, seed, peak, peak_kind, stream, idx):
-    """One measured and parity-checked point: KroQuant (factor sets G: one shared set or one per block), Scale and bare
-    MXFP4 on the same input, each as a CUDA graph of back-to-back calls over rotating buffers (> 3 x L2).  `bits` holds
+    """One measured and parity-checked point: KroQuant (factor sets G: one shared set or one per block; operand images
+    ready-made, and built on chip), Scale and bare MXFP4 on the same input, each as a CUDA graph of back-to-back calls over rotating buffers (> 3 x L2).  `bits` holds
     the first n0 <= tokens host rows; device row r is host row r % n0.  The C oracle then goes over EVERY row in
     chunks of 2048 (that pass is its measured time, all host cores) and all three outputs are compared with it
     (rules P0-P3 of tests/parity.py).  Prints one JSON line."""
@@ -622,6 +622,8 @@ def run_point(torch, B, co, P, args, label, bits, tokens, G, seed, peak, peak_ki
     svh = W.gen_channel_scales(seed, d)
     sv = torch.from_numpy(svh).cuda()
     kernels = (("kroquant", lambda x: B.kroquant_quantize(x, f, q, sc, stream=stream)),
+               # the same kernel with its operand built on chip from the factor scalars (the paper's K2 construction)
+               ("kroquant_onchip", lambda x: B.kroquant_quantize(x, f, q, sc, stream=stream, path="onchip")),
                ("scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
                ("plain_mxfp4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)))
     res, clk = {}, {}
@@ -650,8 +652,9 @@ def run_point(torch, B, co, P, args, label, bits, tokens, G, seed, peak, peak_ki
             for name, fn in kernels:
                 fn(x0)
                 stream.synchronize()
-                if name == "kroquant":
-                    parity[name] = P.check_codes_chunked(q, sc, rows, timed(lambda b: co.quantize(b, G)), tokens, exact=False)
+                if name.startswith("kroquant"):
+                    fn_or = (lambda b: co.quantize(b, G))                 # (its time is taken once, on the first pass)
+                    parity[name] = P.check_codes_chunked(q, sc, rows, timed(fn_or) if name == "kroquant" else fn_or, tokens, exact=False)
                 elif name == "scale":
                     parity[name] = P.check_codes_chunked(q, sc, rows, lambda b: co.scale_quantize(b, svh), tokens, exact=True)
                 else:
@@ -670,6 +673,7 @@ def run_point(torch, B, co, P, args, label, bits, tokens, G, seed, peak, peak_ki
         "tokens_per_s": round(tokens / (res["kroquant"] * 1e-6)),
         "scale_over_kroquant": round(res["scale"] / res["kroquant"], 3),
         "plain_over_kroquant": round(res["plain_mxfp4"] / res["kroquant"], 3),
+        "onchip_over_kroquant": round(res["kroquant_onchip"] / res["kroquant"], 3),
         "parity": parity,
         "cpu_oracle_s": round(oracle_s[0], 3), "cpu_oracle_rows": tokens, "cpu_cores": os.cpu_count(),
         "clocks": clk, "peak": f"{peak} GB/s of {peak_kind}", "buffers": nbuf,
@@ -722,9 +726,10 @@ PAPER_TABLES = {
 
 def run_table(args):
     """The paper's latency tables re-measured on this GPU with FP16 activations: Q4 (bare MXFP4),
-    Scale, K1 (dense 32x32 block handle) and K2 (five-factor handle; here both handles run the same
-    tensor-core kernel on a precomputed operand image).  Back-to-back calls in a CUDA graph over
-    rotating inputs (> 3 x L2).  One JSON line per shape."""
+    Scale, K1 (dense 32x32 block handle: the tensor-core kernel on a ready-made operand image), K2 (five-factor
+    handle, the same kernel on the image made at handle creation) and K2_onchip (five-factor handle, operand built
+    inside the kernel from the 20 scalars, as the paper's K2 kernel does).  Back-to-back calls in a CUDA graph
+    over rotating inputs (> 3 x L2).  One JSON line per shape."""
     import torch
     from paper_2607_21446_b200 import binding as B
     B.load_library()
@@ -747,7 +752,8 @@ def run_table(args):
             kernels = [("Q4", lambda x: B.kroquant_mxfp4_quantize(x, q, sc, stream=stream)),
                        ("Scale", lambda x: B.kroquant_scale_quantize(x, sv, q, sc, stream=stream)),
                        ("K1", lambda x: B.kroquant_quantize(x, f1, q, sc, stream=stream)),
-                       ("K2", lambda x: B.kroquant_quantize(x, f2, q, sc, stream=stream))]
+                       ("K2", lambda x: B.kroquant_quantize(x, f2, q, sc, stream=stream)),
+                       ("K2_onchip", lambda x: B.kroquant_quantize(x, f2, q, sc, stream=stream, path="onchip"))]
             if d & (d - 1) == 0:
                 kernels.append(("FWHT", lambda x: B.kroquant_fwht_quantize(x, q, sc, stream=stream)))
             for name, fn in kernels:
@@ -757,6 +763,7 @@ def run_table(args):
             print(json.dumps({"table": table, "m": m, "d": d, "dtype": "fp16", "us_b200": us,
                               "scale_over_k1": round(us["Scale"] / us["K1"], 3),
                               "scale_over_k2": round(us["Scale"] / us["K2"], 3),
+                              "scale_over_k2_onchip": round(us["Scale"] / us["K2_onchip"], 3),
                               "fwht_over_k2": round(us["FWHT"] / us["K2"], 3) if "FWHT" in us else None,
                               "paper_mi350_us": dict(zip(("Q4", "Scale", "K1", "K2", "FWHT"), paper))}), flush=True)
             del Xs, x0

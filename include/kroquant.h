@@ -64,8 +64,14 @@ typedef enum { KQ_X_BF16 = 0, KQ_X_FP16 = 1 } kq_xdtype_t;
 typedef enum { KQ_SCALES_ROWMAJOR = 0, KQ_SCALES_TILED_128X4 = 1 } kq_scale_layout_t;
 
 /* Which device code applies the transform in kroquant_quantize / kroquant_transform_f32.
- * KQ_PATH_AUTO picks the tensor-core kernel (tcgen05 + TMA) whenever it applies. */
-typedef enum { KQ_PATH_AUTO = 0, KQ_PATH_TENSOR = 1, KQ_PATH_ALU = 2 } kq_path_t;
+ * KQ_PATH_AUTO picks the tensor-core kernel (tcgen05 + TMA) whenever it applies.
+ * KQ_PATH_TENSOR_ONCHIP is the tensor-core kernel with its operand K = G1 (x) ... (x) G5 built inside the kernel
+ * from the 20 scalars of each factor set (Section 3.5, the "K2" kernel; Appendix B) instead of read from the
+ * handle's ready-made 6 KB operand images: handles made from factors only (KQ_ERR_UNSUPPORTED for a dense
+ * handle); the operand holds the same leading bits of K (24 for bf16 activations, 33 of K 2^e for fp16), its
+ * last bit may differ from the ready-made image's, so results may differ from KQ_PATH_TENSOR where a value
+ * lies on a rounding boundary -- as they may between KQ_PATH_TENSOR and KQ_PATH_ALU. */
+typedef enum { KQ_PATH_AUTO = 0, KQ_PATH_TENSOR = 1, KQ_PATH_ALU = 2, KQ_PATH_TENSOR_ONCHIP = 3 } kq_path_t;
 
 /* Opaque, immutable after creation; belongs to the device that was current at creation. */
 typedef struct kroquant_factors kroquant_factors_t;

@@ -18,7 +18,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libkroquant.so")
 
 KQ_OK = 0
-PATHS = {"auto": 0, "tensor": 1, "alu": 2}
+PATHS = {"auto": 0, "tensor": 1, "alu": 2, "onchip": 3}
 EXPORTS = [
     "kroquant_factors_create", "kroquant_factors_create_lu", "kroquant_factors_create_dense",
     "kroquant_factors_destroy", "kroquant_quantize_ex", "kroquant_transform_f32_ex",

@@ -13,6 +13,10 @@
 
 namespace kq {
 
+// One factor set as the kernels read it: g[k] = {G_k[0][0], G_k[0][1], G_k[1][0], G_k[1][1]}.
+struct FactorSet { float4 g[5]; };
+
+
 constexpr int kBlock = 32;  // channels per MX block
 
 __device__ __forceinline__ float bf16lo_to_f32(uint32_t packed) { return __uint_as_float(packed << 16); }

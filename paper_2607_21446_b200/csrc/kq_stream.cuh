@@ -17,9 +17,6 @@ namespace kq {
 
 enum { MODE_PLAIN = 0, MODE_SCALE = 1, MODE_KRON = 2 };
 
-// One factor set as the kernels read it: g[k] = {G_k[0][0], G_k[0][1], G_k[1][0], G_k[1][1]}.
-struct FactorSet { float4 g[5]; };
-
 // y = x K for the 8 channels of this thread (channel index c = 8*quad + i).
 // Factors 3,4,5 mix index bits 2,1,0 (inside the thread); factors 1,2 mix bits 4,3
 // (across the quad, by shuffle).  Stage order k = 1..5 is free (the stages commute).

@@ -83,7 +83,8 @@ enum {
     KQ_DEV_TIMEOUT_MMA_TMEM = 3,
     KQ_DEV_TIMEOUT_EPILOGUE = 4,
     KQ_DEV_TIMEOUT_B = 5,
-    KQ_DEV_TIMEOUT_DRAIN = 6
+    KQ_DEV_TIMEOUT_DRAIN = 6,
+    KQ_DEV_TIMEOUT_BUILD = 7
 };
 
 // ---- PTX wrappers --------------------------------------------------------------
@@ -218,14 +219,18 @@ struct UmmaSmem {
     static constexpr int kStoreTile = kTileRows * 64 + kTileRows * 4;          // one staging tile
     static constexpr int kStoreBytes = PB ? 2 * kStoreTile : 0;                // two of them, used alternately
     static constexpr int kBarOff = kStoreOff + kStoreBytes;
-    // barriers: full[NS], done[NS], tempty[NS], bfull, clc
-    static constexpr int kNumBars = 3 * NS + 2;
+    // barriers: full[NS], done[NS], tempty[NS], bfull, clc, issued[NS] (on-chip image build only)
+    static constexpr int kNumBars = 4 * NS + 2;
     static constexpr int kClcOff = kBarOff + ((8 * kNumBars + 15) & ~15);     // 16-byte response of a cancel request
     static constexpr int kRingOff = kClcOff + 16;                             // kRingEntries ints: work item of local tile n
     static constexpr int kRing2Off = kRingOff + 4 * kRingEntries;             // PB: column group of local tile n
     static constexpr int kTmemSlotOff = kRing2Off + 4 * kRingEntries;
     static constexpr int kAbortOff = kTmemSlotOff + 4;
-    static constexpr int kBytes = kAbortOff + 4;
+    // on-chip image build, per-block sets: the 80 bytes of factor scalars of the tile in each slot (copied by the
+    // producer together with the tile, so that the builders never wait for the L2)
+    static constexpr int kFactorOff = (kAbortOff + 4 + 15) & ~15;
+    static constexpr int kFactorSlot = 96;
+    static constexpr int kBytes = kFactorOff + NS * kFactorSlot;
     static constexpr int kDynBytes = kBytes + 1024;                  // slack for manual alignment
 };
 
@@ -361,6 +366,97 @@ __device__ __forceinline__ float store_block_calib(const uint32_t (&acc)[32], co
     return sq;
 }
 
+// The operand image of one factor set built on chip from its 20 scalars (Section 3.5, the "K2" kernel; Appendix B):
+// K[r][c] = prod_k G_k[bit_{5-k}(r)][bit_{5-k}(c)], written as three bf16 terms of K^T in the 64-byte-swizzled
+// operand layout (element (n = c, k = r) of term t at t*2048 + swz(64 c + 2 r), swz(o) = o ^ (((o >> 7) & 3) << 4)) --
+// the layout and the 8+8+8-bit split of the host-built images, from 80 bytes of input instead of 6 KB.
+// Lane c of a builder warp owns output channel c, i.e. one 64-byte row of each term; PARTS warps share an image, warp
+// `part` building the 32/PARTS input channels r = (32/PARTS) part ...  The products run down the bits of r from G1 to
+// G5 (the values of a thread share every prefix) in compensated single precision: each value is a pair (h, l), the
+// product with the next factor entry is formed exactly by a fused multiply-add and renormalised, so that h + l carries
+// K to about 2^-45 relative -- the three terms then hold its leading 24 bits, as they do in the images made from
+// double products on the host (the last term's last bit may differ from theirs, nothing else).
+__device__ __forceinline__ void kron_mul(float& h, float& l, float g) {
+    const float ph = h * g;
+    const float pe = fmaf(h, g, -ph);          // h g = ph + pe exactly
+    const float pl = fmaf(l, g, pe);
+    const float hh = ph + pl;
+    l = pl - (hh - ph);
+    h = hh;
+}
+// fp16 activations (XF16): terms of K 2^e in fp16 (11 + 11 + 11 bits; e = the set's normalisation exponent, the one the
+// epilogue folds back into the scale byte), otherwise the same steps.
+template <int PARTS, bool XF16>
+__device__ __forceinline__ void build_image_on_chip(uint32_t img, const float4 (&g)[5], int e, int lane, int part) {
+    static_assert(PARTS == 2 || PARTS == 4, "16 or 8 input channels per thread");
+    constexpr int kTop = PARTS == 2 ? 1 : 2;         // leading bits of r fixed by `part`
+    constexpr int kN = 32 / PARTS;                   // values per thread
+    const int c = lane;
+    // entry [rbit][cbit] of factor k (G1 <-> bit 4 ... G5 <-> bit 0), for this thread's column bits
+    float g0[5], g1[5];
+#pragma unroll
+    for (int k = 0; k < 5; ++k) {
+        const bool cb = (c >> (4 - k)) & 1;
+        g0[k] = cb ? g[k].y : g[k].x;
+        g1[k] = cb ? g[k].w : g[k].z;
+    }
+    float h[kN], l[kN];
+    h[0] = ((part >> (kTop - 1)) & 1) ? g1[0] : g0[0];
+    l[0] = 0.f;
+    if (kTop == 2) kron_mul(h[0], l[0], (part & 1) ? g1[1] : g0[1]);
+#pragma unroll
+    for (int k = kTop; k < 5; ++k) {
+#pragma unroll
+        for (int i = kN / 2 - 1; i >= 0; --i) {                  // value i -> values 2i (bit 0) and 2i + 1 (bit 1)
+            if (i >= (1 << (k - kTop))) continue;                // (constant bounds: everything stays in registers)
+            float h1 = h[i], l1 = l[i];
+            kron_mul(h1, l1, g1[k]);
+            kron_mul(h[i], l[i], g0[k]);
+            h[2 * i + 1] = h1; l[2 * i + 1] = l1;
+            h[2 * i] = h[i];   l[2 * i] = l[i];
+        }
+    }
+    // three-term split, two neighbouring input channels per packed conversion (even channel in the low half)
+    uint32_t w[3][kN / 2];
+    const float up = __uint_as_float((uint32_t)(127 + e) << 23);       // 2^e (1 for bf16 images), |e| <= 100
+#pragma unroll
+    for (int i = 0; i < kN / 2; ++i) {
+        float a0 = h[2 * i], a1 = h[2 * i + 1];
+        if (XF16) {
+            a0 *= up; a1 *= up;
+            __half2 t = __floats2half2_rn(a0, a1);
+            w[0][i] = *reinterpret_cast<const uint32_t*>(&t);
+            float2 f = __half22float2(t);
+            a0 = (a0 - f.x) + l[2 * i] * up;                                   // exact difference, then the low part
+            a1 = (a1 - f.y) + l[2 * i + 1] * up;
+            t = __floats2half2_rn(a0, a1);
+            w[1][i] = *reinterpret_cast<const uint32_t*>(&t);
+            f = __half22float2(t);
+            t = __floats2half2_rn(a0 - f.x, a1 - f.y);
+            w[2][i] = *reinterpret_cast<const uint32_t*>(&t);
+        } else {
+            __nv_bfloat162 t = __floats2bfloat162_rn(a0, a1);
+            w[0][i] = *reinterpret_cast<const uint32_t*>(&t);
+            a0 = (a0 - __uint_as_float(w[0][i] << 16)) + l[2 * i];             // exact difference, then the low part
+            a1 = (a1 - __uint_as_float(w[0][i] & 0xFFFF0000u)) + l[2 * i + 1];
+            t = __floats2bfloat162_rn(a0, a1);
+            w[1][i] = *reinterpret_cast<const uint32_t*>(&t);
+            a0 -= __uint_as_float(w[1][i] << 16);
+            a1 -= __uint_as_float(w[1][i] & 0xFFFF0000u);
+            t = __floats2bfloat162_rn(a0, a1);
+            w[2][i] = *reinterpret_cast<const uint32_t*>(&t);
+        }
+    }
+    const uint32_t row = img + 64u * (uint32_t)c, sw = (uint32_t)(c >> 1) & 3u;
+#pragma unroll
+    for (int t = 0; t < 3; ++t)
+#pragma unroll
+        for (int q = 0; q < kN / 8; ++q)                // 16-byte chunk (kN/8) part + q of the row: r = kN part + 8 q ... + 7
+            asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                         ::"r"(row + (uint32_t)(t * kBTermBytes) + 16u * ((uint32_t)(kN / 8 * part + q) ^ sw)),
+                           "r"(w[t][4 * q]), "r"(w[t][4 * q + 1]), "r"(w[t][4 * q + 2]), "r"(w[t][4 * q + 3]) : "memory");
+}
+
 // Work decomposition.  CTA b takes work units b, b + gridDim.x, ...
 //   PB = false (one shared factor set): X is the flat matrix [n_rows = tokens*d/32][32];
 //     unit = tile w = flat rows 128w .. 128w+127; outputs of flat row r: 16 B of codes at
@@ -434,7 +530,15 @@ constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
 //     that the eight lanes of a quarter warp, which hold consecutive columns, read eight different bank groups;
 //     tmap_q is that matrix's map), issued right behind the dependency wait so that it lands with the first tiles;
 //     a thread reads its column's 128 bytes from there.
-constexpr int kOpKron = 0, kOpPlain = 1, kOpScale = 2;
+//   kOpKronBuild  kOpKron with the operand images built on chip from the factor scalars (build_image_on_chip;
+//     handles made from factors) instead of copied from the handle's ready-made images.  b_image then
+//     points at the handle's FactorSet array.  Shared set: one image per CTA, built by the first epilogue warpgroup
+//     (which has nothing to do until the first tile has been through the tensor core) behind a proxy fence -- the
+//     MMA reads shared memory through the async proxy.  Per-block sets (one issuer warp; warps 2 and 3 are the
+//     builders): the image of tile n is built into the tile's own stage while its activations are on their way -- the
+//     producer announces the tile on issued[slot], the builders add their arrivals to the tile's "full" barrier --
+//     so a tile costs 80 bytes of L2 traffic for its operand instead of 6 KB.
+constexpr int kOpKron = 0, kOpPlain = 1, kOpScale = 2, kOpKronBuild = 3;
 template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone, int OP = kOpKron>
 // resident CTAs per SM the register budget must allow: (8,2,2) two; the one-warpgroup shapes three (two with the
 // calibration epilogue)
@@ -445,7 +549,10 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
               uint4* __restrict__ at_out, double* __restrict__ sumsq, const float* __restrict__ chan_scale) {
     constexpr bool DUAL = EXTRA == kExtraDual;
     constexpr bool CALIB = EXTRA == kExtraCalib;
-    constexpr bool TC = OP == kOpKron;            // tensor-core stage present
+    constexpr bool TC = OP == kOpKron || OP == kOpKronBuild;            // tensor-core stage present
+    constexpr bool BUILD = OP == kOpKronBuild;
+    constexpr int NB = PB ? 2 : 4;                // builder warps: warps 2 and 3 (per-block sets) / epilogue group 0
+    static_assert(!BUILD || (EXTRA == kExtraNone && (!PB || NM == 1)), "on-chip images: one output; per-block sets need two free warps");
     static_assert(TC || (!PB && !WRITE_Y && EXTRA == kExtraNone), "comparison kernels: flat view, quantizing path only");
     static_assert(!CALIB || (!XF16 && !WRITE_Y), "calibration outputs: bf16 images, quantizing path");
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
@@ -479,6 +586,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     volatile int* ring = reinterpret_cast<volatile int*>(base_ptr + L::kRingOff);
     volatile int* ring_jg = reinterpret_cast<volatile int*>(base_ptr + L::kRing2Off);
     const uint32_t bar_clc = bar0 + 8u * (3 * NS + 1);
+    auto bar_issued = [&](int s) { return bar0 + 8u * (3 * NS + 2 + s); };
     const uint32_t clc_resp = base + L::kClcOff;
     const int tpu = PB ? kPbCols : prob.unit_tiles;                   // tiles per unit
 
@@ -504,11 +612,15 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
 #ifdef KQ_TIMELINE
         if (n == 0 && blockIdx.x == 0 && g_kq_withhold) return;
 #endif
-        mbar_expect_tx(bar_full(s), L::kStageBytes);
+        mbar_expect_tx(bar_full(s), (PB && BUILD) ? kTileBytes : L::kStageBytes);
         if (PB) {
             const int jb = j < prob.blocks_per_row ? j : prob.blocks_per_row - 1;
             tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));      // zero-filled if j is out of range
-            bulk_load(dst + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(s));
+            if (BUILD) {                                                          // the builders take it from here
+                mbar_expect_tx(bar_issued(s), (uint32_t)sizeof(FactorSet));
+                bulk_load(base + L::kFactorOff + s * L::kFactorSlot, b_image + (size_t)jb * sizeof(FactorSet),
+                          (uint32_t)sizeof(FactorSet), bar_issued(s));
+            } else bulk_load(dst + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(s));
         } else {
             tma_load_2d(dst, &tmap_x, 0, item * kTileRows, bar_full(s));
         }
@@ -601,8 +713,13 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     if (threadIdx.x == 0) {
         // "done" = the stage may be refilled: one tcgen05.commit, or (no tensor-core stage) the four epilogue
         // warps that have read it
-        for (int s = 0; s < NS; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_done(s), TC ? 1 : 4); mbar_init(bar_tempty(s), 4); }
-        mbar_init(bar_b, 1);
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(bar_full(s), (PB && BUILD) ? 1 + NB : 1);
+            mbar_init(bar_done(s), TC ? 1 : 4);
+            mbar_init(bar_tempty(s), 4);
+            mbar_init(bar_issued(s), 1);
+        }
+        mbar_init(bar_b, (!PB && BUILD) ? NB : 1);
         mbar_init(bar_clc, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -614,7 +731,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
         if (PB && !WRITE_Y) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
         if (prob.dynamic) clc_request();       // concerns this grid's own CTAs only
-        if (TC && !PB) {
+        if (TC && !PB && !BUILD) {
             mbar_expect_tx(bar_b, kBImageBytes);
             bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
         }
@@ -680,6 +797,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 }
                 ring[n % kRingEntries] = -1;
                 mbar_arrive(bar_full(n % NS));
+                if (PB && BUILD) mbar_arrive(bar_issued(n % NS));
             }
         }
     } else if (TC && warp <= NM) {
@@ -733,10 +851,50 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc_commit(bar_done(s));
             }
         }
+    } else if (BUILD && PB && warp >= 2 && warp < 4) {
+        // ---------------- image builders (factor sets are immutable: no dependency wait) ----------------
+        const int bw = warp - 2;
+        int sentinels_seen = 0;
+        for (int n = 0;; ++n) {
+            const int s = n % NS;
+            // (the producer has waited for the slot's previous tile to leave the tensor core before it announced this one)
+            if (!mbar_wait(bar_issued(s), (n / NS) & 1, abort_flag)) {
+                if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_BUILD); *abort_flag = 1; }
+                break;
+            }
+            const bool sentinel = ring[n % kRingEntries] < 0;
+            if (!sentinel) {
+                int e_j = 0;
+                if (XF16) {
+                    const int j = ring_jg[n % kRingEntries] * kPbCols + n % kPbCols;
+                    e_j = __ldg(e_norm + (j < prob.blocks_per_row ? j : prob.blocks_per_row - 1));
+                }
+                float4 g[5];
+#pragma unroll
+                for (int k = 0; k < 5; ++k)
+                    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(g[k].x), "=f"(g[k].y), "=f"(g[k].z), "=f"(g[k].w)
+                                 : "r"(base + L::kFactorOff + s * L::kFactorSlot + 16 * k) : "memory");
+                build_image_on_chip<2, XF16>(base + L::kAOff + s * L::kStageBytes + kTileBytes, g, e_j, lane, bw);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_full(s));
+            if (sentinel && ++sentinels_seen == kSentinels) break;
+        }
     } else if (warp >= 4) {
         // ---------------- epilogue warpgroups ----------------
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
+        if (BUILD && !PB && g == 0) {
+            // the shared set's operand image (immutable factors: no dependency wait), a quarter of it per warp
+            float4 g[5];
+#pragma unroll
+            for (int k = 0; k < 5; ++k) g[k] = __ldg(&reinterpret_cast<const FactorSet*>(b_image)->g[k]);
+            build_image_on_chip<4, XF16>(base + L::kBOff, g, XF16 ? __ldg(e_norm) : 0, lane, quarter);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_b);
+        }
         pdl_wait_prior_grid();                     // the outputs may still be read by the previous kernel
         const uint32_t vec_base = (base + (uint32_t)L::kBytes + 1023u) & ~1023u;
         if (OP == kOpScale) {
@@ -943,9 +1101,13 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // memory goes away (load m went to slot m % NS and completes phase (m / NS) & 1)
         int never = 0;
         if ((TC && !PB) || OP == kOpScale) (void)mbar_wait(bar_b, 0, &never);
-        for (int m = (issued > NS ? issued - NS : 0); m < issued; ++m)
+        for (int m = (issued > NS ? issued - NS : 0); m < issued; ++m) {
+            // (on-chip images: the tile's barrier also counts the builders, who may have given up; the copies
+            //  themselves are all that must have landed, and the factor copy reports on the slot's issued barrier)
+            if (PB && BUILD) (void)mbar_wait(bar_issued(m % NS), (m / NS) & 1, &never);
             if (!mbar_wait(bar_full(m % NS), (m / NS) & 1, &never))
                 atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_DRAIN);
+        }
     }
     __syncthreads();
     if (TC && warp == 1) {

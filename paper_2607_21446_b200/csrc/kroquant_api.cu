@@ -268,7 +268,8 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
 // calib_sumsq != null: calibration outputs (bf16 X only): at_out receives Q(y) in bf16, Y the residual y - Q(y)
 template <bool WRITE_Y>
 kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroquant_factors_t* f, uint8_t* q,
-                     uint8_t* scales, bool tiled, float* Y, void* at_out, cudaStream_t st, double* calib_sumsq = nullptr) {
+                     uint8_t* scales, bool tiled, float* Y, void* at_out, cudaStream_t st, double* calib_sumsq = nullptr,
+                     bool onchip = false) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
     const bool pb = f->n_sets != 1;
@@ -338,6 +339,21 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     launch_umma<NS, NM, NG, PB, XF, WRITE_Y>(tmap, tmap_q, b, en, prob, q, scales, Y, nullptr, cps, pdl, st)
 #define KQ_LAUNCH_DUAL(NS, NM, NG, PB, XF) \
     launch_umma<NS, NM, NG, PB, XF, false, kq::kExtraDual>(tmap, tmap_q, b, en, prob, q, scales, nullptr, at_out, cps, pdl, st)
+    if (onchip) {
+        // operand images built on chip from the factor scalars (callers have checked: a handle made from factors, one
+        // output); fixed CTA shapes: the shared-set shapes of the default path; one issuer + two builder warps per block set
+        const uint8_t* g = reinterpret_cast<const uint8_t*>(f->d_G);
+#define KQ_LAUNCH_BUILD(NS, NM, NG, PB, XF) \
+    launch_umma<NS, NM, NG, PB, XF, WRITE_Y, kq::kExtraNone, kq::kOpKronBuild>(tmap, tmap_q, g, en, prob, q, scales, Y, nullptr, \
+                                                                            cps, pdl, st)
+        if (xf16) {
+            if (pb) return KQ_LAUNCH_BUILD(4, 1, 1, true, true);
+            return big_ctas ? KQ_LAUNCH_BUILD(8, 2, 2, false, true) : KQ_LAUNCH_BUILD(4, 2, 1, false, true);
+        }
+        if (pb) return KQ_LAUNCH_BUILD(4, 1, 1, true, false);
+        return big_ctas ? KQ_LAUNCH_BUILD(8, 2, 2, false, false) : KQ_LAUNCH_BUILD(4, 2, 1, false, false);
+#undef KQ_LAUNCH_BUILD
+    }
     if (!WRITE_Y && calib_sumsq != nullptr) {
         if (xf16 || !at_out || !Y) return KQ_ERR_UNSUPPORTED;
         // the calibration epilogue needs about twice the registers: two CTAs per SM.  No programmatic
@@ -356,9 +372,8 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
                         : big_ctas ? KQ_LAUNCH(8, 2, 2, false, true) : KQ_LAUNCH(4, 2, 1, false, true);
     if (pb) {
         switch (t_tuning.config) {
-            default:
+            default: return KQ_LAUNCH(4, 2, 1, true, false);     // two issuers: 6-11 % faster than one on the SANA shapes
             case 4: return KQ_LAUNCH(4, 1, 1, true, false);
-            case 0: return KQ_LAUNCH(4, 2, 1, true, false);
             case 1: return KQ_LAUNCH(8, 2, 1, true, false);
         }
     }
@@ -612,9 +627,12 @@ kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tok
     rc = check_factors_for(f, d);
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(q_packed)) return KQ_ERR_ALIGN;
-    if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
+    if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU && path != KQ_PATH_TENSOR_ONCHIP)
+        return KQ_ERR_UNSUPPORTED;
     if (!valid_xdtype(x_dtype) || !valid_layout(scale_layout)) return KQ_ERR_UNSUPPORTED;
     if (path == KQ_PATH_ALU && f->dense) return KQ_ERR_UNSUPPORTED;
+    // on-chip images: from factor scalars (a dense handle has none)
+    if (path == KQ_PATH_TENSOR_ONCHIP && f->dense) return KQ_ERR_UNSUPPORTED;
     // whole 512-byte scale tiles leave by 16-byte vector stores
     if (scale_layout == KQ_SCALES_TILED_128X4 && !aligned16(scales)) return KQ_ERR_ALIGN;
     if (tokens == 0) return KQ_OK;
@@ -626,7 +644,8 @@ kq_status_t kroquant_quantize_ex(const void* X, kq_xdtype_t x_dtype, int64_t tok
         return run_stream<kq::MODE_PLAIN, false>(X, xf16, tokens, d, nullptr, nullptr, q_packed, scales, tiled, nullptr, st);
     }
     if (path != KQ_PATH_ALU)
-        return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, tiled, nullptr, nullptr, st);
+        return run_umma<false>(X, xf16, tokens, d, f, q_packed, scales, tiled, nullptr, nullptr, st, nullptr,
+                               path == KQ_PATH_TENSOR_ONCHIP);
     return run_stream<kq::MODE_KRON, false>(X, xf16, tokens, d, f, nullptr, q_packed, scales, tiled, nullptr, st);
 }
 
@@ -687,16 +706,19 @@ kq_status_t kroquant_transform_f32_ex(const void* X, kq_xdtype_t x_dtype, int64_
     rc = check_factors_for(f, d);
     if (rc != KQ_OK) return rc;
     if (!aligned16(X) || !aligned16(Y)) return KQ_ERR_ALIGN;
-    if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU) return KQ_ERR_UNSUPPORTED;
+    if (path != KQ_PATH_AUTO && path != KQ_PATH_TENSOR && path != KQ_PATH_ALU && path != KQ_PATH_TENSOR_ONCHIP)
+        return KQ_ERR_UNSUPPORTED;
     if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
     if (path == KQ_PATH_ALU && f->dense) return KQ_ERR_UNSUPPORTED;
+    if (path == KQ_PATH_TENSOR_ONCHIP && f->dense) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool xf16 = x_dtype == KQ_X_FP16;
     if (path == KQ_PATH_AUTO && f->identity)
         return run_stream<kq::MODE_PLAIN, true>(X, xf16, tokens, d, nullptr, nullptr, nullptr, nullptr, false, Y, st);
     if (path != KQ_PATH_ALU)
-        return run_umma<true>(X, xf16, tokens, d, f, nullptr, nullptr, false, Y, nullptr, st);
+        return run_umma<true>(X, xf16, tokens, d, f, nullptr, nullptr, false, Y, nullptr, st, nullptr,
+                              path == KQ_PATH_TENSOR_ONCHIP);
     return run_stream<kq::MODE_KRON, true>(X, xf16, tokens, d, f, nullptr, nullptr, nullptr, false, Y, st);
 }
 

@@ -64,7 +64,8 @@ def test_sweep_point_line_carries_parity():
     assert d["shape"] == "1024x1152" and d["parity"]["status"] == "ok" and d["device_error"] == 0
     assert d["parity"]["scale"]["code_mismatches"] == 0 and d["parity"]["plain_mxfp4"]["code_mismatches"] == 0
     assert d["parity"]["kroquant"]["rows"] == 1024 and d["cpu_oracle_rows"] == 1024 and d["cpu_oracle_s"] > 0
-    assert set(d["us"]) == {"kroquant", "scale", "plain_mxfp4"}
+    assert set(d["us"]) == {"kroquant", "kroquant_onchip", "scale", "plain_mxfp4"}
+    assert d["parity"]["kroquant_onchip"]["rows"] == 1024 and d["onchip_over_kroquant"] > 0
 
 
 def test_reference_arm_line():
