@@ -589,6 +589,10 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     auto bar_issued = [&](int s) { return bar0 + 8u * (3 * NS + 2 + s); };
     const uint32_t clc_resp = base + L::kClcOff;
     const int tpu = PB ? kPbCols : prob.unit_tiles;                   // tiles per unit
+    static_assert(!PB || NS % kPbCols == 0, "a slot must always serve the same column of a group");
+    // producer thread only: column group whose operand image each slot holds (the factor staging area is free
+    // when images are copied)
+    volatile int* slot_jg = reinterpret_cast<volatile int*>(base_ptr + L::kFactorOff);
 
     // PB: unit u, column c of its group -> column j (may be >= blocks_per_row in the last, ragged group: such a
     // tile loads zeros and stores nothing), column group jg, token tile tt
@@ -612,16 +616,25 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
 #ifdef KQ_TIMELINE
         if (n == 0 && blockIdx.x == 0 && g_kq_withhold) return;
 #endif
-        mbar_expect_tx(bar_full(s), (PB && BUILD) ? kTileBytes : L::kStageBytes);
         if (PB) {
             const int jb = j < prob.blocks_per_row ? j : prob.blocks_per_row - 1;
-            tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));      // zero-filled if j is out of range
-            if (BUILD) {                                                          // the builders take it from here
+            if (BUILD) {                                                          // the builders make the image
+                mbar_expect_tx(bar_full(s), kTileBytes);
+                tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));  // zero-filled if j is out of range
                 mbar_expect_tx(bar_issued(s), (uint32_t)sizeof(FactorSet));
                 bulk_load(base + L::kFactorOff + s * L::kFactorSlot, b_image + (size_t)jb * sizeof(FactorSet),
                           (uint32_t)sizeof(FactorSet), bar_issued(s));
-            } else bulk_load(dst + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(s));
+            } else {
+                // a slot always serves the same column of a group (NS is a multiple of kPbCols): when the CTA's
+                // next unit lies in the same column group, the slot's operand image is already in place
+                const bool have = slot_jg[s] == jg;
+                slot_jg[s] = jg;
+                mbar_expect_tx(bar_full(s), have ? kTileBytes : L::kStageBytes);
+                tma_load_2d(dst, &tmap_x, j * 32, tt * kTileRows, bar_full(s));
+                if (!have) bulk_load(dst + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(s));
+            }
         } else {
+            mbar_expect_tx(bar_full(s), L::kStageBytes);
             tma_load_2d(dst, &tmap_x, 0, item * kTileRows, bar_full(s));
         }
     };
@@ -650,7 +663,11 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
 
     // Producer state (thread 0 only).  The work stream of this CTA: its own unit, then static strides or the
     // units of the CTAs it cancels.
-    int64_t unit = blockIdx.x;
+    // (static distribution, per-block sets: CTA b takes the contiguous range [U b / G, U (b + 1) / G) of the units,
+    //  which are ordered column group first -- consecutive units then share their operand images)
+    const bool contiguous = PB && !prob.dynamic;
+    const int64_t u_end = contiguous ? prob.n_units * ((int64_t)blockIdx.x + 1) / gridDim.x : prob.n_units;
+    int64_t unit = contiguous ? prob.n_units * (int64_t)blockIdx.x / gridDim.x : blockIdx.x;
     int unit_left = unit_count(unit);      // tiles of `unit` not yet issued; 0: the next unit has to be fetched
     int t_in = 0;                          // tiles of `unit` already issued
     int issued = 0;                        // tiles whose TMA load the producer thread has issued
@@ -658,8 +675,8 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     bool producer_failed = false;
     auto next_unit = [&]() -> int64_t {
         if (!prob.dynamic) {
-            const int64_t u = unit + gridDim.x;
-            return u < prob.n_units ? u : -1;
+            const int64_t u = contiguous ? unit + 1 : unit + gridDim.x;
+            return u < u_end ? u : -1;
         }
         if (!mbar_wait(bar_clc, clc_parity, abort_flag)) {
             if (!*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_PRODUCER); *abort_flag = 1; }
@@ -720,6 +737,8 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             mbar_init(bar_issued(s), 1);
         }
         mbar_init(bar_b, (!PB && BUILD) ? NB : 1);
+        if (PB && !BUILD)
+            for (int s = 0; s < NS; ++s) slot_jg[s] = -1;
         mbar_init(bar_clc, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -741,14 +760,14 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // (With dynamic distribution nobody knows who will take the units after the first wave; the CTAs of the
         // first wave ask for them by position, prefetch_stride = number of CTAs that run at once: the L2 is shared.)
         if (!prob.dynamic || (int64_t)blockIdx.x < prob.prefetch_stride) {
-            const int64_t stride = prob.dynamic ? prob.prefetch_stride : (int64_t)gridDim.x;
+            const int64_t stride = prob.dynamic ? prob.prefetch_stride : contiguous ? 1 : (int64_t)gridDim.x;
             int64_t u = unit;
             int t = 0, cnt = unit_left;
             for (int k = 0; k < prob.prefetch_tiles; ++k) {
                 prefetch_tile(PB ? (int)u : (int)(u * tpu) + t, t);
                 if (++t == cnt) {
                     u += stride;
-                    if (u >= prob.n_units) break;
+                    if (u >= u_end) break;
                     t = 0;
                     cnt = unit_count(u);
                 }
