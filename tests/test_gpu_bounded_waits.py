@@ -49,6 +49,23 @@ assert err == 4, err
 q3, s3 = B.kroquant_mxfp4_quantize(X)
 torch.cuda.synchronize()
 assert B.kroquant_last_device_error() == 0
+# the kernel that builds its operand on chip (per-block sets): the builder warps wait for the withheld tile's
+# announcement, the issuing warp for the tile itself, the producer for the slot to come back -- whichever limit runs
+# out first reports (7, 2 or 1)
+fp = B.Factors.create(W.gen_factors(0, n_sets=X.shape[1] // 32))
+qk_ref, sk_ref = B.kroquant_quantize(X, fp, path="onchip")
+torch.cuda.synchronize()
+assert B.kroquant_last_device_error() == 0
+B.kroquant_debug_withhold_arrival(True)
+B.kroquant_quantize(X, fp, path="onchip")
+torch.cuda.synchronize()
+err = B.kroquant_last_device_error()
+B.kroquant_debug_withhold_arrival(False)
+assert err in (1, 2, 7), err
+qk, sk = B.kroquant_quantize(X, fp, path="onchip")
+torch.cuda.synchronize()
+assert B.kroquant_last_device_error() == 0
+assert torch.equal(qk, qk_ref) and torch.equal(sk, sk_ref)
 print("ok", round(dt, 3))
 """ % ROOT
 
