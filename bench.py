@@ -1041,6 +1041,54 @@ def run_timeline(args):
     print(json.dumps(out), flush=True)
 
 
+def run_boundary_floor(args):
+    """What the platform charges a dependent launch, apart from anything the quantizer does: chains of ten probe
+    kernels (diagnostic build of the library, kroquant_debug_boundary_probe) whose CTAs only take tensor memory or not,
+    wait for the launch before, idle for a fixed time and leave.  One JSON line per setting: the period of the chain
+    minus the idle time is the cost of the kernel boundary; cta_start says when the next launch's CTAs begin,
+    relative to the end of the last CTA of the launch before."""
+    import torch
+    from paper_2607_21446_b200 import binding as B, build as kbuild
+    B.use_library(kbuild.build_timeline())
+    B.load_library()
+    calls, spin = 10, args.spin_ns
+    stream = torch.cuda.Stream()
+    marks = torch.zeros(calls * 1024 * 4, dtype=torch.int64, device="cuda")
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    settings = [(0, 1, 1), (512, 1, 1), (0, 2, 1), (32, 2, 1), (128, 2, 1), (256, 2, 1), (-1, 2, 1), (0, 3, 1), (128, 3, 1),
+                (0, 2, 0), (256, 2, 0), (0, 3, 0), (128, 3, 0)]
+    for cols, cps, late in settings:
+        with torch.cuda.stream(stream):
+            B.kroquant_debug_boundary_probe(cols, cps, late, spin, calls, marks, stream)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                B.kroquant_debug_boundary_probe(cols, cps, late, spin, calls, marks, stream)
+            for _ in range(5):
+                g.replay()
+            torch.cuda.synchronize()
+            marks.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+        a = marks.cpu().numpy().reshape(calls, 1024, 4)[:, : sms * cps, :].astype(np.float64)
+        ends = a[:, :, 3].max(axis=1)
+        start, ready, setup, periods = np.zeros(3), 0.0, 0.0, []
+        for k in range(2, calls):
+            v = np.sort(a[k, :, 0] - ends[k - 1]) / 1e3
+            start += np.array([v[0], v[len(v) // 2], v[-1]]) / (calls - 2)
+            ready += float(np.median(a[k, :, 2] - ends[k - 1])) / 1e3 / (calls - 2)
+            setup += float(np.median(a[k, :, 1] - a[k, :, 0])) / 1e3 / (calls - 2)
+            periods.append((ends[k] - ends[k - 1]) / 1e3)
+        period = float(np.mean(periods))
+        print(json.dumps({"boundary_floor": {"tmem_cols_per_cta": max(cols, 0), "tcgen05_in_kernel": cols != 0,
+                                             "permit_released": cols > 0 if cols != 0 else None, "ctas_per_sm": cps,
+                                             "completion_signal": "at CTA end" if late else "at CTA start"},
+                          "idle_us": spin / 1e3, "period_us": round(period, 2), "boundary_cost_us": round(period - spin / 1e3, 2),
+                          "cta_start_us_after_previous_launch_ended": [round(float(x), 2) for x in start],
+                          "setup_us": round(setup, 2), "wait_returned_us_after_previous_launch_ended": round(ready, 2),
+                          "ctas": sms * cps}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", action="store_true",
@@ -1049,6 +1097,9 @@ def main():
                     help="tokens x d sweep of KroQuant / Scale / bare MXFP4 (one JSON line per point)")
     ap.add_argument("--timeline", default=None, metavar="TOKENSxD",
                     help="per-CTA timeline of back-to-back calls at the kernel boundary (timeline build of the library)")
+    ap.add_argument("--boundary-floor", action="store_true",
+                    help="platform cost of a dependent launch with and without tensor memory (probe kernels, diagnostic build)")
+    ap.add_argument("--spin-ns", type=int, default=3000, help="with --boundary-floor: idle time of a probe CTA")
     ap.add_argument("--configs", action="store_true",
                     help="the tiny, PixArt-, SANA- (shared and per-block sets) and FLUX-shaped tensors, measured and parity-checked like --sweep")
     ap.add_argument("--points", default=None, metavar="TOKENSxD,...", help="with --sweep: only these points")
@@ -1082,6 +1133,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.timeline:
         run_timeline(args)
+    elif args.boundary_floor:
+        run_boundary_floor(args)
     elif args.table:
         run_table(args)
     elif args.sweep or args.configs:

@@ -274,6 +274,18 @@ kq_status_t kroquant_debug_set_timeline(void *marks);
  * This is how the bounded waits are tested without a fault or a hang. */
 kq_status_t kroquant_debug_withhold_arrival(int on);
 
+/* Diagnostic builds only (KQ_ERR_UNSUPPORTED otherwise): what a dependent launch costs on this platform, with and
+ * without tensor memory.  Launches `calls` (1..16) probe kernels back to back on `stream`, chained by programmatic
+ * dependent launch, ctas_per_sm (1..4) CTAs of 256 threads per SM; each CTA takes tmem_cols columns of tensor memory
+ * (0 = none, and the kernel holds no tensor-memory instruction at all; -1 = none, but the kernel is the one that can
+ * allocate, and the CTA never releases its allocation permit; else a power of two 32..512, ctas_per_sm * tmem_cols
+ * <= 512), waits for the launch before, idles
+ * spin_ns (<= 100000) nanoseconds, signals completion at its start (late_trigger = 0) or at its end, and leaves.
+ * marks: DEVICE int64 [calls][1024][4] = global timer at CTA start, set-up done, dependency wait returned, CTA end.
+ * Touches no other data; `bench.py --boundary-floor` turns the marks into a table. */
+kq_status_t kroquant_debug_boundary_probe(int tmem_cols, int ctas_per_sm, int late_trigger, int spin_ns, int calls,
+                                          void *marks, void *stream);
+
 /* The W4A4 product of the quantized layer (Section 3.4: O = Q(A T) Q(W~)^T + A T L R):
  *     out[m][n] = sum_k a[m][k] 2^(sa[m][k/32] - 127) * b[n][k] 2^(sb[n][k/32] - 127)  (+ add[m][n])
  * on the block-scaled FP4 tensor-core path (fp32 accumulation).  a_codes [M][K/2] and b_codes

@@ -28,7 +28,7 @@ EXPORTS = [
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
     "kroquant_tuning_default", "kroquant_quantize_tuned", "kroquant_quantize_dual_tuned", "kroquant_transform_f32_tuned",
-    "kroquant_scale_quantize_tuned", "kroquant_mxfp4_quantize_tuned", "kroquant_debug_set_timeline", "kroquant_debug_withhold_arrival", "kroquant_launch_count", "kroquant_last_device_error",
+    "kroquant_scale_quantize_tuned", "kroquant_mxfp4_quantize_tuned", "kroquant_debug_set_timeline", "kroquant_debug_withhold_arrival", "kroquant_debug_boundary_probe", "kroquant_launch_count", "kroquant_last_device_error",
     "kroquant_status_string",
     "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
@@ -90,6 +90,7 @@ def load_library() -> C.CDLL:
     L.kroquant_scale_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp]
     L.kroquant_mxfp4_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, vp]
     L.kroquant_debug_set_timeline.argtypes = [vp]
+    L.kroquant_debug_boundary_probe.argtypes = [i32, i32, i32, i32, i32, vp, vp]
     L.kroquant_launch_count.argtypes = []
     L.kroquant_launch_count.restype = i64
     L.kroquant_last_device_error.argtypes = [vp, C.POINTER(i32)]
@@ -350,6 +351,14 @@ def use_library(path: str) -> None:
     """Load another build of the library (the timeline build) instead of libkroquant.so; call before anything else."""
     global LIB_PATH, _lib
     LIB_PATH, _lib = path, None
+
+
+def kroquant_debug_boundary_probe(tmem_cols: int, ctas_per_sm: int, late_trigger: bool, spin_ns: int, calls: int,
+                                  marks: torch.Tensor, stream=None) -> None:
+    """Diagnostic build only: `calls` chained probe launches (see the header); marks: int64 [calls, 1024, 4] on the device."""
+    assert marks.dtype == torch.int64 and marks.numel() >= calls * 1024 * 4 and marks.is_cuda
+    _check(load_library().kroquant_debug_boundary_probe(tmem_cols, ctas_per_sm, 1 if late_trigger else 0, spin_ns, calls,
+                                                        _ptr(marks), C.c_void_p(_stream(stream))), "kroquant_debug_boundary_probe")
 
 
 def kroquant_debug_set_timeline(marks: Optional[torch.Tensor]) -> None:

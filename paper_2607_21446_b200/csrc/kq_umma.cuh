@@ -1137,4 +1137,37 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     }
 }
 
+#ifdef KQ_TIMELINE
+// What a dependent launch costs on this platform, with and without tensor memory: a CTA that (optionally) takes
+// tmem_cols columns of tensor memory, waits for the prerequisite grid, idles for spin_ns, signals completion at its
+// start or at its end, and leaves.  Marks per CTA: start, set-up done (allocation), dependency wait returned, end.
+// TMEM = false: no tcgen05 instruction in the kernel at all.  TMEM = true with tmem_cols <= 0: the instructions are
+// in the kernel but this launch executes none of them, not even the release of the allocation permit.
+template <bool TMEM>
+__global__ void __launch_bounds__(256) boundary_probe(long long* marks, int slot, int tmem_cols, int late_trigger, int spin_ns) {
+    __shared__ uint32_t tslot;
+    auto now = [] { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return (long long)t; };
+    const long long t0 = now();
+    if (!late_trigger) pdl_launch_dependents();
+    if (TMEM && tmem_cols > 0 && threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tslot)), "r"((uint32_t)tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+    const long long t1 = now();
+    pdl_wait_prior_grid();
+    const long long t2 = now();
+    while (now() - t2 < (long long)spin_ns) {}
+    if (late_trigger) pdl_launch_dependents();
+    __syncthreads();
+    if (TMEM && tmem_cols > 0 && threadIdx.x < 32)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tslot), "r"((uint32_t)tmem_cols) : "memory");
+    if (threadIdx.x == 0 && blockIdx.x < 1024) {
+        long long* m = marks + ((size_t)slot * 1024 + blockIdx.x) * 4;
+        m[0] = t0; m[1] = t1; m[2] = t2; m[3] = now();
+    }
+}
+#endif
+
 }  // namespace kq

@@ -959,6 +959,47 @@ kq_status_t kroquant_debug_withhold_arrival(int on) {
 #endif
 }
 
+kq_status_t kroquant_debug_boundary_probe(int tmem_cols, int ctas_per_sm, int late_trigger, int spin_ns, int calls,
+                                          void* marks, void* stream) {
+#ifdef KQ_TIMELINE
+    if (!marks) return KQ_ERR_NULL;
+    const bool cols_ok = tmem_cols == 0 || tmem_cols == -1 ||
+                         (tmem_cols >= 32 && tmem_cols <= 512 && (tmem_cols & (tmem_cols - 1)) == 0);
+    if (!cols_ok || ctas_per_sm < 1 || ctas_per_sm > 4 || tmem_cols * ctas_per_sm > 512 || spin_ns < 0 || spin_ns > 100000 ||
+        calls < 1 || calls > 16)
+        return KQ_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0 || sms * ctas_per_sm > 1024) return KQ_ERR_CUDA;
+    auto kern = tmem_cols == 0 ? kq::boundary_probe<false> : kq::boundary_probe<true>;
+    // residency through the shared memory a CTA asks for: just too much for one more CTA per SM
+    const int smem = ((233472 / (ctas_per_sm + 1) - 1024) & ~127) + 128;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 116224) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KQ_ERR_CUDA;
+    }
+    for (int i = 0; i < calls; ++i) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(sms * ctas_per_sm));
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = (size_t)smem;
+        cfg.stream = static_cast<cudaStream_t>(stream);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kern, static_cast<long long*>(marks), i, tmem_cols, late_trigger, spin_ns) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KQ_ERR_CUDA;
+        }
+    }
+    return KQ_OK;
+#else
+    (void)tmem_cols; (void)ctas_per_sm; (void)late_trigger; (void)spin_ns; (void)calls; (void)marks; (void)stream;
+    return KQ_ERR_UNSUPPORTED;
+#endif
+}
+
 int64_t kroquant_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 kq_status_t kroquant_last_device_error(void* stream, int* code_out) {

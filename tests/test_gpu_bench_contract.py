@@ -74,3 +74,17 @@ def test_reference_arm_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] == d["value"]
     assert d["e2e"] == {"value": d["value"], "unit": d["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert d["higher_is_better"] is True and d["value"] > 0
+
+
+def test_boundary_floor_lines():
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--boundary-floor", "--spin-ns", "2000"],
+                         cwd=ROOT, capture_output=True, text=True, timeout=900)
+    assert res.returncode == 0, res.stderr[-2000:]
+    rows = [json.loads(l) for l in res.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(rows) >= 10
+    for r in rows:
+        assert r["idle_us"] == 2.0 and r["period_us"] > 2.0 and 0.2 < r["boundary_cost_us"] < 20.0
+    plain = [r for r in rows if not r["boundary_floor"]["tcgen05_in_kernel"]]
+    tmem = [r for r in rows if r["boundary_floor"]["permit_released"]]
+    # a launch whose CTAs take tensor memory never costs less than the cheapest one that takes none
+    assert min(r["boundary_cost_us"] for r in tmem) > min(r["boundary_cost_us"] for r in plain)

@@ -81,3 +81,4 @@ def test_ordinary_build_refuses_the_diagnostic_calls():
     L = B.load_library()
     assert L.kroquant_debug_withhold_arrival(1) == 5          # KQ_ERR_UNSUPPORTED
     assert L.kroquant_debug_set_timeline(None) == 5
+    assert L.kroquant_debug_boundary_probe(0, 1, 1, 0, 1, None, None) == 5
