@@ -321,9 +321,18 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     const int cps_set = t_tuning.ctas_per_sm;
     // (a launch that fits the GPU in one wave of the smaller CTAs keeps those: more of them run at once)
     // (the fp16 two-output kernel would spill registers at two large CTAs per SM)
-    const bool big_ctas = main_variant && !(xf16 && at_out != nullptr && !WRITE_Y) && cps_set == 0 &&
+    // (a launch of three to ten tiles per SM is over before a hand-out pays: two small CTAs per SM, static strides,
+    //  single-tile units -- measured 11-12 % faster than the large dynamic shape at 4 to 8 tiles per SM, equal at 10)
+    const bool mid_launch = main_variant && cps_set == 0 && t_tuning.unit_tiles == 0 &&
+                            prob.n_tiles > (int64_t)3 * sm_count() && prob.n_tiles <= (int64_t)10 * sm_count();
+    const bool big_ctas = main_variant && !(xf16 && at_out != nullptr && !WRITE_Y) && cps_set == 0 && !mid_launch &&
                           prob.n_tiles > (int64_t)3 * sm_count();
-    const int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
+    const int cps = cps_set > 0 ? cps_set : ((big_ctas || mid_launch) ? 2 : 3);
+    if (mid_launch) {
+        prob.dynamic = 0;
+        prob.unit_tiles = 1;
+        prob.n_units = prob.n_tiles;
+    }
     const bool pdl = t_tuning.use_pdl != 0;
     // A launch whose units all fit the GPU at once has nothing to hand out: static distribution (no cancel
     // request, no shared-memory padding), and the completion signal goes back to the kernel's start, where it
@@ -423,8 +432,17 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
     const int cps_set = t_tuning.ctas_per_sm;
-    const bool big_ctas = cps_set == 0 && prob.n_tiles > (int64_t)3 * sm_count();
-    int cps = cps_set > 0 ? cps_set : (big_ctas ? 2 : 3);
+    // (the launch shapes follow run_umma's rule: small CTAs for up to three tiles per SM, two small CTAs per SM on
+    //  static strides up to ten, the large dynamic shape above)
+    const bool mid_launch = cps_set == 0 && t_tuning.unit_tiles == 0 &&
+                            prob.n_tiles > (int64_t)3 * sm_count() && prob.n_tiles <= (int64_t)10 * sm_count();
+    const bool big_ctas = cps_set == 0 && !mid_launch && prob.n_tiles > (int64_t)3 * sm_count();
+    int cps = cps_set > 0 ? cps_set : ((big_ctas || mid_launch) ? 2 : 3);
+    if (mid_launch) {
+        prob.dynamic = 0;
+        prob.unit_tiles = 1;
+        prob.n_units = prob.n_tiles;
+    }
     const bool pdl = t_tuning.use_pdl != 0;
     bool big = cps_set == 0 ? big_ctas : t_tuning.config == 2;
     const int box_rows = nb <= 256 ? nb : 128;                 // rows of one TMA box of the multiplier matrix
