@@ -445,6 +445,7 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     }
     const bool pdl = t_tuning.use_pdl != 0;
     bool big = cps_set == 0 ? big_ctas : t_tuning.config == 2;
+    bool six = false;
     const int box_rows = nb <= 256 ? nb : 128;                 // rows of one TMA box of the multiplier matrix
     const int vec = chan_scale ? (nb + box_rows - 1) / box_rows * box_rows * 128 + 1024 : 0;   // whole boxes, 1 KB-aligned
     CUtensorMap tmap_s = tmap;
@@ -460,8 +461,13 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     if (chan_scale) {
         constexpr int kSmemPerSm = 233472, kSmemReserved = 1024;
         const int big_bytes = kq::UmmaSmem<8, false>::kDynBytes + vec, small_bytes = kq::UmmaSmem<4, false>::kDynBytes + vec;
-        if (big && 2 * (big_bytes + kSmemReserved) > kSmemPerSm) big = false;      // eight stages would leave one CTA per SM
-        if (!big) {
+        // eight stages next to a long vector would leave one CTA per SM: six if they fit (no tensor memory here, so the
+        // stage count need not be a power of two), else four
+        if (big && 2 * (big_bytes + kSmemReserved) > kSmemPerSm) {
+            big = false;
+            six = 2 * (kq::UmmaSmem<6, false>::kDynBytes + vec + kSmemReserved) <= kSmemPerSm;
+        }
+        if (!big && !six) {
             if (small_bytes + kSmemReserved > kSmemPerSm / 2) return KQ_ERR_UNSUPPORTED;
             while (cps > 2 && cps * (small_bytes + kSmemReserved) > kSmemPerSm) --cps;
             if (big_ctas) cps = 2;
@@ -476,8 +482,10 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     launch_umma<NS, NM, NG, false, XF, false, kq::kExtraNone, OPC>(tmap, tmap_s, nullptr, nullptr, prob, q, scales, nullptr, \
                                                                    nullptr, cps, pdl, st, nullptr, chan_scale, vec)
     if (chan_scale) {
-        if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true, kq::kOpScale) : KQ_LAUNCH_CMP(4, 2, 2, true, kq::kOpScale);
-        return big ? KQ_LAUNCH_CMP(8, 2, 2, false, kq::kOpScale) : KQ_LAUNCH_CMP(4, 2, 2, false, kq::kOpScale);
+        if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true, kq::kOpScale) : six ? KQ_LAUNCH_CMP(6, 2, 2, true, kq::kOpScale)
+                                                                             : KQ_LAUNCH_CMP(4, 2, 2, true, kq::kOpScale);
+        return big ? KQ_LAUNCH_CMP(8, 2, 2, false, kq::kOpScale) : six ? KQ_LAUNCH_CMP(6, 2, 2, false, kq::kOpScale)
+                                                                 : KQ_LAUNCH_CMP(4, 2, 2, false, kq::kOpScale);
     }
     if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true, kq::kOpPlain) : KQ_LAUNCH_CMP(4, 2, 1, true, kq::kOpPlain);
     return big ? KQ_LAUNCH_CMP(8, 2, 2, false, kq::kOpPlain) : KQ_LAUNCH_CMP(4, 2, 1, false, kq::kOpPlain);
