@@ -259,6 +259,9 @@ kq_status_t kroquant_scale_quantize_tuned(const void *X, kq_xdtype_t x_dtype, in
 kq_status_t kroquant_mxfp4_quantize_tuned(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d,
                                           uint8_t *q_packed, uint8_t *scales, kq_scale_layout_t scale_layout,
                                           const kq_tuning_t *tuning, void *stream);
+/* kroquant_fwht_quantize with a tuning struct (compare_staged = 0 selects the multi-pass kernel for every d). */
+kq_status_t kroquant_fwht_quantize_tuned(const void *X, kq_xdtype_t x_dtype, int64_t tokens, int d, uint8_t *q_packed,
+                                         uint8_t *scales, const kq_tuning_t *tuning, void *stream);
 
 /* Timeline builds only (the library compiled with -DKQ_TIMELINE, `python -m paper_2607_21446_b200.build
  * --timeline`; the ordinary build returns KQ_ERR_UNSUPPORTED): every CTA of the quantizer kernels writes the

@@ -28,7 +28,7 @@ EXPORTS = [
     "kroquant_quantize_path", "kroquant_dequantize", "kroquant_scale_quantize",
     "kroquant_mxfp4_quantize", "kroquant_transform_f32", "kroquant_debug_e2m1_codes",
     "kroquant_tuning_default", "kroquant_quantize_tuned", "kroquant_quantize_dual_tuned", "kroquant_transform_f32_tuned",
-    "kroquant_scale_quantize_tuned", "kroquant_mxfp4_quantize_tuned", "kroquant_debug_set_timeline", "kroquant_debug_withhold_arrival", "kroquant_debug_boundary_probe", "kroquant_launch_count", "kroquant_last_device_error",
+    "kroquant_scale_quantize_tuned", "kroquant_mxfp4_quantize_tuned", "kroquant_fwht_quantize_tuned", "kroquant_debug_set_timeline", "kroquant_debug_withhold_arrival", "kroquant_debug_boundary_probe", "kroquant_launch_count", "kroquant_last_device_error",
     "kroquant_status_string",
     "kroquant_calib_create", "kroquant_calib_destroy", "kroquant_calib_set_theta", "kroquant_calib_get_theta",
     "kroquant_calib_set_lambdas", "kroquant_calib_get_lambdas", "kroquant_calib_get_factors",
@@ -89,6 +89,7 @@ def load_library() -> C.CDLL:
     L.kroquant_transform_f32_tuned.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, vp]
     L.kroquant_scale_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, vp, i32, vp, vp]
     L.kroquant_mxfp4_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, i32, vp, vp]
+    L.kroquant_fwht_quantize_tuned.argtypes = [vp, i32, i64, i32, vp, vp, vp, vp]
     L.kroquant_debug_set_timeline.argtypes = [vp]
     L.kroquant_debug_boundary_probe.argtypes = [i32, i32, i32, i32, i32, vp, vp]
     L.kroquant_launch_count.argtypes = []
@@ -265,15 +266,15 @@ def kroquant_quantize_dual(X: torch.Tensor, factors: Factors, q_packed=None, sca
     return q_packed, scales, AT
 
 
-def kroquant_fwht_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=None):
+def kroquant_fwht_quantize(X: torch.Tensor, q_packed=None, scales=None, stream=None, tuning: Optional[Tuning] = None):
     """Full-d Walsh-Hadamard comparison quantizer (d a power of two, 32..16384)."""
     tokens, d = _x_shape(X)
     if q_packed is None:
         q_packed = torch.empty((tokens, d // 2), dtype=torch.uint8, device=X.device)
     if scales is None:
         scales = torch.empty((tokens, d // 32), dtype=torch.uint8, device=X.device)
-    _check(load_library().kroquant_fwht_quantize(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(q_packed), _ptr(scales),
-                                                 C.c_void_p(_stream(stream))), "kroquant_fwht_quantize")
+    _check(load_library().kroquant_fwht_quantize_tuned(_ptr(X), X_DTYPES[X.dtype], tokens, d, _ptr(q_packed), _ptr(scales),
+                                                       _tuning(tuning), C.c_void_p(_stream(stream))), "kroquant_fwht_quantize")
     return q_packed, scales
 
 

@@ -207,11 +207,11 @@ __device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcon
 // PB = false: one factor image for the whole launch at offset 0, stages of 8 KB (A only).
 // PB = true : every stage carries its own factor image: 8 KB of A + 6 KB of B.
 constexpr int kRingEntries = 32;
-template <int NS, bool PB>
+template <int NS, bool PB, int IMG = 8192>
 struct UmmaSmem {
     static constexpr int kStageBytes = kTileBytes + (PB ? kBImageBytes : 0);   // multiple of 1024
-    static constexpr int kBOff = 0;                                  // shared image (PB = false)
-    static constexpr int kAOff = PB ? 0 : 8192;                      // NS stages
+    static constexpr int kBOff = 0;                                  // shared image (PB = false): IMG bytes reserved
+    static constexpr int kAOff = PB ? 0 : IMG;                       // NS stages
     // PB only: staging of a column group's outputs: 128 rows x 64 B of codes (64-byte
     // swizzle, leaves by TMA store) and 128 x 4 scale bytes; two tiles, so that a group can be staged while
     // the TMA store of the group before still reads its tile
@@ -482,6 +482,7 @@ struct UmmaProblem {
     int64_t n_tiles;     // PB=false: 128-row tiles
     int unit_tiles;      // PB=false: consecutive tiles per work unit (PB: kPbCols)
     int tl_slot;         // timeline builds: which launch slot of the mark buffer this launch writes
+    float norm;          // Hadamard comparison: 1 / sqrt(d)
     int dynamic;         // 1: the grid has one CTA per unit and running CTAs take over the units of CTAs that
                          // have not started yet (cluster launch control); 0: CTA b takes units b, b + gridDim.x, ...
 };
@@ -538,7 +539,16 @@ constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
 //     builders): the image of tile n is built into the tile's own stage while its activations are on their way -- the
 //     producer announces the tile on issued[slot], the builders add their arrivals to the tile's "full" barrier --
 //     so a tile costs 80 bytes of L2 traffic for its operand instead of 6 KB.
-constexpr int kOpKron = 0, kOpPlain = 1, kOpScale = 2, kOpKronBuild = 3;
+//   kOpHadamard  the full-row Walsh-Hadamard comparison (Section 4.4, "FWHT"): y = x H_d / sqrt(d) for a power of two
+//     d <= 4096.  With nb = d/32 blocks per token (a divisor of 128), H_d = H_nb (x) H_32: a tile of 128 flat rows holds
+//     128/nb whole tokens, and the mixing ACROSS the blocks of a token is one tensor-core product with the roles of the
+//     operands exchanged -- A = I_(128/nb) (x) H_nb, a constant 128 x 128 matrix of +-1 and 0 that every CTA writes into
+//     shared memory itself (K-major, 128-byte swizzle, 32 KB), B = the staged tile read as it lies (128 K-rows of 32
+//     channels: an MN-major operand), eight M128 N32 K16 instructions, products exact -- while the mixing INSIDE a
+//     block, H_32 over the 32 values an epilogue thread holds anyway, is a five-stage butterfly in registers.  One pass
+//     over memory instead of log2(d).
+constexpr int kOpKron = 0, kOpPlain = 1, kOpScale = 2, kOpKronBuild = 3, kOpHadamard = 4;
+constexpr int kHadamardImageBytes = 128 * 128 * 2;
 template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone, int OP = kOpKron>
 // resident CTAs per SM the register budget must allow: (8,2,2) two; the one-warpgroup shapes three (two with the
 // calibration epilogue)
@@ -549,8 +559,10 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
               uint4* __restrict__ at_out, double* __restrict__ sumsq, const float* __restrict__ chan_scale) {
     constexpr bool DUAL = EXTRA == kExtraDual;
     constexpr bool CALIB = EXTRA == kExtraCalib;
-    constexpr bool TC = OP == kOpKron || OP == kOpKronBuild;            // tensor-core stage present
+    constexpr bool TC = OP == kOpKron || OP == kOpKronBuild || OP == kOpHadamard;   // tensor-core stage present
     constexpr bool BUILD = OP == kOpKronBuild;
+    constexpr bool HAD = OP == kOpHadamard;
+    static_assert(!HAD || (!PB && EXTRA == kExtraNone), "Hadamard comparison: flat view, one output");
     constexpr int NB = PB ? 2 : 4;                // builder warps: warps 2 and 3 (per-block sets) / epilogue group 0
     static_assert(!BUILD || (EXTRA == kExtraNone && (!PB || NM == 1)), "on-chip images: one output; per-block sets need two free warps");
     static_assert(TC || (!PB && !WRITE_Y && EXTRA == kExtraNone), "comparison kernels: flat view, quantizing path only");
@@ -563,7 +575,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     // only then does program order inside that warp guarantee that a parity wait never
     // runs a whole phase ahead of the barrier it polls.
     static_assert(NS % NM == 0 && NS % NG == 0, "slot ownership must be fixed");
-    using L = UmmaSmem<NS, PB>;
+    using L = UmmaSmem<NS, PB, OP == kOpHadamard ? kHadamardImageBytes : 8192>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -736,7 +748,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             mbar_init(bar_tempty(s), 4);
             mbar_init(bar_issued(s), 1);
         }
-        mbar_init(bar_b, (!PB && BUILD) ? NB : 1);
+        mbar_init(bar_b, (!PB && BUILD) ? NB : HAD ? 4 * NG : 1);
         if (PB && !BUILD)
             for (int s = 0; s < NS; ++s) slot_jg[s] = -1;
         mbar_init(bar_clc, 1);
@@ -750,7 +762,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
         if (PB && !WRITE_Y) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_q) : "memory");
         if (prob.dynamic) clc_request();       // concerns this grid's own CTAs only
-        if (TC && !PB && !BUILD) {
+        if (TC && !PB && !BUILD && !HAD) {
             mbar_expect_tx(bar_b, kBImageBytes);
             bulk_load(base + L::kBOff, b_image, kBImageBytes, bar_b);
         }
@@ -836,6 +848,12 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                     b_desc[t][kk] = smem_desc_sw64(base + (PB ? L::kAOff + kTileBytes : L::kBOff) +
                                                    t * kBTermBytes + kk * 32);
             const uint64_t a_desc0 = smem_desc_sw64(base + L::kAOff);
+            // (Hadamard image: K-major, 128-byte rows, 8-row groups 1024 bytes apart)
+            uint64_t had_desc0 = 0;
+            if (HAD) {
+                had_desc0 = (uint64_t)(((base + L::kBOff) >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+                            ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+            }
             int sentinels_seen = 0;
             for (int n = warp - 1; ok; n += NM) {
                 const int s = n % NS;
@@ -859,6 +877,16 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 const uint64_t slot_off = (uint64_t)((s * L::kStageBytes) >> 4);
                 const uint64_t a_desc = a_desc0 + slot_off;
                 const uint32_t d_addr = tmem_base + (uint32_t)(s * 32);
+                if (HAD) {
+                    // D[row][channel] = sum_k A[row][k] X[k][channel]: A = the +-1 image (K-major, two 64-element halves
+                    // of 16 KB, 32 bytes per K step inside a half), B = the staged tile, 16 K-rows = 1024 bytes per step
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        tc_mma_bf16(d_addr, had_desc0 + (uint64_t)((kk >> 2) * (16384 >> 4) + (kk & 3) * 2),
+                                    a_desc + (uint64_t)(kk * (1024 >> 4)), idesc_m128(XF16, 32u) | (1u << 16), (uint32_t)(kk != 0));
+                    tc_commit(bar_done(s));
+                    continue;
+                }
 #pragma unroll
                 for (int t = 0; t < 3; ++t) {
 #pragma unroll
@@ -904,6 +932,54 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         // ---------------- epilogue warpgroups ----------------
         const int g = (warp - 4) >> 2;             // warpgroup index
         const int quarter = warp & 3;              // TMEM lane quarter this warp may read
+        if (HAD) {
+            // the +-1 operand, written by all epilogue threads: 16-byte chunk (row m, K half h, chunk c) holds
+            // k = 64 h + 8 c ... + 7 and lies at 16384 h + 128 m + 16 (c ^ (m & 7)); entry (m, k) is 0 across tokens and
+            // (-1)^popcount((m mod nb) & (k mod nb)) inside one
+            const uint32_t in_token = (uint32_t)prob.blocks_per_row - 1u;        // nb is a power of two
+            const uint32_t one = XF16 ? 0x3C00u : 0x3F80u;
+            const uint32_t one2 = one | (one << 16);
+            for (int i = threadIdx.x - 128; i < 2048; i += 128 * NG) {
+                const int m = i >> 4, h = (i >> 3) & 1, c = i & 7;
+                uint32_t w[4];
+                if (in_token >= 7u) {
+                    // tokens of eight blocks and more: a chunk lies inside one token or outside it, and its eight signs
+                    // are those of k0 = 64 h + 8 c times row (m mod 8) of H_8
+                    const uint32_t k0 = (uint32_t)(64 * h + 8 * c);
+                    if ((((uint32_t)m ^ k0) & ~in_token) != 0u) {
+                        w[0] = w[1] = w[2] = w[3] = 0u;
+                    } else {
+                        const uint32_t flip = (uint32_t)(__popc((uint32_t)m & k0 & in_token) & 1) * 0x80008000u;
+                        const uint32_t m0 = (uint32_t)m & 1u, m1 = ((uint32_t)m >> 1) & 1u, m2 = ((uint32_t)m >> 2) & 1u;
+                        const uint32_t odd = m0 << 31;                      // sign of the odd element of a pair
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const uint32_t s_e = ((((uint32_t)e & 1u) & m1) ^ ((((uint32_t)e >> 1) & 1u) & m2)) * 0x80008000u;
+                            w[e] = one2 ^ flip ^ s_e ^ odd;
+                        }
+                    }
+                } else
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    uint32_t pair = 0;
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const uint32_t k = (uint32_t)(64 * h + 8 * c + 2 * e + q);
+                        uint32_t v = 0;
+                        if ((((uint32_t)m ^ k) & ~in_token) == 0u)                       // same token
+                            v = one | ((uint32_t)(__popc((uint32_t)m & k & in_token) & 1) << 15);
+                        pair |= v << (16 * q);
+                    }
+                    w[e] = pair;
+                }
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                             ::"r"(base + L::kBOff + (uint32_t)(16384 * h + 128 * m + 16 * (c ^ (m & 7)))),
+                               "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_b);
+        }
         if (BUILD && !PB && g == 0) {
             // the shared set's operand image (immutable factors: no dependency wait), a quarter of it per warp
             float4 g[5];
@@ -919,7 +995,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         if (OP == kOpScale) {
             if (!mbar_wait(bar_b, 0, abort_flag) && !*abort_flag) { atomicCAS(&g_kq_device_error, 0, KQ_DEV_TIMEOUT_B); *abort_flag = 1; }
         }
-        const int e_shared = (PB || !XF16 || !TC) ? 0 : __ldg(e_norm);
+        const int e_shared = (PB || !XF16 || !TC || HAD) ? 0 : __ldg(e_norm);
         double sq_sum = 0.0;                       // CALIB: this thread's sum of squared residuals
         for (int n = g;; n += NG) {
             const int s = n % NS;
@@ -937,6 +1013,35 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty(s));
+                if (HAD) {
+                    // H_32 over the block's 32 channels, then the 1 / sqrt(d) of the orthonormal transform: index bit 0
+                    // inside a register pair, bits 1..4 between pairs with packed adds and subtractions
+                    uint64_t p[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float a = __uint_as_float(acc[2 * i]), c = __uint_as_float(acc[2 * i + 1]);
+                        asm("mov.b64 %0, {%1, %2};" : "=l"(p[i]) : "f"(a + c), "f"(a - c));
+                    }
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (!(i & (1 << b))) {
+                                uint64_t lo, hi;
+                                asm("add.rn.f32x2 %0, %1, %2;" : "=l"(lo) : "l"(p[i]), "l"(p[i | (1 << b)]));
+                                asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(hi) : "l"(p[i]), "l"(p[i | (1 << b)]));
+                                p[i] = lo;
+                                p[i | (1 << b)] = hi;
+                            }
+                    uint64_t n2;
+                    asm("mov.b64 %0, {%1, %1};" : "=l"(n2) : "f"(prob.norm));
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        uint64_t d2;
+                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d2) : "l"(p[i]), "l"(n2));
+                        asm("mov.b64 {%0, %1}, %2;" : "=r"(acc[2 * i]), "=r"(acc[2 * i + 1]) : "l"(d2));
+                    }
+                }
             } else {
                 // the block's 64 bytes straight from the stage: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3)
                 const int r = quarter * 32 + lane;

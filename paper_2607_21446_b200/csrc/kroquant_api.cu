@@ -216,7 +216,7 @@ kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, cons
                         const int* enorm, const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, void* at_out, int ctas_per_sm, bool pdl,
                         cudaStream_t st, double* sumsq = nullptr, const float* chan_scale = nullptr, int extra_smem = 0) {
-    using L = kq::UmmaSmem<NS, PB>;
+    using L = kq::UmmaSmem<NS, PB, OP == kq::kOpHadamard ? kq::kHadamardImageBytes : 8192>;
     auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA, OP>;
     // Dynamic distribution: the grid has one CTA per unit and the hardware decides how many run at once, so the
     // number of resident CTAs per SM is set through the shared memory each CTA asks for: just too much for
@@ -490,6 +490,61 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     if (xf16) return big ? KQ_LAUNCH_CMP(8, 2, 2, true, kq::kOpPlain) : KQ_LAUNCH_CMP(4, 2, 1, true, kq::kOpPlain);
     return big ? KQ_LAUNCH_CMP(8, 2, 2, false, kq::kOpPlain) : KQ_LAUNCH_CMP(4, 2, 1, false, kq::kOpPlain);
 #undef KQ_LAUNCH_CMP
+}
+
+// The full-row Walsh-Hadamard comparison for d <= 4096 on the tensor-core pipeline (kOpHadamard): flat view, the launch
+// shapes of run_umma's shared-set path.
+template <bool WRITE_Y>
+kq_status_t run_fwht_umma(const void* X, bool xf16, int64_t tokens, int d, uint8_t* q, uint8_t* scales, float* Y,
+                          cudaStream_t st) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return KQ_ERR_CUDA;
+    const int nb = d / 32;
+    kq::UmmaProblem prob;
+    prob.blocks_per_row = nb;
+    prob.tiled_scales = 0;
+    prob.early_trigger = t_tuning.use_pdl != 0 ? t_tuning.trigger : 0;
+    prob.prefetch_tiles = t_tuning.use_pdl != 0 ? t_tuning.prefetch_tiles : 0;
+    prob.dynamic = t_tuning.dynamic;
+    prob.tl_slot = g_tl_next.fetch_add(1) % 64;
+    prob.norm = (float)(1.0 / std::sqrt((double)d));
+    prob.unit_tiles = (t_tuning.unit_tiles > 0 ? t_tuning.unit_tiles : 3);
+    prob.n_rows = tokens * (int64_t)nb;
+    prob.n_ttiles = 1;
+    prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
+    if ((t_tuning.unit_tiles == 0) && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
+    prob.n_units = (prob.n_tiles + prob.unit_tiles - 1) / prob.unit_tiles;
+    CUtensorMap tmap;
+    const cuuint64_t dims[2] = {32, (cuuint64_t)prob.n_rows}, strides[1] = {64};
+    const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&tmap, xf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<void*>(X), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return KQ_ERR_CUDA;
+    const int cps_set = t_tuning.ctas_per_sm;
+    const bool mid_launch = cps_set == 0 && t_tuning.unit_tiles == 0 &&
+                            prob.n_tiles > (int64_t)3 * sm_count() && prob.n_tiles <= (int64_t)10 * sm_count();
+    const bool big_ctas = cps_set == 0 ? (!mid_launch && prob.n_tiles > (int64_t)3 * sm_count()) : t_tuning.config == 2;
+    const int cps = cps_set > 0 ? cps_set : 2;          // 32 KB of operand image per CTA: two per SM in either shape
+    if (mid_launch) {
+        prob.dynamic = 0;
+        prob.unit_tiles = 1;
+        prob.n_units = prob.n_tiles;
+    }
+    const bool pdl = t_tuning.use_pdl != 0;
+    prob.prefetch_stride = sm_count() * cps;
+    if (prob.dynamic && prob.n_units <= (int64_t)sm_count() * cps) {
+        prob.dynamic = 0;
+        if (prob.early_trigger == 2) prob.early_trigger = 1;
+    }
+#define KQ_LAUNCH_HAD(NS, NM, NG, XF) \
+    launch_umma<NS, NM, NG, false, XF, WRITE_Y, kq::kExtraNone, kq::kOpHadamard>(tmap, tmap, nullptr, nullptr, prob, q, scales, Y, \
+                                                                              nullptr, cps, pdl, st)
+    if (xf16) return big_ctas ? KQ_LAUNCH_HAD(8, 2, 2, true) : KQ_LAUNCH_HAD(4, 2, 1, true);
+    return big_ctas ? KQ_LAUNCH_HAD(8, 2, 2, false) : KQ_LAUNCH_HAD(4, 2, 1, false);
+#undef KQ_LAUNCH_HAD
 }
 
 template <int MODE, bool WRITE_Y, bool XF16, bool TILED>
@@ -836,6 +891,12 @@ static kq_status_t run_fwht(const void* X, kq_xdtype_t x_dtype, int64_t tokens, 
     if (!aligned16(X) || (Y ? !aligned16(Y) : !aligned16(q_packed))) return KQ_ERR_ALIGN;
     if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
+    // up to d = 4096 a tile of 128 blocks holds whole tokens: the tensor-core kernel; above, the multi-pass kernel
+    if (d <= 4096 && t_tuning.compare_staged != 0) {
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        return Y ? run_fwht_umma<true>(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, nullptr, Y, st)
+                 : run_fwht_umma<false>(X, x_dtype == KQ_X_FP16, tokens, d, q_packed, scales, nullptr, st);
+    }
     const int sms = sm_count();
     if (sms <= 0) return KQ_ERR_CUDA;
     const int tpr = d > 8192 ? 1024 : d / 8;
@@ -962,6 +1023,13 @@ kq_status_t kroquant_mxfp4_quantize_tuned(const void* X, kq_xdtype_t x_dtype, in
     if (!valid_tuning(tuning)) return KQ_ERR_UNSUPPORTED;
     TuningScope scope(tuning);
     return kroquant_mxfp4_quantize_ex(X, x_dtype, tokens, d, q_packed, scales, scale_layout, stream);
+}
+
+kq_status_t kroquant_fwht_quantize_tuned(const void* X, kq_xdtype_t x_dtype, int64_t tokens, int d, uint8_t* q_packed,
+                                         uint8_t* scales, const kq_tuning_t* tuning, void* stream) {
+    if (!valid_tuning(tuning)) return KQ_ERR_UNSUPPORTED;
+    TuningScope scope(tuning);
+    return kroquant_fwht_quantize(X, x_dtype, tokens, d, q_packed, scales, stream);
 }
 
 kq_status_t kroquant_debug_set_timeline(void* marks) {

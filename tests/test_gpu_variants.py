@@ -153,7 +153,8 @@ def test_pixart_shaped_fp16_full_size(B):
 
 # ---- full-d Walsh-Hadamard comparison kernel -------------------------------------------------------------
 @pytest.mark.parametrize("dtype", ["bf16", "fp16"])
-@pytest.mark.parametrize("tokens,d", [(1, 32), (70, 64), (33, 256), (130, 1024), (37, 4096), (9, 8192), (5, 16384)])
+@pytest.mark.parametrize("tokens,d", [(1, 32), (70, 64), (33, 256), (130, 1024), (37, 4096), (9, 8192), (5, 16384),
+                                      (3000, 128), (1111, 2048), (700, 4096), (2500, 512)])
 def test_fwht_quantize(B, dtype, tokens, d):
     Xb = W.gen_activations(spec(tokens, d, seed=d + tokens), dtype)
     X = dev(Xb, dtype)
@@ -162,6 +163,25 @@ def test_fwht_quantize(B, dtype, tokens, d):
     qo, so, Y = co.hadamard_quantize(Xb, dtype)
     print(d, P.check_values(Yg.cpu().numpy(), Y, dtype))
     P.check_codes(q.cpu().numpy(), s.cpu().numpy(), qo, so, Y, exact=False, x_dtype=dtype)
+
+
+def test_fwht_tensor_core_and_multi_pass_kernels_agree(B):
+    """Up to d = 4096 the comparison runs on the tensor-core pipeline (one product across the blocks of a token, a
+    butterfly inside each block); the multi-pass kernel stays reachable through the tuning struct.  Both are held to
+    the oracle, and to each other where no value sits on a rounding boundary."""
+    for tokens, d in [(1500, 1024), (300, 4096)]:
+        Xb = W.gen_activations(spec(tokens, d, seed=d), "bf16")
+        X = dev(Xb, "bf16")
+        qo, so, Y = co.hadamard_quantize(Xb, "bf16")
+        outs = []
+        for staged in (1, 0):
+            n0 = B.kroquant_launch_count()
+            q, s = B.kroquant_fwht_quantize(X, tuning=B.Tuning(compare_staged=staged))
+            assert B.kroquant_launch_count() == n0 + 1
+            P.check_codes(q.cpu().numpy(), s.cpu().numpy(), qo, so, Y, exact=False)
+            outs.append((q, s))
+        assert (outs[0][0] != outs[1][0]).float().mean().item() <= 1e-4
+    assert B.kroquant_last_device_error() == 0
 
 
 def test_fwht_rejects_other_sizes(B):
