@@ -167,6 +167,49 @@ __device__ __forceinline__ void tc_ld_32x32_wait(uint32_t taddr, uint32_t (&r)[3
         : "r"(taddr) : "memory");
 }
 
+// eight columns of this warp's 32 TMEM lanes, without the completion wait; the matching store; the two waits
+__device__ __forceinline__ void tc_ld_32x8_nowait(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_st_32x8(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait_all() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_st_wait_all() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// H_32 over the 32 values of a block held in registers, then the transform's normalisation: index bit 0 inside a
+// register pair, bits 1..4 between pairs with packed adds and subtractions (sm_100 add/sub/mul.f32x2).
+__device__ __forceinline__ void hadamard32_regs(uint32_t (&acc)[32], float norm) {
+    uint64_t p[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float a = __uint_as_float(acc[2 * i]), c = __uint_as_float(acc[2 * i + 1]);
+        asm("mov.b64 %0, {%1, %2};" : "=l"(p[i]) : "f"(a + c), "f"(a - c));
+    }
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (!(i & (1 << b))) {
+                uint64_t lo, hi;
+                asm("add.rn.f32x2 %0, %1, %2;" : "=l"(lo) : "l"(p[i]), "l"(p[i | (1 << b)]));
+                asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(hi) : "l"(p[i]), "l"(p[i | (1 << b)]));
+                p[i] = lo;
+                p[i | (1 << b)] = hi;
+            }
+    uint64_t n2;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(n2) : "f"(norm));
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        uint64_t d2;
+        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d2) : "l"(p[i]), "l"(n2));
+        asm("mov.b64 {%0, %1}, %2;" : "=r"(acc[2 * i]), "=r"(acc[2 * i + 1]) : "l"(d2));
+    }
+}
+
 // K-major operand tile with 64-byte rows in the 64-byte-swizzle layout: 8-row groups
 // 512 bytes apart (stride byte offset), descriptor version 1 (sm_100), swizzle code 4.
 __device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t saddr) {
@@ -207,9 +250,9 @@ __device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcon
 // PB = false: one factor image for the whole launch at offset 0, stages of 8 KB (A only).
 // PB = true : every stage carries its own factor image: 8 KB of A + 6 KB of B.
 constexpr int kRingEntries = 32;
-template <int NS, bool PB, int IMG = 8192>
+template <int NS, bool PB, int IMG = 8192, int STAGE = kTileBytes>
 struct UmmaSmem {
-    static constexpr int kStageBytes = kTileBytes + (PB ? kBImageBytes : 0);   // multiple of 1024
+    static constexpr int kStageBytes = STAGE + (PB ? kBImageBytes : 0);        // multiple of 1024
     static constexpr int kBOff = 0;                                  // shared image (PB = false): IMG bytes reserved
     static constexpr int kAOff = PB ? 0 : IMG;                       // NS stages
     // PB only: staging of a column group's outputs: 128 rows x 64 B of codes (64-byte
@@ -483,6 +526,7 @@ struct UmmaProblem {
     int unit_tiles;      // PB=false: consecutive tiles per work unit (PB: kPbCols)
     int tl_slot;         // timeline builds: which launch slot of the mark buffer this launch writes
     float norm;          // Hadamard comparison: 1 / sqrt(d)
+    int had_rows;        // Hadamard comparison: tile rows that make one token (d/32 up to d = 4096, then 128)
     int dynamic;         // 1: the grid has one CTA per unit and running CTAs take over the units of CTAs that
                          // have not started yet (cluster launch control); 0: CTA b takes units b, b + gridDim.x, ...
 };
@@ -539,17 +583,21 @@ constexpr int kExtraNone = 0, kExtraDual = 1, kExtraCalib = 2;
 //     builders): the image of tile n is built into the tile's own stage while its activations are on their way -- the
 //     producer announces the tile on issued[slot], the builders add their arrivals to the tile's "full" barrier --
 //     so a tile costs 80 bytes of L2 traffic for its operand instead of 6 KB.
-//   kOpHadamard  the full-row Walsh-Hadamard comparison (Section 4.4, "FWHT"): y = x H_d / sqrt(d) for a power of two
-//     d <= 4096.  With nb = d/32 blocks per token (a divisor of 128), H_d = H_nb (x) H_32: a tile of 128 flat rows holds
-//     128/nb whole tokens, and the mixing ACROSS the blocks of a token is one tensor-core product with the roles of the
-//     operands exchanged -- A = I_(128/nb) (x) H_nb, a constant 128 x 128 matrix of +-1 and 0 that every CTA writes into
-//     shared memory itself (K-major, 128-byte swizzle, 32 KB), B = the staged tile read as it lies (128 K-rows of 32
-//     channels: an MN-major operand), eight M128 N32 K16 instructions, products exact -- while the mixing INSIDE a
-//     block, H_32 over the 32 values an epilogue thread holds anyway, is a five-stage butterfly in registers.  One pass
-//     over memory instead of log2(d).
+//   kOpHadamard  the full-row Walsh-Hadamard comparison (Section 4.4, "FWHT"): y = x H_d / sqrt(d), d a power of two.
+//     With nb = d/32 blocks per token, H_d = H_nb (x) H_32.  A tile row is HT adjacent blocks of a token (64 HT contiguous
+//     bytes) and a tile of 128 rows holds whole tokens, so H_nb = H_(nb/HT) (x) H_HT is applied in two steps and H_32
+//     in a third:
+//     (i) across the rows of a token, one tensor-core product with the roles of the operands exchanged -- A =
+//     I (x) H_(nb/HT), a constant 128 x 128 matrix of +-1 and 0 that every CTA writes into shared memory itself (K-major,
+//     128-byte swizzle, 32 KB), B = the staged tile read as it lies (128 K-rows of 32 HT channels: an MN-major operand),
+//     eight M128 N(32 HT) K16 instructions, products exact;
+//     (ii) across the HT blocks of a row (HT > 1), by the thread that owns the row's TMEM lane: eight channels of all HT
+//     blocks are loaded, added and subtracted, and stored back to the accumulator;
+//     (iii) inside a block, H_32 over the 32 values the epilogue thread holds: a five-stage butterfly in registers.
+//     One pass over memory instead of log2(d).
 constexpr int kOpKron = 0, kOpPlain = 1, kOpScale = 2, kOpKronBuild = 3, kOpHadamard = 4;
 constexpr int kHadamardImageBytes = 128 * 128 * 2;
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone, int OP = kOpKron>
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kExtraNone, int OP = kOpKron, int HT = 1>
 // resident CTAs per SM the register budget must allow: (8,2,2) two; the one-warpgroup shapes three (two with the
 // calibration epilogue)
 __global__ void __launch_bounds__(128 + 128 * NG, (NS <= 8 && NG == 2) ? 2 : NG == 1 ? (EXTRA == kExtraCalib ? 2 : 3) : 1)
@@ -563,19 +611,23 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
     constexpr bool BUILD = OP == kOpKronBuild;
     constexpr bool HAD = OP == kOpHadamard;
     static_assert(!HAD || (!PB && EXTRA == kExtraNone), "Hadamard comparison: flat view, one output");
+    // HT > 1 (d = 4096 HT): a tile row is HT adjacent blocks (64 HT contiguous bytes), a tile one whole token
+    static_assert(HT == 1 || (HAD && (HT == 2 || HT == 4)), "wide rows: Hadamard comparison only");
     constexpr int NB = PB ? 2 : 4;                // builder warps: warps 2 and 3 (per-block sets) / epilogue group 0
     static_assert(!BUILD || (EXTRA == kExtraNone && (!PB || NM == 1)), "on-chip images: one output; per-block sets need two free warps");
     static_assert(TC || (!PB && !WRITE_Y && EXTRA == kExtraNone), "comparison kernels: flat view, quantizing path only");
     static_assert(!CALIB || (!XF16 && !WRITE_Y), "calibration outputs: bf16 images, quantizing path");
     static_assert(NM >= 1 && NM <= 3, "MMA issuer warps are warps 1..3");
     // TMEM is handed out in powers of two
-    constexpr int kTmemCols = NS * 32 <= 32 ? 32 : NS * 32 <= 64 ? 64 : NS * 32 <= 128 ? 128 : NS * 32 <= 256 ? 256 : 512;
-    static_assert(NS * 32 <= 512, "at most 16 accumulators of 32 columns");
+    constexpr int kAccCols = 32 * HT;             // columns of one accumulator
+    constexpr int kTmemCols = NS * kAccCols <= 32 ? 32 : NS * kAccCols <= 64 ? 64 : NS * kAccCols <= 128 ? 128
+                              : NS * kAccCols <= 256 ? 256 : 512;
+    static_assert(NS * kAccCols <= 512, "tensor memory has 512 columns");
     // A slot must always be served by the same issuer warp and the same epilogue group:
     // only then does program order inside that warp guarantee that a parity wait never
     // runs a whole phase ahead of the barrier it polls.
     static_assert(NS % NM == 0 && NS % NG == 0, "slot ownership must be fixed");
-    using L = UmmaSmem<NS, PB, OP == kOpHadamard ? kHadamardImageBytes : 8192>;
+    using L = UmmaSmem<NS, PB, OP == kOpHadamard ? kHadamardImageBytes : 8192, HT * kTileBytes>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -648,6 +700,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
         } else {
             mbar_expect_tx(bar_full(s), L::kStageBytes);
             tma_load_2d(dst, &tmap_x, 0, item * kTileRows, bar_full(s));
+            if (HT == 4) tma_load_2d(dst + 2 * kTileBytes, &tmap_x, 64, item * kTileRows, bar_full(s));   // boxes of 128 bytes
         }
     };
     auto prefetch_tile = [&](int item, int c) {
@@ -876,7 +929,20 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
                 tc_fence_after();
                 const uint64_t slot_off = (uint64_t)((s * L::kStageBytes) >> 4);
                 const uint64_t a_desc = a_desc0 + slot_off;
-                const uint32_t d_addr = tmem_base + (uint32_t)(s * 32);
+                const uint32_t d_addr = tmem_base + (uint32_t)(s * kAccCols);
+                if (HAD && HT > 1) {
+                    // wide rows: B = the staged tile, 128 K-rows of 128 bytes per box in the 128-byte swizzle (8-row
+                    // groups 1 KB apart, the second 64 channels one box = 16 KB further), 16 K-rows = 2 KB per step
+                    const uint64_t bw_desc = (uint64_t)(((base + L::kAOff + s * L::kStageBytes) >> 4) & 0x3FFFu) |
+                                             ((uint64_t)(16384 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+                                             ((uint64_t)2 << 61);
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        tc_mma_bf16(d_addr, had_desc0 + (uint64_t)((kk >> 2) * (16384 >> 4) + (kk & 3) * 2),
+                                    bw_desc + (uint64_t)(kk * (2048 >> 4)), idesc_m128(XF16, 32u * HT) | (1u << 16), (uint32_t)(kk != 0));
+                    tc_commit(bar_done(s));
+                    continue;
+                }
                 if (HAD) {
                     // D[row][channel] = sum_k A[row][k] X[k][channel]: A = the +-1 image (K-major, two 64-element halves
                     // of 16 KB, 32 bytes per K step inside a half), B = the staged tile, 16 K-rows = 1024 bytes per step
@@ -936,7 +1002,7 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             // the +-1 operand, written by all epilogue threads: 16-byte chunk (row m, K half h, chunk c) holds
             // k = 64 h + 8 c ... + 7 and lies at 16384 h + 128 m + 16 (c ^ (m & 7)); entry (m, k) is 0 across tokens and
             // (-1)^popcount((m mod nb) & (k mod nb)) inside one
-            const uint32_t in_token = (uint32_t)prob.blocks_per_row - 1u;        // nb is a power of two
+            const uint32_t in_token = (uint32_t)prob.had_rows - 1u;              // tile rows per token: a power of two
             const uint32_t one = XF16 ? 0x3C00u : 0x3F80u;
             const uint32_t one2 = one | (one << 16);
             for (int i = threadIdx.x - 128; i < 2048; i += 128 * NG) {
@@ -1006,42 +1072,72 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             const int item = ring[n % kRingEntries];
             if (n == 0 && threadIdx.x == 128) KQ_TL_MARK(prob.tl_slot, 2);
             if (item < 0) break;
+            if (HAD && HT > 1) {
+                // Wide rows: this thread's TMEM lane holds the HT adjacent blocks of one tile row, already mixed across
+                // the 128 rows of the token.  Pass 1 mixes across the HT blocks (the low bits of the block index), eight
+                // channels at a time, and writes the result back to the accumulator; pass 2 takes one block at a time:
+                // H_32 over its channels, normalisation, encoder.  Nothing leaves the thread's own lane.
+                const uint32_t t0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kAccCols);
+                tc_fence_after();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t w[HT][8];
+#pragma unroll
+                    for (int t = 0; t < HT; ++t) tc_ld_32x8_nowait(t0 + (uint32_t)(t * 32 + ch * 8), w[t]);
+                    tc_ld_wait_all();
+#pragma unroll
+                    for (int b = 0; b < (HT == 4 ? 2 : 1); ++b)
+#pragma unroll
+                        for (int t = 0; t < HT; ++t)
+                            if (!(t & (1 << b)))
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    const float a = __uint_as_float(w[t][i]), c = __uint_as_float(w[t | (1 << b)][i]);
+                                    w[t][i] = __float_as_uint(a + c);
+                                    w[t | (1 << b)][i] = __float_as_uint(a - c);
+                                }
+#pragma unroll
+                    for (int t = 0; t < HT; ++t) tc_st_32x8(t0 + (uint32_t)(t * 32 + ch * 8), w[t]);
+                }
+                tc_st_wait_all();
+                const int64_t sr = (int64_t)item * kTileRows + quarter * 32 + lane;        // tile row = HT blocks
+#pragma unroll
+                for (int t = 0; t < HT; ++t) {
+                    uint32_t acc[32];
+                    tc_ld_32x32_wait(t0 + (uint32_t)(t * 32), acc);
+                    if (t == HT - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_tempty(s));
+                    }
+                    hadamard32_regs(acc, prob.norm);
+                    if (sr < prob.n_rows) {
+                        const int64_t blk = sr * HT + t;
+                        if (WRITE_Y) {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                reinterpret_cast<float4*>(Y + blk * 32)[i] =
+                                    make_float4(__uint_as_float(acc[4 * i]), __uint_as_float(acc[4 * i + 1]),
+                                                __uint_as_float(acc[4 * i + 2]), __uint_as_float(acc[4 * i + 3]));
+                        } else {
+                            uint4 codes;
+                            uint32_t S;
+                            encode_block_regs(acc, 0, codes, S);
+                            st_stream_16(reinterpret_cast<uint4*>(q_packed) + blk, codes);
+                            scales[blk] = (uint8_t)S;
+                        }
+                    }
+                }
+                continue;
+            }
             uint32_t acc[32];
             if (TC) {
                 tc_fence_after();
-                tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * 32), acc);
+                tc_ld_32x32_wait(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(s * kAccCols), acc);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty(s));
-                if (HAD) {
-                    // H_32 over the block's 32 channels, then the 1 / sqrt(d) of the orthonormal transform: index bit 0
-                    // inside a register pair, bits 1..4 between pairs with packed adds and subtractions
-                    uint64_t p[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float a = __uint_as_float(acc[2 * i]), c = __uint_as_float(acc[2 * i + 1]);
-                        asm("mov.b64 %0, {%1, %2};" : "=l"(p[i]) : "f"(a + c), "f"(a - c));
-                    }
-#pragma unroll
-                    for (int b = 0; b < 4; ++b)
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            if (!(i & (1 << b))) {
-                                uint64_t lo, hi;
-                                asm("add.rn.f32x2 %0, %1, %2;" : "=l"(lo) : "l"(p[i]), "l"(p[i | (1 << b)]));
-                                asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(hi) : "l"(p[i]), "l"(p[i | (1 << b)]));
-                                p[i] = lo;
-                                p[i | (1 << b)] = hi;
-                            }
-                    uint64_t n2;
-                    asm("mov.b64 %0, {%1, %1};" : "=l"(n2) : "f"(prob.norm));
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        uint64_t d2;
-                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d2) : "l"(p[i]), "l"(n2));
-                        asm("mov.b64 {%0, %1}, %2;" : "=r"(acc[2 * i]), "=r"(acc[2 * i + 1]) : "l"(d2));
-                    }
-                }
+                if (HAD) hadamard32_regs(acc, prob.norm);      // H_32 over the block's channels and the 1 / sqrt(d)
             } else {
                 // the block's 64 bytes straight from the stage: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3)
                 const int r = quarter * 32 + lane;

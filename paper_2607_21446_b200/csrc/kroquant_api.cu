@@ -5,6 +5,7 @@
 
 #include <atomic>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -211,13 +212,13 @@ kq_status_t finish_factors(kroquant_factors_t* f, const std::vector<double>& K,
     return KQ_OK;
 }
 
-template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kq::kExtraNone, int OP = kq::kOpKron>
+template <int NS, int NM, int NG, bool PB, bool XF16, bool WRITE_Y, int EXTRA = kq::kExtraNone, int OP = kq::kOpKron, int HT = 1>
 kq_status_t launch_umma(const CUtensorMap& tmap, const CUtensorMap& tmap_q, const uint8_t* bimg,
                         const int* enorm, const kq::UmmaProblem& prob,
                         uint8_t* q, uint8_t* scales, float* Y, void* at_out, int ctas_per_sm, bool pdl,
                         cudaStream_t st, double* sumsq = nullptr, const float* chan_scale = nullptr, int extra_smem = 0) {
-    using L = kq::UmmaSmem<NS, PB, OP == kq::kOpHadamard ? kq::kHadamardImageBytes : 8192>;
-    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA, OP>;
+    using L = kq::UmmaSmem<NS, PB, OP == kq::kOpHadamard ? kq::kHadamardImageBytes : 8192, HT * kq::kTileBytes>;
+    auto kern = kq::quantize_umma<NS, NM, NG, PB, XF16, WRITE_Y, EXTRA, OP, HT>;
     // Dynamic distribution: the grid has one CTA per unit and the hardware decides how many run at once, so the
     // number of resident CTAs per SM is set through the shared memory each CTA asks for: just too much for
     // ctas_per_sm + 1 of them (228 KB per SM, 1 KB reserved per CTA).
@@ -500,8 +501,13 @@ kq_status_t run_fwht_umma(const void* X, bool xf16, int64_t tokens, int d, uint8
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
     const int nb = d / 32;
+    // A tile row is ht adjacent blocks (64 ht contiguous bytes): the product across rows then costs 1/ht of the MMAs per
+    // block, the mixing across the ht blocks of a row is a pass through tensor memory.  Measured best: 4 from d = 4096
+    // on (a token is then 32 rows and more), 2 below, single blocks only for d = 32.
+    const int ht = nb >= 128 ? 4 : nb >= 2 ? 2 : 1;
     kq::UmmaProblem prob;
     prob.blocks_per_row = nb;
+    prob.had_rows = nb / ht;
     prob.tiled_scales = 0;
     prob.early_trigger = t_tuning.use_pdl != 0 ? t_tuning.trigger : 0;
     prob.prefetch_tiles = t_tuning.use_pdl != 0 ? t_tuning.prefetch_tiles : 0;
@@ -509,20 +515,38 @@ kq_status_t run_fwht_umma(const void* X, bool xf16, int64_t tokens, int d, uint8
     prob.tl_slot = g_tl_next.fetch_add(1) % 64;
     prob.norm = (float)(1.0 / std::sqrt((double)d));
     prob.unit_tiles = (t_tuning.unit_tiles > 0 ? t_tuning.unit_tiles : 3);
-    prob.n_rows = tokens * (int64_t)nb;
+    prob.n_rows = tokens * (int64_t)nb / ht;
     prob.n_ttiles = 1;
     prob.n_tiles = (prob.n_rows + kq::kTileRows - 1) / kq::kTileRows;
     if ((t_tuning.unit_tiles == 0) && prob.n_tiles < (int64_t)8 * sm_count()) prob.unit_tiles = 1;
     prob.n_units = (prob.n_tiles + prob.unit_tiles - 1) / prob.unit_tiles;
     CUtensorMap tmap;
-    const cuuint64_t dims[2] = {32, (cuuint64_t)prob.n_rows}, strides[1] = {64};
-    const cuuint32_t box[2] = {32, (cuuint32_t)kq::kTileRows};
+    const cuuint64_t dims[2] = {(cuuint64_t)(32 * ht), (cuuint64_t)prob.n_rows}, strides[1] = {(cuuint64_t)(64 * ht)};
+    const cuuint32_t box[2] = {(cuuint32_t)(ht == 1 ? 32 : 64), (cuuint32_t)kq::kTileRows};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(&tmap, xf16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
             const_cast<void*>(X), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            CU_TENSOR_MAP_INTERLEAVE_NONE, ht == 1 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return KQ_ERR_CUDA;
+    if (ht > 1) {
+        // one shape each: four 16 KB stages and two CTAs per SM (rows of two blocks); four 32 KB stages, four epilogue
+        // warpgroups and all 512 accumulator columns in one CTA per SM (rows of four)
+        const int cps_w = ht == 2 ? 2 : 1;
+        const bool pdl_w = t_tuning.use_pdl != 0;
+        prob.prefetch_tiles = 0;                              // (the prefetch helper addresses 64-byte-wide tiles)
+        prob.prefetch_stride = sm_count() * cps_w;
+        if (prob.dynamic && prob.n_units <= (int64_t)sm_count() * cps_w) {
+            prob.dynamic = 0;
+            if (prob.early_trigger == 2) prob.early_trigger = 1;
+        }
+#define KQ_LAUNCH_HADW(NS, NM, NG, XF, HT) \
+    launch_umma<NS, NM, NG, false, XF, WRITE_Y, kq::kExtraNone, kq::kOpHadamard, HT>(tmap, tmap, nullptr, nullptr, prob, q, scales, \
+                                                                                  Y, nullptr, cps_w, pdl_w, st)
+        if (ht == 2) return xf16 ? KQ_LAUNCH_HADW(4, 2, 2, true, 2) : KQ_LAUNCH_HADW(4, 2, 2, false, 2);
+        return xf16 ? KQ_LAUNCH_HADW(4, 2, 4, true, 4) : KQ_LAUNCH_HADW(4, 2, 4, false, 4);
+#undef KQ_LAUNCH_HADW
+    }
     const int cps_set = t_tuning.ctas_per_sm;
     const bool mid_launch = cps_set == 0 && t_tuning.unit_tiles == 0 &&
                             prob.n_tiles > (int64_t)3 * sm_count() && prob.n_tiles <= (int64_t)10 * sm_count();
@@ -891,8 +915,9 @@ static kq_status_t run_fwht(const void* X, kq_xdtype_t x_dtype, int64_t tokens, 
     if (!aligned16(X) || (Y ? !aligned16(Y) : !aligned16(q_packed))) return KQ_ERR_ALIGN;
     if (!valid_xdtype(x_dtype)) return KQ_ERR_UNSUPPORTED;
     if (tokens == 0) return KQ_OK;
-    // up to d = 4096 a tile of 128 blocks holds whole tokens: the tensor-core kernel; above, the multi-pass kernel
-    if (d <= 4096 && t_tuning.compare_staged != 0) {
+    // the tensor-core kernel (a tile of the flat view holds whole tokens; from d = 8192 on one token, in rows of 2 or 4
+    // blocks); the multi-pass kernel only on request
+    if (t_tuning.compare_staged != 0) {
         cudaStream_t st = static_cast<cudaStream_t>(stream);
         return Y ? run_fwht_umma<true>(X, x_dtype == KQ_X_FP16, tokens, d, nullptr, nullptr, Y, st)
                  : run_fwht_umma<false>(X, x_dtype == KQ_X_FP16, tokens, d, q_packed, scales, nullptr, st);

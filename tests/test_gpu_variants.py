@@ -154,7 +154,7 @@ def test_pixart_shaped_fp16_full_size(B):
 # ---- full-d Walsh-Hadamard comparison kernel -------------------------------------------------------------
 @pytest.mark.parametrize("dtype", ["bf16", "fp16"])
 @pytest.mark.parametrize("tokens,d", [(1, 32), (70, 64), (33, 256), (130, 1024), (37, 4096), (9, 8192), (5, 16384),
-                                      (3000, 128), (1111, 2048), (700, 4096), (2500, 512)])
+                                      (3000, 128), (1111, 2048), (700, 4096), (2500, 512), (300, 8192), (200, 16384)])
 def test_fwht_quantize(B, dtype, tokens, d):
     Xb = W.gen_activations(spec(tokens, d, seed=d + tokens), dtype)
     X = dev(Xb, dtype)
@@ -166,10 +166,11 @@ def test_fwht_quantize(B, dtype, tokens, d):
 
 
 def test_fwht_tensor_core_and_multi_pass_kernels_agree(B):
-    """Up to d = 4096 the comparison runs on the tensor-core pipeline (one product across the blocks of a token, a
-    butterfly inside each block); the multi-pass kernel stays reachable through the tuning struct.  Both are held to
+    """The comparison runs on the tensor-core pipeline (one product across the blocks of a token -- from d = 8192 on
+    across its rows of 2 or 4 blocks, which a pass through tensor memory then mixes -- and a butterfly inside each
+    block); the multi-pass kernel stays reachable through the tuning struct.  Both are held to
     the oracle, and to each other where no value sits on a rounding boundary."""
-    for tokens, d in [(1500, 1024), (300, 4096)]:
+    for tokens, d in [(1500, 1024), (300, 4096), (150, 8192), (100, 16384)]:
         Xb = W.gen_activations(spec(tokens, d, seed=d), "bf16")
         X = dev(Xb, "bf16")
         qo, so, Y = co.hadamard_quantize(Xb, "bf16")
