@@ -185,6 +185,20 @@ def test_fwht_tensor_core_and_multi_pass_kernels_agree(B):
     assert B.kroquant_last_device_error() == 0
 
 
+def test_fwht_back_to_back_and_tuned_calls_agree(B):
+    """Chained launches (programmatic dependent launch, dynamic and static tile distribution, several tiles per CTA) of
+    the tensor-core Hadamard kernels must all give the same bytes."""
+    for tokens, d in [(6000, 1024), (3000, 4096), (1200, 16384)]:
+        X = dev(W.gen_activations(spec(tokens, d, seed=tokens), "bf16"), "bf16")
+        ref = B.kroquant_fwht_quantize(X)
+        outs = [B.kroquant_fwht_quantize(X) for _ in range(6)]
+        outs += [B.kroquant_fwht_quantize(X, tuning=B.Tuning(dynamic=dyn, unit_tiles=u, trigger=tr, prefetch_tiles=pf))
+                 for dyn, u, tr, pf in [(0, 1, 1, 0), (1, 2, 2, 4), (0, 3, 0, 1), (1, 1, 1, 2)]]
+        for q, s in outs:
+            assert torch.equal(q, ref[0]) and torch.equal(s, ref[1])
+    assert B.kroquant_last_device_error() == 0
+
+
 def test_fwht_rejects_other_sizes(B):
     import ctypes as C
     L = B.load_library()
