@@ -7,6 +7,7 @@
 //   v_c  = y_c * 2^(127 - S)                        (exact; |v_c| < 8)
 //   code = hardware float -> E2M1 convert (round-to-nearest-even, saturating at 6)
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>

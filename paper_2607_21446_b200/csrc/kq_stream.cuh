@@ -8,7 +8,8 @@
 //                                       transform y = x (G1 (x) .. (x) G5) applied
 //                                       factor by factor (Section 3.2 / 3.5)
 //   transform_stream        the butterfly alone, float output (parity export)
-//   dequantize_stream       decode (+ optional inverse butterfly, Section 3.2)
+//   decode_stream           decode (codes and scales -> values)
+//   dequantize_stream       decode + inverse butterfly (Section 3.2)
 //   fwht_quantize           full-d Walsh-Hadamard + encoder (the paper's FWHT comparison)
 #pragma once
 #include "kq_common.cuh"
@@ -306,6 +307,76 @@ fwht_quantize(const uint4* __restrict__ X, int64_t tokens, int d, float norm,
     }
 }
 
+// codes + scales -> values without an inverse transform, 16 channels (half a block) per thread: 8 bytes of codes in,
+// one full 32-byte sector (bf16) or two (float) out -- full-sector stores write about 1.5 times faster than 16-byte
+// ones here, and a decode is nearly all writes.  n_halves = tokens * d / 16 work items.
+template <bool OUT_BF16>
+__global__ void __launch_bounds__(256)
+decode_stream(const uint2* __restrict__ q_packed, const uint8_t* __restrict__ scales, int64_t n_halves, void* __restrict__ out) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t n_iter = (n_halves + stride * kStreamUnroll - 1) / (stride * kStreamUnroll);
+    int64_t h0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t it = 0; it < n_iter; ++it, h0 += stride * kStreamUnroll) {
+        uint2 codes_u[kStreamUnroll];
+        uint32_t S_u[kStreamUnroll];
+#pragma unroll
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            const int64_t h = h0 + u * stride;
+            codes_u[u] = make_uint2(0u, 0u);
+            S_u[u] = 127;
+            if (h < n_halves) {
+                codes_u[u] = __ldg(q_packed + h);
+                S_u[u] = __ldg(scales + (h >> 1));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kStreamUnroll; ++u) {
+            const int64_t h = h0 + u * stride;
+            if (h >= n_halves) continue;
+            const float sc = scale_from_e8m0(S_u[u]);
+            const uint32_t cw[2] = {codes_u[u].x, codes_u[u].y};
+            float y[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float2 v = e2m1x2_to_float2((cw[i >> 2] >> (8 * (i & 3))) & 0xFFu);
+                y[2 * i] = v.x * sc;
+                y[2 * i + 1] = v.y * sc;
+            }
+            if (OUT_BF16) {
+                uint32_t w[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const __nv_bfloat162 p = __floats2bfloat162_rn(y[2 * i], y[2 * i + 1]);
+                    w[i] = *reinterpret_cast<const uint32_t*>(&p);
+                }
+                uint32_t* op = reinterpret_cast<uint32_t*>(out) + 8 * h;
+                if ((reinterpret_cast<uintptr_t>(op) & 31u) == 0) {
+                    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                 ::"l"(op), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+                } else {
+                    st_stream_16(op, make_uint4(w[0], w[1], w[2], w[3]));
+                    st_stream_16(op + 4, make_uint4(w[4], w[5], w[6], w[7]));
+                }
+            } else {
+                float* op = reinterpret_cast<float*>(out) + 16 * h;
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                    if ((reinterpret_cast<uintptr_t>(op) & 31u) == 0) {
+                        asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                     ::"l"(op + 8 * v), "r"(__float_as_uint(y[8 * v])), "r"(__float_as_uint(y[8 * v + 1])),
+                                       "r"(__float_as_uint(y[8 * v + 2])), "r"(__float_as_uint(y[8 * v + 3])),
+                                       "r"(__float_as_uint(y[8 * v + 4])), "r"(__float_as_uint(y[8 * v + 5])),
+                                       "r"(__float_as_uint(y[8 * v + 6])), "r"(__float_as_uint(y[8 * v + 7])) : "memory");
+                    } else {
+                        reinterpret_cast<float4*>(op + 8 * v)[0] = make_float4(y[8 * v], y[8 * v + 1], y[8 * v + 2], y[8 * v + 3]);
+                        reinterpret_cast<float4*>(op + 8 * v)[1] = make_float4(y[8 * v + 4], y[8 * v + 5], y[8 * v + 6], y[8 * v + 7]);
+                    }
+                }
+            }
+        }
+    }
+}
+
 // codes + scales -> values.  Ginv: inverse factor sets (or nullptr: no inverse transform).
 template <bool OUT_BF16>
 __global__ void __launch_bounds__(256)
@@ -316,27 +387,36 @@ dequantize_stream(const uint32_t* __restrict__ q_packed, const uint8_t* __restri
     const int quad = threadIdx.x & 3;
     FactorSet F;
     if (Ginv != nullptr && n_sets == 1) F = Ginv[0];
-    const int64_t n_iter = (n_quads + stride - 1) / stride;
-    int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    for (int64_t it = 0; it < n_iter; ++it, q += stride) {
+    // kStreamUnroll items per thread and iteration: their loads are issued together (a single 4-byte load per
+    // iteration left the kernel waiting for one memory latency per item: 0.36 of the HBM rate)
+    const int64_t n_iter = (n_quads + stride * kStreamUnroll - 1) / (stride * kStreamUnroll);
+    int64_t q0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (int64_t it = 0; it < n_iter; ++it, q0 += stride * kStreamUnroll) {
+      uint32_t codes_u[kStreamUnroll], S_u[kStreamUnroll];
+#pragma unroll
+      for (int u = 0; u < kStreamUnroll; ++u) {
+          const int64_t qq = q0 + u * stride;
+          codes_u[u] = 0;
+          S_u[u] = 127;
+          if (qq < n_quads) {
+              codes_u[u] = __ldg(q_packed + qq);
+              S_u[u] = __ldg(scales + (qq >> 2));
+          }
+      }
+#pragma unroll
+      for (int u = 0; u < kStreamUnroll; ++u) {
+        const int64_t q = q0 + u * stride;
         const bool live = q < n_quads;
         const int64_t blk = q >> 2;
         float y[8];
-        uint32_t codes = 0, S = 127;
-        if (live) {
-            codes = __ldg(q_packed + q);
-            S = __ldg(scales + blk);
-        }
-        const float sc = scale_from_e8m0(S);
+        const uint32_t codes = codes_u[u];
+        const float sc = scale_from_e8m0(S_u[u]);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const uint32_t c = (codes >> (4 * i)) & 15u;
-            const uint32_t m = c & 7u;
-            // E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6: code 1 is the only subnormal
-            const float mag = (m < 2u) ? 0.5f * (float)m
-                                       : __uint_as_float(((126u + (m >> 1)) << 23) | ((m & 1u) << 22));
-            const float v = mag * sc;
-            y[i] = (c & 8u) ? -v : v;
+        for (int i = 0; i < 4; ++i) {
+            // two E2M1 codes per byte -> two halves by the hardware convert (exact), then the power-of-two scale
+            const float2 v = e2m1x2_to_float2((codes >> (8 * i)) & 0xFFu);
+            y[2 * i] = v.x * sc;
+            y[2 * i + 1] = v.y * sc;
         }
         if (Ginv != nullptr) {
             if (n_sets != 1) {
@@ -359,13 +439,23 @@ dequantize_stream(const uint32_t* __restrict__ q_packed, const uint8_t* __restri
                     b = (b + 0x7FFFu + ((b >> 16) & 1u)) >> 16;
                     w[i] = a | (b << 16);
                 }
-                reinterpret_cast<uint4*>(out)[q] = o;
+                st_stream_16(reinterpret_cast<uint4*>(out) + q, o);
             } else {
-                float4* op = reinterpret_cast<float4*>(out) + 2 * q;
-                op[0] = make_float4(y[0], y[1], y[2], y[3]);
-                op[1] = make_float4(y[4], y[5], y[6], y[7]);
+                // one full 32-byte sector per thread (the output is 16-byte aligned by contract: 32-byte aligned rows
+                // whenever the buffer itself is)
+                float* op = reinterpret_cast<float*>(out) + 8 * q;
+                if ((reinterpret_cast<uintptr_t>(op) & 31u) == 0) {
+                    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                                 ::"l"(op), "r"(__float_as_uint(y[0])), "r"(__float_as_uint(y[1])), "r"(__float_as_uint(y[2])),
+                                   "r"(__float_as_uint(y[3])), "r"(__float_as_uint(y[4])), "r"(__float_as_uint(y[5])),
+                                   "r"(__float_as_uint(y[6])), "r"(__float_as_uint(y[7])) : "memory");
+                } else {
+                    reinterpret_cast<float4*>(op)[0] = make_float4(y[0], y[1], y[2], y[3]);
+                    reinterpret_cast<float4*>(op)[1] = make_float4(y[4], y[5], y[6], y[7]);
+                }
             }
         }
+      }
     }
 }
 

@@ -983,10 +983,22 @@ kq_status_t kroquant_dequantize(const uint8_t* q_packed, const uint8_t* scales, 
     if (tokens == 0) return KQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t n_quads = tokens * (int64_t)(d / 8);
-    const int grid = stream_grid(n_quads);
+    const int grid = stream_grid((n_quads + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
     if (grid <= 0) return KQ_ERR_CUDA;
     const kq::FactorSet* gi = (f && !f->identity) ? f->d_Ginv : nullptr;
     const int ns = f ? f->n_sets : 0;
+    if (gi == nullptr) {
+        // no inverse transform: half a block per thread, full-sector stores
+        const int64_t n_halves = tokens * (int64_t)(d / 16);
+        const int grid_h = stream_grid((n_halves + kq::kStreamUnroll - 1) / kq::kStreamUnroll);
+        if (grid_h <= 0) return KQ_ERR_CUDA;
+        const uint2* q64 = reinterpret_cast<const uint2*>(q_packed);
+        if (out_dtype == KQ_OUT_BF16) kq::decode_stream<true><<<grid_h, 256, 0, st>>>(q64, scales, n_halves, out);
+        else kq::decode_stream<false><<<grid_h, 256, 0, st>>>(q64, scales, n_halves, out);
+        if (cudaGetLastError() != cudaSuccess) return KQ_ERR_CUDA;
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return KQ_OK;
+    }
     const uint32_t* q32 = reinterpret_cast<const uint32_t*>(q_packed);
     if (out_dtype == KQ_OUT_BF16)
         kq::dequantize_stream<true><<<grid, 256, 0, st>>>(q32, scales, n_quads, d / 32, gi, ns, out);
