@@ -114,6 +114,25 @@ def test_onchip_identity_factors_are_exact(B, dtype):
         P.check_codes(q.cpu().numpy(), s.cpu().numpy(), q_or, s_or, Y, exact=True)
 
 
+@pytest.mark.parametrize("per_block", [False, True])
+def test_onchip_factor_sets_of_extreme_scale(B, per_block):
+    """Factor entries far from 1 (K scaled by 2^+-20, one factor nearly singular): the compensated products and the
+    three-term split must hold up, and the scale bytes move with the factor of two."""
+    tokens, d = 300, 1152
+    Xb = W.gen_activations(spec(tokens, d, 17))
+    for pw in (20, -20):
+        G = W.gen_factors(31, n_sets=d // 32 if per_block else 1)
+        G[:, 0] *= np.float32(2.0 ** pw)
+        G[:, 3, 1, :] *= np.float32(1e-3)                      # a small second row: |det G4| shrinks a thousandfold
+        X, f = dev(Xb), B.Factors.create(G)
+        q, s = B.kroquant_quantize(X, f, path="onchip")
+        Yg = B.kroquant_transform_f32(X, f, path="onchip")
+        qo, so, Y = co.quantize(Xb, G)
+        P.check_values(Yg.cpu().numpy(), Y)
+        P.check_codes(q.cpu().numpy(), s.cpu().numpy(), qo, so, Y, exact=False)
+    assert B.kroquant_last_device_error() == 0
+
+
 def test_onchip_back_to_back_and_tuned_calls_agree(B):
     # the builders run ahead of and behind the dependency wait of chained launches: every call must give the same bytes
     tokens, d = 2500, 2240

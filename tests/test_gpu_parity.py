@@ -158,6 +158,34 @@ def test_power_of_two_equivariance_on_gpu(B):
 
 
 # ---- decode ----------------------------------------------------------------------------------
+def test_decode_every_code_under_every_scale_byte(B):
+    """All 256 code bytes under all 255 valid scale bytes (S = 0 decodes to subnormal floats, S = 254 to 6 * 2^127),
+    both output types, bit for bit; and shapes whose size is no multiple of what a thread or a CTA takes."""
+    codes = np.arange(256, dtype=np.uint8)
+    q_or = np.tile(codes, (255, 1)).reshape(255, 16, 16)               # row S: 16 blocks, every byte value once
+    q_or = np.ascontiguousarray(q_or.reshape(255, 256))                # tokens = 255, d = 512
+    s_or = np.repeat(np.arange(255, dtype=np.uint8)[:, None], 16, axis=1)
+    q, s = torch.from_numpy(q_or).cuda(), torch.from_numpy(s_or).cuda()
+    out = host(B.kroquant_dequantize(q, s))
+    ref = co.dequantize(q_or, s_or)
+    assert np.array_equal(out.view(np.uint32), ref.view(np.uint32))     # bit patterns: signed zeros and subnormals included
+    outb = host(B.kroquant_dequantize(q, s, out_dtype=torch.bfloat16).view(torch.int16)).view(np.uint16)
+    assert np.array_equal(outb, co.dequantize(q_or, s_or, out_bf16=True))
+    for tokens, d in [(1, 32), (3, 96), (257, 1152), (1000, 2240)]:
+        rng = np.random.default_rng(tokens)
+        q_or = rng.integers(0, 256, (tokens, d // 2), dtype=np.uint8)
+        s_or = rng.integers(100, 150, (tokens, d // 32), dtype=np.uint8)
+        q, s = torch.from_numpy(q_or).cuda(), torch.from_numpy(s_or).cuda()
+        guard = torch.full((tokens * d + 64,), -7.0, dtype=torch.float32, device="cuda")
+        out = guard[32:32 + tokens * d].view(tokens, d)                 # 128-byte offset: canaries on both sides
+        B.kroquant_dequantize(q, s, out=out)
+        assert np.array_equal(host(out).view(np.uint32), co.dequantize(q_or, s_or).view(np.uint32))
+        assert (guard[:32] == -7.0).all() and (guard[32 + tokens * d:] == -7.0).all()
+        out4 = guard[4:4 + tokens * d].view(tokens, d)                  # 16-byte but not 32-byte aligned: the narrow stores
+        B.kroquant_dequantize(q, s, out=out4)
+        assert np.array_equal(host(out4).view(np.uint32), co.dequantize(q_or, s_or).view(np.uint32))
+
+
 def test_dequantize(B):
     Xb = W.gen_activations(spec(200, 1152, seed=6))
     G = W.gen_factors(6)
