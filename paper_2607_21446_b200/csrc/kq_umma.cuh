@@ -526,6 +526,7 @@ struct UmmaProblem {
     int unit_tiles;      // PB=false: consecutive tiles per work unit (PB: kPbCols)
     int tl_slot;         // timeline builds: which launch slot of the mark buffer this launch writes
     float norm;          // Hadamard comparison: 1 / sqrt(d)
+    int images_early;    // per-block sets: copy the first unit's operand images ahead of the dependency wait
     int had_rows;        // Hadamard comparison: tile rows that make one token (d/32 up to d = 4096, then 128)
     int dynamic;         // 1: the grid has one CTA per unit and running CTAs take over the units of CTAs that
                          // have not started yet (cluster launch control); 0: CTA b takes units b, b + gridDim.x, ...
@@ -839,6 +840,19 @@ quantize_umma(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant_
             }
         } else if (prob.prefetch_tiles > 0) {
             prefetch_tile(PB ? (int)unit : (int)(unit * tpu), 0);
+        }
+        if (PB && !BUILD && prob.images_early) {
+            // The operand images of the CTA's first unit are immutable inputs: their copies go out ahead of the
+            // dependency wait (the tile's barrier is told to expect the bytes, without an arrival; the tile's own
+            // copy, issued behind the wait, finds the image "already in place")
+            int j, jg, tt;
+            for (int c = 0; c < kPbCols && c < NS; ++c) {
+                pb_coords((int)unit, c, j, jg, tt);
+                const int jb = j < prob.blocks_per_row ? j : prob.blocks_per_row - 1;
+                asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar_full(c)), "r"((uint32_t)kBImageBytes) : "memory");
+                bulk_load(base + L::kAOff + c * L::kStageBytes + kTileBytes, b_image + (size_t)jb * kBImageBytes, kBImageBytes, bar_full(c));
+                slot_jg[c] = jg;
+            }
         }
         pdl_wait_prior_grid();
         KQ_TL_MARK(prob.tl_slot, 1);

@@ -5,7 +5,6 @@
 
 #include <atomic>
 #include <cmath>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -275,7 +274,7 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     if (!enc) return KQ_ERR_CUDA;
     const bool pb = f->n_sets != 1;
     const int nb = d / 32;
-    kq::UmmaProblem prob;
+    kq::UmmaProblem prob{};
     prob.blocks_per_row = nb;
     prob.tiled_scales = tiled ? 1 : 0;
     prob.early_trigger = (t_tuning.use_pdl != 0 && calib_sumsq == nullptr) ? t_tuning.trigger : 0;
@@ -283,6 +282,8 @@ kq_status_t run_umma(const void* X, bool xf16, int64_t tokens, int d, const kroq
     prob.dynamic = t_tuning.dynamic;
     prob.tl_slot = g_tl_next.fetch_add(1) % 64;
     prob.unit_tiles = pb ? kq::kPbCols : (t_tuning.unit_tiles > 0 ? t_tuning.unit_tiles : 3);
+    // (the calibration loop writes the operand images in the kernel just before: nothing of them may be read early)
+    prob.images_early = (calib_sumsq == nullptr && t_tuning.use_pdl != 0) ? 1 : 0;
     CUtensorMap tmap;
     cuuint64_t dims[2], strides[1];
     if (pb) {
@@ -410,7 +411,7 @@ kq_status_t run_flat_staged(const void* X, bool xf16, int64_t tokens, int d, con
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return KQ_ERR_CUDA;
     const int nb = d / 32;
-    kq::UmmaProblem prob;
+    kq::UmmaProblem prob{};
     prob.blocks_per_row = nb;
     prob.tiled_scales = tiled ? 1 : 0;
     prob.early_trigger = t_tuning.use_pdl != 0 ? t_tuning.trigger : 0;
@@ -505,7 +506,7 @@ kq_status_t run_fwht_umma(const void* X, bool xf16, int64_t tokens, int d, uint8
     // block, the mixing across the ht blocks of a row is a pass through tensor memory.  Measured best: 4 from d = 4096
     // on (a token is then 32 rows and more), 2 below, single blocks only for d = 32.
     const int ht = nb >= 128 ? 4 : nb >= 2 ? 2 : 1;
-    kq::UmmaProblem prob;
+    kq::UmmaProblem prob{};
     prob.blocks_per_row = nb;
     prob.had_rows = nb / ht;
     prob.tiled_scales = 0;
