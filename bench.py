@@ -71,6 +71,14 @@ class ClockSampler:
         self.index = index
         self.proc = None
         self.lines: list[str] = []
+        self.first = 0            # samples [first, last) were taken between mark_begin() and mark_end()
+        self.last = None
+
+    def mark_begin(self):
+        self.first = len(self.lines)
+
+    def mark_end(self):
+        self.last = len(self.lines)
 
     def start(self):
         try:
@@ -99,7 +107,10 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        # the samples of the marked region and one on either side of it (all of them if nothing was marked)
+        lo = max(0, self.first - 1)
+        hi = len(self.lines) if self.last is None else min(len(self.lines), self.last + 1)
+        for ln in self.lines[lo:hi]:
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 7:
                 continue
@@ -337,30 +348,31 @@ def capture_overlapped(torch, calls, fn, stream, n_streams=3):
 
 def time_graph(torch, dist, g, stream, steps, warmup, sampler=None):
     """W untimed replays, then exactly `steps` timed replays between two events on `stream`.
-    The clock sampler (nvidia-smi, 20 ms period) is started before the warm-up; extra
-    untimed replays keep the GPU under the same load until its first samples arrive and
-    until one more arrives after the timed region, so the samples bracket and cover it."""
+    The clock sampler (nvidia-smi, 20 ms period) is started first and the GPU idles until its first samples have
+    arrived (the tool takes some hundred milliseconds to start); the reported clocks are those of the samples taken
+    during the timed region and of one on either side; untimed replays keep the load up until that last one arrives."""
     with torch.cuda.stream(stream):
         if sampler:
             sampler.start()
+            t_end = time.perf_counter() + 4.0
+            while sampler.proc is not None and sampler.count() < 2 and time.perf_counter() < t_end:
+                time.sleep(0.01)
         for _ in range(warmup):
             g.replay()
-        if sampler and sampler.proc is not None:
-            t_end = time.perf_counter() + 4.0
-            while sampler.count() < 3 and time.perf_counter() < t_end:
-                for _ in range(20):
-                    g.replay()
-                torch.cuda.synchronize()
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if sampler:
+            sampler.mark_begin()
         a.record(stream)
         for _ in range(steps):
             g.replay()
         b.record(stream)
         torch.cuda.synchronize()
+        if sampler:
+            sampler.mark_end()
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
