@@ -601,6 +601,7 @@ def run_single(args):
     sv = torch.from_numpy(W.gen_channel_scales(3, d)).cuda()
     fn = {"kroquant": lambda x: B.kroquant_quantize(x, f, q, sc),
           "kroquant_onchip": lambda x: B.kroquant_quantize(x, f, q, sc, path="onchip"),
+          "fwht": lambda x: B.kroquant_fwht_quantize(x, q, sc),
           "scale": lambda x: B.kroquant_scale_quantize(x, sv, q, sc),
           "plain": lambda x: B.kroquant_mxfp4_quantize(x, q, sc)}[args.kernel]
     torch.cuda.synchronize()
@@ -1117,7 +1118,7 @@ def main():
     ap.add_argument("--points", default=None, metavar="TOKENSxD,...", help="with --sweep: only these points")
     ap.add_argument("--single", default=None, metavar="TOKENSxD",
                     help="profiling aid: a few eager launches of one shape, e.g. 4608x12288")
-    ap.add_argument("--kernel", default="kroquant", choices=["kroquant", "kroquant_onchip", "scale", "plain"])
+    ap.add_argument("--kernel", default="kroquant", choices=["kroquant", "kroquant_onchip", "fwht", "scale", "plain"])
     ap.add_argument("--calls", type=int, default=8)
     ap.add_argument("--per-block", action="store_true", help="with --single: one factor set per 32-channel block")
     ap.add_argument("--calib", default=None, metavar="MxOxD",
