@@ -29,6 +29,11 @@
 // Every mbarrier wait is bounded; a wait that gives up records a code in
 // g_kq_device_error, raises the CTA's abort flag and the CTA drains and frees
 // its TMEM before returning.
+//
+// The same kernel template also serves (template parameters PB, EXTRA, OP, HT; each described at the kernel):
+// per-block factor sets, the second 16-bit output and the calibration outputs, the operand built on chip from the
+// factor scalars, the comparison quantizers on the same pipeline without the tensor-core stage (bare MXFP4, per-channel
+// scale), and the full-row Walsh-Hadamard comparison.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
